@@ -1,0 +1,284 @@
+// Decoding: interpolate the product polynomial from the evaluations of the nodes in use and
+// keep the wanted coefficients (Theorem 2's proof; the Vandermonde system of the decoding
+// appendix).  Done as one small FP64 factorisation followed by a bandwidth-bound streaming pass:
+//
+//   1. decode_matrix_kernel (one warp): Householder QR of the |S| x Q Vandermonde matrix of the
+//      nodes in use; row w of D = e_w^T R^-1 Q^T is the linear functional that reads coefficient
+//      w of the least-squares polynomial off the node values.  Normal equations are never
+//      formed (the Vandermonde matrix is too ill-conditioned for that at thresholds near 30).
+//   2. decode_stream_kernel: out_block(w)[pos] = sum_p D[w][p] * Z[p][pos], each worker output
+//      read once with 16-byte loads, FP64 accumulation, FP32 store into the right block of the
+//      result; optional fused activation (step C1).
+#include "gpd_internal.h"
+
+namespace gpd {
+
+namespace {
+
+struct MatrixParams {
+    const double* points;            // [P]
+    double* D;                       // [n_wanted][P]
+    int* gate;                       // [0] = 1 if the stream kernel may run
+    const gpd_locate_result* result; // used when have_mask == 0
+    unsigned long long use_mask;
+    int have_mask;
+    int P, Q, n_wanted;
+    int wanted[kMaxWanted];
+};
+
+__global__ void __launch_bounds__(32) decode_matrix_kernel(MatrixParams prm) {
+    __shared__ double A[kMaxNodes][kMaxQ + 1];       // Vandermonde rows of the nodes in use -> R
+    __shared__ double Vh[kMaxNodes][kMaxQ + 1];      // Householder vectors (column k = reflector k)
+    __shared__ int node_of[kMaxNodes];
+    __shared__ int s_rows;
+    const int lane = threadIdx.x;
+    const int P = prm.P, Q = prm.Q;
+    if (lane == 0) {
+        int rows = 0;
+        bool ok = true;
+        if (prm.have_mask) {
+            for (int p = 0; p < P; ++p)
+                if ((prm.use_mask >> p) & 1ULL) node_of[rows++] = p;
+        } else {
+            ok = prm.result->outcome != GPD_DECODE_FAILURE;
+            for (int p = 0; p < P; ++p)
+                if (!prm.result->flagged[p]) node_of[rows++] = p;
+        }
+        if (rows < Q) ok = false;                    // fewer clean nodes than the threshold
+        s_rows = ok ? rows : 0;
+        prm.gate[0] = ok ? 1 : 0;
+    }
+    __syncwarp();
+    const int rows = s_rows;
+    for (int i = lane; i < prm.n_wanted * P; i += 32) prm.D[i] = 0.0;
+    if (rows == 0) return;
+    for (int r = lane; r < rows; r += 32) {
+        const double b = prm.points[node_of[r]];
+        double acc = 1.0;
+        for (int c = 0; c < Q; ++c) { A[r][c] = acc; acc *= b; }
+    }
+    __syncwarp();
+    // Householder triangularisation; lane c owns column c
+    for (int k = 0; k < Q; ++k) {
+        double sigma = 0.0;
+        for (int r = k; r < rows; ++r) sigma += A[r][k] * A[r][k];     // every lane, same value
+        const double akk = A[k][k];
+        const double alpha = akk >= 0.0 ? -sqrt(sigma) : sqrt(sigma);
+        const double vnorm = sqrt(fmax(sigma - 2.0 * alpha * akk + alpha * alpha, 1e-300));
+        __syncwarp();
+        for (int r = k + lane; r < rows; r += 32) Vh[r][k] = (A[r][k] - (r == k ? alpha : 0.0)) / vnorm;
+        __syncwarp();
+        if (lane >= k && lane < Q) {
+            double dot = 0.0;
+            for (int r = k; r < rows; ++r) dot += Vh[r][k] * A[r][lane];
+            for (int r = k; r < rows; ++r) A[r][lane] -= 2.0 * dot * Vh[r][k];
+        }
+        __syncwarp();
+    }
+    // row w of the pseudo-inverse: solve R^T y = e_w, then x = H_0 H_1 ... H_{Q-1} [y; 0]
+    for (int wi = lane; wi < prm.n_wanted; wi += 32) {
+        const int w = prm.wanted[wi];
+        double y[kMaxQ];
+        for (int i = 0; i < Q; ++i) {
+            double rhs = i == w ? 1.0 : 0.0;
+            for (int j = 0; j < i; ++j) rhs -= A[j][i] * y[j];
+            y[i] = rhs / A[i][i];
+        }
+        double x[kMaxNodes];
+        for (int r = 0; r < rows; ++r) x[r] = r < Q ? y[r] : 0.0;
+        for (int k = Q - 1; k >= 0; --k) {
+            double dot = 0.0;
+            for (int r = k; r < rows; ++r) dot += Vh[r][k] * x[r];
+            for (int r = k; r < rows; ++r) x[r] -= 2.0 * dot * Vh[r][k];
+        }
+        for (int r = 0; r < rows; ++r) prm.D[wi * P + node_of[r]] = x[r];
+    }
+}
+
+struct StreamParams {
+    const void* Z;             // [P][br*bc]
+    const double* D;           // [n_wanted][P]
+    const int* gate;
+    float* out;                // result matrix, leading dimension ldo
+    float* act_out;            // optional
+    int64_t br, bc, ldo;
+    int P, n_wanted, grid_cols;
+    int activation;
+};
+
+__device__ __forceinline__ float apply_act(float v, int kind) {
+    if (kind == GPD_ACT_RELU) return v > 0.f ? v : 0.f;
+    if (kind == GPD_ACT_SIGMOID) return 1.f / (1.f + __expf(-v));
+    return v;
+}
+
+template <typename T> struct Vec;
+template <> struct Vec<float> {
+    static constexpr int N = 4;
+    __device__ static void load(const float* p, double (&v)[4]) {
+        const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+};
+template <> struct Vec<double> {
+    static constexpr int N = 2;
+    __device__ static void load(const double* p, double (&v)[2]) {
+        const double2 t = __ldcs(reinterpret_cast<const double2*>(p));
+        v[0] = t.x; v[1] = t.y;
+    }
+};
+
+// NW wanted coefficients per pass over the inputs; VECTOR: 16-byte loads of N positions.
+template <typename T, int NW, bool VECTOR>
+__global__ void __launch_bounds__(256) decode_stream_kernel(StreamParams prm) {
+    if (prm.gate[0] == 0) return;
+    extern __shared__ double sD[];                   // [n_wanted][P]
+    __shared__ int s_nodes[kMaxNodes];
+    __shared__ int s_nused;
+    for (int i = threadIdx.x; i < prm.n_wanted * prm.P; i += blockDim.x) sD[i] = prm.D[i];
+    __syncthreads();
+    if (threadIdx.x == 0) {                          // nodes with an all-zero column are not read
+        int n = 0;
+        for (int p = 0; p < prm.P; ++p) {
+            bool used = false;
+            for (int w = 0; w < prm.n_wanted; ++w) used |= sD[w * prm.P + p] != 0.0;
+            if (used) s_nodes[n++] = p;
+        }
+        s_nused = n;
+    }
+    __syncthreads();
+    constexpr int N = VECTOR ? Vec<T>::N : 1;
+    const T* Z = reinterpret_cast<const T*>(prm.Z);
+    const int64_t L = prm.br * prm.bc;
+    const int64_t groups = VECTOR ? L / N : L;
+    for (int64_t gidx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; gidx < groups;
+         gidx += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t pos = gidx * N;
+        const int64_t row = pos / prm.bc, col = pos - row * prm.bc;
+        for (int w0 = 0; w0 < prm.n_wanted; w0 += NW) {
+            double acc[NW][N];
+#pragma unroll
+            for (int w = 0; w < NW; ++w)
+#pragma unroll
+                for (int v = 0; v < N; ++v) acc[w][v] = 0.0;
+            for (int i = 0; i < s_nused; ++i) {
+                const int p = s_nodes[i];
+                double z[N];
+                if constexpr (VECTOR) Vec<T>::load(Z + (int64_t)p * L + pos, z);
+                else z[0] = (double)__ldcs(Z + (int64_t)p * L + pos);
+#pragma unroll
+                for (int w = 0; w < NW; ++w) {
+                    const double d = (w0 + w < prm.n_wanted) ? sD[(w0 + w) * prm.P + p] : 0.0;
+#pragma unroll
+                    for (int v = 0; v < N; ++v) acc[w][v] = fma(d, z[v], acc[w][v]);
+                }
+            }
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const int wi = w0 + w;
+                if (wi >= prm.n_wanted) break;
+                const int gr = wi / prm.grid_cols, gc = wi - gr * prm.grid_cols;
+                const int64_t o = (gr * prm.br + row) * prm.ldo + gc * prm.bc + col;
+                if constexpr (VECTOR && N == 4) {
+                    const float4 v = make_float4((float)acc[w][0], (float)acc[w][1], (float)acc[w][2], (float)acc[w][3]);
+                    *reinterpret_cast<float4*>(prm.out + o) = v;
+                    if (prm.act_out)
+                        *reinterpret_cast<float4*>(prm.act_out + o) =
+                            make_float4(apply_act(v.x, prm.activation), apply_act(v.y, prm.activation),
+                                        apply_act(v.z, prm.activation), apply_act(v.w, prm.activation));
+                } else if constexpr (VECTOR && N == 2) {
+                    const float2 v = make_float2((float)acc[w][0], (float)acc[w][1]);
+                    *reinterpret_cast<float2*>(prm.out + o) = v;
+                    if (prm.act_out)
+                        *reinterpret_cast<float2*>(prm.act_out + o) =
+                            make_float2(apply_act(v.x, prm.activation), apply_act(v.y, prm.activation));
+                } else {
+                    prm.out[o] = (float)acc[w][0];
+                    if (prm.act_out) prm.act_out[o] = apply_act((float)acc[w][0], prm.activation);
+                }
+            }
+        }
+    }
+}
+
+template <typename T, int NW, bool VECTOR>
+void launch_stream(const StreamParams& prm, cudaStream_t st) {
+    constexpr int N = VECTOR ? Vec<T>::N : 1;
+    const int64_t groups = prm.br * prm.bc / N;
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((groups + 255) / 256, 148 * 8));
+    decode_stream_kernel<T, NW, VECTOR><<<grid, 256, sizeof(double) * prm.n_wanted * prm.P, st>>>(prm);
+}
+
+template <typename T>
+gpd_status dispatch_stream(const StreamParams& prm, cudaStream_t st) {
+    constexpr int N = Vec<T>::N;
+    const bool vec = (prm.bc % N == 0) && (prm.ldo % N == 0) &&
+                     (reinterpret_cast<uintptr_t>(prm.Z) % 16 == 0) &&
+                     (reinterpret_cast<uintptr_t>(prm.out) % 16 == 0) &&
+                     (!prm.act_out || reinterpret_cast<uintptr_t>(prm.act_out) % 16 == 0) &&
+                     ((prm.br * prm.bc) % N == 0);
+    if (vec) {
+        if (prm.n_wanted <= 4) launch_stream<T, 4, true>(prm, st);
+        else if (prm.n_wanted <= 8) launch_stream<T, 8, true>(prm, st);
+        else launch_stream<T, 16, true>(prm, st);
+    } else {
+        if (prm.n_wanted <= 4) launch_stream<T, 4, false>(prm, st);
+        else launch_stream<T, 16, false>(prm, st);
+    }
+    return launch_ok();
+}
+
+}  // namespace
+
+gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, bool have_mask,
+                         uint64_t use_mask, const gpd_locate_result* result, float* out, float* act_out,
+                         int activation, void* workspace, cudaStream_t st) {
+    if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
+    const ProductInfo& pi = plan->prod[which];
+    if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
+    gpd_status rc = ensure_device(plan);
+    if (rc != GPD_OK) return rc;
+    const WorkspaceLayout wl = workspace_layout();
+    char* ws = reinterpret_cast<char*>(workspace);
+    MatrixParams mp{};
+    mp.points = plan->dev.base + plan->dev.off_points;
+    mp.D = reinterpret_cast<double*>(ws + wl.off_decode);
+    mp.gate = reinterpret_cast<int*>(ws + wl.off_flags);
+    mp.result = result;
+    mp.use_mask = use_mask;
+    mp.have_mask = have_mask ? 1 : 0;
+    mp.P = plan->P; mp.Q = pi.Q; mp.n_wanted = pi.grid_rows * pi.grid_cols;
+    for (int i = 0; i < mp.n_wanted; ++i) mp.wanted[i] = pi.wanted[i];
+    decode_matrix_kernel<<<1, 32, 0, st>>>(mp);
+    rc = launch_ok();
+    if (rc != GPD_OK) return rc;
+    StreamParams sp{};
+    sp.Z = outputs; sp.D = mp.D; sp.gate = mp.gate; sp.out = out; sp.act_out = act_out;
+    sp.br = pi.br; sp.bc = pi.bc; sp.ldo = pi.bc * pi.grid_cols;
+    sp.P = plan->P; sp.n_wanted = mp.n_wanted; sp.grid_cols = pi.grid_cols;
+    sp.activation = activation;
+    return plan->elem_size == 4 ? dispatch_stream<float>(sp, st) : dispatch_stream<double>(sp, st);
+}
+
+}  // namespace gpd
+
+using namespace gpd;
+
+extern "C" gpd_status gpd_decode(gpd_plan_t plan, gpd_product which, const void* outputs_dev,
+                                 const uint8_t* use_mask_host, const gpd_locate_result* result_dev,
+                                 float* out_dev, float* act_out_dev, gpd_activation_kind activation,
+                                 void* workspace_dev, void* stream) {
+    if (!plan || !outputs_dev || !out_dev) return GPD_ERR_ARG;
+    if (!use_mask_host && !result_dev) return GPD_ERR_ARG;
+    if (!workspace_dev) return GPD_ERR_WORKSPACE;
+    uint64_t mask = 0;
+    if (use_mask_host) {
+        int n = 0;
+        for (int p = 0; p < plan->P; ++p)
+            if (use_mask_host[p]) { mask |= 1ULL << p; ++n; }
+        if (which >= 0 && which <= GPD_AUDIT && which != GPD_UPD && n < plan->prod[which].Q)
+            return GPD_ERR_P_TOO_SMALL;
+    }
+    return decode_launch(plan, which, outputs_dev, use_mask_host != nullptr, mask, result_dev, out_dev,
+                         act_out_dev, (int)activation, workspace_dev, as_stream(stream));
+}

@@ -1,0 +1,191 @@
+// FP64 worker products on the FP64 tensor-core path (mma.sync m8n8k4 f64), batched over the
+// P nodes.  Used when the recovery threshold is large enough that interpolation amplifies
+// FP32-level noise beyond the 1e-4 accuracy target (thresholds above 9), so shares, products
+// and outputs stay in FP64.  tcgen05 has no FP64 kind; this is the chip's native FP64 matrix path.
+//
+// CTA tile 128 x 128, K step 16, 8 warps (2 x 4), warp tile 64 x 32 = 8 x 4 MMA tiles.
+// Operands are staged with 16-byte cp.async into a 3-stage ring; rows are padded by 4 doubles
+// so that the 64-bit fragment loads of each half-warp hit 16 distinct bank pairs.
+#include "gemm_common.h"
+
+namespace gpd {
+
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 16, STAGES = 3;
+constexpr int A_LD = BK + 4;                  // A tile  [BM][A_LD]
+constexpr int BK_LD = BK + 4;                 // B tile, K-major source: [BN][BK_LD]
+constexpr int BN_LD = BN + 4;                 // B tile, N-major source: [BK][BN_LD]
+constexpr int A_STAGE = BM * A_LD;
+constexpr int B_STAGE_KMAJOR = BN * BK_LD;
+constexpr int B_STAGE_NMAJOR = BK * BN_LD;
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem, bool valid) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    const int bytes = valid ? 16 : 0;         // src-size 0: destination is zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+__device__ __forceinline__ void dmma(double& d0, double& d1, double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};\n"
+                 : "+d"(d0), "+d"(d1)
+                 : "d"(a), "d"(b));
+}
+
+template <bool B_KMAJOR, bool UPDATE>
+__global__ void __launch_bounds__(256, 1) dgemm_mma_kernel(GemmParams prm) {
+    if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
+    extern __shared__ __align__(16) double smem[];
+    constexpr int B_STAGE = B_KMAJOR ? B_STAGE_KMAJOR : B_STAGE_NMAJOR;
+    double* sA = smem;
+    double* sB = smem + STAGES * A_STAGE;
+
+    const int p = blockIdx.z;
+    const double* A = reinterpret_cast<const double*>(prm.A) + (int64_t)p * prm.M * prm.K;
+    const double* B = reinterpret_cast<const double*>(prm.B) + (int64_t)p * prm.K * prm.N;
+    double* C = reinterpret_cast<double*>(prm.C) + (int64_t)p * prm.M * prm.N;
+    const int64_t m0 = (int64_t)blockIdx.y * BM, n0 = (int64_t)blockIdx.x * BN;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int wm = warp >> 2, wn = warp & 3;
+    const int g = lane >> 2, t = lane & 3;
+
+    auto load_stage = [&](int stage, int64_t k0) {
+        double* a = sA + stage * A_STAGE;
+        double* b = sB + stage * B_STAGE;
+        // A tile: 128 rows x 8 chunks of 2 doubles
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = tid + i * 256;
+            const int row = c >> 3, ch = c & 7;
+            const int64_t gm = m0 + row, gk = k0 + ch * 2;
+            const bool ok = gm < prm.M && gk < prm.K;
+            cp_async16(a + row * A_LD + ch * 2, ok ? (const void*)(A + gm * prm.K + gk) : (const void*)A, ok);
+        }
+        if (B_KMAJOR) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int c = tid + i * 256;
+                const int row = c >> 3, ch = c & 7;
+                const int64_t gn = n0 + row, gk = k0 + ch * 2;
+                const bool ok = gn < prm.N && gk < prm.K;
+                cp_async16(b + row * BK_LD + ch * 2, ok ? (const void*)(B + gn * prm.K + gk) : (const void*)B, ok);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int c = tid + i * 256;
+                const int kr = c >> 6, ch = c & 63;
+                const int64_t gk = k0 + kr, gn = n0 + ch * 2;
+                const bool ok = gk < prm.K && gn < prm.N;
+                cp_async16(b + kr * BN_LD + ch * 2, ok ? (const void*)(B + gk * prm.N + gn) : (const void*)B, ok);
+            }
+        }
+    };
+
+    double acc[8][4][2];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+
+    const int64_t ktiles = (prm.K + BK - 1) / BK;
+#pragma unroll
+    for (int s = 0; s < STAGES - 1; ++s) {
+        if (s < ktiles) load_stage(s, (int64_t)s * BK);
+        cp_async_commit();
+    }
+    for (int64_t kt = 0; kt < ktiles; ++kt) {
+        cp_async_wait<STAGES - 2>();
+        __syncthreads();
+        const int64_t nxt = kt + STAGES - 1;
+        if (nxt < ktiles) load_stage((int)(nxt % STAGES), nxt * BK);
+        cp_async_commit();
+        const double* a = sA + (kt % STAGES) * A_STAGE + (wm * 64 + g) * A_LD + t;
+        const double* b = sB + (kt % STAGES) * B_STAGE;
+#pragma unroll
+        for (int kk = 0; kk < BK; kk += 4) {
+            double af[8], bf[4];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) af[i] = a[i * 8 * A_LD + kk];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int col = wn * 32 + j * 8 + g;
+                bf[j] = B_KMAJOR ? b[col * BK_LD + kk + t] : b[(kk + t) * BN_LD + col];
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) dmma(acc[i][j][0], acc[i][j][1], af[i], bf[j]);
+        }
+    }
+    cp_async_wait<0>();
+
+    // epilogue: each thread owns two adjacent columns of one row per MMA tile
+    const bool n_even = (prm.N & 1) == 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int64_t gm = m0 + wm * 64 + i * 8 + g;
+        if (gm >= prm.M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t gn = n0 + wn * 32 + j * 8 + t * 2;
+            if (gn >= prm.N) continue;
+            double* c = C + gm * prm.N + gn;
+            double v0 = acc[i][j][0], v1 = acc[i][j][1];
+            if (n_even) {                                   // gn even and N even: 16-byte aligned pair
+                if (UPDATE) {
+                    const double2 old = *reinterpret_cast<const double2*>(c);
+                    v0 = prm.shrink * old.x + prm.eta * v0;
+                    v1 = prm.shrink * old.y + prm.eta * v1;
+                }
+                *reinterpret_cast<double2*>(c) = make_double2(v0, v1);
+            } else {
+                if (UPDATE) v0 = prm.shrink * c[0] + prm.eta * v0;
+                c[0] = v0;
+                if (gn + 1 < prm.N) {
+                    if (UPDATE) v1 = prm.shrink * c[1] + prm.eta * v1;
+                    c[1] = v1;
+                }
+            }
+        }
+    }
+}
+
+template <bool B_KMAJOR, bool UPDATE>
+gpd_status launch(const GemmParams& prm, cudaStream_t st) {
+    constexpr int B_STAGE = B_KMAJOR ? B_STAGE_KMAJOR : B_STAGE_NMAJOR;
+    constexpr size_t smem = sizeof(double) * STAGES * (A_STAGE + B_STAGE);
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(dgemm_mma_kernel<B_KMAJOR, UPDATE>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return GPD_ERR_CUDA;
+        configured = true;
+    }
+    dim3 grid((unsigned)((prm.N + BN - 1) / BN), (unsigned)((prm.M + BM - 1) / BM), (unsigned)prm.P);
+    dgemm_mma_kernel<B_KMAJOR, UPDATE><<<grid, 256, smem, st>>>(prm);
+    return launch_ok();
+}
+
+}  // namespace
+
+bool dgemm_mma_supported(const GemmParams& prm) {
+    // 16-byte cp.async needs even leading dimensions and 16-byte aligned bases
+    const bool aligned = reinterpret_cast<uintptr_t>(prm.A) % 16 == 0 &&
+                         reinterpret_cast<uintptr_t>(prm.B) % 16 == 0 &&
+                         reinterpret_cast<uintptr_t>(prm.C) % 16 == 0;
+    const bool lds = (prm.K % 2 == 0) && (prm.b_kmajor || prm.N % 2 == 0);
+    // (K even makes every per-node operand base 16-byte aligned; an odd N takes scalar stores)
+    return aligned && lds && prm.M >= 16 && prm.N >= 8;
+}
+
+gpd_status dgemm_mma_launch(const GemmParams& prm, cudaStream_t st) {
+    if (prm.b_kmajor)
+        return prm.update ? launch<true, true>(prm, st) : launch<true, false>(prm, st);
+    return prm.update ? launch<false, true>(prm, st) : launch<false, false>(prm, st);
+}
+
+}  // namespace gpd

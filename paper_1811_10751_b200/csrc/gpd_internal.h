@@ -1,0 +1,103 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <mutex>
+#include <vector>
+
+#include "gpd.h"
+
+namespace gpd {
+
+constexpr int kMaxNodes = GPD_MAX_NODES;
+constexpr int kMaxQ = GPD_MAX_THRESHOLD;
+constexpr int kMaxR = GPD_MAX_PARITY;
+constexpr int kMaxBlocks = 64;   // blocks combined by one encoding polynomial (m*n, n*d1, d2*m)
+constexpr int kMaxWanted = 64;   // wanted coefficients of one product (m*d1, d2*n, m*n)
+
+// Zero tests of the locator in floating point (engineering constants, chosen from the noise
+// floor of each storage type; the paper works in exact real arithmetic).
+constexpr double kTauColFp32 = 1.220703125e-4;           // 2^-13
+constexpr double kTauInFp32 = 3.0517578125e-5;           // 2^-15
+constexpr double kTauColFp64 = 9.5367431640625e-7;       // 2^-20
+constexpr double kTauInFp64 = 9.313225746154785e-10;     // 2^-30
+
+// Geometry of one decodable product (forward, backward or audit).
+struct ProductInfo {
+    int Q = 0;             // recovery threshold = number of polynomial coefficients
+    int R = 0;             // P - Q parity checks
+    int grid_rows = 0;     // wanted block grid (m x d1, d2 x n, m x n)
+    int grid_cols = 0;
+    int64_t br = 0;        // rows / cols of one worker output = one result block
+    int64_t bc = 0;
+    int wanted[kMaxWanted] = {0};   // exponent of block (r, c), row-major over the grid
+    std::vector<double> H;          // R x P, orthonormal rows, H * Vandermonde(points, Q) = 0
+    // offsets (in doubles) into the device table buffer
+    int64_t off_H = 0;
+};
+
+// Device-resident tables of a plan (one allocation).
+struct DeviceTables {
+    double* base = nullptr;
+    int64_t n_doubles = 0;
+    int64_t off_points = 0;
+    int64_t off_coefW = 0, off_coefX = 0, off_coefDT = 0, off_coefDup = 0, off_coefXup = 0;
+};
+
+}  // namespace gpd
+
+struct gpd_plan_s {
+    gpd_shape shape;
+    gpd_split split;
+    int P = 0;
+    gpd_precision prec = GPD_PREC_FP32;
+    int elem_size = 4;
+    double tau_col = 0, tau_in = 0;
+    std::vector<double> points;
+    std::vector<double> coefW, coefX, coefDT, coefDup, coefXup;   // [P][blocks]
+    gpd::ProductInfo prod[4];    // indexed by gpd_product (GPD_UPD unused)
+    // device side
+    std::mutex mu;
+    bool uploaded = false;
+    int device = -1;
+    gpd::DeviceTables dev;
+};
+
+namespace gpd {
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+// Uploads the plan's tables on first use (cudaMalloc + cudaMemcpy on the current device).
+gpd_status ensure_device(gpd_plan_s* plan);
+
+inline gpd_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? GPD_OK : GPD_ERR_CUDA; }
+inline gpd_status launch_ok() { return cuda_ok(cudaGetLastError()); }
+
+// Workspace layout for locate / decode (bytes, 256-aligned sections).
+struct WorkspaceLayout {
+    int64_t off_gram;      // double[kMaxR * kMaxR]   syndrome Gram matrix
+    int64_t off_counts;    // unsigned long long[4]   n_active, nonfinite mask, spare
+    int64_t off_decode;    // double[kMaxWanted * kMaxNodes] decode matrix D
+    int64_t off_flags;     // int[4] decode gate
+    int64_t total;
+};
+WorkspaceLayout workspace_layout();
+
+// Entry points used by coded_layer_step and by the public wrappers (all asynchronous).
+gpd_status encode_launch(gpd_plan_s* plan, int operand_or_A, const float* src, void* dst, cudaStream_t st);
+gpd_status worker_gemm_launch(gpd_plan_s* plan, gpd_product which, const void* W_sh, const void* other,
+                              void* out, cudaStream_t st);
+gpd_status update_launch(gpd_plan_s* plan, void* W_sh, const void* Dhat, const void* Xhat, float eta,
+                         float lambda, const gpd_locate_result* gate, cudaStream_t st);
+gpd_status inject_launch(gpd_plan_s* plan, gpd_product which, void* outputs, uint64_t seed, int mode,
+                         double prob, uint64_t node_mask, int count, double scale, uint64_t* hit_mask,
+                         cudaStream_t st);
+gpd_status locate_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, uint64_t erased_mask,
+                         gpd_locate_result* result, void* workspace, cudaStream_t st);
+gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, bool have_mask,
+                         uint64_t use_mask, const gpd_locate_result* result, float* out, float* act_out,
+                         int activation, void* workspace, cudaStream_t st);
+
+}  // namespace gpd

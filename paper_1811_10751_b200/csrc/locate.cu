@@ -1,0 +1,396 @@
+// Error detection and location over the P worker outputs: Algorithm 1 (Section V-A) taken at
+// node level, in the polynomial-time form the decoding appendix allows.
+//
+// Pass 1 (streaming, bandwidth-bound): every output position l holds one codeword z_l (the P
+// values the nodes produced there).  Its syndrome s_l = H z_l is formed in FP64 from H held in
+// shared memory; the codeword passes Algorithm 1's zero test when ||s_l||^2 <= tau^2 ||z_l||^2.
+// Failing ("active") codewords contribute s_l s_l^T / ||z_l||^2 to a Gram matrix G, reduced per
+// CTA through a shared-memory SYRK and added to global memory with one atomic per entry.
+// Non-finite values and erased nodes count as zero and their node is flagged up front.
+//
+// Pass 2 (one warp): eigen-decomposition of G by cyclic Jacobi; numerical rank rho; the error
+// support is the set of nodes whose parity-check column H_p lies in the span of the top-rho
+// eigenvectors (any P-Q columns of H are independent, so for at most P-Q-1 erroneous nodes no
+// other column does); the support is verified by the syndrome energy left outside span(H_A).
+// More than P-Q-1 nodes, a rank-deficient error matrix or an ambiguous geometry end in a
+// declared decoding failure (Theorem 3, third claim).
+#include "gpd_internal.h"
+
+namespace gpd {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct SyndromeParams {
+    const void* Z;              // [P][L]
+    const double* H;            // [R][P]
+    int64_t L;
+    int P, R;
+    double tau2;                // tau_col^2
+    unsigned long long erased;  // bit p set: node p is ignored (treated as zero)
+    double* gram;               // [R][R], zero on entry
+    unsigned long long* counts; // [0] n_active, [1] mask of nodes holding a non-finite value
+};
+
+template <typename T, int RT>
+__global__ void __launch_bounds__(kThreads) syndrome_gram_kernel(SyndromeParams prm) {
+    extern __shared__ __align__(16) double sm[];
+    double* sH = sm;                                   // [RT][P], rows >= R are zero
+    double* sS = sm + RT * prm.P;                      // [kThreads][RT + 1]
+    __shared__ unsigned long long s_nonfinite;
+    __shared__ unsigned int s_active;
+    for (int i = threadIdx.x; i < RT * prm.P; i += kThreads)
+        sH[i] = (i < prm.R * prm.P) ? prm.H[i] : 0.0;
+    if (threadIdx.x == 0) { s_nonfinite = 0ULL; s_active = 0u; }
+    __syncthreads();
+
+    constexpr int kPairs = RT * (RT + 1) / 2;
+    constexpr int kOwn = (kPairs + kThreads - 1) / kThreads;
+    double g_own[kOwn];
+    int own_i[kOwn], own_j[kOwn];
+#pragma unroll
+    for (int e = 0; e < kOwn; ++e) {
+        g_own[e] = 0.0;
+        int idx = threadIdx.x + e * kThreads, i = 0;
+        if (idx >= kPairs) { own_i[e] = -1; own_j[e] = 0; continue; }
+        while (idx >= RT - i) { idx -= RT - i; ++i; }   // row-major upper triangle
+        own_i[e] = i;
+        own_j[e] = i + idx;
+    }
+
+    const T* Z = reinterpret_cast<const T*>(prm.Z);
+    const int64_t n_batches = (prm.L + kThreads - 1) / kThreads;
+    unsigned int my_active = 0;
+    for (int64_t batch = blockIdx.x; batch < n_batches; batch += gridDim.x) {
+        const int64_t l = batch * kThreads + threadIdx.x;
+        double s[RT];
+#pragma unroll
+        for (int r = 0; r < RT; ++r) s[r] = 0.0;
+        double nz = 0.0;
+        unsigned long long bad = 0ULL;
+        if (l < prm.L) {
+            for (int p = 0; p < prm.P; ++p) {
+                double z = (double)__ldcs(Z + (int64_t)p * prm.L + l);
+                if (!isfinite(z)) { bad |= 1ULL << p; z = 0.0; }
+                if ((prm.erased >> p) & 1ULL) z = 0.0;
+                nz = fma(z, z, nz);
+#pragma unroll
+                for (int r = 0; r < RT; ++r) s[r] = fma(sH[r * prm.P + p], z, s[r]);
+            }
+        }
+        double ns = 0.0;
+#pragma unroll
+        for (int r = 0; r < RT; ++r) ns = fma(s[r], s[r], ns);
+        const bool active = (nz > 0.0) && (ns > prm.tau2 * nz);
+        if (bad) atomicOr(&s_nonfinite, bad);
+        my_active += active ? 1u : 0u;
+        if (__syncthreads_or(active ? 1 : 0)) {
+            const double w = active ? rsqrt(nz) : 0.0;
+            double* mine = sS + threadIdx.x * (RT + 1);
+#pragma unroll
+            for (int r = 0; r < RT; ++r) mine[r] = s[r] * w;
+            __syncthreads();
+#pragma unroll
+            for (int e = 0; e < kOwn; ++e) {
+                if (own_i[e] < 0) continue;
+                double acc = 0.0;
+                for (int c = 0; c < kThreads; ++c)
+                    acc = fma(sS[c * (RT + 1) + own_i[e]], sS[c * (RT + 1) + own_j[e]], acc);
+                g_own[e] += acc;
+            }
+            __syncthreads();
+        }
+    }
+    // CTA totals -> global
+    if (my_active) atomicAdd(&s_active, my_active);
+#pragma unroll
+    for (int e = 0; e < kOwn; ++e) {
+        if (own_i[e] < 0 || own_i[e] >= prm.R || own_j[e] >= prm.R || g_own[e] == 0.0) continue;
+        atomicAdd(&prm.gram[own_i[e] * prm.R + own_j[e]], g_own[e]);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (s_active) atomicAdd(&prm.counts[0], (unsigned long long)s_active);
+        if (s_nonfinite) atomicOr(&prm.counts[1], s_nonfinite);
+    }
+}
+
+struct FinishParams {
+    const double* H;            // [R][P]
+    const double* gram;         // upper triangle filled
+    const unsigned long long* counts;
+    gpd_locate_result* result;
+    int P, R;
+    double tau2, tau_in;
+    unsigned long long erased;
+};
+
+// One warp.  Shared: G[R][R], V[R][R] (eigenvectors in columns), Hs[R][P], Qa[R][R], lam[R].
+__global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
+    __shared__ double G[kMaxR][kMaxR + 1];
+    __shared__ double V[kMaxR][kMaxR + 1];
+    __shared__ double Qa[kMaxR][kMaxR + 1];
+    __shared__ double Hs[kMaxR][kMaxNodes];
+    __shared__ double lam[kMaxR];
+    __shared__ int order[kMaxR];
+    __shared__ unsigned char inside[kMaxNodes];
+    __shared__ double dist[kMaxNodes];
+    const int lane = threadIdx.x;
+    const int R = prm.R, P = prm.P;
+    gpd_locate_result* res = prm.result;
+    const unsigned long long n_active = prm.counts[0];
+    const unsigned long long forced = prm.counts[1] | prm.erased;
+    const int n_forced = __popcll(forced);
+
+    // header fields common to every exit
+    for (int p = lane; p < kMaxNodes; p += 32) {
+        res->forced[p] = (p < P && ((forced >> p) & 1ULL)) ? 1 : 0;
+        res->flagged[p] = res->forced[p];
+    }
+    if (lane == 0) {
+        res->n_active = (int64_t)n_active;
+        res->device_status = 0;
+        res->rank = 0;
+        res->residual = 0.0;
+        res->max_inside = 0.0;
+        res->min_outside = 0.0;
+        res->n_flagged = n_forced;
+    }
+    if (n_active == 0ULL && forced == 0ULL) {
+        if (lane == 0) res->outcome = GPD_NO_ERROR;
+        return;
+    }
+    const int budget = R - 1;
+    if (n_forced > budget) {
+        if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
+        return;
+    }
+    for (int i = lane; i < R * P; i += 32) Hs[i / P][i % P] = prm.H[i];
+    for (int i = lane; i < R * R; i += 32) {
+        const int r = i / R, c = i % R;
+        G[r][c] = prm.gram[r <= c ? r * R + c : c * R + r];
+        V[r][c] = r == c ? 1.0 : 0.0;
+    }
+    __syncwarp();
+
+    int rank = 0;
+    unsigned long long flagged = forced;
+    double max_in = 0.0, min_out = 1e300;
+    if (n_active > 0ULL) {
+        // ---- cyclic Jacobi: G <- J^T G J, V <- V J --------------------------------------
+        double tr = 0.0;
+        for (int i = 0; i < R; ++i) tr += G[i][i];
+        for (int sweep = 0; sweep < 40; ++sweep) {
+            double off = 0.0;
+            for (int i = lane; i < R * R; i += 32) {
+                const int r = i / R, c = i % R;
+                if (r != c) off += G[r][c] * G[r][c];
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
+            if (off <= 1e-34 * tr * tr) break;
+            for (int p = 0; p < R - 1; ++p) {
+                for (int q = p + 1; q < R; ++q) {
+                    const double gpq = G[p][q];
+                    const double gpp = G[p][p], gqq = G[q][q];
+                    __syncwarp();
+                    if (fabs(gpq) <= 1e-300 || fabs(gpq) <= 1e-20 * sqrt(fabs(gpp * gqq))) continue;
+                    const double th = (gqq - gpp) / (2.0 * gpq);
+                    const double t = (th >= 0.0 ? 1.0 : -1.0) / (fabs(th) + sqrt(th * th + 1.0));
+                    const double c = 1.0 / sqrt(t * t + 1.0), s = t * c;
+                    if (lane < R) {                          // G <- G J   (columns p, q)
+                        const double a = G[lane][p], b = G[lane][q];
+                        G[lane][p] = c * a - s * b;
+                        G[lane][q] = s * a + c * b;
+                        const double va = V[lane][p], vb = V[lane][q];
+                        V[lane][p] = c * va - s * vb;
+                        V[lane][q] = s * va + c * vb;
+                    }
+                    __syncwarp();
+                    if (lane < R) {                          // G <- J^T G (rows p, q)
+                        const double a = G[p][lane], b = G[q][lane];
+                        G[p][lane] = c * a - s * b;
+                        G[q][lane] = s * a + c * b;
+                    }
+                    __syncwarp();
+                    if (lane == 0) { G[p][q] = 0.0; G[q][p] = 0.0; }
+                    __syncwarp();
+                }
+            }
+        }
+        // ---- eigenvalues in descending order ---------------------------------------------
+        if (lane == 0) {
+            for (int i = 0; i < R; ++i) { lam[i] = G[i][i]; order[i] = i; }
+            for (int i = 1; i < R; ++i) {                    // insertion sort, R <= 32
+                const int oi = order[i];
+                int j = i - 1;
+                while (j >= 0 && lam[order[j]] < lam[oi]) { order[j + 1] = order[j]; --j; }
+                order[j + 1] = oi;
+            }
+        }
+        __syncwarp();
+        const double theta = prm.tau2 * (double)n_active / (double)R;
+        for (int i = 0; i < R; ++i) rank += lam[order[i]] > theta ? 1 : 0;
+        if (lane == 0) res->rank = rank;
+        if (rank > budget) {
+            if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
+            return;
+        }
+        // ---- distance of every H_p to span of the top-rank eigenvectors --------------------
+        for (int p = lane; p < P; p += 32) {
+            double hn = 0.0;
+            for (int r = 0; r < R; ++r) hn += Hs[r][p] * Hs[r][p];
+            double resid[kMaxR];
+            for (int r = 0; r < R; ++r) resid[r] = Hs[r][p];
+            for (int pass = 0; pass < 2; ++pass) {           // project twice (re-orthogonalisation)
+                for (int e = 0; e < rank; ++e) {
+                    const int col = order[e];
+                    double dot = 0.0;
+                    for (int r = 0; r < R; ++r) dot += V[r][col] * resid[r];
+                    for (int r = 0; r < R; ++r) resid[r] -= dot * V[r][col];
+                }
+            }
+            double rn = 0.0;
+            for (int r = 0; r < R; ++r) rn += resid[r] * resid[r];
+            dist[p] = sqrt(rn / hn);
+            inside[p] = dist[p] <= prm.tau_in ? 1 : 0;
+        }
+        __syncwarp();
+        int n_inside = 0;
+        for (int p = 0; p < P; ++p) {
+            if (inside[p]) { ++n_inside; flagged |= 1ULL << p; max_in = fmax(max_in, dist[p]); }
+            else min_out = fmin(min_out, dist[p]);
+        }
+        if (lane == 0) { res->max_inside = max_in; res->min_outside = min_out; }
+        if (n_inside != rank) {
+            if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
+            return;
+        }
+    }
+    const int n_flagged = __popcll(flagged);
+    if (n_flagged > budget) {
+        if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
+        return;
+    }
+    // ---- verification: syndrome energy outside span(H_A), A = flagged nodes ------------------
+    // Orthonormal basis of span(H_A) by twice-applied modified Gram-Schmidt (columns of Qa).
+    int na = 0;
+    for (int p = 0; p < P; ++p) {
+        if (!((flagged >> p) & 1ULL)) continue;
+        if (lane < R) Qa[lane][na] = Hs[lane][p];
+        __syncwarp();
+        for (int pass = 0; pass < 2; ++pass) {
+            for (int e = 0; e < na; ++e) {
+                double part = lane < R ? Qa[lane][e] * Qa[lane][na] : 0.0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                if (lane < R) Qa[lane][na] -= part * Qa[lane][e];
+                __syncwarp();
+            }
+        }
+        double nn = lane < R ? Qa[lane][na] * Qa[lane][na] : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(0xffffffffu, nn, o);
+        if (lane < R) Qa[lane][na] *= rsqrt(nn);
+        __syncwarp();
+        ++na;
+    }
+    double residual = 0.0;
+    if (n_active > 0ULL) {
+        // tr((I-Pi) G (I-Pi)) = sum_i lambda_i ||(I-Pi) u_i||^2, every term non-negative
+        for (int i = 0; i < R; ++i) {
+            double u = lane < R ? V[lane][i] : 0.0;
+            for (int pass = 0; pass < 2; ++pass) {
+                for (int e = 0; e < na; ++e) {
+                    double part = lane < R ? Qa[lane][e] * u : 0.0;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                    if (lane < R) u -= part * Qa[lane][e];
+                }
+            }
+            double un = u * u;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) un += __shfl_xor_sync(0xffffffffu, un, o);
+            residual += fmax(G[i][i], 0.0) * un;
+        }
+    }
+    const double limit = prm.tau2 * (double)(n_active > 0ULL ? n_active : 1ULL);
+    if (lane == 0) {
+        res->residual = residual / (double)(n_active > 0ULL ? n_active : 1ULL);
+        res->n_flagged = residual > limit ? n_forced : n_flagged;
+        res->outcome = residual > limit ? GPD_DECODE_FAILURE : GPD_CORRECTED;
+    }
+    if (residual <= limit)
+        for (int p = lane; p < P; p += 32) res->flagged[p] = (flagged >> p) & 1ULL ? 1 : 0;
+}
+
+template <typename T, int RT>
+gpd_status launch_syndrome(const SyndromeParams& prm, cudaStream_t st) {
+    const size_t smem = sizeof(double) * ((size_t)RT * prm.P + (size_t)kThreads * (RT + 1));
+    if (smem > 48 * 1024) {
+        if (cudaFuncSetAttribute(syndrome_gram_kernel<T, RT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem) != cudaSuccess)
+            return GPD_ERR_CUDA;
+    }
+    const int64_t batches = (prm.L + kThreads - 1) / kThreads;
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(batches, 148 * 4));
+    syndrome_gram_kernel<T, RT><<<grid, kThreads, smem, st>>>(prm);
+    return launch_ok();
+}
+
+template <typename T>
+gpd_status dispatch_syndrome(const SyndromeParams& prm, cudaStream_t st) {
+    if (prm.R <= 8) return launch_syndrome<T, 8>(prm, st);
+    if (prm.R <= 16) return launch_syndrome<T, 16>(prm, st);
+    return launch_syndrome<T, 32>(prm, st);
+}
+
+}  // namespace
+
+gpd_status locate_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, uint64_t erased_mask,
+                         gpd_locate_result* result, void* workspace, cudaStream_t st) {
+    if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
+    const ProductInfo& pi = plan->prod[which];
+    if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
+    gpd_status rc = ensure_device(plan);
+    if (rc != GPD_OK) return rc;
+    const WorkspaceLayout wl = workspace_layout();
+    char* ws = reinterpret_cast<char*>(workspace);
+    double* gram = reinterpret_cast<double*>(ws + wl.off_gram);
+    unsigned long long* counts = reinterpret_cast<unsigned long long*>(ws + wl.off_counts);
+    // Gram matrix and counters start at zero (they sit next to each other in the workspace)
+    if (cudaMemsetAsync(ws + wl.off_gram, 0, (size_t)(wl.off_decode - wl.off_gram), st) != cudaSuccess)
+        return GPD_ERR_CUDA;
+    const double* H = plan->dev.base + pi.off_H;
+    if (pi.R > 0) {
+        SyndromeParams sp{};
+        sp.Z = outputs; sp.H = H; sp.L = pi.br * pi.bc; sp.P = plan->P; sp.R = pi.R;
+        sp.tau2 = plan->tau_col * plan->tau_col; sp.erased = erased_mask;
+        sp.gram = gram; sp.counts = counts;
+        rc = plan->elem_size == 4 ? dispatch_syndrome<float>(sp, st) : dispatch_syndrome<double>(sp, st);
+        if (rc != GPD_OK) return rc;
+    }
+    FinishParams fp{};
+    fp.H = H; fp.gram = gram; fp.counts = counts; fp.result = result;
+    fp.P = plan->P; fp.R = pi.R; fp.tau2 = plan->tau_col * plan->tau_col; fp.tau_in = plan->tau_in;
+    fp.erased = erased_mask;
+    locate_finish_kernel<<<1, 32, 0, st>>>(fp);
+    return launch_ok();
+}
+
+}  // namespace gpd
+
+using namespace gpd;
+
+extern "C" gpd_status gpd_locate_errors(gpd_plan_t plan, gpd_product which, const void* outputs_dev,
+                                        const uint8_t* erased_host, gpd_locate_result* result_dev,
+                                        void* workspace_dev, void* stream) {
+    if (!plan || !outputs_dev || !result_dev) return GPD_ERR_ARG;
+    if (!workspace_dev) return GPD_ERR_WORKSPACE;
+    uint64_t mask = 0;
+    if (erased_host)
+        for (int p = 0; p < plan->P; ++p)
+            if (erased_host[p]) mask |= 1ULL << p;
+    return locate_launch(plan, which, outputs_dev, mask, result_dev, workspace_dev, as_stream(stream));
+}

@@ -1,0 +1,294 @@
+// Code construction on the host in FP64: evaluation points, exponent maps, coefficient tables,
+// recovery thresholds and parity-check matrices (Section IV, Theorems 1-2; Section V-A).
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "gpd_internal.h"
+
+namespace gpd {
+
+namespace {
+
+// V[p][e] = b_p^e by repeated multiplication.
+std::vector<double> power_table(const std::vector<double>& b, int count) {
+    const int P = (int)b.size();
+    std::vector<double> V((size_t)P * count);
+    for (int p = 0; p < P; ++p) {
+        double acc = 1.0;
+        for (int e = 0; e < count; ++e) {
+            V[(size_t)p * count + e] = acc;
+            acc *= b[p];
+        }
+    }
+    return V;
+}
+
+// Orthonormal basis (rows of H, R x P) of the left null space of the P x Q Vandermonde matrix:
+// Householder-triangularise V, then push the unit vectors e_Q .. e_{P-1} back through the
+// reflectors; the images are the last P-Q columns of the full orthogonal factor.
+std::vector<double> left_null_space(const std::vector<double>& b, int Q) {
+    const int P = (int)b.size();
+    const int R = P - Q;
+    std::vector<double> H((size_t)std::max(R, 0) * P, 0.0);
+    if (R <= 0) return H;
+    std::vector<double> A = power_table(b, Q);            // P x Q, row-major
+    std::vector<double> vs((size_t)Q * P, 0.0);           // reflector k in vs[k*P + k .. k*P + P-1]
+    for (int k = 0; k < Q; ++k) {
+        double nrm = 0.0;
+        for (int r = k; r < P; ++r) nrm += A[(size_t)r * Q + k] * A[(size_t)r * Q + k];
+        nrm = std::sqrt(nrm);
+        double* v = &vs[(size_t)k * P];
+        const double akk = A[(size_t)k * Q + k];
+        const double alpha = akk >= 0.0 ? -nrm : nrm;
+        for (int r = k; r < P; ++r) v[r] = A[(size_t)r * Q + k];
+        v[k] -= alpha;
+        double vn = 0.0;
+        for (int r = k; r < P; ++r) vn += v[r] * v[r];
+        vn = std::sqrt(vn);
+        if (vn > 0.0)
+            for (int r = k; r < P; ++r) v[r] /= vn;
+        for (int c = k; c < Q; ++c) {                     // A <- (I - 2 v v^T) A
+            double dot = 0.0;
+            for (int r = k; r < P; ++r) dot += v[r] * A[(size_t)r * Q + c];
+            for (int r = k; r < P; ++r) A[(size_t)r * Q + c] -= 2.0 * dot * v[r];
+        }
+    }
+    std::vector<double> x(P);
+    for (int j = 0; j < R; ++j) {
+        std::fill(x.begin(), x.end(), 0.0);
+        x[Q + j] = 1.0;
+        for (int k = Q - 1; k >= 0; --k) {                // x <- H_0 H_1 ... H_{Q-1} e_{Q+j}
+            const double* v = &vs[(size_t)k * P];
+            double dot = 0.0;
+            for (int r = k; r < P; ++r) dot += v[r] * x[r];
+            for (int r = k; r < P; ++r) x[r] -= 2.0 * dot * v[r];
+        }
+        for (int p = 0; p < P; ++p) H[(size_t)j * P + p] = x[p];
+    }
+    return H;
+}
+
+int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+WorkspaceLayout workspace_layout() {
+    WorkspaceLayout w{};
+    int64_t off = 0;
+    w.off_gram = off;   off = align_up(off + (int64_t)sizeof(double) * kMaxR * kMaxR, 256);
+    w.off_counts = off; off = align_up(off + (int64_t)sizeof(unsigned long long) * 8, 256);
+    w.off_decode = off; off = align_up(off + (int64_t)sizeof(double) * kMaxWanted * kMaxNodes, 256);
+    w.off_flags = off;  off = align_up(off + (int64_t)sizeof(int) * 8, 256);
+    w.total = off;
+    return w;
+}
+
+gpd_status ensure_device(gpd_plan_s* plan) {
+    std::lock_guard<std::mutex> lock(plan->mu);
+    if (plan->uploaded) return GPD_OK;
+    std::vector<double> host;
+    auto push = [&](const std::vector<double>& v) {
+        int64_t off = (int64_t)host.size();
+        host.insert(host.end(), v.begin(), v.end());
+        while (host.size() % 32) host.push_back(0.0);      // keep every table 256-byte aligned
+        return off;
+    };
+    DeviceTables& d = plan->dev;
+    d.off_points = push(plan->points);
+    d.off_coefW = push(plan->coefW);
+    d.off_coefX = push(plan->coefX);
+    d.off_coefDT = push(plan->coefDT);
+    d.off_coefDup = push(plan->coefDup);
+    d.off_coefXup = push(plan->coefXup);
+    for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT}) plan->prod[w].off_H = push(plan->prod[w].H);
+    d.n_doubles = (int64_t)host.size();
+    if (cudaGetDevice(&plan->device) != cudaSuccess) return GPD_ERR_CUDA;
+    if (cudaMalloc(&d.base, sizeof(double) * host.size()) != cudaSuccess) return GPD_ERR_CUDA;
+    if (cudaMemcpy(d.base, host.data(), sizeof(double) * host.size(), cudaMemcpyHostToDevice) !=
+        cudaSuccess) {
+        cudaFree(d.base);
+        d.base = nullptr;
+        return GPD_ERR_CUDA;
+    }
+    plan->uploaded = true;
+    return GPD_OK;
+}
+
+}  // namespace gpd
+
+using namespace gpd;
+
+extern "C" const char* gpd_status_string(gpd_status s) {
+    switch (s) {
+        case GPD_OK: return "ok";
+        case GPD_ERR_ARG: return "invalid argument";
+        case GPD_ERR_SHAPE: return "splits do not divide the matrix dimensions";
+        case GPD_ERR_POINTS: return "evaluation points repeated or non-finite";
+        case GPD_ERR_P_TOO_SMALL: return "fewer nodes than the recovery threshold";
+        case GPD_ERR_Q_TOO_LARGE: return "threshold, node count or parity count above the supported maximum";
+        case GPD_ERR_WORKSPACE: return "workspace missing";
+        case GPD_ERR_CUDA: return "CUDA runtime error";
+        case GPD_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case GPD_ERR_UNSUPPORTED: return "unsupported combination";
+    }
+    return "unknown status";
+}
+
+extern "C" gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, int32_t P,
+                               const double* points_host, gpd_precision precision, gpd_plan_t* out) {
+    if (!shape || !split || !out) return GPD_ERR_ARG;
+    *out = nullptr;
+    if (precision != GPD_PREC_AUTO && precision != GPD_PREC_FP32 && precision != GPD_PREC_FP64)
+        return GPD_ERR_ARG;
+    const int m = split->m, n = split->n, d1 = split->d1, d2 = split->d2;
+    if (shape->N1 <= 0 || shape->N0 <= 0 || shape->B <= 0 || m <= 0 || n <= 0 || d1 <= 0 || d2 <= 0)
+        return GPD_ERR_SHAPE;
+    if (shape->N1 % m || shape->N0 % n || shape->B % d1 || shape->B % d2) return GPD_ERR_SHAPE;
+    if (P <= 0) return GPD_ERR_P_TOO_SMALL;
+    const int64_t Qf = (int64_t)m * n * d1 + n - 1;        // Theorem 2
+    const int64_t Qb = (int64_t)m * n * (d2 + 1) - n;      // coefficients of C~^T(v)
+    const int64_t Qw = (int64_t)m * n;                     // coefficients of W~(v)
+    if (P > kMaxNodes || Qf > kMaxQ) return GPD_ERR_Q_TOO_LARGE;
+    if (m * n > kMaxBlocks || n * d1 > kMaxBlocks || d2 * m > kMaxBlocks || m * d1 > kMaxWanted ||
+        d2 * n > kMaxWanted)
+        return GPD_ERR_Q_TOO_LARGE;
+    if (P < Qf) return GPD_ERR_P_TOO_SMALL;
+    if (P - Qf > kMaxR) return GPD_ERR_Q_TOO_LARGE;
+
+    gpd_plan_s* plan = new (std::nothrow) gpd_plan_s();
+    if (!plan) return GPD_ERR_ARG;
+    plan->shape = *shape;
+    plan->split = *split;
+    plan->P = P;
+    plan->points.resize(P);
+    if (points_host) {
+        for (int p = 0; p < P; ++p) plan->points[p] = points_host[p];
+    } else {
+        const double pi = 3.14159265358979323846;
+        for (int p = 0; p < P; ++p) plan->points[p] = std::cos((2.0 * p + 1.0) * pi / (2.0 * P));
+    }
+    for (int p = 0; p < P; ++p) {
+        if (!std::isfinite(plan->points[p])) { delete plan; return GPD_ERR_POINTS; }
+        for (int q = 0; q < p; ++q)
+            if (plan->points[p] == plan->points[q]) { delete plan; return GPD_ERR_POINTS; }
+    }
+    const bool bwd_ok = (P >= Qb) && (Qb <= kMaxQ) && (P - Qb <= kMaxR);
+    const bool audit_ok = (P - Qw <= kMaxR);
+    const int64_t q_for_prec = bwd_ok ? std::max(Qf, Qb) : Qf;
+    plan->prec = precision == GPD_PREC_AUTO ? (q_for_prec <= 9 ? GPD_PREC_FP32 : GPD_PREC_FP64) : precision;
+    plan->elem_size = plan->prec == GPD_PREC_FP32 ? 4 : 8;
+    plan->tau_col = plan->prec == GPD_PREC_FP32 ? kTauColFp32 : kTauColFp64;
+    plan->tau_in = plan->prec == GPD_PREC_FP32 ? kTauInFp32 : kTauInFp64;
+
+    // powers up to the largest exponent used by any encoding
+    const int max_exp = (int)std::max<int64_t>(std::max(Qf, Qb), Qw) + 1;
+    const std::vector<double> pw = power_table(plan->points, max_exp);
+    auto at = [&](int p, int e) { return pw[(size_t)p * max_exp + e]; };
+    plan->coefW.resize((size_t)P * m * n);
+    plan->coefX.resize((size_t)P * n * d1);
+    plan->coefDT.resize((size_t)P * d2 * m);
+    plan->coefDup.resize((size_t)P * m);
+    plan->coefXup.resize((size_t)P * n);
+    for (int p = 0; p < P; ++p) {
+        for (int i = 0; i < m; ++i)
+            for (int j = 0; j < n; ++j) plan->coefW[((size_t)p * m + i) * n + j] = at(p, n * i + j);
+        for (int j = 0; j < n; ++j)
+            for (int k = 0; k < d1; ++k)
+                plan->coefX[((size_t)p * n + j) * d1 + k] = at(p, (n - 1 - j) + m * n * k);
+        for (int k = 0; k < d2; ++k)
+            for (int i = 0; i < m; ++i)
+                plan->coefDT[((size_t)p * d2 + k) * m + i] = at(p, m * n * k + n * (m - 1 - i));
+        for (int i = 0; i < m; ++i) plan->coefDup[(size_t)p * m + i] = at(p, n * i);
+        for (int j = 0; j < n; ++j) plan->coefXup[(size_t)p * n + j] = at(p, j);
+    }
+    // products
+    ProductInfo& f = plan->prod[GPD_FWD];
+    f.Q = (int)Qf; f.R = P - f.Q; f.grid_rows = m; f.grid_cols = d1;
+    f.br = shape->N1 / m; f.bc = shape->B / d1;
+    for (int i = 0; i < m; ++i)
+        for (int k = 0; k < d1; ++k) f.wanted[i * d1 + k] = n * i + m * n * k + n - 1;
+    f.H = left_null_space(plan->points, f.Q);
+    ProductInfo& b = plan->prod[GPD_BWD];
+    if (bwd_ok) {
+        b.Q = (int)Qb; b.R = P - b.Q; b.grid_rows = d2; b.grid_cols = n;
+        b.br = shape->B / d2; b.bc = shape->N0 / n;
+        for (int k = 0; k < d2; ++k)
+            for (int j = 0; j < n; ++j) b.wanted[k * n + j] = m * n * k + n * (m - 1) + j;
+        b.H = left_null_space(plan->points, b.Q);
+    }
+    ProductInfo& a = plan->prod[GPD_AUDIT];
+    if (audit_ok) {
+        a.Q = (int)Qw; a.R = P - a.Q; a.grid_rows = m; a.grid_cols = n;
+        a.br = shape->N1 / m; a.bc = shape->N0 / n;
+        for (int i = 0; i < m; ++i)
+            for (int j = 0; j < n; ++j) a.wanted[i * n + j] = n * i + j;
+        a.H = left_null_space(plan->points, a.Q);
+    }
+    *out = plan;
+    return GPD_OK;
+}
+
+extern "C" gpd_status gpd_plan_destroy(gpd_plan_t plan) {
+    if (!plan) return GPD_ERR_ARG;
+    if (plan->uploaded && plan->dev.base) cudaFree(plan->dev.base);
+    delete plan;
+    return GPD_OK;
+}
+
+extern "C" gpd_status gpd_plan_query(gpd_plan_t plan, gpd_query what, int64_t* value) {
+    if (!plan || !value) return GPD_ERR_ARG;
+    const gpd_shape& s = plan->shape;
+    const gpd_split& c = plan->split;
+    const int64_t P = plan->P;
+    switch (what) {
+        case GPD_Q_THRESHOLD_FWD: *value = plan->prod[GPD_FWD].Q; break;
+        case GPD_Q_THRESHOLD_BWD: *value = (int64_t)c.m * c.n * (c.d2 + 1) - c.n; break;
+        case GPD_Q_THRESHOLD_AUDIT: *value = (int64_t)c.m * c.n; break;
+        case GPD_Q_ELEMENT_SIZE: *value = plan->elem_size; break;
+        case GPD_Q_W_SHARE_ELEMS: *value = P * (s.N1 / c.m) * (s.N0 / c.n); break;
+        case GPD_Q_X_SHARE_ELEMS: *value = P * (s.N0 / c.n) * (s.B / c.d1); break;
+        case GPD_Q_DT_SHARE_ELEMS: *value = P * (s.B / c.d2) * (s.N1 / c.m); break;
+        case GPD_Q_DHAT_ELEMS: *value = P * (s.N1 / c.m) * s.B; break;
+        case GPD_Q_XHAT_ELEMS: *value = P * (s.N0 / c.n) * s.B; break;
+        case GPD_Q_OUT_ELEMS_FWD: *value = P * (s.N1 / c.m) * (s.B / c.d1); break;
+        case GPD_Q_OUT_ELEMS_BWD: *value = P * (s.B / c.d2) * (s.N0 / c.n); break;
+        case GPD_Q_WORKSPACE_BYTES: *value = workspace_layout().total; break;
+        case GPD_Q_STEP_WORKSPACE_BYTES: {
+            // locate/decode scratch + the larger of {X~ + S~} and {Delta~^T + C~^T} and {Delta^ + X^}
+            const int64_t e = plan->elem_size;
+            const int64_t fwd = P * (s.N0 / c.n) * (s.B / c.d1) + P * (s.N1 / c.m) * (s.B / c.d1);
+            const int64_t bwd = P * (s.B / c.d2) * (s.N1 / c.m) + P * (s.B / c.d2) * (s.N0 / c.n);
+            const int64_t upd = P * (s.N1 / c.m) * s.B + P * (s.N0 / c.n) * s.B;
+            const int64_t big = std::max(fwd, std::max(bwd, upd));
+            *value = workspace_layout().total + ((big * e + 255) / 256 + 2) * 256;
+            break;
+        }
+        case GPD_Q_PRECISION: *value = plan->prec; break;
+        case GPD_Q_NODES: *value = P; break;
+        default: return GPD_ERR_ARG;
+    }
+    return GPD_OK;
+}
+
+extern "C" gpd_status gpd_plan_table(gpd_plan_t plan, gpd_table which, double* host_out,
+                                     int64_t capacity, int64_t* count) {
+    if (!plan || !count) return GPD_ERR_ARG;
+    const std::vector<double>* src = nullptr;
+    switch (which) {
+        case GPD_TABLE_POINTS: src = &plan->points; break;
+        case GPD_TABLE_PARITY_FWD: src = &plan->prod[GPD_FWD].H; break;
+        case GPD_TABLE_PARITY_BWD: src = &plan->prod[GPD_BWD].H; break;
+        case GPD_TABLE_PARITY_AUDIT: src = &plan->prod[GPD_AUDIT].H; break;
+        case GPD_TABLE_COEF_W: src = &plan->coefW; break;
+        case GPD_TABLE_COEF_X: src = &plan->coefX; break;
+        case GPD_TABLE_COEF_DT: src = &plan->coefDT; break;
+        default: return GPD_ERR_ARG;
+    }
+    *count = (int64_t)src->size();
+    if (host_out) {
+        if (capacity < *count) return GPD_ERR_ARG;
+        std::memcpy(host_out, src->data(), sizeof(double) * src->size());
+    }
+    return GPD_OK;
+}

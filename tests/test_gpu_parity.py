@@ -1,0 +1,327 @@
+"""GPU parity: every stage of the CUDA path against the CPU FP64 oracle, through the C ABI.
+
+Bars: integer / index work (error-location outcome, flag vectors, bit flips, which entries an
+injector touches) bit-exact; decoded floating point within 1e-4 relative Frobenius error (the
+target the workloads state); intermediate FP64 quantities much tighter, as written per test.
+"""
+
+import itertools
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+if not torch.cuda.is_available():                       # collected on a CPU machine: nothing to run
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+import paper_1811_10751_b200 as g                        # noqa: E402
+import workloads as wl                                   # noqa: E402
+from oracle import inject as oinj                        # noqa: E402
+from oracle import product as op                         # noqa: E402
+from oracle.code import GPCode, FWD, BWD, AUDIT          # noqa: E402
+from oracle.locate import (CORRECTED, DECODE_FAILURE, NO_ERROR, locate_subspace,  # noqa: E402
+                           tolerances_for)
+from tests.gpu_pipeline import CodedProduct, dev, host, make_code   # noqa: E402
+
+REL_TOL = 1e-4                                           # decoded outputs, relative Frobenius
+
+
+def rms(a):
+    return float(np.sqrt(np.mean(np.asarray(a, dtype=np.float64) ** 2)))
+
+
+def rand(shape, seed, dist="gauss"):
+    r = np.random.default_rng(seed)
+    a = r.standard_normal(shape) if dist == "gauss" else r.uniform(-1, 1, shape)
+    return a.astype(np.float32)
+
+
+# --------------------------------------------------------------------------------------------------
+# encode
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N1,N0,B,m,n,d1,d2,P,prec", [
+    (64, 64, 64, 2, 2, 2, 1, 11, g.GPD_PREC_FP32),
+    (512, 1024, 128, 2, 4, 2, 1, 25, g.GPD_PREC_FP64),
+    (96, 60, 6, 3, 2, 2, 3, 20, g.GPD_PREC_FP64),            # block widths not multiples of 4
+    (10, 4096, 256, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),        # 5-row blocks
+    (4096, 4096, 1, 4, 2, 1, 1, 13, g.GPD_PREC_FP32),        # matrix-vector
+    (256, 128, 64, 4, 4, 1, 1, 36, g.GPD_PREC_FP64),
+])
+def test_encode_matches_oracle(N1, N0, B, m, n, d1, d2, P, prec):
+    code = GPCode(N1, N0, B, m, n, d1, d2, P)
+    cp = CodedProduct(code, prec)
+    W, X, DT = rand((N1, N0), 1), rand((N0, B), 2), rand((B, N1), 3)
+    f32 = cp.np_dtype == np.float32
+    rtol = 2e-7 if f32 else 1e-14
+    cases = [(cp.encode_W(W), op.encode_W(W, code)),
+             (cp.encode(g.GPD_OPERAND_X_FWD, X), op.encode_X(X, code))]
+    if P >= code.Q_b:
+        cases.append((cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT), op.encode_DeltaT(DT, code)))
+    Dh, Xh = op.encode_update_operands(DT.T.copy(), X, code)
+    cases.append((cp.encode(g.GPD_OPERAND_DELTA_UPD, DT.T.copy()), Dh))
+    cases.append((cp.encode(g.GPD_OPERAND_X_UPD, X), Xh))
+    for got, want in cases:
+        got = host(got).reshape(want.shape).astype(np.float64)
+        scale = np.abs(want).max()
+        assert np.abs(got - want).max() <= rtol * scale * 4
+
+
+# --------------------------------------------------------------------------------------------------
+# worker products and coded update
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N1,N0,B,m,n,d1,d2,P,prec", [
+    (512, 512, 256, 2, 2, 2, 2, 16, g.GPD_PREC_FP64),        # tensor-core FP64 tiles, exact multiples
+    (400, 200, 144, 2, 2, 2, 2, 16, g.GPD_PREC_FP64),        # ragged tails in M, N and K
+    (66, 50, 14, 2, 2, 2, 2, 16, g.GPD_PREC_FP64),           # odd sizes -> CUDA-core kernel
+    (512, 512, 256, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),
+    (10, 512, 64, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),          # 5-row blocks
+    (1024, 512, 1, 4, 2, 1, 1, 13, g.GPD_PREC_FP32),         # matrix-vector
+    (1024, 512, 1, 4, 2, 1, 1, 13, g.GPD_PREC_FP64),
+])
+def test_worker_products_and_update_match_oracle(N1, N0, B, m, n, d1, d2, P, prec):
+    code = GPCode(N1, N0, B, m, n, d1, d2, P)
+    cp = CodedProduct(code, prec)
+    W, X, DT = rand((N1, N0), 4), rand((N0, B), 5), rand((B, N1), 6)
+    tol = 2e-6 if cp.np_dtype == np.float32 else 1e-13
+    Wsh = cp.encode_W(W)
+    Ws_o = host(Wsh).reshape(P, N1 // m, N0 // n).astype(np.float64)      # same stored shares
+    Xsh = cp.encode(g.GPD_OPERAND_X_FWD, X)
+    Z = cp.outputs_as_array(g.GPD_FWD, cp.products(g.GPD_FWD, Xsh))
+    want = op.worker_products(Ws_o, host(Xsh).reshape(P, N0 // n, B // d1).astype(np.float64))
+    assert np.isfinite(Z).all() and np.abs(Z - want).max() <= tol * rms(want) * 8
+    if P >= code.Q_b:
+        Dsh = cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT)
+        Zb = cp.outputs_as_array(g.GPD_BWD, cp.products(g.GPD_BWD, Dsh))
+        want = op.worker_products(host(Dsh).reshape(P, B // d2, N1 // m).astype(np.float64), Ws_o)
+        assert np.isfinite(Zb).all() and np.abs(Zb - want).max() <= tol * rms(want) * 8
+    # coded update in place, with weight decay
+    Delta = DT.T.copy()
+    Dh, Xh = cp.encode(g.GPD_OPERAND_DELTA_UPD, Delta), cp.encode(g.GPD_OPERAND_X_UPD, X)
+    want = op.update_shares(Ws_o, host(Dh).reshape(P, N1 // m, B).astype(np.float64),
+                            host(Xh).reshape(P, N0 // n, B).astype(np.float64), eta=0.05, lam=0.1)
+    g.gpd_update_shares(cp.plan, Wsh, Dh, Xh, 0.05, 0.1)
+    got = host(Wsh).reshape(want.shape).astype(np.float64)
+    assert np.abs(got - want).max() <= max(tol, 2e-7) * rms(want) * 8
+
+
+# --------------------------------------------------------------------------------------------------
+# injection: same clean buffer on both sides
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("prec", [g.GPD_PREC_FP32, g.GPD_PREC_FP64])
+def test_injectors_match_oracle(prec):
+    code = GPCode(96, 64, 40, 2, 2, 2, 1, 14)
+    cp = CodedProduct(code, prec)
+    L = (96 // 2) * (40 // 2)
+    clean = np.random.default_rng(7).standard_normal((14, L)).astype(cp.np_dtype)
+    hit = torch.zeros(1, dtype=torch.int64, device="cuda")
+
+    def mask_of(h):
+        return np.array([(int(h.item()) >> p) & 1 for p in range(14)], dtype=bool)
+
+    for seed in (1, 2, 3):
+        Z = dev(clean)
+        g.gpd_inject(cp.plan, g.GPD_FWD, Z, seed, g.GPD_INJECT_BITFLIP, count=3, scale=1.0, hit_mask=hit)
+        ref = clean.copy()
+        sel = oinj.inject_bitflip(ref, seed, 3, 1.0)
+        itype = np.uint32 if prec == g.GPD_PREC_FP32 else np.uint64
+        assert np.array_equal(host(Z).view(itype), ref.view(itype))            # bit-exact
+        assert np.array_equal(mask_of(hit), sel)
+
+        Z = dev(clean)
+        g.gpd_inject(cp.plan, g.GPD_FWD, Z, seed, g.GPD_INJECT_ADDITIVE, prob=0.3, scale=2.0, hit_mask=hit)
+        ref = clean.copy()
+        sel = oinj.inject_additive(ref, seed, 2.0, prob=0.3)
+        assert np.array_equal(host(Z).view(itype), ref.view(itype))            # bit-exact
+        assert np.array_equal(mask_of(hit), sel)
+
+        Z = dev(clean)
+        nodes = np.zeros(14, dtype=bool)
+        nodes[[2, 9]] = True
+        g.gpd_inject(cp.plan, g.GPD_FWD, Z, seed, g.GPD_INJECT_GAUSS, prob=-1.0,
+                     node_mask=(1 << 2) | (1 << 9), scale=1.5, hit_mask=hit)
+        ref = clean.copy()
+        oinj.inject_gauss(ref, seed, 1.5, nodes=nodes)
+        assert np.array_equal(mask_of(hit), nodes)
+        assert np.array_equal(host(Z)[~nodes], clean[~nodes])
+        tol = 1e-6 if prec == g.GPD_PREC_FP32 else 1e-12
+        assert np.abs(host(Z).astype(np.float64) - ref.astype(np.float64)).max() < tol * 8
+
+
+# --------------------------------------------------------------------------------------------------
+# config 1: tiny matmul, no errors, every threshold-sized subset
+# --------------------------------------------------------------------------------------------------
+def test_config1_all_subsets():
+    cfg = wl.CONFIG_1_TINY
+    W, X = wl.matmul_inputs(cfg)
+    code = make_code(cfg)
+    cp = CodedProduct(code)
+    assert cp.np_dtype == np.float32
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    r = cp.locate(g.GPD_FWD, Z)
+    assert r.outcome == NO_ERROR and r.n_flagged == 0 and r.n_active == 0
+    ref = op.ref_forward(W, X)
+    Zo = op.worker_products(op.encode_W(W, code), op.encode_X(X, code))
+    assert op.rel_fro(cp.decode(g.GPD_FWD, Z), ref) < REL_TOL
+    worst = 0.0
+    for keep in itertools.combinations(range(cfg.P), code.Q_f):
+        use = np.zeros(cfg.P, dtype=bool)
+        use[list(keep)] = True
+        S = cp.decode(g.GPD_FWD, Z, use_mask=use)
+        worst = max(worst, op.rel_fro(S, ref))
+        assert op.rel_fro(S, op.decode(Zo, code, FWD, use)) < REL_TOL
+    assert worst < REL_TOL
+
+
+# --------------------------------------------------------------------------------------------------
+# config 2: matrix-vector with two bit flips (full size)
+# --------------------------------------------------------------------------------------------------
+def test_config2_matvec_two_bitflips():
+    cfg = wl.CONFIG_2_MATVEC
+    W, X = wl.matmul_inputs(cfg)
+    code = make_code(cfg)
+    cp = CodedProduct(code)
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    ref = op.ref_forward(W, X)
+    # oracle pipeline on its own outputs
+    Zo = op.worker_products(op.encode_W(W, code), op.encode_X(X, code)).astype(np.float32)
+    scale = rms(Zo)
+    for seed in cfg.inject_seeds + (5, 6, 7):
+        Zg = Z.clone()
+        hit = torch.zeros(1, dtype=torch.int64, device="cuda")
+        g.gpd_inject(cp.plan, g.GPD_FWD, Zg, seed, g.GPD_INJECT_BITFLIP, count=cfg.inject_count, scale=scale,
+                     hit_mask=hit)
+        Zr = Zo.copy()
+        sel = oinj.inject_bitflip(Zr, seed, cfg.inject_count, scale)
+        ro = locate_subspace(Zr, code.points, code.Q_f, tolerances_for(np.float32))
+        r = cp.locate(g.GPD_FWD, Zg)
+        assert r.outcome == ro.outcome == CORRECTED
+        assert np.array_equal(cp.flags(r), ro.flagged) and np.array_equal(ro.flagged, sel)
+        assert sel.sum() == 2 and r.n_flagged == 2
+        S = cp.decode(g.GPD_FWD, Zg)
+        assert op.rel_fro(S, ref) < REL_TOL
+        assert op.rel_fro(S, op.decode(Zr, code, FWD, use=~ro.flagged)) < REL_TOL
+
+
+# --------------------------------------------------------------------------------------------------
+# config 3 at reduced size: additive errors on random nodes, several seeds, failure included
+# --------------------------------------------------------------------------------------------------
+def _run_additive_case(cfg, seeds, check_against_full_oracle=True):
+    W, X = wl.matmul_inputs(cfg)
+    code = make_code(cfg)
+    cp = CodedProduct(code)
+    assert cp.np_dtype == np.float64
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    ref = op.ref_forward(W, X)
+    Zo = op.worker_products(op.encode_W(W, code), op.encode_X(X, code))
+    scale = rms(Zo)
+    outcomes = []
+    for seed in seeds:
+        Zg = Z.clone()
+        g.gpd_inject(cp.plan, g.GPD_FWD, Zg, seed, g.GPD_INJECT_ADDITIVE, prob=cfg.inject_prob, scale=scale)
+        Zr = Zo.copy()
+        sel = oinj.inject_additive(Zr, seed, scale, prob=cfg.inject_prob)
+        ro = locate_subspace(Zr, code.points, code.Q_f, tolerances_for(np.float64))
+        r = cp.locate(g.GPD_FWD, Zg)
+        assert r.outcome == ro.outcome, (seed, r.outcome, ro.outcome, sel.sum())
+        assert np.array_equal(cp.flags(r), ro.flagged)
+        outcomes.append(r.outcome)
+        S = cp.decode(g.GPD_FWD, Zg, fill=-7.0)
+        if r.outcome == DECODE_FAILURE:
+            assert (S == -7.0).all()                                   # nothing written
+            continue
+        assert np.array_equal(ro.flagged, sel)
+        assert op.rel_fro(S, ref) < REL_TOL
+        assert op.rel_fro(S, op.decode(Zr, code, FWD, use=~ro.flagged)) < REL_TOL
+    return outcomes
+
+
+def test_config3_scaled_additive_errors():
+    cfg = wl.scaled_down(wl.CONFIG_3_MATMUL, 8)                         # 1024 x 1024 x 64, same code
+    outcomes = _run_additive_case(cfg, cfg.inject_seeds)
+    assert CORRECTED in outcomes
+
+
+def test_too_many_errors_is_a_declared_failure():
+    cfg = wl.scaled_down(wl.CONFIG_3_MATMUL, 16)
+    W, X = wl.matmul_inputs(cfg)
+    code = make_code(cfg)
+    cp = CodedProduct(code)
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    Zo = op.worker_products(op.encode_W(W, code), op.encode_X(X, code))
+    for n_bad in (6, 9):                                                # P - Q = 6: budget is 5
+        mask = sum(1 << p for p in range(0, 2 * n_bad, 2))
+        nodes = np.array([(mask >> p) & 1 for p in range(cfg.P)], dtype=bool)
+        Zg = Z.clone()
+        g.gpd_inject(cp.plan, g.GPD_FWD, Zg, 11, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=mask, scale=1.0)
+        Zr = Zo.copy()
+        oinj.inject_gauss(Zr, 11, 1.0, nodes=nodes)
+        ro = locate_subspace(Zr, code.points, code.Q_f, tolerances_for(np.float64))
+        r = cp.locate(g.GPD_FWD, Zg)
+        assert r.outcome == ro.outcome == DECODE_FAILURE
+        S = cp.decode(g.GPD_FWD, Zg, fill=3.0)
+        assert (S == 3.0).all()
+
+
+def test_erasures_and_nonfinite_values():
+    cfg = wl.scaled_down(wl.CONFIG_3_MATMUL, 16)
+    W, X = wl.matmul_inputs(cfg)
+    code = make_code(cfg)
+    cp = CodedProduct(code)
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    ref = op.ref_forward(W, X)
+    Zg = Z.clone()
+    L = Zg.numel() // cfg.P
+    Zg[3 * L + 17] = float("inf")
+    Zg[20 * L + 5] = float("nan")
+    erased = np.zeros(cfg.P, dtype=bool)
+    erased[[7, 8]] = True
+    r = cp.locate(g.GPD_FWD, Zg, erased=erased)
+    Zr = cp.outputs_as_array(g.GPD_FWD, Zg)
+    ro = locate_subspace(Zr, code.points, code.Q_f, tolerances_for(np.float64), erased=erased)
+    assert r.outcome == ro.outcome == CORRECTED
+    assert np.array_equal(cp.flags(r), ro.flagged)
+    assert sorted(np.flatnonzero(ro.flagged)) == [3, 7, 8, 20]
+    assert np.array_equal(np.array(list(r.forced)[:cfg.P], dtype=bool), ro.forced)
+    assert op.rel_fro(cp.decode(g.GPD_FWD, Zg), ref) < REL_TOL
+
+
+# --------------------------------------------------------------------------------------------------
+# backward product and audit of the shares
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N1,N0,B,m,n,d2,P,prec", [
+    (512, 512, 64, 2, 2, 1, 10, g.GPD_PREC_AUTO),              # FP32 path (thresholds 5/6/4)
+    (256, 512, 128, 4, 4, 1, 36, g.GPD_PREC_AUTO),             # FP64 path (thresholds 19/28/16)
+    (128, 96, 24, 2, 3, 3, 24, g.GPD_PREC_AUTO),               # d2 = 3: Q_b = 21
+])
+def test_backward_and_audit(N1, N0, B, m, n, d2, P, prec):
+    code = GPCode(N1, N0, B, m, n, 1, d2, P)
+    cp = CodedProduct(code, prec)
+    W, DT = rand((N1, N0), 8) / np.sqrt(N0), rand((B, N1), 9)
+    Wsh = cp.encode_W(W)
+    Dsh = cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT)
+    Z = cp.products(g.GPD_BWD, Dsh)
+    nodes = np.zeros(P, dtype=bool)
+    nodes[[1, P - 2]] = True
+    g.gpd_inject(cp.plan, g.GPD_BWD, Z, 21, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=(1 << 1) | (1 << (P - 2)),
+                 scale=1.0)
+    r = cp.locate(g.GPD_BWD, Z)
+    Zr = op.worker_products(op.encode_DeltaT(DT, code), op.encode_W(W, code)).astype(cp.np_dtype)
+    oinj.inject_gauss(Zr, 21, 1.0, nodes=nodes)
+    ro = locate_subspace(Zr, code.points, code.Q_b, tolerances_for(cp.np_dtype))
+    assert r.outcome == ro.outcome == CORRECTED and np.array_equal(cp.flags(r), ro.flagged)
+    assert np.array_equal(ro.flagged, nodes)
+    CT = cp.decode(g.GPD_BWD, Z)
+    assert op.rel_fro(CT, op.ref_backward(DT, W)) < REL_TOL
+    assert op.rel_fro(CT, op.decode(Zr, code, BWD, use=~ro.flagged)) < REL_TOL
+    # audit: corrupt one stored share, find it, read W back
+    g.gpd_inject(cp.plan, g.GPD_AUDIT, Wsh, 22, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=1 << 4, scale=0.1)
+    r = cp.locate(g.GPD_AUDIT, Wsh)
+    assert r.outcome == CORRECTED and list(np.flatnonzero(cp.flags(r))) == [4]
+    assert op.rel_fro(cp.decode(g.GPD_AUDIT, Wsh), W) < REL_TOL
