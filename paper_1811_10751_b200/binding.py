@@ -103,14 +103,19 @@ def _check(status: int, where: str):
         raise GpdError(status, where)
 
 
-def _ptr(t: Optional[torch.Tensor]):
+def _ptr(t: Optional[torch.Tensor], dtype: Optional[torch.dtype] = None):
     if t is None:
         return None
     if not t.is_cuda:
         raise ValueError("device tensor expected")
     if not t.is_contiguous():
         raise ValueError("contiguous tensor expected")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"tensor of dtype {dtype} expected, got {t.dtype}")
     return C.c_void_p(t.data_ptr())
+
+
+_F32 = torch.float32
 
 
 def _stream(stream) -> C.c_void_p:
@@ -195,11 +200,11 @@ def gpd_plan_destroy(plan: Plan):
 
 
 def gpd_encode_A(plan: Plan, W, W_shares, stream=None):
-    _check(lib.gpd_encode_A(plan.handle, _ptr(W), _ptr(W_shares), _stream(stream)), "gpd_encode_A")
+    _check(lib.gpd_encode_A(plan.handle, _ptr(W, _F32), _ptr(W_shares, plan.dtype), _stream(stream)), "gpd_encode_A")
 
 
 def gpd_encode_B(plan: Plan, operand: int, src, shares, stream=None):
-    _check(lib.gpd_encode_B(plan.handle, operand, _ptr(src), _ptr(shares), _stream(stream)), "gpd_encode_B")
+    _check(lib.gpd_encode_B(plan.handle, operand, _ptr(src, _F32), _ptr(shares, plan.dtype), _stream(stream)), "gpd_encode_B")
 
 
 def gpd_worker_gemm(plan: Plan, which: int, W_shares, other_shares, outputs, stream=None):
@@ -226,8 +231,8 @@ def gpd_locate_errors(plan: Plan, which: int, outputs, result, workspace, erased
 
 def gpd_decode(plan: Plan, which: int, outputs, out, workspace, result=None, use_mask=None, act_out=None,
                activation: int = GPD_ACT_IDENTITY, stream=None):
-    _check(lib.gpd_decode(plan.handle, which, _ptr(outputs), _mask(use_mask, plan.P), _ptr(result), _ptr(out),
-                          _ptr(act_out), activation, _ptr(workspace), _stream(stream)), "gpd_decode")
+    _check(lib.gpd_decode(plan.handle, which, _ptr(outputs), _mask(use_mask, plan.P), _ptr(result), _ptr(out, _F32),
+                          _ptr(act_out, _F32), activation, _ptr(workspace), _stream(stream)), "gpd_decode")
 
 
 def gpd_activation(kind: int, S, X_next, stream=None):
@@ -262,7 +267,7 @@ def coded_layer_step(plan: Plan, phases: int, W_shares, X=None, Delta=None, Delt
                      activation: int = GPD_ACT_IDENTITY, eta: float = 0.0, lam: float = 0.0,
                      inject_seed: int = 0, inject_prob: float = 0.0, inject_scale: float = 1.0,
                      S_out=None, Xnext_out=None, CT_out=None, results=None, workspace=None, stream=None):
-    _check(lib.coded_layer_step(plan.handle, phases, _ptr(W_shares), _ptr(X), _ptr(Delta), _ptr(DeltaT),
+    _check(lib.coded_layer_step(plan.handle, phases, _ptr(W_shares), _ptr(X, _F32), _ptr(Delta, _F32), _ptr(DeltaT, _F32),
                                 activation, eta, lam, inject_seed & 0xFFFFFFFFFFFFFFFF, inject_prob, inject_scale,
                                 _ptr(S_out), _ptr(Xnext_out), _ptr(CT_out), _ptr(results), _ptr(workspace),
                                 _stream(stream)), "coded_layer_step")

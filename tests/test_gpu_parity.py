@@ -303,7 +303,7 @@ def test_erasures_and_nonfinite_values():
 def test_backward_and_audit(N1, N0, B, m, n, d2, P, prec):
     code = GPCode(N1, N0, B, m, n, 1, d2, P)
     cp = CodedProduct(code, prec)
-    W, DT = rand((N1, N0), 8) / np.sqrt(N0), rand((B, N1), 9)
+    W, DT = (rand((N1, N0), 8) / np.sqrt(N0)).astype(np.float32), rand((B, N1), 9)
     Wsh = cp.encode_W(W)
     Dsh = cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT)
     Z = cp.products(g.GPD_BWD, Dsh)
