@@ -164,6 +164,21 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def max_over_ranks(values_ms, world: int, device: str):
+    """Every rank times its own replica on its device; the job's time is the slowest rank's."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values_ms, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def whole_job_tflops(flops_per_step_per_rank: float, steps: int, world: int, ms: float) -> float:
+    """Aggregate over all replicas: units all ranks processed / slowest rank's time."""
+    return flops_per_step_per_rank * steps * world / (ms * 1e-3) / 1e12
+
+
 def measure_fp64_matmul_peak(torch) -> float:
     """cuBLAS FP64 GEMM 8192^3, best of 10 (the recipe that produced the bf16 figure, for FP64)."""
     n = 8192
@@ -316,12 +331,9 @@ def run_ours(args, cfg):
     check = {"outcome": int(r.outcome), "flagged": [p for p in range(cfg.P) if r.flagged[p]],
              "rel_err_sampled_rows": rel}
 
-    times = torch.tensor([ms, e2e_ms, gemm_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms, e2e_ms, gemm_ms = (float(v) for v in times.cpu())
-    value = useful_flops * args.steps * world / (ms * 1e-3) / 1e12
-    e2e_value = useful_flops * args.steps * world / (e2e_ms * 1e-3) / 1e12
+    ms, e2e_ms, gemm_ms = max_over_ranks([ms, e2e_ms, gemm_ms], world, "cuda")
+    value = whole_job_tflops(useful_flops, args.steps, world, ms)
+    e2e_value = whole_job_tflops(useful_flops, args.steps, world, e2e_ms)
 
     # FP64 tensor peak: MEASURED_PEAKS.json has no FP64 figure, and scaling its power-capped bf16
     # number by the nominal ratio gives a value below what the FP64 path delivers (FP64 does not

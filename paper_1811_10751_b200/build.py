@@ -1,6 +1,7 @@
 """Builds libgpd.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-Usage:  python -m paper_1811_10751_b200.build [--force] [--verbose]
+Usage:  python paper_1811_10751_b200/build.py [--force] [--verbose] [--ptxas]
+(run as a script so that the package, which needs the built library, is not imported)
 """
 
 from __future__ import annotations
