@@ -36,6 +36,7 @@ extern "C" {
 #define GPD_MAX_NODES 64        /* P <= 64 */
 #define GPD_MAX_THRESHOLD 32    /* every recovery threshold of the plan <= 32 */
 #define GPD_MAX_PARITY 32       /* P - Q <= 32 for every product of the plan */
+#define GPD_STATIC_MAX_PARITY 16 /* P - Q <= 16 for gpd_locate_errors_static (built-in scratch) */
 
 typedef struct gpd_plan_s* gpd_plan_t;
 
@@ -49,7 +50,8 @@ typedef enum {
     GPD_ERR_WORKSPACE = 6,      /* NULL workspace */
     GPD_ERR_CUDA = 7,           /* a CUDA runtime call failed (no device, launch failure) */
     GPD_ERR_TIMEOUT = 8,        /* a bounded device-side wait expired (reported through status words) */
-    GPD_ERR_UNSUPPORTED = 9     /* combination not implemented */
+    GPD_ERR_UNSUPPORTED = 9,    /* combination not implemented */
+    GPD_ERR_STATIC_LIMIT = 10   /* problem exceeds the built-in scratch of a no-allocation entry point */
 } gpd_status;
 
 /* The three exits of Algorithm 1 (Section V-A). */
@@ -207,6 +209,34 @@ gpd_status gpd_inject(gpd_plan_t plan, gpd_product which, void* outputs_dev, uin
 gpd_status gpd_locate_errors(gpd_plan_t plan, gpd_product which, const void* outputs_dev,
                              const uint8_t* erased_host, gpd_locate_result* result_dev,
                              void* workspace_dev, void* stream);
+
+/*
+ * gpd_locate_errors_static — gpd_locate_errors for callers that must not allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of the call above, same arithmetic,
+ * same result.)
+ *
+ * Who needs it: a fault-detection hook that runs inside a job whose framework has already handed
+ * all of HBM to its own memory pool, so that a cudaMalloc made on the library's behalf fails or
+ * eats into someone else's budget; and latency-critical loops that cannot afford the device-wide
+ * synchronisation an allocation implies.  gpd_locate_errors itself asks the caller for a workspace
+ * and, on a plan's first use, uploads the plan's tables into memory it allocates.  This variant
+ * does neither: its scratch (Gram matrix, counters and the parity-check matrix, about 10 KB) is a
+ * fixed array compiled into the library, present once on every GPU that loads the library until
+ * the process exits, and the parity-check matrix is copied into it from the plan's host tables on
+ * every call.  No cudaMalloc, cudaFree or allocating library routine is called on its path.
+ *
+ * Limit: products with P - Q <= GPD_STATIC_MAX_PARITY (16); beyond that the call returns
+ * GPD_ERR_STATIC_LIMIT and does nothing.
+ * Set-up: the first call on a device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture.
+ * Sharing: every call on a GPU uses the same array.  It is cleared by the call itself, but two
+ * calls whose work overlaps on the GPU (different streams, different threads) race on it: keep
+ * calls to this entry point ordered on one stream per GPU.
+ * Arguments as for gpd_locate_errors, without the workspace.
+ */
+gpd_status gpd_locate_errors_static(gpd_plan_t plan, gpd_product which, const void* outputs_dev,
+                                    const uint8_t* erased_host, gpd_locate_result* result_dev,
+                                    void* stream);
 
 /*
  * gpd_decode — interpolation of the wanted coefficients from the clean evaluations

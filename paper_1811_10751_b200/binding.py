@@ -17,14 +17,14 @@ import torch
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgpd.so")
 if not os.path.exists(_LIB_PATH):
     raise ImportError(
-        f"{_LIB_PATH} not found: build it with `python -m paper_1811_10751_b200.build` "
+        f"{_LIB_PATH} not found: build it with `python paper_1811_10751_b200/build.py` "
         "(nvcc, sm_100a). This package has no CPU fallback.")
 lib = C.CDLL(_LIB_PATH)
 
 # ---- enums ------------------------------------------------------------------------------------
 GPD_OK = 0
 (GPD_ERR_ARG, GPD_ERR_SHAPE, GPD_ERR_POINTS, GPD_ERR_P_TOO_SMALL, GPD_ERR_Q_TOO_LARGE,
- GPD_ERR_WORKSPACE, GPD_ERR_CUDA, GPD_ERR_TIMEOUT, GPD_ERR_UNSUPPORTED) = range(1, 10)
+ GPD_ERR_WORKSPACE, GPD_ERR_CUDA, GPD_ERR_TIMEOUT, GPD_ERR_UNSUPPORTED, GPD_ERR_STATIC_LIMIT) = range(1, 11)
 GPD_NO_ERROR, GPD_CORRECTED, GPD_DECODE_FAILURE = 0, 1, 2
 GPD_FWD, GPD_BWD, GPD_UPD, GPD_AUDIT = 0, 1, 2, 3
 GPD_OPERAND_X_FWD, GPD_OPERAND_DELTAT_BWD, GPD_OPERAND_DELTA_UPD, GPD_OPERAND_X_UPD = 0, 1, 2, 3
@@ -43,7 +43,7 @@ GPD_MAX_NODES = 64
 EXPORTED = [
     "gpd_status_string", "gpd_plan", "gpd_plan_destroy", "gpd_plan_query", "gpd_plan_table",
     "gpd_encode_A", "gpd_encode_B", "gpd_worker_gemm", "gpd_update_shares", "gpd_inject",
-    "gpd_locate_errors", "gpd_decode", "gpd_activation", "gpd_softmax_xent_delta",
+    "gpd_locate_errors", "gpd_locate_errors_static", "gpd_decode", "gpd_activation", "gpd_softmax_xent_delta",
     "gpd_backprop_hadamard", "gpd_sae_output_delta", "gpd_sae_hidden_delta", "coded_layer_step",
 ]
 
@@ -79,6 +79,7 @@ lib.gpd_worker_gemm.argtypes = [_vp, C.c_int, _vp, _vp, _vp, _vp]
 lib.gpd_update_shares.argtypes = [_vp, _vp, _vp, _vp, _f, _f, _vp, _vp]
 lib.gpd_inject.argtypes = [_vp, C.c_int, _vp, _u64, C.c_int, _d, _u64, _i32, _d, _vp, _vp]
 lib.gpd_locate_errors.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp, _vp]
+lib.gpd_locate_errors_static.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp]
 lib.gpd_decode.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp, _vp, C.c_int, _vp, _vp]
 lib.gpd_activation.argtypes = [C.c_int, _vp, _vp, _i64, _vp]
 lib.gpd_softmax_xent_delta.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _vp]
@@ -227,6 +228,14 @@ def gpd_inject(plan: Plan, which: int, outputs, seed: int, mode: int, prob: floa
 def gpd_locate_errors(plan: Plan, which: int, outputs, result, workspace, erased=None, stream=None):
     _check(lib.gpd_locate_errors(plan.handle, which, _ptr(outputs), _mask(erased, plan.P), _ptr(result),
                                  _ptr(workspace), _stream(stream)), "gpd_locate_errors")
+
+
+def gpd_locate_errors_static(plan: Plan, which: int, outputs, result, erased=None, stream=None):
+    """gpd_locate_errors without a workspace and without any device allocation on its path: the
+    scratch is a fixed array inside the library (products with P - Q <= 16 only).  Calls on one GPU
+    share that array, so keep them ordered on one stream."""
+    _check(lib.gpd_locate_errors_static(plan.handle, which, _ptr(outputs), _mask(erased, plan.P), _ptr(result),
+                                        _stream(stream)), "gpd_locate_errors_static")
 
 
 def gpd_decode(plan: Plan, which: int, outputs, out, workspace, result=None, use_mask=None, act_out=None,

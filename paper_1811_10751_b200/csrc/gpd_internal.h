@@ -96,6 +96,8 @@ gpd_status inject_launch(gpd_plan_s* plan, gpd_product which, void* outputs, uin
                          cudaStream_t st);
 gpd_status locate_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, uint64_t erased_mask,
                          gpd_locate_result* result, void* workspace, cudaStream_t st);
+gpd_status locate_static_launch(gpd_plan_s* plan, gpd_product which, const void* outputs,
+                                uint64_t erased_mask, gpd_locate_result* result, cudaStream_t st);
 gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, bool have_mask,
                          uint64_t use_mask, const gpd_locate_result* result, float* out, float* act_out,
                          int activation, void* workspace, cudaStream_t st);

@@ -379,6 +379,77 @@ gpd_status locate_launch(gpd_plan_s* plan, gpd_product which, const void* output
     return launch_ok();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Variant with built-in scratch: no device allocation anywhere on its path.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxR = GPD_STATIC_MAX_PARITY;
+constexpr size_t kStaticGramBytes = sizeof(double) * kStaticMaxR * kStaticMaxR;        // Gram matrix
+constexpr size_t kStaticCountBytes = 256;                                               // counters
+constexpr size_t kStaticHBytes = sizeof(double) * kStaticMaxR * kMaxNodes;              // parity checks
+constexpr size_t kStaticBytes = kStaticGramBytes + kStaticCountBytes + kStaticHBytes;
+
+// One copy per GPU that loads the library, held until the process exits.  Shared by every call of
+// gpd_locate_errors_static on that GPU.
+static __device__ __align__(256) unsigned char g_locate_scratch[kStaticBytes];
+
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[64] = {nullptr};      // device address of g_locate_scratch, per device
+
+// In host code `g_locate_scratch` is only a handle; the device address has to be asked for, with
+// the device current, once per device.
+gpd_status static_scratch(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GPD_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_locate_scratch) != cudaSuccess || !p) return GPD_ERR_CUDA;
+        g_static_ptr[dev] = reinterpret_cast<unsigned char*>(p);
+    }
+    *out = g_static_ptr[dev];
+    return GPD_OK;
+}
+
+}  // namespace
+
+gpd_status locate_static_launch(gpd_plan_s* plan, gpd_product which, const void* outputs,
+                                uint64_t erased_mask, gpd_locate_result* result, cudaStream_t st) {
+    if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
+    const ProductInfo& pi = plan->prod[which];
+    if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
+    if (pi.R > kStaticMaxR) return GPD_ERR_STATIC_LIMIT;
+    unsigned char* base = nullptr;
+    gpd_status rc = static_scratch(&base);
+    if (rc != GPD_OK) return rc;
+    double* gram = reinterpret_cast<double*>(base);
+    unsigned long long* counts = reinterpret_cast<unsigned long long*>(base + kStaticGramBytes);
+    double* H = reinterpret_cast<double*>(base + kStaticGramBytes + kStaticCountBytes);
+    // the array keeps the previous call's contents: Gram matrix and counters must start at zero
+    if (cudaMemsetAsync(base, 0, kStaticGramBytes + kStaticCountBytes, st) != cudaSuccess) return GPD_ERR_CUDA;
+    if (pi.R > 0 &&
+        cudaMemcpyAsync(H, pi.H.data(), sizeof(double) * pi.R * plan->P, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return GPD_ERR_CUDA;
+    if (pi.R > 0) {
+        SyndromeParams sp{};
+        sp.Z = outputs; sp.H = H; sp.L = pi.br * pi.bc; sp.P = plan->P; sp.R = pi.R;
+        sp.tau2 = plan->tau_col * plan->tau_col; sp.erased = erased_mask;
+        sp.gram = gram; sp.counts = counts;
+        if (plan->elem_size == 4)
+            rc = pi.R <= 8 ? launch_syndrome<float, 8>(sp, st) : launch_syndrome<float, 16>(sp, st);
+        else
+            rc = pi.R <= 8 ? launch_syndrome<double, 8>(sp, st) : launch_syndrome<double, 16>(sp, st);
+        if (rc != GPD_OK) return rc;
+    }
+    FinishParams fp{};
+    fp.H = H; fp.gram = gram; fp.counts = counts; fp.result = result;
+    fp.P = plan->P; fp.R = pi.R; fp.tau2 = plan->tau_col * plan->tau_col; fp.tau_in = plan->tau_in;
+    fp.erased = erased_mask;
+    locate_finish_kernel<<<1, 32, 0, st>>>(fp);
+    return launch_ok();
+}
+
 }  // namespace gpd
 
 using namespace gpd;
@@ -393,4 +464,15 @@ extern "C" gpd_status gpd_locate_errors(gpd_plan_t plan, gpd_product which, cons
         for (int p = 0; p < plan->P; ++p)
             if (erased_host[p]) mask |= 1ULL << p;
     return locate_launch(plan, which, outputs_dev, mask, result_dev, workspace_dev, as_stream(stream));
+}
+
+extern "C" gpd_status gpd_locate_errors_static(gpd_plan_t plan, gpd_product which, const void* outputs_dev,
+                                               const uint8_t* erased_host, gpd_locate_result* result_dev,
+                                               void* stream) {
+    if (!plan || !outputs_dev || !result_dev) return GPD_ERR_ARG;
+    uint64_t mask = 0;
+    if (erased_host)
+        for (int p = 0; p < plan->P; ++p)
+            if (erased_host[p]) mask |= 1ULL << p;
+    return locate_static_launch(plan, which, outputs_dev, mask, result_dev, as_stream(stream));
 }

@@ -131,6 +131,9 @@ extern "C" const char* gpd_status_string(gpd_status s) {
         case GPD_ERR_CUDA: return "CUDA runtime error";
         case GPD_ERR_TIMEOUT: return "bounded device-side wait expired";
         case GPD_ERR_UNSUPPORTED: return "unsupported combination";
+        case GPD_ERR_STATIC_LIMIT:
+            return "parity count above GPD_STATIC_MAX_PARITY: the built-in scratch of the no-allocation "
+                   "entry point is too small for this product; use gpd_locate_errors with a workspace";
     }
     return "unknown status";
 }
