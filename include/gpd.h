@@ -179,6 +179,13 @@ gpd_status gpd_worker_gemm(gpd_plan_t plan, gpd_product which, const void* W_sha
                            const void* other_shares_dev, void* outputs_dev, void* stream);
 
 /*
+ * gpd_device_status — kernels that wait on hardware barriers (the tensor-core product path) bound
+ * every wait; a wait that expires raises a device-side status word instead of hanging.  This call
+ * synchronises the device, returns that word in *status_host (0, or GPD_ERR_TIMEOUT) and clears it.
+ */
+gpd_status gpd_device_status(int32_t* status_host);
+
+/*
  * gpd_update_shares — coded update (step O3, Eq. 10 and its weight-decay form):
  *   W~_p <- (1 - eta*lambda) W~_p + eta * Delta^_p X^_p^T   for all p, in place.
  * If gate_dev is non-NULL and gate_dev->outcome == GPD_DECODE_FAILURE the shares are left

@@ -42,7 +42,7 @@ GPD_MAX_NODES = 64
 
 EXPORTED = [
     "gpd_status_string", "gpd_plan", "gpd_plan_destroy", "gpd_plan_query", "gpd_plan_table",
-    "gpd_encode_A", "gpd_encode_B", "gpd_worker_gemm", "gpd_update_shares", "gpd_inject",
+    "gpd_encode_A", "gpd_encode_B", "gpd_worker_gemm", "gpd_device_status", "gpd_update_shares", "gpd_inject",
     "gpd_locate_errors", "gpd_locate_errors_static", "gpd_decode", "gpd_activation", "gpd_softmax_xent_delta",
     "gpd_backprop_hadamard", "gpd_sae_output_delta", "gpd_sae_hidden_delta", "coded_layer_step",
 ]
@@ -76,6 +76,7 @@ lib.gpd_plan_table.argtypes = [_vp, C.c_int, C.POINTER(C.c_double), _i64, C.POIN
 lib.gpd_encode_A.argtypes = [_vp, _vp, _vp, _vp]
 lib.gpd_encode_B.argtypes = [_vp, C.c_int, _vp, _vp, _vp]
 lib.gpd_worker_gemm.argtypes = [_vp, C.c_int, _vp, _vp, _vp, _vp]
+lib.gpd_device_status.argtypes = [C.POINTER(_i32)]
 lib.gpd_update_shares.argtypes = [_vp, _vp, _vp, _vp, _f, _f, _vp, _vp]
 lib.gpd_inject.argtypes = [_vp, C.c_int, _vp, _u64, C.c_int, _d, _u64, _i32, _d, _vp, _vp]
 lib.gpd_locate_errors.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp, _vp]
@@ -211,6 +212,13 @@ def gpd_encode_B(plan: Plan, operand: int, src, shares, stream=None):
 def gpd_worker_gemm(plan: Plan, which: int, W_shares, other_shares, outputs, stream=None):
     _check(lib.gpd_worker_gemm(plan.handle, which, _ptr(W_shares), _ptr(other_shares), _ptr(outputs),
                                _stream(stream)), "gpd_worker_gemm")
+
+
+def gpd_device_status() -> int:
+    """Synchronises the device and returns (then clears) the tensor-path status word."""
+    v = _i32(0)
+    _check(lib.gpd_device_status(C.byref(v)), "gpd_device_status")
+    return int(v.value)
 
 
 def gpd_update_shares(plan: Plan, W_shares, Dhat, Xhat, eta: float, lam: float = 0.0, gate=None, stream=None):

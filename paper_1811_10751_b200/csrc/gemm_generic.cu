@@ -195,3 +195,10 @@ extern "C" gpd_status gpd_update_shares(gpd_plan_t plan, void* W_shares_dev, con
     if (!plan || !W_shares_dev || !Dhat_dev || !Xhat_dev) return GPD_ERR_ARG;
     return update_launch(plan, W_shares_dev, Dhat_dev, Xhat_dev, eta, lambda, gate_dev, as_stream(stream));
 }
+
+extern "C" gpd_status gpd_device_status(int32_t* status_host) {
+    if (!status_host) return GPD_ERR_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return GPD_ERR_CUDA;
+    *status_host = tf32_device_status_fetch_and_clear();
+    return GPD_OK;
+}

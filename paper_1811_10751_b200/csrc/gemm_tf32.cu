@@ -1,9 +1,365 @@
-// FP32-storage worker products on the tcgen05 tensor cores with 3xTF32 splitting.
+// FP32-storage worker products (steps O1, O2) and coded update (O3) on the 5th-generation tensor
+// cores: tcgen05.mma kind::tf32 with the accumulator in tensor memory, operands brought into
+// shared memory by TMA, and 3xTF32 splitting so that the result keeps FP32-level accuracy:
+//     a = a_hi + a_lo (both exactly representable in TF32),   a*b ~ a_lo*b_hi + a_hi*b_lo + a_hi*b_hi.
+//
+// One CTA computes one 128 x 128 tile of one node's product.  Warp roles:
+//   warp 0      : TMA producer (one lane) - raw FP32 tiles of A and B into a 3-stage ring
+//   warp 1      : allocates tensor memory; one lane issues the MMAs and commits them to mbarriers
+//   warps 2..5  : split every landed tile in place into hi (overwrites the raw tile) and lo (second
+//                 tile), then, after the last k-block, read the accumulator back (tcgen05.ld) and
+//                 write the tile (plain store, or read-modify-write for the coded update)
+// Operand tiles use the 128-byte swizzle; A is K-major; B is K-major for the update (X^_p is
+// [N][K]) and MN-major for the forward / backward products (X~_p, W~_p are [K][N]).
+// Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains its copies,
+// frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "gemm_common.h"
 
 namespace gpd {
 
-bool sgemm_3xtf32_supported(const GemmParams&) { return false; }
-gpd_status sgemm_3xtf32_launch(const GemmParams&, cudaStream_t) { return GPD_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int BM = 128, BN = 128, BK = 32, STAGES = 3;
+constexpr int UMMA_K = 8;
+constexpr int A_TILE_BYTES = BM * BK * 4;            // 16 KB, rows of 128 B
+constexpr int B_TILE_BYTES = BN * BK * 4;            // 16 KB
+constexpr int STAGE_BYTES = 2 * A_TILE_BYTES + 2 * B_TILE_BYTES;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
+constexpr int TMEM_COLS = 128;
+constexpr int kThreads = 192;
+constexpr long long kWaitCycles = 2000000000LL;      // about one second
+
+__device__ int g_tf32_status = 0;                    // GPD_ERR_TIMEOUT if a bounded wait expired
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within about a second or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicExch(&g_tf32_status, (int)GPD_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// Shared-memory matrix descriptor: start address, leading / stride byte offsets in 16-byte units,
+// descriptor version 1, layout type (2 = 128-byte swizzle of 16-byte chunks, used for K-major
+// operands; 1 = 128-byte swizzle of 32-byte chunks, the only layout an MN-major 32-bit operand
+// may use).
+constexpr uint32_t kLayoutSw128 = 2, kLayoutSw128Base32 = 1;
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)layout << 61;
+    return d;
+}
+// K-major tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) { return smem_desc(addr, 16, 1024, kLayoutSw128); }
+// MN-major tile: [k][32 columns] rows of 128 bytes; 4-row swizzle groups 512 bytes apart (two per
+// MMA of K = 8); the next 32 columns start BK rows (BK * 128 bytes) further.
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) { return smem_desc(addr, BK * 128, 512, kLayoutSw128Base32); }
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ float to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+template <bool B_KMAJOR, bool UPDATE>
+__global__ void __launch_bounds__(kThreads, 1)
+sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams prm) {
+    if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t full_bar[STAGES], conv_bar[STAGES], empty_bar[STAGES], acc_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int p = blockIdx.z;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int num_kb = (int)((prm.K + BK - 1) / BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&conv_bar[s], 4);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(&acc_bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_slot;
+    volatile int* abort_p = &abort_flag;
+
+    auto A_hi = [&](int s) { return smem + s * STAGE_BYTES; };
+    auto A_lo = [&](int s) { return smem + s * STAGE_BYTES + A_TILE_BYTES; };
+    auto B_hi = [&](int s) { return smem + s * STAGE_BYTES + 2 * A_TILE_BYTES; };
+    auto B_lo = [&](int s) { return smem + s * STAGE_BYTES + 2 * A_TILE_BYTES + B_TILE_BYTES; };
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) break;
+                mbar_expect_tx(&full_bar[s], A_TILE_BYTES + B_TILE_BYTES);
+                tma_load_3d(A_hi(s), &tmA, kb * BK, m0, p, &full_bar[s]);
+                if (B_KMAJOR) {
+                    tma_load_3d(B_hi(s), &tmB, kb * BK, n0, p, &full_bar[s]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < BN / 32; ++c)
+                        tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, n0 + 32 * c, kb * BK, p, &full_bar[s]);
+                }
+                ++issued;
+            }
+            if (*abort_p) {                      // let copies still in flight land before the CTA exits
+                for (int kb = issued > STAGES ? issued - STAGES : 0; kb < issued; ++kb) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&full_bar[kb % STAGES], (kb / STAGES) & 1) && clock64() - t0 < kWaitCycles) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
+                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                if (!mbar_wait(&conv_bar[s], ph, abort_p)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_hi = smem_u32(A_hi(s)), a_lo = smem_u32(A_lo(s));
+                const uint32_t b_hi = smem_u32(B_hi(s)), b_lo = smem_u32(B_lo(s));
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k) {
+                    // K-major: next 8 elements of K are 32 bytes further inside the swizzled row;
+                    // MN-major: next 8 k-rows are 8 * 128 bytes further in every 32-column chunk
+                    const uint32_t a_off = k * UMMA_K * 4;
+                    const uint32_t b_off = B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128;
+                    const uint64_t da_hi = desc_kmajor(a_hi + a_off);
+                    const uint64_t da_lo = desc_kmajor(a_lo + a_off);
+                    const uint64_t db_hi = B_KMAJOR ? desc_kmajor(b_hi + b_off) : desc_mnmajor(b_hi + b_off);
+                    const uint64_t db_lo = B_KMAJOR ? desc_kmajor(b_lo + b_off) : desc_mnmajor(b_lo + b_off);
+                    umma_tf32(tmem_base, da_lo, db_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);   // small terms first
+                    umma_tf32(tmem_base, da_hi, db_lo, idesc, 1u);
+                    umma_tf32(tmem_base, da_hi, db_hi, idesc, 1u);
+                }
+                umma_commit(&empty_bar[s]);          // stage reusable once these MMAs have read it
+            }
+            if (ok) umma_commit(&acc_bar);           // accumulator complete
+        }
+    } else {
+        // ------------------------------ split hi / lo, then epilogue ------------------------------
+        const int tc = threadIdx.x - 64;             // 0..127
+        bool ok = true;
+        for (int kb = 0; kb < num_kb; ++kb) {
+            const int s = kb % STAGES;
+            const uint32_t ph = (kb / STAGES) & 1;
+            if (!mbar_wait(&full_bar[s], ph, abort_p)) { ok = false; break; }
+            float4* hi[2] = {reinterpret_cast<float4*>(A_hi(s)), reinterpret_cast<float4*>(B_hi(s))};
+            float4* lo[2] = {reinterpret_cast<float4*>(A_lo(s)), reinterpret_cast<float4*>(B_lo(s))};
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+#pragma unroll
+                for (int i = 0; i < A_TILE_BYTES / 16 / 128; ++i) {
+                    const int idx = tc + 128 * i;
+                    const float4 v = hi[t][idx];
+                    float4 h, l;
+                    h.x = to_tf32(v.x); h.y = to_tf32(v.y); h.z = to_tf32(v.z); h.w = to_tf32(v.w);
+                    l.x = to_tf32(v.x - h.x); l.y = to_tf32(v.y - h.y); l.z = to_tf32(v.z - h.z); l.w = to_tf32(v.w - h.w);
+                    hi[t][idx] = h;
+                    lo[t][idx] = l;
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the tiles visible to the MMA unit
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&conv_bar[s]);
+        }
+        const bool acc_ready = ok && mbar_wait(&acc_bar, 0, abort_p);
+        __syncwarp();
+        if (__all_sync(0xffffffffu, acc_ready)) {    // tcgen05.ld is warp-collective: all lanes or none
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int q = warp & 3;                  // this warp may touch TMEM lanes 32q .. 32q+31
+            const int64_t gm = (int64_t)m0 + q * 32 + lane;
+            float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
+            const float shrink = (float)prm.shrink, eta = (float)prm.eta;
+            const bool vec = (prm.N % 4 == 0);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0;
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                    : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                      "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                      "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                      "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                    : "r"(taddr));
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (gm < prm.M) {
+                    float* crow = C + gm * prm.N + n0 + c0;
+                    if (vec && n0 + c0 + 32 <= prm.N) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                   __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                            if (UPDATE) {
+                                const float4 o = *reinterpret_cast<const float4*>(crow + j);
+                                v.x = shrink * o.x + eta * v.x; v.y = shrink * o.y + eta * v.y;
+                                v.z = shrink * o.z + eta * v.z; v.w = shrink * o.w + eta * v.w;
+                            }
+                            *reinterpret_cast<float4*>(crow + j) = v;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (n0 + c0 + j < prm.N) {
+                                float v = __uint_as_float(r[j]);
+                                if (UPDATE) v = shrink * crow[j] + eta * v;
+                                crow[j] = v;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 3-D FP32 tensor [batch][rows][cols] (cols contiguous), box {box_cols, box_rows, 1}, given
+// 128-byte swizzle flavour, out-of-range elements read as zero.
+bool make_map(CUtensorMap* map, const void* base, int64_t batch, int64_t rows, int64_t cols, int box_cols, int box_rows,
+              CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 4, (cuuint64_t)rows * (cuuint64_t)cols * 4};
+    cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool B_KMAJOR, bool UPDATE>
+gpd_status launch(const GemmParams& prm, cudaStream_t st) {
+    CUtensorMap tmA, tmB;
+    if (!make_map(&tmA, prm.A, prm.P, prm.M, prm.K, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B)) return GPD_ERR_CUDA;
+    const bool okB = B_KMAJOR ? make_map(&tmB, prm.B, prm.P, prm.N, prm.K, BK, BN, CU_TENSOR_MAP_SWIZZLE_128B)
+                              : make_map(&tmB, prm.B, prm.P, prm.K, prm.N, 32, BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
+    if (!okB) return GPD_ERR_CUDA;
+    if (cudaFuncSetAttribute(sgemm_3xtf32_kernel<B_KMAJOR, UPDATE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             SMEM_BYTES) != cudaSuccess)
+        return GPD_ERR_CUDA;
+    dim3 grid((unsigned)((prm.N + BN - 1) / BN), (unsigned)((prm.M + BM - 1) / BM), (unsigned)prm.P);
+    sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<grid, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm);
+    return launch_ok();
+}
+
+}  // namespace
+
+bool sgemm_3xtf32_supported(const GemmParams& prm) {
+    // TMA: 16-byte aligned bases and row pitches; big enough that a 128 x 128 tile is not mostly padding
+    const bool aligned = reinterpret_cast<uintptr_t>(prm.A) % 16 == 0 && reinterpret_cast<uintptr_t>(prm.B) % 16 == 0 &&
+                         reinterpret_cast<uintptr_t>(prm.C) % 16 == 0;
+    const bool pitches = (prm.K % 4 == 0) && (prm.b_kmajor || prm.N % 4 == 0);
+    return aligned && pitches && prm.M >= 64 && prm.N >= 64 && prm.K >= 32 && encode_tiled_fn() != nullptr;
+}
+
+gpd_status sgemm_3xtf32_launch(const GemmParams& prm, cudaStream_t st) {
+    if (prm.b_kmajor) return prm.update ? launch<true, true>(prm, st) : launch<true, false>(prm, st);
+    return prm.update ? launch<false, true>(prm, st) : launch<false, false>(prm, st);
+}
+
+int tf32_device_status_fetch_and_clear() {
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_tf32_status, sizeof(int)) != cudaSuccess) return (int)GPD_ERR_CUDA;
+    if (v != 0) cudaMemcpyToSymbol(g_tf32_status, &zero, sizeof(int));
+    return v;
+}
 
 }  // namespace gpd
