@@ -376,6 +376,110 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def measure_tf32_matmul_peak(torch) -> float:
+    """cuBLAS TF32 GEMM 8192^3, best of 10 (same recipe as the bf16 figure)."""
+    n = 8192
+    a = torch.randn((n, n), device="cuda")
+    b = torch.randn((n, n), device="cuda")
+    c = torch.empty((n, n), device="cuda")
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    for _ in range(2):
+        torch.matmul(a, b, out=c)
+    best = float("inf")
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        torch.matmul(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    torch.backends.cuda.matmul.allow_tf32 = old
+    return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+
+
+def run_mlp_layer(args):
+    """Secondary workload (not the headline line): one hidden layer of the coded MLP step,
+    4096 x 4096 weights, batch 256, split 2 x 2, P = 10, FP32 shares, tensor-core 3xTF32 products;
+    step = coded forward + coded backward + coded update through coded_layer_step."""
+    import torch
+    import paper_1811_10751_b200 as g
+    import workloads as wl
+    c4 = wl.CONFIG_4_MLP
+    N, B, P = c4.widths[1], c4.B, c4.P
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    gen = torch.Generator(device="cuda").manual_seed(c4.seed)
+    W = torch.randn((N, N), device="cuda", generator=gen) * (2.0 / N) ** 0.5
+    X = torch.randn((N, B), device="cuda", generator=gen).clamp_(min=0)
+    D = torch.randn((N, B), device="cuda", generator=gen) / B
+    DT = D.t().contiguous()
+    plan = g.gpd_plan((N, N, B), (c4.m, c4.n, 1, 1), P)
+    Wsh = plan.empty(g.GPD_Q_W_SHARE_ELEMS)
+    g.gpd_encode_A(plan, W, Wsh)
+    ws, res = plan.workspace(step=True), g.new_results(3)
+    S, Xn = torch.empty((N, B), device="cuda"), torch.empty((N, B), device="cuda")
+    CT = torch.empty((B, N), device="cuda")
+    stream = torch.cuda.Stream()
+
+    def step(i):
+        g.coded_layer_step(plan, g.GPD_PHASE_FWD, Wsh, X=X, activation=g.GPD_ACT_RELU, inject_seed=1000 + 16 * i,
+                           inject_prob=c4.inject_prob, S_out=S, Xnext_out=Xn, CT_out=CT, results=res, workspace=ws,
+                           stream=stream)
+        g.coded_layer_step(plan, g.GPD_PHASE_BWD | g.GPD_PHASE_UPD, Wsh, X=X, Delta=D, DeltaT=DT, eta=1e-4,
+                           inject_seed=1000 + 16 * i, inject_prob=c4.inject_prob, S_out=S, Xnext_out=Xn, CT_out=CT,
+                           results=res, workspace=ws, stream=stream)
+
+    with torch.cuda.stream(stream):
+        for i in range(max(args.warmup, 3)):
+            step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    # the three tensor-core launches on their own
+    Xsh, Dsh = plan.empty(g.GPD_Q_X_SHARE_ELEMS), plan.empty(g.GPD_Q_DT_SHARE_ELEMS)
+    Dh, Xh = plan.empty(g.GPD_Q_DHAT_ELEMS), plan.empty(g.GPD_Q_XHAT_ELEMS)
+    Zf, Zb = plan.empty(g.GPD_Q_OUT_ELEMS_FWD), plan.empty(g.GPD_Q_OUT_ELEMS_BWD)
+    g.gpd_encode_B(plan, g.GPD_OPERAND_X_FWD, X, Xsh)
+    g.gpd_encode_B(plan, g.GPD_OPERAND_DELTAT_BWD, DT, Dsh)
+    g.gpd_encode_B(plan, g.GPD_OPERAND_DELTA_UPD, D, Dh)
+    g.gpd_encode_B(plan, g.GPD_OPERAND_X_UPD, X, Xh)
+    kern = {}
+    for name, fn in (("forward", lambda: g.gpd_worker_gemm(plan, g.GPD_FWD, Wsh, Xsh, Zf)),
+                     ("backward", lambda: g.gpd_worker_gemm(plan, g.GPD_BWD, Wsh, Dsh, Zb)),
+                     ("update", lambda: g.gpd_update_shares(plan, Wsh, Dh, Xh, 1e-6, 0.0))):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(args.steps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        kern[name] = a.elapsed_time(b) / args.steps
+    status = g.gpd_device_status()
+    peak = measure_tf32_matmul_peak(torch) / 3.0
+    flops = 2.0 * P * (N // c4.m) * (N // c4.n) * B            # FP32-equivalent flops of one product
+    useful = 3 * 2.0 * N * N * B
+    line = {"metric": METRIC, "value": useful / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32 (3xTF32 products, FP64 encode/locate/decode arithmetic)",
+            "data": "synthetic",
+            "config": {"workload": "cfg4_mlp_hidden_layer_4096x4096_b256", "split": [c4.m, c4.n, 1, 1], "nodes": P,
+                       "step": "coded forward + backward + update of one layer", "l2": "shares 168 MB > L2"},
+            "kernel_ms": kern, "device_status": status,
+            "roofline": {"bound": "tensor", "kernel": "sgemm_3xtf32_kernel (forward products)",
+                         "achieved": flops / (kern["forward"] * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
+                         "frac": flops / (kern["forward"] * 1e-3) / 1e12 / peak, "traffic": None,
+                         "peak_source": "measured here: torch.matmul TF32 8192^3 best of 10, divided by 3 (3xTF32)"}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -384,7 +488,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-down", type=int, default=1,
                     help="profiling aid: same code on matrices this many times smaller per side")
+    ap.add_argument("--workload", default="matmul", choices=["matmul", "mlp_layer"],
+                    help="matmul: the headline 8192 x 8192 x 512 coded product; mlp_layer: secondary, FP32 path")
     args = ap.parse_args()
+    if args.workload == "mlp_layer" and args.impl == "ours":
+        run_mlp_layer(args)
+        return
     import workloads as wl
     cfg = wl.CONFIG_3_MATMUL
     if args.scale_down > 1:

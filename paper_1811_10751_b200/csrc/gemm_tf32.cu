@@ -6,7 +6,7 @@
 // One CTA computes one 128 x 128 tile of one node's product.  Warp roles:
 //   warp 0      : TMA producer (one lane) - raw FP32 tiles of A and B into a 3-stage ring
 //   warp 1      : allocates tensor memory; one lane issues the MMAs and commits them to mbarriers
-//   warps 2..5  : split every landed tile in place into hi (overwrites the raw tile) and lo (second
+//   warps 2..9  : split every landed tile in place into hi (overwrites the raw tile) and lo (second
 //                 tile), then, after the last k-block, read the accumulator back (tcgen05.ld) and
 //                 write the tile (plain store, or read-modify-write for the coded update)
 // Operand tiles use the 128-byte swizzle; A is K-major; B is K-major for the update (X^_p is
@@ -28,7 +28,9 @@ constexpr int B_TILE_BYTES = BN * BK * 4;            // 16 KB
 constexpr int STAGE_BYTES = 2 * A_TILE_BYTES + 2 * B_TILE_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
 constexpr int TMEM_COLS = 128;
-constexpr int kThreads = 192;
+constexpr int kConvWarps = 8;                        // warps 2..9: split tiles, then drain tensor memory
+constexpr int kConvThreads = kConvWarps * 32;
+constexpr int kThreads = 64 + kConvThreads;
 constexpr long long kWaitCycles = 2000000000LL;      // about one second
 
 __device__ int g_tf32_status = 0;                    // GPD_ERR_TIMEOUT if a bounded wait expired
@@ -101,10 +103,10 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// Round to the nearest TF32 value (10 explicit mantissa bits) with integer arithmetic: add half
+// a TF32 ulp to the magnitude and clear the 13 low bits (ties away from zero; Inf stays Inf).
 __device__ __forceinline__ float to_tf32(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return __uint_as_float(r);
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
 }
 
 template <bool B_KMAJOR, bool UPDATE>
@@ -125,7 +127,7 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&conv_bar[s], 4);
+            mbar_init(&conv_bar[s], kConvWarps);
             mbar_init(&empty_bar[s], 1);
         }
         mbar_init(&acc_bar, 1);
@@ -206,7 +208,7 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
     } else {
         // ------------------------------ split hi / lo, then epilogue ------------------------------
-        const int tc = threadIdx.x - 64;             // 0..127
+        const int tc = threadIdx.x - 64;             // 0..kConvThreads-1
         bool ok = true;
         for (int kb = 0; kb < num_kb; ++kb) {
             const int s = kb % STAGES;
@@ -217,8 +219,8 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
 #pragma unroll
-                for (int i = 0; i < A_TILE_BYTES / 16 / 128; ++i) {
-                    const int idx = tc + 128 * i;
+                for (int i = 0; i < A_TILE_BYTES / 16 / kConvThreads; ++i) {
+                    const int idx = tc + kConvThreads * i;
                     const float4 v = hi[t][idx];
                     float4 h, l;
                     h.x = to_tf32(v.x); h.y = to_tf32(v.y); h.z = to_tf32(v.z); h.w = to_tf32(v.w);
@@ -236,12 +238,13 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (__all_sync(0xffffffffu, acc_ready)) {    // tcgen05.ld is warp-collective: all lanes or none
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int q = warp & 3;                  // this warp may touch TMEM lanes 32q .. 32q+31
+            const int half = (warp - 2) >> 2;        // two warps share a lane quarter: 64 columns each
             const int64_t gm = (int64_t)m0 + q * 32 + lane;
             float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
             const float shrink = (float)prm.shrink, eta = (float)prm.eta;
             const bool vec = (prm.N % 4 == 0);
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0;
                 asm volatile(
