@@ -296,7 +296,10 @@ def test_erasures_and_nonfinite_values():
     erased = np.zeros(cfg.P, dtype=bool)
     erased[[7, 8]] = True
     r = cp.locate(g.GPD_FWD, Zg, erased=erased)
-    Zr = cp.outputs_as_array(g.GPD_FWD, Zg)
+    # the oracle works on its own outputs, with the same two values planted
+    Zr = op.worker_products(op.encode_W(W, code), op.encode_X(X, code)).reshape(cfg.P, L)
+    Zr[3, 17] = np.inf
+    Zr[20, 5] = np.nan
     ro = locate_subspace(Zr, code.points, code.Q_f, tolerances_for(np.float64), erased=erased)
     assert r.outcome == ro.outcome == CORRECTED
     assert np.array_equal(cp.flags(r), ro.flagged)
@@ -369,11 +372,18 @@ def test_config4_full_size_layer():
     assert r.outcome == CORRECTED and list(np.flatnonzero(cp.flags(r))) == [9]
     CT = cp.decode(g.GPD_BWD, Zb)
     assert op.rel_fro(CT, op.ref_backward(DT, W)) < REL_TOL
-    # oracle decisions on the same corrupted buffers
-    for which, Z, Q in ((g.GPD_FWD, Zf, code.Q_f), (g.GPD_BWD, Zb, code.Q_b)):
-        ro = locate_subspace(cp.outputs_as_array(which, Z), code.points, Q, tolerances_for(np.float32))
+    # the oracle's own pipeline on the same inputs, seeds and nodes
+    Ws_o = op.encode_W(W, code)
+    for which, Z, Q, seed, mask, Zo in (
+            (g.GPD_FWD, Zf, code.Q_f, 41, nodes_f, op.worker_products(Ws_o, op.encode_X(X, code))),
+            (g.GPD_BWD, Zb, code.Q_b, 42, nodes_b, op.worker_products(op.encode_DeltaT(DT, code), Ws_o))):
+        Zo = Zo.astype(np.float32)
+        oinj.inject_gauss(Zo, seed, 1.0, nodes=[(mask >> p) & 1 for p in range(P)])
+        ro = locate_subspace(Zo, code.points, Q, tolerances_for(np.float32))
         rg = cp.locate(which, Z)
         assert ro.outcome == rg.outcome and np.array_equal(ro.flagged, cp.flags(rg))
+        got = S if which == g.GPD_FWD else CT
+        assert op.rel_fro(got, op.decode(Zo, code, FWD if which == g.GPD_FWD else BWD, use=~ro.flagged)) < REL_TOL
     # coded update, then audit
     Dh, Xh = cp.encode(g.GPD_OPERAND_DELTA_UPD, Delta), cp.encode(g.GPD_OPERAND_X_UPD, X)
     g.gpd_update_shares(cp.plan, Wsh, Dh, Xh, c4.lr, 0.0)
@@ -384,3 +394,45 @@ def test_config4_full_size_layer():
     assert op.rel_fro(W_new, ref_new) < REL_TOL
     assert op.rel_fro(W_new.astype(np.float64) - W, ref_new - W) < 5e-3
     assert g.gpd_device_status() == 0
+
+
+# --------------------------------------------------------------------------------------------------
+# config 3 at full size, in the launch configuration bench.py times: decisions against the oracle's
+# (tests/golden/cfg3_full_expected.json, written by make_cfg3_expected.py from oracle/ alone),
+# sampled worker outputs and sampled rows of the decoded product against FP64 definitions
+# --------------------------------------------------------------------------------------------------
+def test_config3_full_size_against_oracle_decisions():
+    import json
+    import os
+    gold = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "cfg3_full_expected.json")))
+    cfg = wl.CONFIG_3_MATMUL
+    assert gold["config"] == cfg.name
+    W, X = wl.matmul_inputs(cfg)
+    code = make_code(cfg)
+    cp = CodedProduct(code)
+    assert cp.np_dtype == np.float64
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    L = Z.numel() // cfg.P
+    pos = np.array(gold["sample_positions"])
+    got = host(Z.reshape(cfg.P, L)[:, torch.from_numpy(pos).cuda()])
+    want = np.array(gold["clean_outputs_at_samples"])
+    assert np.abs(got - want).max() <= 1e-12 * gold["scale"] * 8          # FP64 products, K = 2048
+    rows = np.arange(0, cfg.N1, cfg.N1 // 32)
+    ref_rows = op.ref_forward(W[rows], X)
+    for seed in cfg.inject_seeds:
+        e = gold["seeds"][str(seed)]
+        Zg = Z.clone()
+        g.gpd_inject(cp.plan, g.GPD_FWD, Zg, seed, g.GPD_INJECT_ADDITIVE, prob=cfg.inject_prob, scale=gold["scale"])
+        r = cp.locate(g.GPD_FWD, Zg)
+        assert r.outcome == e["outcome"] and r.rank == e["rank"] and r.n_active == e["n_active"]
+        assert list(np.flatnonzero(cp.flags(r))) == e["flagged"] == e["injected"]
+        S = cp.decode(g.GPD_FWD, Zg)
+        assert np.isfinite(S).all()
+        assert op.rel_fro(S[rows], ref_rows) < REL_TOL
+        # the decoded product must not depend on which nodes were hit: compare with the clean decode
+        if seed == cfg.inject_seeds[0]:
+            r0 = cp.locate(g.GPD_FWD, Z)
+            assert r0.outcome == NO_ERROR
+            S_clean = cp.decode(g.GPD_FWD, Z)
+        assert op.rel_fro(S, S_clean) < REL_TOL
