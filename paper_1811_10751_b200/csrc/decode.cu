@@ -161,16 +161,30 @@ __global__ void __launch_bounds__(256) decode_stream_kernel(StreamParams prm) {
             for (int w = 0; w < NW; ++w)
 #pragma unroll
                 for (int v = 0; v < N; ++v) acc[w][v] = 0.0;
-            for (int i = 0; i < s_nused; ++i) {
-                const int p = s_nodes[i];
-                double z[N];
-                if constexpr (VECTOR) Vec<T>::load(Z + (int64_t)p * L + pos, z);
-                else z[0] = (double)__ldcs(Z + (int64_t)p * L + pos);
+            constexpr int U = 6;                         // nodes per trip, loads issued first
+            for (int i0 = 0; i0 < s_nused; i0 += U) {
+                double z[U][N];
+                int pn[U];
 #pragma unroll
-                for (int w = 0; w < NW; ++w) {
-                    const double d = (w0 + w < prm.n_wanted) ? sD[(w0 + w) * prm.P + p] : 0.0;
+                for (int u = 0; u < U; ++u) {
+                    const bool live = i0 + u < s_nused;
+                    pn[u] = s_nodes[live ? i0 + u : 0];
+                    if (live) {
+                        if constexpr (VECTOR) Vec<T>::load(Z + (int64_t)pn[u] * L + pos, z[u]);
+                        else z[u][0] = (double)__ldcs(Z + (int64_t)pn[u] * L + pos);
+                    } else {
 #pragma unroll
-                    for (int v = 0; v < N; ++v) acc[w][v] = fma(d, z[v], acc[w][v]);
+                        for (int v = 0; v < N; ++v) z[u][v] = 0.0;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+#pragma unroll
+                    for (int w = 0; w < NW; ++w) {
+                        const double d = (w0 + w < prm.n_wanted) ? sD[(w0 + w) * prm.P + pn[u]] : 0.0;
+#pragma unroll
+                        for (int v = 0; v < N; ++v) acc[w][v] = fma(d, z[u][v], acc[w][v]);
+                    }
                 }
             }
 #pragma unroll

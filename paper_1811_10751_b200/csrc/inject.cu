@@ -34,6 +34,8 @@ __host__ __device__ __forceinline__ double unit(unsigned long long r) {
 }
 
 struct InjectParams {
+    int n_sel;             // additive / gauss: number of selected nodes, listed in sel[]
+    unsigned char sel[kMaxNodes];
     void* out;             // [P][L]
     int64_t L;
     int P;
@@ -46,25 +48,16 @@ struct InjectParams {
     unsigned long long* hit_mask;
 };
 
-__device__ __forceinline__ bool node_selected(const InjectParams& prm, int p) {
+__host__ __device__ __forceinline__ bool node_selected(const InjectParams& prm, int p) {
     if (prm.prob < 0.0) return (prm.node_mask >> p) & 1ULL;
     return unit(draw(make_key(prm.seed, TAG_NODE, 0), (unsigned long long)p)) < prm.prob;
 }
 
-__device__ __forceinline__ void write_hit_mask(const InjectParams& prm) {
-    if (prm.hit_mask && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
-        unsigned long long m = 0;
-        for (int p = 0; p < prm.P; ++p)
-            if (node_selected(prm, p)) m |= 1ULL << p;
-        *prm.hit_mask = m;
-    }
-}
+__global__ void write_mask_kernel(unsigned long long* dst, unsigned long long value) { *dst = value; }
 
 template <typename T>
 __global__ void __launch_bounds__(256) inject_additive_kernel(InjectParams prm) {
-    write_hit_mask(prm);
-    const int p = blockIdx.y;
-    if (!node_selected(prm, p)) return;
+    const int p = prm.sel[blockIdx.y];
     const double phi = 1.0 - unit(draw(make_key(prm.seed, TAG_PHI, 0), (unsigned long long)p));
     const unsigned long long first = draw(make_key(prm.seed, TAG_FIRST, 0), (unsigned long long)p) %
                                      (unsigned long long)prm.L;
@@ -86,9 +79,7 @@ __global__ void __launch_bounds__(256) inject_additive_kernel(InjectParams prm) 
 
 template <typename T>
 __global__ void __launch_bounds__(256) inject_gauss_kernel(InjectParams prm) {
-    write_hit_mask(prm);
-    const int p = blockIdx.y;
-    if (!node_selected(prm, p)) return;
+    const int p = prm.sel[blockIdx.y];
     const unsigned long long key = make_key(prm.seed, TAG_GAUSS, (unsigned long long)p);
     T* out = reinterpret_cast<T*>(prm.out) + (int64_t)p * prm.L;
     for (int64_t l = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; l < prm.L;
@@ -159,7 +150,18 @@ gpd_status inject_launch(gpd_plan_s* plan, gpd_product which, void* outputs, uin
         else inject_bitflip_kernel<double, unsigned long long><<<1, 32, 0, st>>>(prm);
         return launch_ok();
     }
-    dim3 grid((unsigned)std::min<int64_t>((prm.L + 255) / 256, 2048), (unsigned)prm.P);
+    if (mode != GPD_INJECT_ADDITIVE && mode != GPD_INJECT_GAUSS) return GPD_ERR_ARG;
+    // Which nodes are hit is a pure function of (seed, node): evaluated here with the same
+    // generator, so that only the selected nodes get thread blocks.
+    unsigned long long mask = 0;
+    for (int p = 0; p < prm.P; ++p)
+        if (node_selected(prm, p)) { prm.sel[prm.n_sel++] = (unsigned char)p; mask |= 1ULL << p; }
+    if (prm.hit_mask) {
+        write_mask_kernel<<<1, 1, 0, st>>>(prm.hit_mask, mask);
+        if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+    }
+    if (prm.n_sel == 0) return GPD_OK;
+    dim3 grid((unsigned)std::min<int64_t>((prm.L + 1023) / 1024, 1024), (unsigned)prm.n_sel);
     if (mode == GPD_INJECT_ADDITIVE) {
         if (f32) inject_additive_kernel<float><<<grid, 256, 0, st>>>(prm);
         else inject_additive_kernel<double><<<grid, 256, 0, st>>>(prm);

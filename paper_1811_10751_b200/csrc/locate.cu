@@ -33,86 +33,124 @@ struct SyndromeParams {
     unsigned long long* counts; // [0] n_active, [1] mask of nodes holding a non-finite value
 };
 
+__device__ __forceinline__ void dmma_m8n8k4(double& d0, double& d1, double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};\n"
+                 : "+d"(d0), "+d"(d1)
+                 : "d"(a), "d"(b));
+}
+
+// One thread per output position (codeword): P coalesced loads (issued four at a time), the
+// syndrome in RT registers, the zero test.  The Gram matrix of the failing codewords is formed
+// warp by warp on the FP64 tensor cores: the 32 scaled syndromes of a warp are staged in shared
+// memory and fed to mma.m8n8k4 as both operands (G += S S^T, four codewords per instruction), so
+// the accumulator costs two registers per 8 x 8 tile and the streaming loop needs no CTA barrier.
 template <typename T, int RT>
 __global__ void __launch_bounds__(kThreads) syndrome_gram_kernel(SyndromeParams prm) {
+    constexpr int NT = RT / 8;                          // 8 x 8 tiles per side of the Gram matrix
+    constexpr int LD = RT + 4;                          // row pitch of the staging buffer (bank spread)
+    constexpr int kWarps = kThreads / 32;
     extern __shared__ __align__(16) double sm[];
-    double* sH = sm;                                   // [RT][P], rows >= R are zero
-    double* sS = sm + RT * prm.P;                      // [kThreads][RT + 1]
-    __shared__ unsigned long long s_nonfinite;
-    __shared__ unsigned int s_active;
-    for (int i = threadIdx.x; i < RT * prm.P; i += kThreads)
-        sH[i] = (i < prm.R * prm.P) ? prm.H[i] : 0.0;
-    if (threadIdx.x == 0) { s_nonfinite = 0ULL; s_active = 0u; }
+    double* sH = sm;                                    // [P][RT] node-major, rows >= R are zero
+    double* sS = sm + RT * prm.P;                       // [kWarps][32][LD]
+    double* sG = sS + kWarps * 32 * LD;                 // [RT][RT] CTA total
+    for (int i = threadIdx.x; i < RT * prm.P; i += kThreads) {
+        const int pnode = i / RT, r = i % RT;
+        sH[i] = r < prm.R ? prm.H[r * prm.P + pnode] : 0.0;
+    }
+    for (int i = threadIdx.x; i < RT * RT; i += kThreads) sG[i] = 0.0;
     __syncthreads();
 
-    constexpr int kPairs = RT * (RT + 1) / 2;
-    constexpr int kOwn = (kPairs + kThreads - 1) / kThreads;
-    double g_own[kOwn];
-    int own_i[kOwn], own_j[kOwn];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double* myS = sS + warp * 32 * LD;
+    double acc[NT][NT][2];
 #pragma unroll
-    for (int e = 0; e < kOwn; ++e) {
-        g_own[e] = 0.0;
-        int idx = threadIdx.x + e * kThreads, i = 0;
-        if (idx >= kPairs) { own_i[e] = -1; own_j[e] = 0; continue; }
-        while (idx >= RT - i) { idx -= RT - i; ++i; }   // row-major upper triangle
-        own_i[e] = i;
-        own_j[e] = i + idx;
-    }
-
+    for (int a = 0; a < NT; ++a)
+#pragma unroll
+        for (int b = 0; b < NT; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
+    unsigned long long bad_all = 0ULL;
+    unsigned int my_active = 0;
     const T* Z = reinterpret_cast<const T*>(prm.Z);
     const int64_t n_batches = (prm.L + kThreads - 1) / kThreads;
-    unsigned int my_active = 0;
     for (int64_t batch = blockIdx.x; batch < n_batches; batch += gridDim.x) {
         const int64_t l = batch * kThreads + threadIdx.x;
         double s[RT];
 #pragma unroll
         for (int r = 0; r < RT; ++r) s[r] = 0.0;
         double nz = 0.0;
-        unsigned long long bad = 0ULL;
         if (l < prm.L) {
-            for (int p = 0; p < prm.P; ++p) {
-                double z = (double)__ldcs(Z + (int64_t)p * prm.L + l);
-                if (!isfinite(z)) { bad |= 1ULL << p; z = 0.0; }
-                if ((prm.erased >> p) & 1ULL) z = 0.0;
-                nz = fma(z, z, nz);
+            const T* zp = Z + l;
+            for (int p0 = 0; p0 < prm.P; p0 += 4) {
+                double z[4];
 #pragma unroll
-                for (int r = 0; r < RT; ++r) s[r] = fma(sH[r * prm.P + p], z, s[r]);
+                for (int u = 0; u < 4; ++u)
+                    z[u] = (p0 + u < prm.P) ? (double)__ldcs(zp + (int64_t)(p0 + u) * prm.L) : 0.0;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int pnode = p0 + u;
+                    if (pnode < prm.P) {
+                        double zz = z[u];
+                        if (!isfinite(zz)) { bad_all |= 1ULL << pnode; zz = 0.0; }
+                        if ((prm.erased >> pnode) & 1ULL) zz = 0.0;
+                        nz = fma(zz, zz, nz);
+                        const double2* h = reinterpret_cast<const double2*>(sH + pnode * RT);
+#pragma unroll
+                        for (int r = 0; r < RT / 2; ++r) {
+                            const double2 hv = h[r];
+                            s[2 * r] = fma(hv.x, zz, s[2 * r]);
+                            s[2 * r + 1] = fma(hv.y, zz, s[2 * r + 1]);
+                        }
+                    }
+                }
             }
         }
         double ns = 0.0;
 #pragma unroll
         for (int r = 0; r < RT; ++r) ns = fma(s[r], s[r], ns);
         const bool active = (nz > 0.0) && (ns > prm.tau2 * nz);
-        if (bad) atomicOr(&s_nonfinite, bad);
         my_active += active ? 1u : 0u;
-        if (__syncthreads_or(active ? 1 : 0)) {
+        if (__any_sync(0xffffffffu, active)) {           // G += sum over the warp's codewords of s s^T / ||z||^2
             const double w = active ? rsqrt(nz) : 0.0;
-            double* mine = sS + threadIdx.x * (RT + 1);
+            double2* row = reinterpret_cast<double2*>(myS + lane * LD);
 #pragma unroll
-            for (int r = 0; r < RT; ++r) mine[r] = s[r] * w;
-            __syncthreads();
+            for (int r = 0; r < RT / 2; ++r) row[r] = make_double2(s[2 * r] * w, s[2 * r + 1] * w);
+            __syncwarp();
 #pragma unroll
-            for (int e = 0; e < kOwn; ++e) {
-                if (own_i[e] < 0) continue;
-                double acc = 0.0;
-                for (int c = 0; c < kThreads; ++c)
-                    acc = fma(sS[c * (RT + 1) + own_i[e]], sS[c * (RT + 1) + own_j[e]], acc);
-                g_own[e] += acc;
+            for (int j = 0; j < 8; ++j) {                // codewords 4j .. 4j+3 of the warp
+                const double* src = myS + (4 * j + (lane & 3)) * LD + (lane >> 2);
+                double f[NT];
+#pragma unroll
+                for (int a = 0; a < NT; ++a) f[a] = src[8 * a];
+#pragma unroll
+                for (int a = 0; a < NT; ++a)
+#pragma unroll
+                    for (int b = 0; b < NT; ++b) dmma_m8n8k4(acc[a][b][0], acc[a][b][1], f[a], f[b]);
             }
-            __syncthreads();
+            __syncwarp();
         }
     }
-    // CTA totals -> global
-    if (my_active) atomicAdd(&s_active, my_active);
+    // warp fragments -> CTA total (shared atomics) -> global (one atomic per upper-triangle entry)
 #pragma unroll
-    for (int e = 0; e < kOwn; ++e) {
-        if (own_i[e] < 0 || own_i[e] >= prm.R || own_j[e] >= prm.R || g_own[e] == 0.0) continue;
-        atomicAdd(&prm.gram[own_i[e] * prm.R + own_j[e]], g_own[e]);
+    for (int a = 0; a < NT; ++a)
+#pragma unroll
+        for (int b = 0; b < NT; ++b) {
+            const int r = 8 * a + (lane >> 2), c = 8 * b + 2 * (lane & 3);
+            if (acc[a][b][0] != 0.0) atomicAdd(&sG[r * RT + c], acc[a][b][0]);
+            if (acc[a][b][1] != 0.0) atomicAdd(&sG[r * RT + c + 1], acc[a][b][1]);
+        }
+    unsigned int act = my_active;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        act += __shfl_xor_sync(0xffffffffu, act, o);
+        bad_all |= __shfl_xor_sync(0xffffffffu, bad_all, o);
+    }
+    if (lane == 0) {
+        if (act) atomicAdd(&prm.counts[0], (unsigned long long)act);
+        if (bad_all) atomicOr(&prm.counts[1], bad_all);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        if (s_active) atomicAdd(&prm.counts[0], (unsigned long long)s_active);
-        if (s_nonfinite) atomicOr(&prm.counts[1], s_nonfinite);
+    for (int i = threadIdx.x; i < prm.R * prm.R; i += kThreads) {
+        const int r = i / prm.R, c = i % prm.R;
+        if (r <= c && sG[r * RT + c] != 0.0) atomicAdd(&prm.gram[r * prm.R + c], sG[r * RT + c]);
     }
 }
 
@@ -189,7 +227,7 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
-            if (off <= 1e-34 * tr * tr) break;
+            if (off <= 1e-27 * tr * tr) break;          // off-diagonal mass at the FP64 rounding floor
             for (int p = 0; p < R - 1; ++p) {
                 for (int q = p + 1; q < R; ++q) {
                     const double gpq = G[p][q];
@@ -327,7 +365,7 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
 
 template <typename T, int RT>
 gpd_status launch_syndrome(const SyndromeParams& prm, cudaStream_t st) {
-    const size_t smem = sizeof(double) * ((size_t)RT * prm.P + (size_t)kThreads * (RT + 1));
+    const size_t smem = sizeof(double) * ((size_t)RT * prm.P + (size_t)kThreads * (RT + 4) + (size_t)RT * RT);
     if (smem > 48 * 1024) {
         if (cudaFuncSetAttribute(syndrome_gram_kernel<T, RT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem) != cudaSuccess)
