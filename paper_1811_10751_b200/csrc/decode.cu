@@ -219,7 +219,7 @@ template <typename T, int NW, bool VECTOR>
 void launch_stream(const StreamParams& prm, cudaStream_t st) {
     constexpr int N = VECTOR ? Vec<T>::N : 1;
     const int64_t groups = prm.br * prm.bc / N;
-    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((groups + 255) / 256, 148 * 8));
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((groups + 255) / 256, 148 * 4));
     decode_stream_kernel<T, NW, VECTOR><<<grid, 256, sizeof(double) * prm.n_wanted * prm.P, st>>>(prm);
 }
 

@@ -39,7 +39,7 @@ __device__ __forceinline__ void dmma_m8n8k4(double& d0, double& d1, double a, do
                  : "d"(a), "d"(b));
 }
 
-// One thread per output position (codeword): P coalesced loads (issued four at a time), the
+// One thread per output position (codeword): P coalesced loads (issued eight at a time), the
 // syndrome in RT registers, the zero test.  The Gram matrix of the failing codewords is formed
 // warp by warp on the FP64 tensor cores: the 32 scaled syndromes of a warp are staged in shared
 // memory and fed to mma.m8n8k4 as both operands (G += S S^T, four codewords per instruction), so
@@ -79,13 +79,14 @@ __global__ void __launch_bounds__(kThreads) syndrome_gram_kernel(SyndromeParams 
         double nz = 0.0;
         if (l < prm.L) {
             const T* zp = Z + l;
-            for (int p0 = 0; p0 < prm.P; p0 += 4) {
-                double z[4];
+            constexpr int U = 8;                         // loads issued together: bytes in flight
+            for (int p0 = 0; p0 < prm.P; p0 += U) {
+                double z[U];
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
+                for (int u = 0; u < U; ++u)
                     z[u] = (p0 + u < prm.P) ? (double)__ldcs(zp + (int64_t)(p0 + u) * prm.L) : 0.0;
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < U; ++u) {
                     const int pnode = p0 + u;
                     if (pnode < prm.P) {
                         double zz = z[u];
