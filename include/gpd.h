@@ -89,7 +89,9 @@ typedef enum {
 typedef enum { GPD_ACT_IDENTITY = 0, GPD_ACT_RELU = 1, GPD_ACT_SIGMOID = 2 } gpd_activation_kind;
 
 typedef enum {
-    GPD_PHASE_FWD = 1, GPD_PHASE_BWD = 2, GPD_PHASE_UPD = 4
+    GPD_PHASE_FWD = 1, GPD_PHASE_BWD = 2, GPD_PHASE_UPD = 4,
+    GPD_PHASE_REGEN = 8,          /* with FWD: regenerate the stored shares of the nodes the forward product flagged */
+    GPD_PHASE_INJECT_SHARES = 16  /* with UPD: soft errors of the update stage, written into the updated shares */
 } gpd_phase;
 
 typedef struct { int64_t N1, N0, B; } gpd_shape;
@@ -258,6 +260,17 @@ gpd_status gpd_decode(gpd_plan_t plan, gpd_product which, const void* outputs_de
                       float* out_dev, float* act_out_dev, gpd_activation_kind activation,
                       void* workspace_dev, void* stream);
 
+/*
+ * gpd_regenerate_shares — regeneration of erroneous nodes (Section VI, "Regeneration"): the share
+ * W~_p is the evaluation at b_p of a polynomial of degree mn-1 whose coefficients are the blocks
+ * W_ij, so the share of every node flagged in result_dev is recomputed from the shares of the
+ * clean nodes (interpolation over all of them, least squares, then evaluation at b_p), in place.
+ * Needs at least mn clean nodes; does nothing when result_dev reports no flagged node or a
+ * decoding failure.  workspace_dev: GPD_Q_WORKSPACE_BYTES bytes.
+ */
+gpd_status gpd_regenerate_shares(gpd_plan_t plan, void* W_shares_dev, const gpd_locate_result* result_dev,
+                                 void* workspace_dev, void* stream);
+
 /* Element-wise steps C1 / C2 and the last-layer transitions (Section II-B; Section IX). */
 gpd_status gpd_activation(gpd_activation_kind kind, const float* S_dev, float* X_next_dev,
                           int64_t count, void* stream);
@@ -286,11 +299,13 @@ gpd_status gpd_sae_hidden_delta(const float* C2T_dev, const float* Y1_dev, float
  * coded_layer_step — one layer of the coded training step (Sections VI and VIII), composed from
  * the calls above on one stream with no host synchronisation:
  *   GPD_PHASE_FWD: encode X -> P products -> inject -> locate -> decode S (-> activation)
+ *                  (+ GPD_PHASE_REGEN: then regenerate the shares of the nodes just flagged, which is
+ *                  how errors left in the shares by an earlier update are repaired, Section VI)
  *   GPD_PHASE_BWD: encode Delta^T -> P products -> inject -> locate -> decode C^T
  *   GPD_PHASE_UPD: encode Delta, X ascending -> W~_p += eta Delta^_p X^_p^T;
  *                  skipped on the device if this call's backward product declared a decoding failure.
- *                  (Errors of the update stage live in the shares; inject them with
- *                  gpd_inject(GPD_AUDIT) and find them with the audit product or the next forward.)
+ *                  (+ GPD_PHASE_INJECT_SHARES: Gaussian node errors written into the updated shares,
+ *                  seed inject_seed + 2; they surface at the next forward product of the layer.)
  * X_dev: N0 x B.  Delta_dev: N1 x B and DeltaT_dev: B x N1 (needed for BWD / UPD).
  * S_out_dev, Xnext_out_dev: N1 x B (FWD; Xnext optional).  CT_out_dev: B x N0 (BWD).
  * inject_prob <= 0 disables injection; product k of the call uses seed inject_seed + k

@@ -27,7 +27,7 @@ from . import inject as inj
 from .code import GPCode, FWD, BWD, AUDIT
 from .locate import LocateResult, locate_subspace, tolerances_for, DECODE_FAILURE
 from .product import (decode, encode_DeltaT, encode_update_operands, encode_W, encode_X,
-                      update_shares, worker_products)
+                      regenerate_shares, update_shares, worker_products)
 
 
 # ------------------------------------------------------------------------------------------
@@ -155,6 +155,8 @@ class CodedLayer:
     inject_mode: str = "none"            # "none" | "gauss" | "additive"
     inject_prob: float = 0.0
     inject_scale: float = 1.0
+    regenerate: bool = False             # after a forward product, regenerate the shares of flagged nodes
+    inject_shares: bool = False          # the update stage leaves Gaussian node errors in the shares
     log: List[LocateResult] = field(default_factory=list)
 
     @classmethod
@@ -175,16 +177,21 @@ class CodedLayer:
     def forward(self, X, seed: Optional[int] = None, scale: float = 1.0):
         """S = W X through encode -> P products -> locate -> decode."""
         Z = worker_products(self.W_shares, encode_X(X, self.code))
-        return self._finish(Z, FWD, seed, scale)
+        S, res = self._finish(Z, FWD, seed, scale)
+        if self.regenerate and S is not None and res.flagged.any():
+            self.W_shares = regenerate_shares(self.W_shares, self.code, res.flagged)
+        return S, res
 
     def backward(self, DeltaT, seed: Optional[int] = None, scale: float = 1.0):
         """C^T = Delta^T W through the same four stages."""
         Z = worker_products(encode_DeltaT(DeltaT, self.code), self.W_shares)
         return self._finish(Z, BWD, seed, scale)
 
-    def update(self, Delta, X, eta: float, lam: float = 0.0):
+    def update(self, Delta, X, eta: float, lam: float = 0.0, seed: Optional[int] = None, scale: float = 1.0):
         Dh, Xh = encode_update_operands(Delta, X, self.code)
         self.W_shares = update_shares(self.W_shares, Dh, Xh, eta, lam)
+        if self.inject_shares and seed is not None and self.inject_prob > 0:
+            inj.inject_gauss(self.W_shares, seed, scale, prob=self.inject_prob)
 
     def audit(self, seed: Optional[int] = None, scale: float = 1.0):
         """Decode W itself from the shares (each share is a degree mn-1 polynomial evaluation)."""
@@ -231,7 +238,7 @@ def mlp_step_coded(layers: Sequence[CodedLayer], X1, labels, lr: float,
         if l > 0:
             Delta = (CT * relu_g(Xs[l]).T).T
     for l in range(L):
-        layers[l].update(Deltas[l], Xs[l], lr)
+        layers[l].update(Deltas[l], Xs[l], lr, seed=sd(l, 2))
     return {"X": Xs, "S": Ss, "Delta": Deltas, "CT": CTs, "loss": softmax_ce_loss(Ss[-1], labels)}
 
 
@@ -266,6 +273,6 @@ def autoencoder_step_coded(enc: CodedLayer, dec: CodedLayer, X, lr: float, rho: 
     rho_hat = np.clip(Y1.mean(axis=1), RHO_CLAMP, 1.0 - RHO_CLAMP)
     kl = rho * np.log(rho / rho_hat) + (1.0 - rho) * np.log((1.0 - rho) / (1.0 - rho_hat))
     loss = float(((S2 - X) ** 2).sum() / B + beta * kl.sum())
-    enc.update(Delta1, X, lr)
-    dec.update(Delta2, Y1, lr)
+    enc.update(Delta1, X, lr, seed=sd(0, 2))
+    dec.update(Delta2, Y1, lr, seed=sd(1, 2))
     return {"S1": S1, "S2": S2, "Delta1": Delta1, "Delta2": Delta2, "C1T": C1T, "loss": loss}

@@ -133,6 +133,29 @@ def decode(outputs: np.ndarray, code: GPCode, which: int, use: Optional[Sequence
     return out
 
 
+def regenerate_shares(W_shares: np.ndarray, code: GPCode, flagged: Sequence[bool]) -> np.ndarray:
+    """Regeneration (Section VI): every share is the evaluation at b_p of the polynomial
+    sum_ij W_ij v^(n i + j) of degree mn - 1, so the shares of the flagged nodes are recomputed
+    by interpolating that polynomial from the clean nodes (all of them, least squares) and
+    evaluating it at the flagged nodes' points.  Only the polynomial's values are needed, not its
+    monomial coefficients, so the fit is done in the Chebyshev basis (numpy.polynomial.chebyshev),
+    which keeps the system well conditioned on [-1,1].  Returns a new array."""
+    flagged = np.asarray(flagged, dtype=bool)
+    use = ~flagged
+    Q = code.Q_w
+    if use.sum() < Q:
+        raise ValueError("fewer clean nodes than mn")
+    out = _f64(W_shares).copy()
+    if not flagged.any():
+        return out
+    shape = out.shape[1:]
+    V = np.polynomial.chebyshev.chebvander(code.points, Q - 1)                 # T_c(b_p)
+    Qm, R = np.linalg.qr(V[use])
+    coeffs = np.linalg.solve(R, Qm.T @ out[use].reshape(int(use.sum()), -1))   # Q x L Chebyshev coefficients
+    out[flagged] = (V[flagged] @ coeffs).reshape((int(flagged.sum()),) + shape)
+    return out
+
+
 def rel_fro(a, b) -> float:
     """Relative Frobenius error ||a - b||_F / ||b||_F."""
     a, b = _f64(a), _f64(b)

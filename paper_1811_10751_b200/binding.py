@@ -31,7 +31,7 @@ GPD_OPERAND_X_FWD, GPD_OPERAND_DELTAT_BWD, GPD_OPERAND_DELTA_UPD, GPD_OPERAND_X_
 GPD_PREC_AUTO, GPD_PREC_FP32, GPD_PREC_FP64 = 0, 1, 2
 GPD_INJECT_BITFLIP, GPD_INJECT_ADDITIVE, GPD_INJECT_GAUSS = 0, 1, 2
 GPD_ACT_IDENTITY, GPD_ACT_RELU, GPD_ACT_SIGMOID = 0, 1, 2
-GPD_PHASE_FWD, GPD_PHASE_BWD, GPD_PHASE_UPD = 1, 2, 4
+GPD_PHASE_FWD, GPD_PHASE_BWD, GPD_PHASE_UPD, GPD_PHASE_REGEN, GPD_PHASE_INJECT_SHARES = 1, 2, 4, 8, 16
 (GPD_Q_THRESHOLD_FWD, GPD_Q_THRESHOLD_BWD, GPD_Q_THRESHOLD_AUDIT, GPD_Q_ELEMENT_SIZE,
  GPD_Q_W_SHARE_ELEMS, GPD_Q_X_SHARE_ELEMS, GPD_Q_DT_SHARE_ELEMS, GPD_Q_DHAT_ELEMS, GPD_Q_XHAT_ELEMS,
  GPD_Q_OUT_ELEMS_FWD, GPD_Q_OUT_ELEMS_BWD, GPD_Q_WORKSPACE_BYTES, GPD_Q_STEP_WORKSPACE_BYTES,
@@ -43,7 +43,7 @@ GPD_MAX_NODES = 64
 EXPORTED = [
     "gpd_status_string", "gpd_plan", "gpd_plan_destroy", "gpd_plan_query", "gpd_plan_table",
     "gpd_encode_A", "gpd_encode_B", "gpd_worker_gemm", "gpd_device_status", "gpd_update_shares", "gpd_inject",
-    "gpd_locate_errors", "gpd_locate_errors_static", "gpd_decode", "gpd_activation", "gpd_softmax_xent_delta",
+    "gpd_locate_errors", "gpd_locate_errors_static", "gpd_decode", "gpd_regenerate_shares", "gpd_activation", "gpd_softmax_xent_delta",
     "gpd_backprop_hadamard", "gpd_sae_output_delta", "gpd_sae_hidden_delta", "coded_layer_step",
 ]
 
@@ -82,6 +82,7 @@ lib.gpd_inject.argtypes = [_vp, C.c_int, _vp, _u64, C.c_int, _d, _u64, _i32, _d,
 lib.gpd_locate_errors.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp, _vp]
 lib.gpd_locate_errors_static.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp]
 lib.gpd_decode.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp, _vp, C.c_int, _vp, _vp]
+lib.gpd_regenerate_shares.argtypes = [_vp, _vp, _vp, _vp, _vp]
 lib.gpd_activation.argtypes = [C.c_int, _vp, _vp, _i64, _vp]
 lib.gpd_softmax_xent_delta.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _vp]
 lib.gpd_backprop_hadamard.argtypes = [C.c_int, _vp, _vp, _vp, _vp, _i64, _i64, _vp]
@@ -250,6 +251,11 @@ def gpd_decode(plan: Plan, which: int, outputs, out, workspace, result=None, use
                activation: int = GPD_ACT_IDENTITY, stream=None):
     _check(lib.gpd_decode(plan.handle, which, _ptr(outputs), _mask(use_mask, plan.P), _ptr(result), _ptr(out, _F32),
                           _ptr(act_out, _F32), activation, _ptr(workspace), _stream(stream)), "gpd_decode")
+
+
+def gpd_regenerate_shares(plan: Plan, W_shares, result, workspace, stream=None):
+    _check(lib.gpd_regenerate_shares(plan.handle, _ptr(W_shares, plan.dtype), _ptr(result), _ptr(workspace),
+                                     _stream(stream)), "gpd_regenerate_shares")
 
 
 def gpd_activation(kind: int, S, X_next, stream=None):

@@ -24,6 +24,8 @@ struct MatrixParams {
     int have_mask;
     int P, Q, n_wanted;
     int wanted[kMaxWanted];
+    double* regen;                   // optional [n_flagged][P]: re-evaluation of the interpolated
+                                     // polynomial at the flagged nodes' points (share regeneration)
 };
 
 __global__ void __launch_bounds__(32) decode_matrix_kernel(MatrixParams prm) {
@@ -54,8 +56,15 @@ __global__ void __launch_bounds__(32) decode_matrix_kernel(MatrixParams prm) {
     if (rows == 0) return;
     for (int r = lane; r < rows; r += 32) {
         const double b = prm.points[node_of[r]];
-        double acc = 1.0;
-        for (int c = 0; c < Q; ++c) { A[r][c] = acc; acc *= b; }
+        if (prm.regen) {
+            // regeneration only needs the polynomial's values, not its monomial coefficients: the
+            // Chebyshev basis T_c keeps this least-squares system well conditioned on [-1,1]
+            double t0 = 1.0, t1 = b;
+            for (int c = 0; c < Q; ++c) { A[r][c] = t0; const double t2 = 2.0 * b * t1 - t0; t0 = t1; t1 = t2; }
+        } else {
+            double acc = 1.0;
+            for (int c = 0; c < Q; ++c) { A[r][c] = acc; acc *= b; }
+        }
     }
     __syncwarp();
     // Householder triangularisation; lane c owns column c
@@ -92,6 +101,28 @@ __global__ void __launch_bounds__(32) decode_matrix_kernel(MatrixParams prm) {
             for (int r = k; r < rows; ++r) x[r] -= 2.0 * dot * Vh[r][k];
         }
         for (int r = 0; r < rows; ++r) prm.D[wi * P + node_of[r]] = x[r];
+    }
+    if (prm.regen) {
+        // Regeneration (Section VI): node f's share is a polynomial of degree Q-1 evaluated at b_f.
+        // With D[c][q] the functional giving its c-th Chebyshev coefficient from the clean nodes q,
+        // share_f = sum_q (sum_c T_c(b_f) D[c][q]) share_q.  Needs n_wanted == Q, wanted[c] == c.
+        __syncwarp();
+        __threadfence_block();
+        int nf = 0;
+        for (int f = 0; f < P; ++f) {
+            if (!prm.result->flagged[f]) continue;
+            const double b = prm.points[f];
+            for (int q = lane; q < P; q += 32) {
+                double acc = 0.0, t0 = 1.0, t1 = b;
+                for (int c = 0; c < Q; ++c) {
+                    acc = fma(t0, prm.D[c * P + q], acc);
+                    const double t2 = 2.0 * b * t1 - t0; t0 = t1; t1 = t2;
+                }
+                prm.regen[nf * P + q] = acc;
+            }
+            ++nf;
+        }
+        if (lane == 0) prm.gate[1] = nf;
     }
 }
 
@@ -274,6 +305,86 @@ gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* output
     return plan->elem_size == 4 ? dispatch_stream<float>(sp, st) : dispatch_stream<double>(sp, st);
 }
 
+namespace {
+
+struct RegenParams {
+    void* shares;                    // [P][L] in/out
+    const double* Rg;                // [n_flagged][P], zero columns for flagged nodes
+    const int* gate;                 // [0] run?, [1] n_flagged
+    const gpd_locate_result* result;
+    int64_t L;
+    int P;
+};
+
+// share_f[pos] = sum over clean q of Rg[f][q] * share_q[pos]; clean shares are read once, flagged
+// shares are overwritten in place (the two sets are disjoint, so in-place is safe).
+template <typename T>
+__global__ void __launch_bounds__(256) regen_stream_kernel(RegenParams prm) {
+    if (prm.gate[0] == 0 || prm.gate[1] == 0) return;
+    extern __shared__ double sR[];                   // [n_flagged][P]
+    __shared__ int s_flag[kMaxNodes], s_clean[kMaxNodes];
+    __shared__ int s_nf, s_nc;
+    if (threadIdx.x == 0) {
+        int nf = 0, nc = 0;
+        for (int p = 0; p < prm.P; ++p) {
+            if (prm.result->flagged[p]) s_flag[nf++] = p; else s_clean[nc++] = p;
+        }
+        s_nf = nf; s_nc = nc;
+    }
+    __syncthreads();
+    const int nf = s_nf, nc = s_nc;
+    for (int i = threadIdx.x; i < nf * prm.P; i += blockDim.x) sR[i] = prm.Rg[i];
+    __syncthreads();
+    T* S = reinterpret_cast<T*>(prm.shares);
+    for (int64_t pos = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; pos < prm.L;
+         pos += (int64_t)gridDim.x * blockDim.x) {
+        for (int f0 = 0; f0 < nf; f0 += 4) {
+            double acc[4] = {0.0, 0.0, 0.0, 0.0};
+            for (int i = 0; i < nc; ++i) {
+                const int q = s_clean[i];
+                const double z = (double)__ldcs(S + (int64_t)q * prm.L + pos);
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (f0 + u < nf) acc[u] = fma(sR[(f0 + u) * prm.P + q], z, acc[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (f0 + u < nf) S[(int64_t)s_flag[f0 + u] * prm.L + pos] = (T)acc[u];
+        }
+    }
+}
+
+}  // namespace
+
+gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_result* result, void* workspace,
+                             cudaStream_t st) {
+    const ProductInfo& pi = plan->prod[GPD_AUDIT];
+    if (pi.Q == 0) return GPD_ERR_UNSUPPORTED;
+    gpd_status rc = ensure_device(plan);
+    if (rc != GPD_OK) return rc;
+    const WorkspaceLayout wl = workspace_layout();
+    char* ws = reinterpret_cast<char*>(workspace);
+    MatrixParams mp{};
+    mp.points = plan->dev.base + plan->dev.off_points;
+    mp.D = reinterpret_cast<double*>(ws + wl.off_decode);
+    mp.gate = reinterpret_cast<int*>(ws + wl.off_flags);
+    mp.result = result;
+    mp.have_mask = 0;
+    mp.P = plan->P; mp.Q = pi.Q; mp.n_wanted = pi.Q;
+    for (int c = 0; c < pi.Q; ++c) mp.wanted[c] = c;
+    mp.regen = reinterpret_cast<double*>(ws + wl.off_regen);
+    decode_matrix_kernel<<<1, 32, 0, st>>>(mp);
+    if ((rc = launch_ok()) != GPD_OK) return rc;
+    RegenParams rp{};
+    rp.shares = shares; rp.Rg = mp.regen; rp.gate = mp.gate; rp.result = result;
+    rp.L = pi.br * pi.bc; rp.P = plan->P;
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((rp.L + 255) / 256, 148 * 8));
+    const size_t smem = sizeof(double) * (size_t)plan->P * plan->P;
+    if (plan->elem_size == 4) regen_stream_kernel<float><<<grid, 256, smem, st>>>(rp);
+    else regen_stream_kernel<double><<<grid, 256, smem, st>>>(rp);
+    return launch_ok();
+}
+
 }  // namespace gpd
 
 using namespace gpd;
@@ -295,4 +406,11 @@ extern "C" gpd_status gpd_decode(gpd_plan_t plan, gpd_product which, const void*
     }
     return decode_launch(plan, which, outputs_dev, use_mask_host != nullptr, mask, result_dev, out_dev,
                          act_out_dev, (int)activation, workspace_dev, as_stream(stream));
+}
+
+extern "C" gpd_status gpd_regenerate_shares(gpd_plan_t plan, void* W_shares_dev, const gpd_locate_result* result_dev,
+                                            void* workspace_dev, void* stream) {
+    if (!plan || !W_shares_dev || !result_dev) return GPD_ERR_ARG;
+    if (!workspace_dev) return GPD_ERR_WORKSPACE;
+    return regenerate_launch(plan, W_shares_dev, result_dev, workspace_dev, as_stream(stream));
 }

@@ -80,7 +80,8 @@ struct WorkspaceLayout {
     int64_t off_gram;      // double[kMaxR * kMaxR]   syndrome Gram matrix
     int64_t off_counts;    // unsigned long long[4]   n_active, nonfinite mask, spare
     int64_t off_decode;    // double[kMaxWanted * kMaxNodes] decode matrix D
-    int64_t off_flags;     // int[4] decode gate
+    int64_t off_flags;     // int[8] decode gate, number of regenerated nodes
+    int64_t off_regen;     // double[kMaxNodes * kMaxNodes] regeneration matrix
     int64_t total;
 };
 WorkspaceLayout workspace_layout();
@@ -98,6 +99,8 @@ gpd_status locate_launch(gpd_plan_s* plan, gpd_product which, const void* output
                          gpd_locate_result* result, void* workspace, cudaStream_t st);
 gpd_status locate_static_launch(gpd_plan_s* plan, gpd_product which, const void* outputs,
                                 uint64_t erased_mask, gpd_locate_result* result, cudaStream_t st);
+gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_result* result, void* workspace,
+                             cudaStream_t st);
 gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, bool have_mask,
                          uint64_t use_mask, const gpd_locate_result* result, float* out, float* act_out,
                          int activation, void* workspace, cudaStream_t st);

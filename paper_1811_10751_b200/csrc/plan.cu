@@ -80,6 +80,7 @@ WorkspaceLayout workspace_layout() {
     w.off_counts = off; off = align_up(off + (int64_t)sizeof(unsigned long long) * 8, 256);
     w.off_decode = off; off = align_up(off + (int64_t)sizeof(double) * kMaxWanted * kMaxNodes, 256);
     w.off_flags = off;  off = align_up(off + (int64_t)sizeof(int) * 8, 256);
+    w.off_regen = off;  off = align_up(off + (int64_t)sizeof(double) * kMaxNodes * kMaxNodes, 256);
     w.total = off;
     return w;
 }

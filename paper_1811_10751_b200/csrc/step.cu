@@ -21,7 +21,9 @@ extern "C" gpd_status coded_layer_step(gpd_plan_t plan, int32_t phases, void* W_
                                        gpd_locate_result* results_dev, void* workspace_dev, void* stream) {
     if (!plan || !W_shares_dev || !results_dev) return GPD_ERR_ARG;
     if (!workspace_dev) return GPD_ERR_WORKSPACE;
-    if ((phases & ~(GPD_PHASE_FWD | GPD_PHASE_BWD | GPD_PHASE_UPD)) || phases == 0) return GPD_ERR_ARG;
+    if ((phases & ~(GPD_PHASE_FWD | GPD_PHASE_BWD | GPD_PHASE_UPD | GPD_PHASE_REGEN | GPD_PHASE_INJECT_SHARES)) ||
+        !(phases & (GPD_PHASE_FWD | GPD_PHASE_BWD | GPD_PHASE_UPD)))
+        return GPD_ERR_ARG;
     cudaStream_t st = as_stream(stream);
     const gpd_shape& s = plan->shape;
     const gpd_split& c = plan->split;
@@ -44,6 +46,9 @@ extern "C" gpd_status coded_layer_step(gpd_plan_t plan, int32_t phases, void* W_
         if ((rc = locate_launch(plan, GPD_FWD, Z, 0, &results_dev[0], small, st)) != GPD_OK) return rc;
         if ((rc = decode_launch(plan, GPD_FWD, Z, false, 0, &results_dev[0], S_out_dev, Xnext_out_dev,
                                 (int)activation, small, st)) != GPD_OK)
+            return rc;
+        if ((phases & GPD_PHASE_REGEN) &&
+            (rc = regenerate_launch(plan, W_shares_dev, &results_dev[0], small, st)) != GPD_OK)
             return rc;
     }
     if (phases & GPD_PHASE_BWD) {
@@ -69,6 +74,10 @@ extern "C" gpd_status coded_layer_step(gpd_plan_t plan, int32_t phases, void* W_
         if ((rc = encode_launch(plan, GPD_OPERAND_X_UPD, X_dev, Xhat, st)) != GPD_OK) return rc;
         const gpd_locate_result* gate = (phases & GPD_PHASE_BWD) ? &results_dev[1] : nullptr;
         if ((rc = update_launch(plan, W_shares_dev, Dhat, Xhat, eta, lambda, gate, st)) != GPD_OK) return rc;
+        if ((phases & GPD_PHASE_INJECT_SHARES) && inject_prob > 0.0 &&
+            (rc = inject_launch(plan, GPD_AUDIT, W_shares_dev, inject_seed + 2, GPD_INJECT_GAUSS, inject_prob, 0, 0,
+                                inject_scale, nullptr, st)) != GPD_OK)
+            return rc;
     }
     return GPD_OK;
 }

@@ -186,3 +186,95 @@ def test_sparse_autoencoder_steps_match_oracle():
     assert len(enc_o.log) == 2 * steps and len(dec_o.log) == 2 * steps
     assert op.rel_fro(enc.audit(), U1) < REL_TOL and op.rel_fro(dec.audit(), U2) < REL_TOL
     assert op.rel_fro(enc.audit().astype(np.float64) - W1, U1 - W1) < 5e-3
+
+
+@pytest.mark.parametrize("N1,N0,B,m,n,P,nodes", [
+    (256, 256, 16, 2, 2, 10, (3, 8)),                      # FP32 storage, mn = 4
+    (256, 128, 64, 4, 4, 36, (0, 5, 17, 30)),              # FP64 storage, mn = 16
+])
+def test_regenerate_shares_matches_oracle(N1, N0, B, m, n, P, nodes):
+    W = (np.random.default_rng(31).standard_normal((N1, N0)) / np.sqrt(N0)).astype(np.float32)
+    layer = GpuLayer(W, B, m, n, P)
+    code = GPCode(N1, N0, B, m, n, 1, 1, P)
+    clean = layer.W_shares.clone()
+    mask = sum(1 << p for p in nodes)
+    g.gpd_inject(layer.plan, g.GPD_AUDIT, layer.W_shares, 5, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=mask, scale=0.3)
+    small, r = layer.plan.workspace(), g.new_results(1)
+    g.gpd_locate_errors(layer.plan, g.GPD_AUDIT, layer.W_shares, r, small)
+    res = g.read_results(r)[0]
+    assert res.outcome == g.GPD_CORRECTED and list(np.flatnonzero(_flags(res, P))) == list(nodes)
+    g.gpd_regenerate_shares(layer.plan, layer.W_shares, r, small)
+    got = host(layer.W_shares).reshape(P, N1 // m, N0 // n).astype(np.float64)
+    # oracle: its own encoding, the same nodes overwritten by anything, regenerated
+    sh = op.encode_W(W, code)
+    flagged = np.zeros(P, dtype=bool)
+    flagged[list(nodes)] = True
+    bad = sh.copy()
+    bad[flagged] = 123.0
+    want = op.regenerate_shares(bad, code, flagged)
+    # a regenerated share must be as good as an encoded one (a few units of the storage rounding):
+    # later products amplify any excess by up to 1e8 at thresholds near 30
+    eps = 6e-8 if layer.np_dtype == np.float32 else 1.2e-16
+    assert np.abs(got - want).max() <= 32 * eps * np.abs(want).max()
+    assert np.abs(got - sh).max() <= 32 * eps * np.abs(sh).max()
+    assert torch.equal(layer.W_shares.reshape(P, -1)[~torch.from_numpy(flagged).cuda()],
+                       clean.reshape(P, -1)[~torch.from_numpy(flagged).cuda()])      # clean shares untouched
+    # a clean audit regenerates nothing
+    g.gpd_locate_errors(layer.plan, g.GPD_AUDIT, layer.W_shares, r, small)
+    assert g.read_results(r)[0].outcome == g.GPD_NO_ERROR
+    before = layer.W_shares.clone()
+    g.gpd_regenerate_shares(layer.plan, layer.W_shares, r, small)
+    assert torch.equal(layer.W_shares, before)
+
+
+def test_training_with_share_errors_and_regeneration():
+    """Several coded MLP iterations with soft errors in the products and in the updated shares;
+    forward products locate the damaged nodes and their shares are regenerated (Section VI)."""
+    cfg = wl.scaled_down(wl.CONFIG_4_MLP, 16)
+    Ws, X1, labels = wl.mlp_inputs(cfg)
+    L, prob, steps = len(Ws), 0.05, 4
+    o_layers = [odnn.CodedLayer.from_weights(W, GPCode(W.shape[0], W.shape[1], cfg.B, cfg.m, cfg.n, 1, 1, cfg.P),
+                                             out_dtype=np.float32, inject_mode="gauss", inject_prob=prob,
+                                             regenerate=True, inject_shares=True) for W in Ws]
+    layers = [GpuLayer(W, cfg.B, cfg.m, cfg.n, cfg.P) for W in Ws]
+    U = [w.astype(np.float64) for w in Ws]
+    labels_d = dev(labels.astype(np.int32))
+    n_corrected = 0
+    for it in range(steps):
+        seed = 7000 + 100 * it
+        o_out = odnn.mlp_step_coded(o_layers, X1, labels, cfg.lr, step_seed=seed)
+        assert o_out is not None
+        U, ref = odnn.mlp_step_uncoded(U, X1, labels, cfg.lr)
+        Xs = [dev(X1)]
+        for l in range(L):
+            act = g.GPD_ACT_RELU if l < L - 1 else g.GPD_ACT_IDENTITY
+            layers[l].step(g.GPD_PHASE_FWD | g.GPD_PHASE_REGEN, X=Xs[l], act=act, seed=odnn.product_seed(seed, l, 0),
+                           prob=prob)
+            Xs.append(layers[l].Xnext.clone())
+        C = Ws[-1].shape[0]
+        Delta = torch.empty((C, cfg.B), dtype=torch.float32, device="cuda")
+        DeltaT = torch.empty((cfg.B, C), dtype=torch.float32, device="cuda")
+        g.gpd_softmax_xent_delta(layers[-1].S, labels_d, Delta, DeltaT, None)
+        for l in range(L - 1, -1, -1):
+            layers[l].step(g.GPD_PHASE_BWD | g.GPD_PHASE_UPD | g.GPD_PHASE_INJECT_SHARES, X=Xs[l], Delta=Delta,
+                           DeltaT=DeltaT, eta=cfg.lr, seed=odnn.product_seed(seed, l, 0), prob=prob)
+            if l > 0:
+                N = Ws[l].shape[1]
+                Delta = torch.empty((N, cfg.B), dtype=torch.float32, device="cuda")
+                DeltaT = torch.empty((cfg.B, N), dtype=torch.float32, device="cuda")
+                g.gpd_backprop_hadamard(g.GPD_ACT_RELU, layers[l].CT, Xs[l], Delta, DeltaT)
+        torch.cuda.synchronize()
+        for l in range(L):
+            rf, rb, _ = layers[l].results()
+            of, ob = o_layers[l].log[2 * it], o_layers[l].log[2 * it + 1]
+            assert rf.outcome == of.outcome and np.array_equal(_flags(rf, cfg.P), of.flagged), (it, l)
+            assert rb.outcome == ob.outcome and np.array_equal(_flags(rb, cfg.P), ob.flagged), (it, l)
+            n_corrected += (rf.outcome == g.GPD_CORRECTED) + (rb.outcome == g.GPD_CORRECTED)
+            assert op.rel_fro(host(layers[l].S), ref["S"][l]) < REL_TOL
+            assert op.rel_fro(host(layers[l].CT), ref["CT"][l]) < REL_TOL
+    assert n_corrected >= 3
+    # one more forward pass repairs what the last update left in the shares; then the audit is clean
+    for l in range(L):
+        layers[l].step(g.GPD_PHASE_FWD | g.GPD_PHASE_REGEN, X=dev(ref["X"][l].astype(np.float32)))
+        torch.cuda.synchronize()
+        assert op.rel_fro(layers[l].audit(), U[l]) < REL_TOL

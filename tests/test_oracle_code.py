@@ -280,3 +280,30 @@ def test_parity_check_is_mds_on_small_codes():
     H = parity_check(chebyshev_points(P), Q)
     for cols in itertools.combinations(range(P), P - Q):
         assert np.linalg.svd(H[:, cols], compute_uv=False)[-1] > 1e-6
+
+
+# ----------------------------------------------------------------------------------------------
+# regeneration of erroneous nodes' shares
+# ----------------------------------------------------------------------------------------------
+def test_regeneration_restores_any_set_of_up_to_P_minus_mn_shares():
+    """A share is the evaluation of a degree mn-1 polynomial: whatever was stored at up to P - mn
+    nodes, interpolating from the others and re-evaluating gives back the encoding of W."""
+    code = GPCode(8, 6, 2, 2, 3, 1, 1, 9)                      # mn = 6: any 3 shares can be lost
+    W = _rand((8, 6), 21)
+    clean = op.encode_W(W, code)
+    rng = np.random.default_rng(22)
+    for size in range(0, 4):
+        for nodes in itertools.combinations(range(9), size):
+            bad = clean.copy()
+            flagged = np.zeros(9, dtype=bool)
+            flagged[list(nodes)] = True
+            bad[flagged] = rng.standard_normal(bad[flagged].shape) * 7
+            assert np.allclose(op.regenerate_shares(bad, code, flagged), clean, atol=1e-10)
+    # the regenerated value is the polynomial's value: with one block per monomial it is W~(b_p) itself
+    flagged = np.zeros(9, dtype=bool)
+    flagged[4] = True
+    again = op.regenerate_shares(clean, code, flagged)
+    coeffs = [W[4 * i + 1, 2 * j + 1] for i in range(2) for j in range(3)]
+    assert np.isclose(again[4, 1, 1], np.polyval(coeffs[::-1], code.points[4]), rtol=1e-12)
+    with pytest.raises(ValueError):
+        op.regenerate_shares(clean, code, np.array([True] * 4 + [False] * 5))

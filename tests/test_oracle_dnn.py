@@ -106,3 +106,29 @@ def test_coded_autoencoder_steps_track_uncoded_training():
         losses.append(loss)
     assert losses[-1] < losses[0]
     assert rel_fro(enc.audit()[0], U1) < 1e-9 and rel_fro(dec.audit()[0], U2) < 1e-9
+
+
+def test_training_with_share_errors_and_regeneration_tracks_uncoded_training():
+    """Errors left in the shares by the update stage surface at the next forward product, are
+    located there and the shares regenerated (Section VI); the decoded weights keep following
+    the uncoded SGD trajectory over several iterations."""
+    widths, B = (16, 12, 8, 4), 6
+    Ws, X, labels = _mlp(seed=6, widths=widths, B=B)
+    layers = [dnn.CodedLayer.from_weights(W, GPCode(W.shape[0], W.shape[1], B, 2, 2, 1, 1, 10), inject_mode="gauss",
+                                          inject_prob=0.08, regenerate=True, inject_shares=True) for W in Ws]
+    U = [w.copy() for w in Ws]
+    hits = 0
+    for step in range(6):
+        out = dnn.mlp_step_coded(layers, X, labels, 0.05, step_seed=5000 + 100 * step)
+        assert out is not None
+        U, info = dnn.mlp_step_uncoded(U, X, labels, 0.05)
+        for l in range(len(Ws)):
+            assert rel_fro(out["S"][l], info["S"][l]) < 1e-8
+    for lay in layers:
+        hits += sum(r.outcome == CORRECTED for r in lay.log)
+    assert hits >= 3
+    # one last forward pass repairs whatever the last update left behind, then the shares are clean
+    for l, lay in enumerate(layers):
+        lay.forward(info["X"][l] if l < len(info["X"]) else info["X"][-1], seed=None)
+        W_dec, res = lay.audit()
+        assert res.outcome == NO_ERROR and rel_fro(W_dec, U[l]) < 1e-8
