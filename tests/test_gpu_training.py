@@ -278,3 +278,51 @@ def test_training_with_share_errors_and_regeneration():
         layers[l].step(g.GPD_PHASE_FWD | g.GPD_PHASE_REGEN, X=dev(ref["X"][l].astype(np.float32)))
         torch.cuda.synchronize()
         assert op.rel_fro(layers[l].audit(), U[l]) < REL_TOL
+
+
+def test_config5_full_size_two_steps():
+    """The sparse-autoencoder workload at full size (1024 <-> 8192, batch 1024, split 4 x 4, P = 36,
+    thresholds 19 / 28 / 16, FP64 path), two coded SGD steps with Gaussian node errors."""
+    cfg = wl.CONFIG_5_AUTOENCODER
+    W1, W2, X = wl.autoencoder_inputs(cfg)
+    enc_o = odnn.CodedLayer.from_weights(W1, GPCode(cfg.n_hidden, cfg.n_visible, cfg.B, cfg.m, cfg.n, 1, 1, cfg.P),
+                                         inject_mode="gauss", inject_prob=cfg.inject_prob)
+    dec_o = odnn.CodedLayer.from_weights(W2, GPCode(cfg.n_visible, cfg.n_hidden, cfg.B, cfg.m, cfg.n, 1, 1, cfg.P),
+                                         inject_mode="gauss", inject_prob=cfg.inject_prob)
+    enc, dec = GpuLayer(W1, cfg.B, cfg.m, cfg.n, cfg.P), GpuLayer(W2, cfg.B, cfg.m, cfg.n, cfg.P)
+    assert enc.np_dtype == np.float64
+    Xd = dev(X)
+    U1, U2 = W1.astype(np.float64), W2.astype(np.float64)
+    f32 = dict(dtype=torch.float32, device="cuda")
+    D2, D2T = torch.empty((cfg.n_visible, cfg.B), **f32), torch.empty((cfg.B, cfg.n_visible), **f32)
+    D1, D1T = torch.empty((cfg.n_hidden, cfg.B), **f32), torch.empty((cfg.B, cfg.n_hidden), **f32)
+    mse, kl = torch.zeros(1, **f32), torch.zeros(1, **f32)
+    n_corrected = 0
+    for s in range(2):
+        seed = 8800 + 100 * s
+        o = odnn.autoencoder_step_coded(enc_o, dec_o, X, cfg.lr, cfg.rho, cfg.beta, step_seed=seed)
+        assert o is not None
+        U1, U2, loss_ref = odnn.autoencoder_step_uncoded(U1, U2, X, cfg.lr, cfg.rho, cfg.beta)
+        enc.step(g.GPD_PHASE_FWD, X=Xd, act=g.GPD_ACT_SIGMOID, seed=odnn.product_seed(seed, 0, 0), prob=cfg.inject_prob)
+        dec.step(g.GPD_PHASE_FWD, X=enc.Xnext, seed=odnn.product_seed(seed, 1, 0), prob=cfg.inject_prob)
+        g.gpd_sae_output_delta(dec.S, Xd, D2, D2T, mse)
+        dec.step(g.GPD_PHASE_BWD, DeltaT=D2T, seed=odnn.product_seed(seed, 1, 0), prob=cfg.inject_prob)
+        g.gpd_sae_hidden_delta(dec.CT, enc.Xnext, cfg.rho, cfg.beta, D1, D1T, kl)
+        enc.step(g.GPD_PHASE_BWD | g.GPD_PHASE_UPD, X=Xd, Delta=D1, DeltaT=D1T, eta=cfg.lr,
+                 seed=odnn.product_seed(seed, 0, 0), prob=cfg.inject_prob)
+        dec.step(g.GPD_PHASE_UPD, X=enc.Xnext, Delta=D2, eta=cfg.lr)
+        torch.cuda.synchronize()
+        loss = float(mse.item() + kl.item())
+        assert abs(loss - loss_ref) < 1e-4 * abs(loss_ref)
+        for lay, olay in ((enc, enc_o), (dec, dec_o)):
+            rf, rb, _ = lay.results()
+            of, ob = olay.log[2 * s], olay.log[2 * s + 1]
+            assert rf.outcome == of.outcome and np.array_equal(_flags(rf, cfg.P), of.flagged)
+            assert rb.outcome == ob.outcome and np.array_equal(_flags(rb, cfg.P), ob.flagged)
+            n_corrected += (rf.outcome == g.GPD_CORRECTED) + (rb.outcome == g.GPD_CORRECTED)
+        assert op.rel_fro(host(enc.S), o["S1"]) < REL_TOL and op.rel_fro(host(dec.S), o["S2"]) < REL_TOL
+        assert op.rel_fro(host(D1), o["Delta1"]) < REL_TOL and op.rel_fro(host(D2), o["Delta2"]) < REL_TOL
+        assert op.rel_fro(host(enc.CT), o["C1T"]) < REL_TOL
+    assert n_corrected >= 1
+    assert op.rel_fro(enc.audit(), U1) < REL_TOL and op.rel_fro(dec.audit(), U2) < REL_TOL
+    assert g.gpd_device_status() == 0
