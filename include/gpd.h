@@ -86,6 +86,12 @@ typedef enum {
     GPD_INJECT_GAUSS = 2        /* selected nodes: scale * N(0,1) added to every entry (Error Model 2) */
 } gpd_inject_mode;
 
+/* Garbage-alignment substitution (Section VI, "we use one of the substitutions ..."; Tables I, III). */
+typedef enum {
+    GPD_SUBST_U_EQ_VN = 0,      /* u = v^n, w = v^(mn): Q_f = mn d1 + n - 1,      Q_b = mn d2 + mn - n  */
+    GPD_SUBST_V_EQ_UM = 1       /* v = u^m, w = u^(mn): Q_f = mn d1 + mn - m,     Q_b = mn d2 + m - 1   */
+} gpd_substitution;
+
 typedef enum { GPD_ACT_IDENTITY = 0, GPD_ACT_RELU = 1, GPD_ACT_SIGMOID = 2 } gpd_activation_kind;
 
 typedef enum {
@@ -113,8 +119,8 @@ typedef struct {
 
 /* What gpd_plan_query returns. */
 typedef enum {
-    GPD_Q_THRESHOLD_FWD = 0,    /* mn d1 + n - 1            (Theorem 2)            */
-    GPD_Q_THRESHOLD_BWD = 1,    /* mn (d2 + 1) - n          (proof of Theorem 6)   */
+    GPD_Q_THRESHOLD_FWD = 0,    /* mn d1 + n - 1   (Theorem 2)          or, alternate substitution, mn d1 + mn - m */
+    GPD_Q_THRESHOLD_BWD = 1,    /* mn (d2 + 1) - n (proof of Theorem 6) or, alternate substitution, mn d2 + m - 1  */
     GPD_Q_THRESHOLD_AUDIT = 2,  /* mn                                               */
     GPD_Q_ELEMENT_SIZE = 3,     /* bytes per share / worker-output element (4 or 8) */
     GPD_Q_W_SHARE_ELEMS = 4,    /* P * (N1/m) * (N0/n)                              */
@@ -152,6 +158,12 @@ const char* gpd_status_string(gpd_status s);
  */
 gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, int32_t P,
                     const double* points_host, gpd_precision precision, gpd_plan_t* out);
+/* Same with the substitution chosen by the caller (gpd_plan uses GPD_SUBST_U_EQ_VN).  The alternate
+ * substitution moves error tolerance from the forward to the backward product (proofs of Theorems
+ * 4 and 6); exponent maps: W_ij at u^(i + m j), X_jk at u^(m(n-1-j) + mn k), Delta^T_ki at
+ * u^(mn k + m-1-i), update operands Delta_i at u^i and X_j at u^(m j). */
+gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* split, gpd_substitution subst, int32_t P,
+                          const double* points_host, gpd_precision precision, gpd_plan_t* out);
 gpd_status gpd_plan_destroy(gpd_plan_t plan);
 gpd_status gpd_plan_query(gpd_plan_t plan, gpd_query what, int64_t* value);
 /* Copies a host table into host_out (capacity in doubles); *count receives its length. */

@@ -4,8 +4,8 @@ Follows Section IV (Theorems 1 and 2), the DNN versions of Sections VI and VIII
 and the single-variable forms in the proofs of Theorems 4 and 6 (appendix on
 error tolerances), with the substitution u = v^n, w = v^{mn}.
 
-Everything below is a polynomial in the single variable v evaluated at the
-node's point b_p:
+With the default substitution everything below is a polynomial in the single
+variable v evaluated at the node's point b_p:
 
     W block (i,j)         -> exponent n*i + j                      (Eq. 1 with u=v^n)
     X block (j,k)         -> exponent (n-1-j) + m*n*k              (Theorem 2 encoding, w=v^{mn})
@@ -13,6 +13,15 @@ node's point b_p:
     Delta^T block (k,i)   -> exponent m*n*k + n*(m-1-i)            (backpropagation encoding)
     wanted C^T block (k,j)-> exponent m*n*k + n*(m-1) + j          (proof of Theorem 6)
     update operands       -> Delta_i at n*i, X_j at j (ascending)  (update stage)
+
+The alternate substitution v = u^m, w = u^{mn} (second rows of Tables I and III; proofs of
+Theorems 4 and 6) makes everything a polynomial in u instead and trades forward for backward
+error tolerance:
+
+    W block (i,j) -> i + m*j            X block (j,k) -> m*(n-1-j) + m*n*k
+    wanted S (i,k) -> i + m*(n-1) + m*n*k           Q_f = m n d1 + m n - m
+    Delta^T block (k,i) -> m*n*k + (m-1-i)          wanted C^T (k,j) -> m*n*k + (m-1) + m*j
+    Q_b = m n d2 + m - 1                            update operands: Delta_i at i, X_j at m*j
 """
 
 from __future__ import annotations
@@ -23,6 +32,7 @@ from typing import Optional
 import numpy as np
 
 FWD, BWD, UPD, AUDIT = 0, 1, 2, 3
+SUBST_U_VN, SUBST_V_UM = 0, 1          # u = v^n, w = v^{mn}   |   v = u^m, w = u^{mn}
 
 
 def chebyshev_points(P: int) -> np.ndarray:
@@ -56,6 +66,7 @@ class GPCode:
     d2: int = 1
     P: int = 0
     points: Optional[np.ndarray] = None
+    subst: int = SUBST_U_VN
 
     def __post_init__(self):
         if self.N1 % self.m or self.N0 % self.n or self.B % self.d1 or self.B % self.d2:
@@ -71,12 +82,16 @@ class GPCode:
     # ---- recovery thresholds -------------------------------------------------
     @property
     def Q_f(self) -> int:
-        """Theorem 2: number of coefficients of S~(v), m n d1 + n - 1."""
+        """Theorem 2: number of coefficients of S~(v), m n d1 + n - 1 (alternate: m n d1 + m n - m)."""
+        if self.subst == SUBST_V_UM:
+            return self.m * self.n * self.d1 + self.m * self.n - self.m
         return self.m * self.n * self.d1 + self.n - 1
 
     @property
     def Q_b(self) -> int:
-        """Backpropagation polynomial C~^T(v): m n d2 + m n - n coefficients."""
+        """Backpropagation polynomial C~^T(v): m n d2 + m n - n coefficients (alternate: m n d2 + m - 1)."""
+        if self.subst == SUBST_V_UM:
+            return self.m * self.n * self.d2 + self.m - 1
         return self.m * self.n * (self.d2 + 1) - self.n
 
     @property
@@ -91,27 +106,44 @@ class GPCode:
     def exp_W(self) -> np.ndarray:
         i = np.arange(self.m)[:, None]
         j = np.arange(self.n)[None, :]
+        if self.subst == SUBST_V_UM:
+            return i + self.m * j
         return self.n * i + j                                   # [m, n]
 
     def exp_X(self) -> np.ndarray:
         j = np.arange(self.n)[:, None]
         k = np.arange(self.d1)[None, :]
+        if self.subst == SUBST_V_UM:
+            return self.m * (self.n - 1 - j) + self.m * self.n * k
         return (self.n - 1 - j) + self.m * self.n * k           # [n, d1]
 
     def exp_DeltaT(self) -> np.ndarray:
         k = np.arange(self.d2)[:, None]
         i = np.arange(self.m)[None, :]
+        if self.subst == SUBST_V_UM:
+            return self.m * self.n * k + (self.m - 1 - i)
         return self.m * self.n * k + self.n * (self.m - 1 - i)  # [d2, m]
+
+    def exp_update(self):
+        """Exponents of the ascending update-stage encodings: (Delta_i, X_j)."""
+        i, j = np.arange(self.m), np.arange(self.n)
+        if self.subst == SUBST_V_UM:
+            return i, self.m * j
+        return self.n * i, j
 
     def wanted(self, which: int) -> np.ndarray:
         """Exponent whose coefficient is block (row, col) of the result."""
         if which == FWD:
             i = np.arange(self.m)[:, None]
             k = np.arange(self.d1)[None, :]
+            if self.subst == SUBST_V_UM:
+                return i + self.m * (self.n - 1) + self.m * self.n * k
             return self.n * i + self.m * self.n * k + self.n - 1      # [m, d1]
         if which == BWD:
             k = np.arange(self.d2)[:, None]
             j = np.arange(self.n)[None, :]
+            if self.subst == SUBST_V_UM:
+                return self.m * self.n * k + (self.m - 1) + self.m * j
             return self.m * self.n * k + self.n * (self.m - 1) + j    # [d2, n]
         if which == AUDIT:
             return self.exp_W()                                       # [m, n]

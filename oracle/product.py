@@ -70,8 +70,8 @@ def encode_DeltaT(DeltaT, code: GPCode) -> np.ndarray:
 def encode_update_operands(Delta, X, code: GPCode):
     """Ascending-power encodings of the update stage:
     Delta^_p = sum_i Delta_i a_p^i  ([P][N1/m][B]),  X^_p = sum_j X_j b_p^j  ([P][N0/n][B])."""
-    eD = (code.n * np.arange(code.m))[:, None]
-    eX = np.arange(code.n)[:, None]
+    eD, eX = code.exp_update()
+    eD, eX = eD[:, None], eX[:, None]
     Dh = _encode_blocks(Delta, code.m, 1, eD, code)
     Xh = _encode_blocks(X, code.n, 1, eX, code)
     return Dh, Xh

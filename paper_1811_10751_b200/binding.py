@@ -39,9 +39,10 @@ GPD_PHASE_FWD, GPD_PHASE_BWD, GPD_PHASE_UPD, GPD_PHASE_REGEN, GPD_PHASE_INJECT_S
 (GPD_TABLE_POINTS, GPD_TABLE_PARITY_FWD, GPD_TABLE_PARITY_BWD, GPD_TABLE_PARITY_AUDIT,
  GPD_TABLE_COEF_W, GPD_TABLE_COEF_X, GPD_TABLE_COEF_DT) = range(7)
 GPD_MAX_NODES = 64
+GPD_SUBST_U_EQ_VN, GPD_SUBST_V_EQ_UM = 0, 1
 
 EXPORTED = [
-    "gpd_status_string", "gpd_plan", "gpd_plan_destroy", "gpd_plan_query", "gpd_plan_table",
+    "gpd_status_string", "gpd_plan", "gpd_plan_subst", "gpd_plan_destroy", "gpd_plan_query", "gpd_plan_table",
     "gpd_encode_A", "gpd_encode_B", "gpd_worker_gemm", "gpd_device_status", "gpd_update_shares", "gpd_inject",
     "gpd_locate_errors", "gpd_locate_errors_static", "gpd_decode", "gpd_regenerate_shares", "gpd_activation", "gpd_softmax_xent_delta",
     "gpd_backprop_hadamard", "gpd_sae_output_delta", "gpd_sae_hidden_delta", "coded_layer_step",
@@ -70,6 +71,8 @@ lib.gpd_status_string.restype = C.c_char_p
 lib.gpd_status_string.argtypes = [C.c_int]
 lib.gpd_plan.argtypes = [C.POINTER(gpd_shape), C.POINTER(gpd_split), _i32, C.POINTER(C.c_double), C.c_int,
                          C.POINTER(_vp)]
+lib.gpd_plan_subst.argtypes = [C.POINTER(gpd_shape), C.POINTER(gpd_split), C.c_int, _i32, C.POINTER(C.c_double),
+                               C.c_int, C.POINTER(_vp)]
 lib.gpd_plan_destroy.argtypes = [_vp]
 lib.gpd_plan_query.argtypes = [_vp, C.c_int, C.POINTER(_i64)]
 lib.gpd_plan_table.argtypes = [_vp, C.c_int, C.POINTER(C.c_double), _i64, C.POINTER(_i64)]
@@ -183,8 +186,10 @@ def gpd_status_string(status: int) -> str:
     return lib.gpd_status_string(status).decode()
 
 
-def gpd_plan(shape, split, P: int, points=None, precision: int = GPD_PREC_AUTO) -> Plan:
-    """shape = (N1, N0, B); split = (m, n, d1, d2); points: P doubles or None (Chebyshev)."""
+def gpd_plan(shape, split, P: int, points=None, precision: int = GPD_PREC_AUTO,
+             subst: int = GPD_SUBST_U_EQ_VN) -> Plan:
+    """shape = (N1, N0, B); split = (m, n, d1, d2); points: P doubles or None (Chebyshev);
+    subst other than the default goes through gpd_plan_subst."""
     sh = gpd_shape(*[int(v) for v in shape])
     sp = gpd_split(*[int(v) for v in split])
     pts = None
@@ -194,8 +199,16 @@ def gpd_plan(shape, split, P: int, points=None, precision: int = GPD_PREC_AUTO) 
             raise ValueError("need exactly P points")
         pts = arr.ctypes.data_as(C.POINTER(C.c_double))
     h = _vp(0)
-    _check(lib.gpd_plan(C.byref(sh), C.byref(sp), int(P), pts, int(precision), C.byref(h)), "gpd_plan")
+    if subst == GPD_SUBST_U_EQ_VN:
+        _check(lib.gpd_plan(C.byref(sh), C.byref(sp), int(P), pts, int(precision), C.byref(h)), "gpd_plan")
+    else:
+        _check(lib.gpd_plan_subst(C.byref(sh), C.byref(sp), int(subst), int(P), pts, int(precision), C.byref(h)),
+               "gpd_plan_subst")
     return Plan(h.value, tuple(shape), tuple(split), int(P))
+
+
+def gpd_plan_subst(shape, split, subst: int, P: int, points=None, precision: int = GPD_PREC_AUTO) -> Plan:
+    return gpd_plan(shape, split, P, points=points, precision=precision, subst=subst)
 
 
 def gpd_plan_destroy(plan: Plan):

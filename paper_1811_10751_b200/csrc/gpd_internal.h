@@ -52,6 +52,7 @@ struct gpd_plan_s {
     gpd_shape shape;
     gpd_split split;
     int P = 0;
+    int Qf = 0, Qb = 0, Qw = 0;  // thresholds under the plan's substitution
     gpd_precision prec = GPD_PREC_FP32;
     int elem_size = 4;
     double tau_col = 0, tau_in = 0;

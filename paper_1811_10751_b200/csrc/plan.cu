@@ -141,8 +141,16 @@ extern "C" const char* gpd_status_string(gpd_status s) {
 
 extern "C" gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, int32_t P,
                                const double* points_host, gpd_precision precision, gpd_plan_t* out) {
+    return gpd_plan_subst(shape, split, GPD_SUBST_U_EQ_VN, P, points_host, precision, out);
+}
+
+extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* split, gpd_substitution subst,
+                                     int32_t P, const double* points_host, gpd_precision precision,
+                                     gpd_plan_t* out) {
     if (!shape || !split || !out) return GPD_ERR_ARG;
     *out = nullptr;
+    if (subst != GPD_SUBST_U_EQ_VN && subst != GPD_SUBST_V_EQ_UM) return GPD_ERR_ARG;
+    const bool alt = subst == GPD_SUBST_V_EQ_UM;
     if (precision != GPD_PREC_AUTO && precision != GPD_PREC_FP32 && precision != GPD_PREC_FP64)
         return GPD_ERR_ARG;
     const int m = split->m, n = split->n, d1 = split->d1, d2 = split->d2;
@@ -150,9 +158,11 @@ extern "C" gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, i
         return GPD_ERR_SHAPE;
     if (shape->N1 % m || shape->N0 % n || shape->B % d1 || shape->B % d2) return GPD_ERR_SHAPE;
     if (P <= 0) return GPD_ERR_P_TOO_SMALL;
-    const int64_t Qf = (int64_t)m * n * d1 + n - 1;        // Theorem 2
-    const int64_t Qb = (int64_t)m * n * (d2 + 1) - n;      // coefficients of C~^T(v)
-    const int64_t Qw = (int64_t)m * n;                     // coefficients of W~(v)
+    // u = v^n, w = v^(mn): Theorem 2 and the proof of Theorem 6, first case;
+    // v = u^m, w = u^(mn): second case (forward and backward tolerances swap roles)
+    const int64_t Qf = alt ? (int64_t)m * n * d1 + (int64_t)m * n - m : (int64_t)m * n * d1 + n - 1;
+    const int64_t Qb = alt ? (int64_t)m * n * d2 + m - 1 : (int64_t)m * n * (d2 + 1) - n;
+    const int64_t Qw = (int64_t)m * n;                     // coefficients of the share polynomial
     if (P > kMaxNodes || Qf > kMaxQ) return GPD_ERR_Q_TOO_LARGE;
     if (m * n > kMaxBlocks || n * d1 > kMaxBlocks || d2 * m > kMaxBlocks || m * d1 > kMaxWanted ||
         d2 * n > kMaxWanted)
@@ -165,6 +175,7 @@ extern "C" gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, i
     plan->shape = *shape;
     plan->split = *split;
     plan->P = P;
+    plan->Qf = (int)Qf; plan->Qb = (int)Qb; plan->Qw = (int)Qw;
     plan->points.resize(P);
     if (points_host) {
         for (int p = 0; p < P; ++p) plan->points[p] = points_host[p];
@@ -196,29 +207,34 @@ extern "C" gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, i
     plan->coefXup.resize((size_t)P * n);
     for (int p = 0; p < P; ++p) {
         for (int i = 0; i < m; ++i)
-            for (int j = 0; j < n; ++j) plan->coefW[((size_t)p * m + i) * n + j] = at(p, n * i + j);
+            for (int j = 0; j < n; ++j)
+                plan->coefW[((size_t)p * m + i) * n + j] = at(p, alt ? i + m * j : n * i + j);
         for (int j = 0; j < n; ++j)
             for (int k = 0; k < d1; ++k)
-                plan->coefX[((size_t)p * n + j) * d1 + k] = at(p, (n - 1 - j) + m * n * k);
+                plan->coefX[((size_t)p * n + j) * d1 + k] =
+                    at(p, alt ? m * (n - 1 - j) + m * n * k : (n - 1 - j) + m * n * k);
         for (int k = 0; k < d2; ++k)
             for (int i = 0; i < m; ++i)
-                plan->coefDT[((size_t)p * d2 + k) * m + i] = at(p, m * n * k + n * (m - 1 - i));
-        for (int i = 0; i < m; ++i) plan->coefDup[(size_t)p * m + i] = at(p, n * i);
-        for (int j = 0; j < n; ++j) plan->coefXup[(size_t)p * n + j] = at(p, j);
+                plan->coefDT[((size_t)p * d2 + k) * m + i] =
+                    at(p, alt ? m * n * k + (m - 1 - i) : m * n * k + n * (m - 1 - i));
+        for (int i = 0; i < m; ++i) plan->coefDup[(size_t)p * m + i] = at(p, alt ? i : n * i);
+        for (int j = 0; j < n; ++j) plan->coefXup[(size_t)p * n + j] = at(p, alt ? m * j : j);
     }
     // products
     ProductInfo& f = plan->prod[GPD_FWD];
     f.Q = (int)Qf; f.R = P - f.Q; f.grid_rows = m; f.grid_cols = d1;
     f.br = shape->N1 / m; f.bc = shape->B / d1;
     for (int i = 0; i < m; ++i)
-        for (int k = 0; k < d1; ++k) f.wanted[i * d1 + k] = n * i + m * n * k + n - 1;
+        for (int k = 0; k < d1; ++k)
+            f.wanted[i * d1 + k] = alt ? i + m * (n - 1) + m * n * k : n * i + m * n * k + n - 1;
     f.H = left_null_space(plan->points, f.Q);
     ProductInfo& b = plan->prod[GPD_BWD];
     if (bwd_ok) {
         b.Q = (int)Qb; b.R = P - b.Q; b.grid_rows = d2; b.grid_cols = n;
         b.br = shape->B / d2; b.bc = shape->N0 / n;
         for (int k = 0; k < d2; ++k)
-            for (int j = 0; j < n; ++j) b.wanted[k * n + j] = m * n * k + n * (m - 1) + j;
+            for (int j = 0; j < n; ++j)
+                b.wanted[k * n + j] = alt ? m * n * k + (m - 1) + m * j : m * n * k + n * (m - 1) + j;
         b.H = left_null_space(plan->points, b.Q);
     }
     ProductInfo& a = plan->prod[GPD_AUDIT];
@@ -226,7 +242,7 @@ extern "C" gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, i
         a.Q = (int)Qw; a.R = P - a.Q; a.grid_rows = m; a.grid_cols = n;
         a.br = shape->N1 / m; a.bc = shape->N0 / n;
         for (int i = 0; i < m; ++i)
-            for (int j = 0; j < n; ++j) a.wanted[i * n + j] = n * i + j;
+            for (int j = 0; j < n; ++j) a.wanted[i * n + j] = alt ? i + m * j : n * i + j;
         a.H = left_null_space(plan->points, a.Q);
     }
     *out = plan;
@@ -247,8 +263,8 @@ extern "C" gpd_status gpd_plan_query(gpd_plan_t plan, gpd_query what, int64_t* v
     const int64_t P = plan->P;
     switch (what) {
         case GPD_Q_THRESHOLD_FWD: *value = plan->prod[GPD_FWD].Q; break;
-        case GPD_Q_THRESHOLD_BWD: *value = (int64_t)c.m * c.n * (c.d2 + 1) - c.n; break;
-        case GPD_Q_THRESHOLD_AUDIT: *value = (int64_t)c.m * c.n; break;
+        case GPD_Q_THRESHOLD_BWD: *value = plan->Qb; break;
+        case GPD_Q_THRESHOLD_AUDIT: *value = plan->Qw; break;
         case GPD_Q_ELEMENT_SIZE: *value = plan->elem_size; break;
         case GPD_Q_W_SHARE_ELEMS: *value = P * (s.N1 / c.m) * (s.N0 / c.n); break;
         case GPD_Q_X_SHARE_ELEMS: *value = P * (s.N0 / c.n) * (s.B / c.d1); break;

@@ -27,7 +27,7 @@ class CodedProduct:
     def __init__(self, code: GPCode, precision: int = g.GPD_PREC_AUTO):
         self.code = code
         self.plan = g.gpd_plan((code.N1, code.N0, code.B), (code.m, code.n, code.d1, code.d2), code.P,
-                               points=code.points, precision=precision)
+                               points=code.points, precision=precision, subst=code.subst)
         self.np_dtype = np.float32 if self.plan.query(g.GPD_Q_ELEMENT_SIZE) == 4 else np.float64
         self.ws = self.plan.workspace()
         self.res = g.new_results(1)

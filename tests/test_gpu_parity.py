@@ -436,3 +436,40 @@ def test_config3_full_size_against_oracle_decisions():
             assert r0.outcome == NO_ERROR
             S_clean = cp.decode(g.GPD_FWD, Z)
         assert op.rel_fro(S, S_clean) < REL_TOL
+
+
+# --------------------------------------------------------------------------------------------------
+# alternate substitution v = u^m, w = u^(mn): same kernels, other exponent tables
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("N1,N0,B,m,n,d1,d2,P", [(384, 256, 64, 3, 2, 2, 2, 22), (512, 512, 64, 2, 2, 1, 1, 10)])
+def test_alternate_substitution_products(N1, N0, B, m, n, d1, d2, P):
+    from oracle.code import SUBST_V_UM
+    code = GPCode(N1, N0, B, m, n, d1, d2, P, subst=SUBST_V_UM)
+    assert P >= max(code.Q_f, code.Q_b) + 2
+    cp = CodedProduct(code)
+    W = (rand((N1, N0), 51) / np.sqrt(N0)).astype(np.float32)
+    X, DT = rand((N0, B), 52), rand((B, N1), 53)
+    Wsh = cp.encode_W(W)
+    assert np.allclose(host(Wsh).reshape(P, N1 // m, N0 // n), op.encode_W(W, code), rtol=0, atol=1e-6)
+    for which, operand, src, Q, ref, Zo in (
+            (g.GPD_FWD, g.GPD_OPERAND_X_FWD, X, code.Q_f, op.ref_forward(W, X),
+             op.worker_products(op.encode_W(W, code), op.encode_X(X, code))),
+            (g.GPD_BWD, g.GPD_OPERAND_DELTAT_BWD, DT, code.Q_b, op.ref_backward(DT, W),
+             op.worker_products(op.encode_DeltaT(DT, code), op.encode_W(W, code)))):
+        Z = cp.products(which, cp.encode(operand, src))
+        nodes = np.zeros(P, dtype=bool)
+        nodes[[2]] = True
+        g.gpd_inject(cp.plan, which, Z, 61, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=1 << 2, scale=1.0)
+        Zo = Zo.astype(cp.np_dtype)
+        oinj.inject_gauss(Zo, 61, 1.0, nodes=nodes)
+        ro = locate_subspace(Zo, code.points, Q, tolerances_for(cp.np_dtype))
+        r = cp.locate(which, Z)
+        assert r.outcome == ro.outcome == CORRECTED and np.array_equal(cp.flags(r), ro.flagged)
+        out = cp.decode(which, Z)
+        assert op.rel_fro(out, ref) < REL_TOL
+        assert op.rel_fro(out, op.decode(Zo, code, FWD if which == g.GPD_FWD else BWD, use=~ro.flagged)) < REL_TOL
+    Delta = np.ascontiguousarray(DT.T)
+    g.gpd_update_shares(cp.plan, Wsh, cp.encode(g.GPD_OPERAND_DELTA_UPD, Delta), cp.encode(g.GPD_OPERAND_X_UPD, X),
+                        0.05, 0.0)
+    assert cp.locate(g.GPD_AUDIT, Wsh).outcome == NO_ERROR
+    assert op.rel_fro(cp.decode(g.GPD_AUDIT, Wsh), op.ref_update(W, Delta, X, 0.05)) < REL_TOL

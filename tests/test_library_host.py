@@ -100,3 +100,23 @@ def test_custom_points_are_kept():
     plan = g.gpd_plan((8, 8, 4), (2, 2, 1, 1), 7, points=pts)
     assert np.array_equal(plan.table(g.GPD_TABLE_POINTS), pts)
     plan.destroy()
+
+
+@pytest.mark.parametrize("shape,split,P", [((12, 8, 6), (3, 2, 2, 3), 26), ((4096, 4096, 256), (2, 2, 1, 1), 10),
+                                           ((8192, 1024, 1024), (4, 4, 1, 1), 36)])
+def test_alternate_substitution_plan_matches_oracle(shape, split, P):
+    from oracle.code import SUBST_V_UM
+    plan = g.gpd_plan_subst(shape, split, g.GPD_SUBST_V_EQ_UM, P)
+    code = GPCode(shape[0], shape[1], shape[2], split[0], split[1], split[2], split[3], P, subst=SUBST_V_UM)
+    assert plan.query(g.GPD_Q_THRESHOLD_FWD) == code.Q_f
+    assert plan.query(g.GPD_Q_THRESHOLD_BWD) == code.Q_b
+    assert plan.query(g.GPD_Q_THRESHOLD_AUDIT) == code.Q_w
+    pw = powers(plan.table(g.GPD_TABLE_POINTS), 64)
+    for tab, ex in ((g.GPD_TABLE_COEF_W, code.exp_W()), (g.GPD_TABLE_COEF_X, code.exp_X()),
+                    (g.GPD_TABLE_COEF_DT, code.exp_DeltaT())):
+        assert np.allclose(plan.table(tab).reshape(P, -1), pw[:, ex.reshape(-1)], rtol=1e-14, atol=0)
+    H = plan.table(g.GPD_TABLE_PARITY_BWD).reshape(P - code.Q_b, P)
+    assert np.abs(H @ powers(plan.table(g.GPD_TABLE_POINTS), code.Q_b)).max() < 1e-13
+    plan.destroy()
+    with pytest.raises(g.GpdError):
+        g.gpd_plan_subst(shape, split, 7, P)

@@ -307,3 +307,45 @@ def test_regeneration_restores_any_set_of_up_to_P_minus_mn_shares():
     assert np.isclose(again[4, 1, 1], np.polyval(coeffs[::-1], code.points[4]), rtol=1e-12)
     with pytest.raises(ValueError):
         op.regenerate_shares(clean, code, np.array([True] * 4 + [False] * 5))
+
+
+# ----------------------------------------------------------------------------------------------
+# alternate substitution v = u^m, w = u^{mn}
+# ----------------------------------------------------------------------------------------------
+from oracle.code import SUBST_V_UM   # noqa: E402
+
+
+@pytest.mark.parametrize("m,n,d", [(m, n, d) for m in range(1, 5) for n in range(1, 5) for d in range(1, 4)])
+def test_alternate_substitution_thresholds_by_brute_force(m, n, d):
+    code = GPCode(m, n, d, m, n, d, d, 64, points=np.linspace(-1, 1, 64), subst=SUBST_V_UM)
+    eW, eX, eD = code.exp_W(), code.exp_X(), code.exp_DeltaT()
+    terms = {}
+    for i, j, jp, k in itertools.product(range(m), range(n), range(n), range(d)):
+        terms.setdefault(int(eW[i, j] + eX[jp, k]), []).append((i, j, jp, k))
+    assert max(terms) + 1 == code.Q_f == m * n * d + m * n - m            # proof of Theorem 6, second case
+    want = code.wanted(FWD)
+    for i, k in itertools.product(range(m), range(d)):
+        assert sorted(terms[int(want[i, k])]) == [(i, j, j, k) for j in range(n)]
+    terms = {}
+    for k, ip, i, j in itertools.product(range(d), range(m), range(m), range(n)):
+        terms.setdefault(int(eD[k, ip] + eW[i, j]), []).append((k, ip, i, j))
+    assert max(terms) + 1 == code.Q_b == m * n * d + m - 1
+    want = code.wanted(BWD)
+    for k, j in itertools.product(range(d), range(n)):
+        assert sorted(terms[int(want[k, j])]) == [(k, i, i, j) for i in range(m)]
+    assert sorted(eW.reshape(-1).tolist()) == list(range(m * n))
+
+
+def test_alternate_substitution_tolerances_and_products():
+    # Table I, second row, at P = 180, m = n = 6: (t_f, t_b) swap roles
+    code = GPCode(6, 6, 1, 6, 6, 1, 1, 180, subst=SUBST_V_UM)
+    assert ((180 - code.Q_f) // 2, (180 - code.Q_b) // 2) == (57, 69)
+    assert (180 - code.Q_f - 1, 180 - code.Q_b - 1) == (113, 138)
+    code = GPCode(12, 8, 6, 3, 2, 2, 3, 26, subst=SUBST_V_UM)
+    W, X, DT = _rand((12, 8), 31), _rand((8, 6), 32), _rand((6, 12), 33)
+    Ws = op.encode_W(W, code)
+    assert op.rel_fro(op.decode(op.worker_products(Ws, op.encode_X(X, code)), code, FWD), W @ X) < 1e-8
+    assert op.rel_fro(op.decode(op.worker_products(op.encode_DeltaT(DT, code), Ws), code, BWD), DT @ W) < 1e-8
+    Dh, Xh = op.encode_update_operands(DT.T.copy(), X, code)
+    new = op.update_shares(Ws, Dh, Xh, eta=0.1)
+    assert op.rel_fro(op.decode(new, code, AUDIT), op.ref_update(W, DT.T, X, 0.1)) < 1e-10
