@@ -473,3 +473,63 @@ def test_alternate_substitution_products(N1, N0, B, m, n, d1, d2, P):
                         0.05, 0.0)
     assert cp.locate(g.GPD_AUDIT, Wsh).outcome == NO_ERROR
     assert op.rel_fro(cp.decode(g.GPD_AUDIT, Wsh), op.ref_update(W, Delta, X, 0.05)) < REL_TOL
+
+
+# --------------------------------------------------------------------------------------------------
+# limits and degenerate shapes
+# --------------------------------------------------------------------------------------------------
+def test_maximum_nodes_threshold_and_parity():
+    """P = 64 nodes, threshold 32, 32 parity checks: the largest code a plan accepts."""
+    N1, N0, B, m, n, d1 = 160, 96, 32, 5, 3, 2                        # Q_f = 5*3*2 + 3 - 1 = 32
+    code = GPCode(N1, N0, B, m, n, d1, 1, 64)
+    assert code.Q_f == 32
+    cp = CodedProduct(code)
+    assert cp.np_dtype == np.float64
+    W, X = rand((N1, N0), 71), rand((N0, B), 72)
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    r = cp.locate(g.GPD_FWD, Z)
+    assert r.outcome == NO_ERROR
+    nodes = np.zeros(64, dtype=bool)
+    nodes[[4, 33, 60]] = True
+    mask = sum(1 << int(p) for p in np.flatnonzero(nodes))
+    g.gpd_inject(cp.plan, g.GPD_FWD, Z, 73, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=mask, scale=1.0)
+    Zo = op.worker_products(op.encode_W(W, code), op.encode_X(X, code))
+    oinj.inject_gauss(Zo, 73, 1.0, nodes=nodes)
+    ro = locate_subspace(Zo, code.points, code.Q_f, tolerances_for(np.float64))
+    r = cp.locate(g.GPD_FWD, Z)
+    assert r.outcome == ro.outcome == CORRECTED and np.array_equal(cp.flags(r), ro.flagged)
+    assert np.array_equal(ro.flagged, nodes)
+    # threshold 32 amplifies rounding by about 1e10: the decoded product is compared with the
+    # oracle's decode of the same polynomial and, more loosely, with the uncoded product
+    S = cp.decode(g.GPD_FWD, Z)
+    assert op.rel_fro(S, op.decode(Zo, code, FWD, use=~ro.flagged)) < 1e-3
+    assert op.rel_fro(S, op.ref_forward(W, X)) < 1e-3
+
+
+def test_tiny_and_skinny_shapes():
+    """One-element blocks, a single output position per node, and a mini-batch of one in the
+    backward product (a 1 x K by K x N worker product)."""
+    code = GPCode(2, 2, 1, 2, 2, 1, 1, 9)                            # blocks are 1 x 1, L = 1
+    cp = CodedProduct(code, g.GPD_PREC_FP64)
+    W, X, DT = rand((2, 2), 81), rand((2, 1), 82), rand((1, 2), 83)
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    assert cp.locate(g.GPD_FWD, Z).outcome == NO_ERROR
+    assert np.allclose(cp.decode(g.GPD_FWD, Z), W.astype(np.float64) @ X, atol=1e-6)
+    Zb = cp.products(g.GPD_BWD, cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT))
+    assert np.allclose(cp.decode(g.GPD_BWD, Zb, use_mask=[True] * 9), DT.astype(np.float64) @ W, atol=1e-6)
+    # one corrupted node with a single codeword: located (rank 1, one column of H in its range)
+    Zg = Z.clone()
+    Zg[5] += 3.0
+    r = cp.locate(g.GPD_FWD, Zg)
+    assert r.outcome == CORRECTED and list(np.flatnonzero(cp.flags(r))) == [5]
+    # mini-batch of one, backward, FP32 path (thresholds 5 / 6): M = 1
+    code = GPCode(256, 512, 1, 2, 2, 1, 1, 10)
+    cp = CodedProduct(code)
+    assert cp.np_dtype == np.float32
+    W, DT = (rand((256, 512), 84) / 16).astype(np.float32), rand((1, 256), 85)
+    cp.encode_W(W)
+    Zb = cp.products(g.GPD_BWD, cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT))
+    assert cp.locate(g.GPD_BWD, Zb).outcome == NO_ERROR
+    assert op.rel_fro(cp.decode(g.GPD_BWD, Zb), op.ref_backward(DT, W)) < REL_TOL
