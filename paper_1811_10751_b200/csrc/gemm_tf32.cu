@@ -3,7 +3,8 @@
 // shared memory by TMA, and 3xTF32 splitting so that the result keeps FP32-level accuracy:
 //     a = a_hi + a_lo (both exactly representable in TF32),   a*b ~ a_lo*b_hi + a_hi*b_lo + a_hi*b_hi.
 //
-// One CTA computes one 128 x 128 tile of one node's product.  Warp roles:
+// One CTA computes one 128 x 128 tile of one node's product (column strips of it for the tiles
+// left over after the last full round over the SMs).  Warp roles:
 //   warp 0      : TMA producer (one lane) - raw FP32 tiles of A and B into a 3-stage ring
 //   warp 1      : allocates tensor memory; one lane issues the MMAs and commits them to mbarriers
 //   warps 2..9  : split every landed tile in place into hi (overwrites the raw tile) and lo (second
@@ -111,7 +112,8 @@ __device__ __forceinline__ float to_tf32(float x) {
 
 template <bool B_KMAJOR, bool UPDATE>
 __global__ void __launch_bounds__(kThreads, 1)
-sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams prm) {
+sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams prm,
+                    int tiles_m, int tiles_n, int full_tiles, int split) {
     if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -120,9 +122,21 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int p = blockIdx.z;
-    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    // Tile schedule: CTAs 0 .. full_tiles-1 take whole 128 x 128 tiles; the tiles left over after the
+    // last full round over the SMs are cut into `split` column strips, one per CTA, so that the
+    // final, partly filled round is short (128 x 32 strips when split = 4).
+    int tile = blockIdx.x, sub = 0, bn = BN;
+    if (tile >= full_tiles) {
+        const int piece = tile - full_tiles;
+        tile = full_tiles + piece / split;
+        sub = piece % split;
+        bn = BN / split;
+    }
+    const int tn = tile % tiles_n, tm = (tile / tiles_n) % tiles_m;
+    const int p = tile / (tiles_n * tiles_m);
+    const int m0 = tm * BM, n0 = tn * BN + sub * bn;
     const int num_kb = (int)((prm.K + BK - 1) / BK);
+    const int b_float4 = bn * BK / 4;                // 16-byte units of one B tile
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -157,13 +171,12 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const int s = kb % STAGES;
                 const uint32_t ph = (kb / STAGES) & 1;
                 if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) break;
-                mbar_expect_tx(&full_bar[s], A_TILE_BYTES + B_TILE_BYTES);
+                mbar_expect_tx(&full_bar[s], A_TILE_BYTES + bn * BK * 4);
                 tma_load_3d(A_hi(s), &tmA, kb * BK, m0, p, &full_bar[s]);
-                if (B_KMAJOR) {
-                    tma_load_3d(B_hi(s), &tmB, kb * BK, n0, p, &full_bar[s]);
-                } else {
-#pragma unroll
-                    for (int c = 0; c < BN / 32; ++c)
+                for (int c = 0; c < bn / 32; ++c) {      // B arrives in boxes of 32 columns (or 32 rows of X^_p)
+                    if (B_KMAJOR)
+                        tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, kb * BK, n0 + 32 * c, p, &full_bar[s]);
+                    else
                         tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, n0 + 32 * c, kb * BK, p, &full_bar[s]);
                 }
                 ++issued;
@@ -179,7 +192,7 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
-                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                                   ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; ++kb) {
                 const int s = kb % STAGES;
@@ -216,11 +229,11 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (!mbar_wait(&full_bar[s], ph, abort_p)) { ok = false; break; }
             float4* hi[2] = {reinterpret_cast<float4*>(A_hi(s)), reinterpret_cast<float4*>(B_hi(s))};
             float4* lo[2] = {reinterpret_cast<float4*>(A_lo(s)), reinterpret_cast<float4*>(B_lo(s))};
+            const int count[2] = {A_TILE_BYTES / 16, b_float4};
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
-#pragma unroll
-                for (int i = 0; i < A_TILE_BYTES / 16 / kConvThreads; ++i) {
-                    const int idx = tc + kConvThreads * i;
+#pragma unroll 4
+                for (int idx = tc; idx < count[t]; idx += kConvThreads) {
                     const float4 v = hi[t][idx];
                     float4 h, l;
                     h.x = to_tf32(v.x); h.y = to_tf32(v.y); h.z = to_tf32(v.z); h.w = to_tf32(v.w);
@@ -238,13 +251,15 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (__all_sync(0xffffffffu, acc_ready)) {    // tcgen05.ld is warp-collective: all lanes or none
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int q = warp & 3;                  // this warp may touch TMEM lanes 32q .. 32q+31
-            const int half = (warp - 2) >> 2;        // two warps share a lane quarter: 64 columns each
+            const int half = (warp - 2) >> 2;        // two warps share a lane quarter: half the columns each
+            const int c_begin = bn >= 64 ? half * (bn / 2) : (half == 0 ? 0 : bn);
+            const int c_end = bn >= 64 ? (half + 1) * (bn / 2) : bn;
             const int64_t gm = (int64_t)m0 + q * 32 + lane;
             float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
             const float shrink = (float)prm.shrink, eta = (float)prm.eta;
             const bool vec = (prm.N % 4 == 0);
 #pragma unroll 1
-            for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
+            for (int c0 = c_begin; c0 < c_end; c0 += 32) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0;
                 asm volatile(
@@ -328,18 +343,40 @@ bool make_map(CUtensorMap* map, const void* base, int64_t batch, int64_t rows, i
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
 template <bool B_KMAJOR, bool UPDATE>
 gpd_status launch(const GemmParams& prm, cudaStream_t st) {
     CUtensorMap tmA, tmB;
     if (!make_map(&tmA, prm.A, prm.P, prm.M, prm.K, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B)) return GPD_ERR_CUDA;
-    const bool okB = B_KMAJOR ? make_map(&tmB, prm.B, prm.P, prm.N, prm.K, BK, BN, CU_TENSOR_MAP_SWIZZLE_128B)
+    const bool okB = B_KMAJOR ? make_map(&tmB, prm.B, prm.P, prm.N, prm.K, BK, 32, CU_TENSOR_MAP_SWIZZLE_128B)
                               : make_map(&tmB, prm.B, prm.P, prm.K, prm.N, 32, BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
     if (!okB) return GPD_ERR_CUDA;
     if (cudaFuncSetAttribute(sgemm_3xtf32_kernel<B_KMAJOR, UPDATE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              SMEM_BYTES) != cudaSuccess)
         return GPD_ERR_CUDA;
-    dim3 grid((unsigned)((prm.N + BN - 1) / BN), (unsigned)((prm.M + BM - 1) / BM), (unsigned)prm.P);
-    sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<grid, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm);
+    const int tiles_n = (int)((prm.N + BN - 1) / BN), tiles_m = (int)((prm.M + BM - 1) / BM);
+    const int64_t tiles = (int64_t)tiles_n * tiles_m * prm.P;
+    // One CTA per SM at a time.  After the last full round, `rem` tiles are left: cutting them into
+    // 2 or 4 strips shortens that last round if the strips still fit in one round.
+    const int sms = sm_count();
+    const int rem = (int)(tiles % sms);
+    int split = 1;
+    if (rem > 0 && rem * 4 <= sms) split = 4;
+    else if (rem > 0 && rem * 2 <= sms) split = 2;
+    const int full_tiles = (int)(tiles - (split > 1 ? rem : 0));
+    const int64_t ctas = full_tiles + (int64_t)(split > 1 ? rem : 0) * split;
+    sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<(unsigned)ctas, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n,
+                                                                                         full_tiles, split);
     return launch_ok();
 }
 
