@@ -77,7 +77,20 @@ typedef enum {
 typedef enum {
     GPD_PREC_AUTO = 0,          /* FP32 if every threshold of the plan is <= 9, else FP64 */
     GPD_PREC_FP32 = 1,          /* shares/outputs float; products in 3xTF32 (tensor cores) or FP32 FMA */
-    GPD_PREC_FP64 = 2           /* shares/outputs double; products in FP64 */
+    GPD_PREC_FP64 = 2,          /* shares/outputs double; products in FP64 */
+    GPD_PREC_FP64_SLICED = 3    /* forward product only (gpd_encode_A, gpd_encode_B with GPD_OPERAND_X_FWD,
+                                   gpd_worker_gemm with GPD_FWD, then inject / locate / decode as for
+                                   GPD_PREC_FP64).  The shares W~_p (Eq. 1), X~_p (Theorem 2) are evaluated in
+                                   FP64 and stored as six signed 7-bit digit planes plus one power-of-two
+                                   scale per row of W~_p / column of X~_p, in buffers of the same byte size as
+                                   the FP64 shares (opaque to the caller); the worker products are exact
+                                   int8 x int8 -> int32 tensor-core contractions of digit planes, recombined
+                                   in FP64 (terms below 2^-49 of row scale x column scale dropped); worker
+                                   outputs are double.  Needs N0/n divisible by 16 and finite inputs (a row
+                                   holding a non-finite value encodes as zeros).  Every other call that takes
+                                   shares returns GPD_ERR_UNSUPPORTED; gpd_plan returns it when the shapes
+                                   do not fit.  An implementation choice of this library: the paper
+                                   prescribes no arithmetic for the nodes' products. */
 } gpd_precision;
 
 typedef enum {

@@ -279,6 +279,7 @@ gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* output
                          uint64_t use_mask, const gpd_locate_result* result, float* out, float* act_out,
                          int activation, void* workspace, cudaStream_t st) {
     if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
+    if (plan->sliced && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward product only
     const ProductInfo& pi = plan->prod[which];
     if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
     gpd_status rc = ensure_device(plan);
@@ -359,7 +360,7 @@ __global__ void __launch_bounds__(256) regen_stream_kernel(RegenParams prm) {
 gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_result* result, void* workspace,
                              cudaStream_t st) {
     const ProductInfo& pi = plan->prod[GPD_AUDIT];
-    if (pi.Q == 0) return GPD_ERR_UNSUPPORTED;
+    if (pi.Q == 0 || plan->sliced) return GPD_ERR_UNSUPPORTED;
     gpd_status rc = ensure_device(plan);
     if (rc != GPD_OK) return rc;
     const WorkspaceLayout wl = workspace_layout();

@@ -3,6 +3,7 @@
 // and update encodings).  Bandwidth-bound: each source element is read once, all P shares of
 // that element are produced from registers and streamed out with 16-byte stores.
 #include "gpd_internal.h"
+#include "slice_common.h"
 
 namespace gpd {
 
@@ -128,6 +129,11 @@ gpd_status dispatch(const EncodeParams& prm, cudaStream_t st) {
 
 gpd_status encode_launch(gpd_plan_s* plan, int operand_or_A, const float* src, void* dst,
                          cudaStream_t st) {
+    if (plan->sliced) {
+        if (operand_or_A == -1) return encode_sliced_launch(plan, true, src, dst, st);
+        if (operand_or_A == GPD_OPERAND_X_FWD) return encode_sliced_launch(plan, false, src, dst, st);
+        return GPD_ERR_UNSUPPORTED;
+    }
     gpd_status rc = ensure_device(plan);
     if (rc != GPD_OK) return rc;
     const gpd_shape& s = plan->shape;

@@ -2,6 +2,7 @@
 // shape-agnostic CUDA-core kernels used for blocks the tensor-core paths do not take
 // (matrix-vector products, 5-row blocks, dimensions that break 16-byte alignment).
 #include "gemm_common.h"
+#include "slice_common.h"
 
 namespace gpd {
 
@@ -140,6 +141,8 @@ gpd_status worker_gemm_launch(gpd_plan_s* plan, gpd_product which, const void* W
                               void* out, cudaStream_t st) {
     const gpd_shape& s = plan->shape;
     const gpd_split& c = plan->split;
+    if (plan->sliced)
+        return which == GPD_FWD ? gemm_sliced_launch(plan, W_sh, other, out, st) : GPD_ERR_UNSUPPORTED;
     GemmParams prm{};
     prm.P = plan->P;
     prm.C = out;
@@ -165,6 +168,7 @@ gpd_status update_launch(gpd_plan_s* plan, void* W_sh, const void* Dhat, const v
                          float lambda, const gpd_locate_result* gate, cudaStream_t st) {
     const gpd_shape& s = plan->shape;
     const gpd_split& c = plan->split;
+    if (plan->sliced) return GPD_ERR_UNSUPPORTED;
     GemmParams prm{};
     prm.P = plan->P;
     prm.A = Dhat; prm.B = Xhat; prm.C = W_sh;
@@ -199,6 +203,7 @@ extern "C" gpd_status gpd_update_shares(gpd_plan_t plan, void* W_shares_dev, con
 extern "C" gpd_status gpd_device_status(int32_t* status_host) {
     if (!status_host) return GPD_ERR_ARG;
     if (cudaDeviceSynchronize() != cudaSuccess) return GPD_ERR_CUDA;
-    *status_host = tf32_device_status_fetch_and_clear();
+    const int a = tf32_device_status_fetch_and_clear(), b = i8_device_status_fetch_and_clear();
+    *status_host = a != 0 ? a : b;
     return GPD_OK;
 }

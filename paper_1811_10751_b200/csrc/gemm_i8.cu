@@ -1,0 +1,339 @@
+// FP64-class forward worker products (step O1) on the integer tensor cores.
+//
+// Both operands arrive cut into six signed 7-bit digit planes (slice.cu):
+//     W~_p[i][k] = 2^ea[i] * sum_s A_s[i][k] 128^-(s+1),   X~_p[k][j] = 2^eb[j] * sum_t B_t[j][k] 128^-(t+1).
+// A digit-plane product A_s B_t^T is an int8 x int8 -> int32 contraction, exact on the tensor
+// cores (|digit| <= 64, so K up to 87381 cannot overflow six summed pairs).  Pairs with
+// s + t <= 5 (weight >= 128^-7) are kept: 21 of 36, the rest lie below 2^-49 of the row/column
+// scales.  Pairs of equal weight share one accumulator, so a 128 x 64 output tile owns six
+// 128 x 64 int32 accumulators in tensor memory (384 of 512 columns), group g = s + t at columns
+// 64 g.  For a fixed s the planes t = 0 .. 5-s are adjacent in shared memory and their
+// accumulators are adjacent in tensor memory, so one tcgen05.mma of N = 64 (6 - s) columns
+// (two when that exceeds 256) covers all pairs of plane s: 8 instructions per 32 elements of K.
+//
+// Warp roles: warp 0 one lane issues the TMA copies (12 per 64-element k-block, 3-stage ring),
+// warp 1 allocates tensor memory and one lane issues the MMAs, warps 2..5 read the accumulators
+// back, combine them in FP64 (sum_g acc_g 2^-7g, then the row and column powers of two) and store.
+// Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains its copies,
+// frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "slice_common.h"
+
+namespace gpd {
+
+namespace {
+
+constexpr int BM = 128, BN = 64, BK = 64, STAGES = 3;
+constexpr int UMMA_K = 32;                            // int8 elements per MMA along K
+constexpr int A_PLANE_BYTES = BM * BK;                // 8 KB, rows of 64 B
+constexpr int B_PLANE_BYTES = BN * BK;                // 4 KB
+constexpr int STAGE_BYTES = kSlices * (A_PLANE_BYTES + B_PLANE_BYTES);   // 72 KB
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
+constexpr int TMEM_COLS = 512;                        // 6 x 64 used; allocations are powers of two
+constexpr int kEpiWarps = 4;
+constexpr int kThreads = 64 + kEpiWarps * 32;
+constexpr long long kWaitCycles = 2000000000LL;       // about one second
+
+__device__ int g_i8_status = 0;                       // GPD_ERR_TIMEOUT if a bounded wait expired
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicExch(&g_i8_status, (int)GPD_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+// K-major tile with rows of 64 bytes under the 64-byte swizzle: 8-row groups 512 bytes apart
+// (descriptor version 1, layout type 4).
+__device__ __forceinline__ uint64_t desc_sw64(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)(16 >> 4) << 16;
+    d |= (uint64_t)(512 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)4 << 61;
+    return d;
+}
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// instruction descriptor: int32 accumulator, signed 8-bit A and B, both K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t idesc_i8(int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+// 2^e as a double (0 below the normal range: only the all-zero marker gets there)
+__device__ __forceinline__ double exp2i(int e) {
+    if (e < -1022) return 0.0;
+    if (e > 1023) e = 1023;
+    return __longlong_as_double((long long)(e + 1023) << 52);
+}
+// int32 -> double without the conversion unit: 2^52 + 2^31 + x has x ^ 0x80000000 as its low word
+__device__ __forceinline__ double i2d(uint32_t x) {
+    return __hiloint2double(0x43300000, (int)(x ^ 0x80000000u)) - 4503601774854144.0;
+}
+
+struct I8Params {
+    const int* ea;     // [P][M]
+    const int* eb;     // [P][N]
+    double* C;         // [P][M][N]
+    int64_t M, N, K;
+    int P;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, I8Params prm,
+                      int tiles_m, int tiles_n) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ double col_scale[BN];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x;
+    const int tn = tile % tiles_n, tm = (tile / tiles_n) % tiles_m;
+    const int p = tile / (tiles_n * tiles_m);
+    const int m0 = tm * BM, n0 = tn * BN;
+    const int num_kb = (int)((prm.K + BK - 1) / BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(&acc_bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + BN) {
+        const int j = threadIdx.x - 64;
+        col_scale[j] = (n0 + j < prm.N) ? exp2i(prm.eb[(int64_t)p * prm.N + n0 + j]) : 0.0;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_slot;
+    volatile int* abort_p = &abort_flag;
+
+    auto A_plane = [&](int s, int t) { return smem + s * STAGE_BYTES + t * A_PLANE_BYTES; };
+    auto B_plane = [&](int s, int t) { return smem + s * STAGE_BYTES + kSlices * A_PLANE_BYTES + t * B_PLANE_BYTES; };
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) break;
+                mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+#pragma unroll
+                for (int t = 0; t < kSlices; ++t) {
+                    tma_load_3d(A_plane(s, t), &tmA, kb * BK, m0, t * prm.P + p, &full_bar[s]);
+                    tma_load_3d(B_plane(s, t), &tmB, kb * BK, n0, t * prm.P + p, &full_bar[s]);
+                }
+                ++issued;
+            }
+            if (*abort_p) {                      // let copies still in flight land before the CTA exits
+                for (int kb = issued > STAGES ? issued - STAGES : 0; kb < issued; ++kb) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&full_bar[kb % STAGES], (kb / STAGES) & 1) && clock64() - t0 < kWaitCycles) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; ++kb) {
+                const int s = kb % STAGES;
+                const uint32_t ph = (kb / STAGES) & 1;
+                if (!mbar_wait(&full_bar[s], ph, abort_p)) { ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a0 = smem_u32(A_plane(s, 0)), b0 = smem_u32(B_plane(s, 0));
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k) {
+#pragma unroll
+                    for (int ta = 0; ta < kSlices; ++ta) {
+                        // planes tb = 0 .. 5-ta of B in one operand of 64 (6 - ta) rows, at most 256 per MMA;
+                        // the pair (ta, tb) lands in accumulator group ta + tb = columns 64 (ta + tb)
+                        const uint64_t da = desc_sw64(a0 + ta * A_PLANE_BYTES + k * UMMA_K);
+                        const int n_total = BN * (kSlices - ta);
+                        const int n_first = n_total > 256 ? 256 : n_total;
+                        // the plane-0 instruction of the first k-step overwrites all six groups
+                        const uint32_t acc = (kb > 0 || k > 0 || ta > 0) ? 1u : 0u;
+                        umma_i8(tmem_base + BN * ta, da, desc_sw64(b0 + k * UMMA_K), idesc_i8(n_first), acc);
+                        if (n_total > 256)
+                            umma_i8(tmem_base + BN * ta + 256, da, desc_sw64(b0 + 4 * B_PLANE_BYTES + k * UMMA_K),
+                                    idesc_i8(n_total - 256), acc);
+                    }
+                }
+                umma_commit(&empty_bar[s]);          // stage reusable once these MMAs have read it
+            }
+            if (ok) umma_commit(&acc_bar);           // accumulators complete
+        }
+    } else {
+        // ------------------------------ epilogue ------------------------------
+        const bool acc_ready = mbar_wait(&acc_bar, 0, abort_p);
+        __syncwarp();
+        if (__all_sync(0xffffffffu, acc_ready)) {    // tcgen05.ld is warp-collective: all lanes or none
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int q = warp & 3;                  // this warp may touch TMEM lanes 32q .. 32q+31
+            const int64_t gm = (int64_t)m0 + q * 32 + lane;
+            const double row_scale = gm < prm.M ? exp2i(prm.ea[(int64_t)p * prm.M + gm] - 2 * kDigitBits) : 0.0;
+            double* C = prm.C + (int64_t)p * prm.M * prm.N;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                double v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = 0.0;
+#pragma unroll
+                for (int g = kSlices - 1; g >= 0; --g) {             // smallest weight first
+                    uint32_t r[32];
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(BN * g + c0);
+                    asm volatile(
+                        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                        : "r"(taddr));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    const double w = exp2i(-kDigitBits * g);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = fma(i2d(r[j]), w, v[j]);
+                }
+                if (gm < prm.M) {
+                    double* crow = C + gm * prm.N + n0 + c0;
+                    if ((prm.N & 1) == 0 && n0 + c0 + 32 <= prm.N) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            double2 o;
+                            o.x = v[j] * row_scale * col_scale[c0 + j];
+                            o.y = v[j + 1] * row_scale * col_scale[c0 + j + 1];
+                            __stcs(reinterpret_cast<double2*>(crow + j), o);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (n0 + c0 + j < prm.N) crow[j] = v[j] * row_scale * col_scale[c0 + j];
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 3-D byte tensor [batch][rows][K] (K contiguous), box {BK, box_rows, 1}, 64-byte swizzle,
+// out-of-range elements read as zero.
+bool make_map(CUtensorMap* map, const void* base, int64_t batch, int64_t rows, int64_t K, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t strides[2] = {(cuuint64_t)K, (cuuint64_t)rows * (cuuint64_t)K};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+gpd_status gemm_sliced_launch(gpd_plan_s* plan, const void* W_sliced, const void* X_sliced, void* out,
+                              cudaStream_t st) {
+    const gpd_shape& s = plan->shape;
+    const gpd_split& c = plan->split;
+    I8Params prm{};
+    prm.P = plan->P;
+    prm.M = s.N1 / c.m; prm.K = s.N0 / c.n; prm.N = s.B / c.d1;
+    const SlicedLayout la = sliced_layout(prm.P, prm.M, prm.K), lb = sliced_layout(prm.P, prm.N, prm.K);
+    prm.ea = reinterpret_cast<const int*>(reinterpret_cast<const char*>(W_sliced) + la.expo_offset);
+    prm.eb = reinterpret_cast<const int*>(reinterpret_cast<const char*>(X_sliced) + lb.expo_offset);
+    prm.C = reinterpret_cast<double*>(out);
+    if (reinterpret_cast<uintptr_t>(W_sliced) % 16 || reinterpret_cast<uintptr_t>(X_sliced) % 16 ||
+        reinterpret_cast<uintptr_t>(out) % 16)
+        return GPD_ERR_ARG;
+    CUtensorMap tmA, tmB;
+    if (!make_map(&tmA, W_sliced, (int64_t)kSlices * prm.P, prm.M, prm.K, BM)) return GPD_ERR_CUDA;
+    if (!make_map(&tmB, X_sliced, (int64_t)kSlices * prm.P, prm.N, prm.K, BN)) return GPD_ERR_CUDA;
+    if (cudaFuncSetAttribute(gemm_i8_sliced_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+        return GPD_ERR_CUDA;
+    const int tiles_n = (int)((prm.N + BN - 1) / BN), tiles_m = (int)((prm.M + BM - 1) / BM);
+    const int64_t tiles = (int64_t)tiles_n * tiles_m * prm.P;
+    gemm_i8_sliced_kernel<<<(unsigned)tiles, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n);
+    return launch_ok();
+}
+
+int i8_device_status_fetch_and_clear() {
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_i8_status, sizeof(int)) != cudaSuccess) return (int)GPD_ERR_CUDA;
+    if (v != 0) cudaMemcpyToSymbol(g_i8_status, &zero, sizeof(int));
+    return v;
+}
+
+}  // namespace gpd

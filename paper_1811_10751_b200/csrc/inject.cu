@@ -130,6 +130,7 @@ gpd_status inject_launch(gpd_plan_s* plan, gpd_product which, void* outputs, uin
                          double prob, uint64_t node_mask, int count, double scale, uint64_t* hit_mask,
                          cudaStream_t st) {
     if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
+    if (plan->sliced && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward product only
     const ProductInfo& pi = plan->prod[which];
     if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
     InjectParams prm{};

@@ -5,6 +5,7 @@
 #include <new>
 
 #include "gpd_internal.h"
+#include "slice_common.h"
 
 namespace gpd {
 
@@ -151,7 +152,8 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
     *out = nullptr;
     if (subst != GPD_SUBST_U_EQ_VN && subst != GPD_SUBST_V_EQ_UM) return GPD_ERR_ARG;
     const bool alt = subst == GPD_SUBST_V_EQ_UM;
-    if (precision != GPD_PREC_AUTO && precision != GPD_PREC_FP32 && precision != GPD_PREC_FP64)
+    if (precision != GPD_PREC_AUTO && precision != GPD_PREC_FP32 && precision != GPD_PREC_FP64 &&
+        precision != GPD_PREC_FP64_SLICED)
         return GPD_ERR_ARG;
     const int m = split->m, n = split->n, d1 = split->d1, d2 = split->d2;
     if (shape->N1 <= 0 || shape->N0 <= 0 || shape->B <= 0 || m <= 0 || n <= 0 || d1 <= 0 || d2 <= 0)
@@ -195,6 +197,7 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
     plan->elem_size = plan->prec == GPD_PREC_FP32 ? 4 : 8;
     plan->tau_col = plan->prec == GPD_PREC_FP32 ? kTauColFp32 : kTauColFp64;
     plan->tau_in = plan->prec == GPD_PREC_FP32 ? kTauInFp32 : kTauInFp64;
+    plan->sliced = plan->prec == GPD_PREC_FP64_SLICED;
 
     // powers up to the largest exponent used by any encoding
     const int max_exp = (int)std::max<int64_t>(std::max(Qf, Qb), Qw) + 1;
@@ -245,6 +248,7 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
             for (int j = 0; j < n; ++j) a.wanted[i * n + j] = alt ? i + m * j : n * i + j;
         a.H = left_null_space(plan->points, a.Q);
     }
+    if (plan->sliced && !sliced_supported(plan)) { delete plan; return GPD_ERR_UNSUPPORTED; }
     *out = plan;
     return GPD_OK;
 }

@@ -1,0 +1,338 @@
+// Encoding for the integer-slice product path (GPD_PREC_FP64_SLICED).
+//
+// The shares W~_p (Eq. 1) and X~_p (Theorem 2) are evaluated in FP64 exactly as in encode.cu, but
+// instead of being stored as doubles each value a is stored as six signed 7-bit digits:
+//     a = 2^e * sum_{t=1..6} q_t * 128^-t  (+ remainder below 2^(e-43)),   q_t in [-64, 64],
+// with one exponent e per row of W~_p (per column of X~_p) chosen so that |a| < 2^(e-1).  The
+// digits of one operand form six int8 planes; products of planes are exact in int32 on the tensor
+// cores (gemm_i8.cu), which gives FP64-class worker products at integer-tensor-core speed.
+// Both operands are written K-major: W planes [6][P][M][K], X planes [6][P][N][K] (transposed).
+// Layout of a sliced share buffer: planes, then the int32 exponents (256-byte aligned).
+#include <cmath>
+
+#include "gpd_internal.h"
+#include "slice_common.h"
+
+namespace gpd {
+
+namespace {
+
+struct SliceParams {
+    const float* src;      // source matrix, row-major, leading dimension ld
+    const double* coef;    // [P][nblk]
+    int8_t* planes;        // [kSlices][P][R][K]   (R = rows of the K-major operand)
+    int* expo;             // [P][R]
+    unsigned int* amax;    // [P][R] scratch of the X side: largest |value| per operand row (high word)
+    int64_t ld;            // leading dimension of src
+    int64_t br, bc;        // block rows / cols of src
+    int gc, nblk, P;
+};
+
+// Largest magnitudes are tracked as the high 32 bits of |a| (non-negative doubles order like
+// their bit patterns); hi + 1 with a zero low word is an upper bound within 2^-20 relative.
+__device__ __forceinline__ unsigned int abs_hi(double a) { return (unsigned int)__double2hiint(a) & 0x7FFFFFFFu; }
+__device__ __forceinline__ unsigned int abs_hi_max4(const double (&a)[4]) {
+    return max(max(abs_hi(a[0]), abs_hi(a[1])), max(abs_hi(a[2]), abs_hi(a[3])));
+}
+
+// Exponent e such that every |a| <= amax has |a| 2^-e < 0.4923, which keeps the biased fixed-point
+// value of digits4() inside 42 bits; amax is given by its high word as above.  Magnitudes below
+// 2^-900 (and non-finite ones) get the marker -1000: all digits zero.
+__device__ __forceinline__ int slice_exponent(unsigned int amax_hi) {
+    if (amax_hi < 0x07B00000u || amax_hi >= 0x7FF00000u) return -1000;
+    const double amax = __hiloint2double((int)(amax_hi + 1u), 0);
+    int x;
+    frexp(amax * 1.015625, &x);   // amax (1 + 1/64) = f 2^x, f in [0.5, 1)
+    return x + 1;
+}
+// 2^(42 - e) as a double, 0 for the all-zero marker
+__device__ __forceinline__ double slice_scale(int e) {
+    if (e <= -1000) return 0.0;
+    return __longlong_as_double((long long)(42 - e + 1023) << 52);
+}
+
+// Digits of four values at once.  U = rint(a 2^(42-e)) + sum_i 64 * 128^i lies in [0, 2^42); its
+// 7-bit fields minus 64 are the digits (each in [-64, 63]), most significant first.  U is read
+// from the mantissa of a 2^(42-e) + 2^52 + bias (one FMA); the fields of the four values are
+// gathered bytewise; word[t] holds digit t of values 0..3 in bytes 0..3.
+__device__ __forceinline__ void digits4(const double (&a)[4], double scale, unsigned int (&word)[kSlices]) {
+    const double magic = 4503599627370496.0 + 2216338399296.0;   // 2^52 + 64 (128^6 - 1) / 127
+    unsigned int lo[4], hi[4];
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+        const double t = fma(scale != 0.0 ? a[v] : 0.0, scale, magic);
+        lo[v] = (unsigned int)__double2loint(t);
+        hi[v] = (unsigned int)__double2hiint(t);
+    }
+#pragma unroll
+    for (int t = 0; t < kSlices; ++t) {
+        unsigned int x[4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int bit = kDigitBits * (kSlices - 1 - t);              // position of digit t in U
+            x[v] = bit == 0 ? lo[v] : bit < 28 ? lo[v] >> bit : bit == 28 ? __funnelshift_r(lo[v], hi[v], 28) : hi[v] >> (bit - 32);
+        }
+        const unsigned int p01 = __byte_perm(x[0], x[1], 0x0040), p23 = __byte_perm(x[2], x[3], 0x0040);
+        const unsigned int u = __byte_perm(p01, p23, 0x5410) & 0x7F7F7F7Fu;
+        word[t] = (u + 0x40404040u) ^ 0x80808080u;                        // bytewise u - 64
+    }
+}
+
+// ---- W side: operand rows are rows of the share (K = block columns, contiguous in the source) ----
+// Pass 1: one CTA per share row r; an upper bound of max_c |W~_p[r][c]| for every p.  The share
+// values are evaluated in FP32 here (they only fix a power-of-two scale); the bound adds the
+// worst-case FP32 evaluation error (NBLK + 1) 2^-23 sum_b |coef_pb| max_c |W_b[r][c]|.
+template <int NBLK>
+__global__ void __launch_bounds__(256) rowmax_kernel(SliceParams prm) {
+    __shared__ unsigned int sMax[kMaxNodes];     // bit patterns of non-negative floats order like integers
+    __shared__ unsigned int sBlk[NBLK];
+    extern __shared__ double s_coef[];           // [P][NBLK]
+    float* s_cf32 = reinterpret_cast<float*>(s_coef + prm.P * NBLK);
+    for (int i = threadIdx.x; i < prm.P * NBLK; i += 256) {
+        const double c = prm.coef[i];
+        s_coef[i] = c;
+        s_cf32[i] = (float)c;
+    }
+    if (threadIdx.x < kMaxNodes) sMax[threadIdx.x] = 0u;
+    if (threadIdx.x < NBLK) sBlk[threadIdx.x] = 0u;
+    __syncthreads();
+    const int64_t r = blockIdx.x;
+    const int lane = threadIdx.x & 31;
+    // every lane of a warp runs the same number of rounds (the warp reductions need all 32)
+    for (int64_t c0 = 0; c0 < prm.bc; c0 += 1024) {
+        const int64_t c = c0 + (int64_t)threadIdx.x * 4;
+        float4 x[NBLK];
+#pragma unroll
+        for (int b = 0; b < NBLK; ++b) {
+            const int gi = b / prm.gc, gj = b - gi * prm.gc;
+            x[b] = c < prm.bc ? __ldg(reinterpret_cast<const float4*>(prm.src + (gi * prm.br + r) * prm.ld + gj * prm.bc + c))
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int b = 0; b < NBLK; ++b) {
+            const unsigned int m = max(max(__float_as_uint(fabsf(x[b].x)), __float_as_uint(fabsf(x[b].y))),
+                                       max(__float_as_uint(fabsf(x[b].z)), __float_as_uint(fabsf(x[b].w))));
+            const unsigned int w = __reduce_max_sync(0xffffffffu, m);
+            if (lane == 0) atomicMax(&sBlk[b], w);
+        }
+#pragma unroll 2
+        for (int p = 0; p < prm.P; ++p) {
+            const float* cf = s_cf32 + p * NBLK;
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+            for (int b = 0; b < NBLK; ++b) {
+                const float k = cf[b];
+                a0 = fmaf(k, x[b].x, a0); a1 = fmaf(k, x[b].y, a1);
+                a2 = fmaf(k, x[b].z, a2); a3 = fmaf(k, x[b].w, a3);
+            }
+            const unsigned int m = max(max(__float_as_uint(fabsf(a0)), __float_as_uint(fabsf(a1))),
+                                       max(__float_as_uint(fabsf(a2)), __float_as_uint(fabsf(a3))));
+            const unsigned int w = __reduce_max_sync(0xffffffffu, m);
+            if (lane == 0) atomicMax(&sMax[p], w);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < prm.P) {
+        const int p = threadIdx.x;
+        double spread = 0.0;
+        for (int b = 0; b < NBLK; ++b) spread += fabs(s_coef[p * NBLK + b]) * (double)__uint_as_float(sBlk[b]);
+        const double bound = (double)__uint_as_float(sMax[p]) + (NBLK + 1) * 1.1920928955078125e-7 * spread;
+        prm.expo[(int64_t)p * prm.br + r] = slice_exponent(abs_hi(bound));
+    }
+}
+
+// Pass 2: one thread per 4 consecutive columns of a share row: recompute the share values, cut
+// them into digits with the row's exponent, store 4 digits (one 32-bit word) per plane.
+template <int NBLK>
+__global__ void __launch_bounds__(256) rowslice_kernel(SliceParams prm) {
+    extern __shared__ double s_coef[];
+    for (int i = threadIdx.x; i < prm.P * NBLK; i += 256) s_coef[i] = prm.coef[i];
+    __syncthreads();
+    const int64_t bc4 = prm.bc >> 2, total = prm.br * bc4;
+    const int64_t plane_stride = (int64_t)prm.P * prm.br * prm.bc;
+    for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < total; t += (int64_t)gridDim.x * 256) {
+        const int64_t r = t / bc4, c = (t - r * bc4) << 2;
+        double x[NBLK][4];                       // converted once, used by every node
+#pragma unroll
+        for (int b = 0; b < NBLK; ++b) {
+            const int gi = b / prm.gc, gj = b - gi * prm.gc;
+            const float4 v = __ldg(reinterpret_cast<const float4*>(prm.src + (gi * prm.br + r) * prm.ld + gj * prm.bc + c));
+            x[b][0] = v.x; x[b][1] = v.y; x[b][2] = v.z; x[b][3] = v.w;
+        }
+#pragma unroll 2
+        for (int p = 0; p < prm.P; ++p) {
+            const double* cf = s_coef + p * NBLK;
+            double a[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int b = 0; b < NBLK; ++b) {
+                const double k = cf[b];
+                a[0] = fma(k, x[b][0], a[0]); a[1] = fma(k, x[b][1], a[1]);
+                a[2] = fma(k, x[b][2], a[2]); a[3] = fma(k, x[b][3], a[3]);
+            }
+            unsigned int word[kSlices];
+            digits4(a, slice_scale(__ldg(prm.expo + (int64_t)p * prm.br + r)), word);
+            int8_t* dst = prm.planes + ((int64_t)p * prm.br + r) * prm.bc + c;
+#pragma unroll
+            for (int s = 0; s < kSlices; ++s)
+                __stcs(reinterpret_cast<unsigned int*>(dst + s * plane_stride), word[s]);
+        }
+    }
+}
+
+// ---- X side: operand rows are columns of the share (K = block rows, strided in the source) ----
+// A CTA stages the source values of a tile (128 rows kk x 8 columns n of every block) in shared
+// memory, transposed, so that a thread owns 4 consecutive kk of one column (warp = column,
+// lane = kk / 4): it converts its values once and runs over the nodes.
+//   SLICE = false: largest |X~_p[kk][n]| over kk, met in amax[p][n] (high words, zeroed before the launch)
+//   SLICE = true : digits with the column's exponent, written K-major (128 bytes per warp and plane);
+//                  the CTAs of the first row slab also publish the exponents.
+constexpr int XT_K = 128, XT_N = 8, XT_PITCH = XT_K + 4;
+
+template <int NBLK, bool SLICE>
+__global__ void __launch_bounds__(256) colpass_kernel(SliceParams prm) {
+    extern __shared__ double s_coef[];                             // [P][NBLK], then the tile
+    float* xs = reinterpret_cast<float*>(s_coef + prm.P * NBLK);   // [NBLK][XT_N][XT_PITCH]
+    for (int i = threadIdx.x; i < prm.P * NBLK; i += 256) s_coef[i] = prm.coef[i];
+    const int64_t n0 = (int64_t)blockIdx.x * XT_N, k0 = (int64_t)blockIdx.y * XT_K;
+    {   // stage the tile: thread = (column nn, rows kq + 32 j); all loads issued before the stores
+        const int nn = threadIdx.x % XT_N, kq = threadIdx.x / XT_N;
+        const int64_t gn = n0 + nn;
+        float v[NBLK][XT_K / 32];
+#pragma unroll
+        for (int b = 0; b < NBLK; ++b) {
+            const int gi = b / prm.gc, gj = b - gi * prm.gc;
+#pragma unroll
+            for (int j = 0; j < XT_K / 32; ++j) {
+                const int64_t gk = k0 + kq + 32 * j;
+                v[b][j] = (gk < prm.br && gn < prm.bc) ? __ldg(prm.src + (gi * prm.br + gk) * prm.ld + gj * prm.bc + gn) : 0.f;
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < NBLK; ++b)
+#pragma unroll
+            for (int j = 0; j < XT_K / 32; ++j) xs[(b * XT_N + nn) * XT_PITCH + kq + 32 * j] = v[b][j];
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t gn = n0 + warp, gk = k0 + 4 * lane;
+    if (gn >= prm.bc) return;                                      // whole warp
+    double x[NBLK][4];
+#pragma unroll
+    for (int b = 0; b < NBLK; ++b) {
+        const float4 v = *reinterpret_cast<const float4*>(xs + (b * XT_N + warp) * XT_PITCH + 4 * lane);
+        x[b][0] = v.x; x[b][1] = v.y; x[b][2] = v.z; x[b][3] = v.w;
+    }
+    const int64_t plane_stride = (int64_t)prm.P * prm.bc * prm.br;
+#pragma unroll 2
+    for (int p = 0; p < prm.P; ++p) {
+        const double* cf = s_coef + p * NBLK;
+        double a[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int b = 0; b < NBLK; ++b) {
+            const double k = cf[b];
+            a[0] = fma(k, x[b][0], a[0]); a[1] = fma(k, x[b][1], a[1]);
+            a[2] = fma(k, x[b][2], a[2]); a[3] = fma(k, x[b][3], a[3]);
+        }
+        if (!SLICE) {
+            const unsigned int mx = __reduce_max_sync(0xffffffffu, abs_hi_max4(a));
+            if (lane == 0) atomicMax(prm.amax + (int64_t)p * prm.bc + gn, mx);
+        } else {
+            const int e = slice_exponent(prm.amax[(int64_t)p * prm.bc + gn]);
+            if (blockIdx.y == 0 && lane == 0) prm.expo[(int64_t)p * prm.bc + gn] = e;
+            unsigned int word[kSlices];
+            digits4(a, slice_scale(e), word);
+            if (gk < prm.br) {                                     // br is a multiple of 16: whole words
+                int8_t* dst = prm.planes + ((int64_t)p * prm.bc + gn) * prm.br + gk;
+#pragma unroll
+                for (int s = 0; s < kSlices; ++s) *reinterpret_cast<unsigned int*>(dst + s * plane_stride) = word[s];
+            }
+        }
+    }
+}
+
+template <int NBLK>
+gpd_status launch_rows(const SliceParams& prm, cudaStream_t st) {
+    const size_t smem = sizeof(double) * prm.P * NBLK;
+    rowmax_kernel<NBLK><<<(unsigned)prm.br, 256, smem + sizeof(float) * prm.P * NBLK, st>>>(prm);
+    if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+    const int64_t work = prm.br * (prm.bc / 4);
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, 148 * 16));
+    rowslice_kernel<NBLK><<<grid, 256, smem, st>>>(prm);
+    return launch_ok();
+}
+
+template <int NBLK>
+gpd_status launch_cols(const SliceParams& prm, cudaStream_t st) {
+    if (cudaMemsetAsync(prm.amax, 0, sizeof(unsigned int) * prm.P * prm.bc, st) != cudaSuccess) return GPD_ERR_CUDA;
+    const size_t smem = sizeof(double) * prm.P * NBLK + sizeof(float) * NBLK * XT_N * XT_PITCH;
+    if (smem > 48 * 1024 &&
+        (cudaFuncSetAttribute(colpass_kernel<NBLK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+         cudaFuncSetAttribute(colpass_kernel<NBLK, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess))
+        return GPD_ERR_CUDA;
+    dim3 grid((unsigned)((prm.bc + XT_N - 1) / XT_N), (unsigned)((prm.br + XT_K - 1) / XT_K));
+    colpass_kernel<NBLK, false><<<grid, 256, smem, st>>>(prm);
+    if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+    colpass_kernel<NBLK, true><<<grid, 256, smem, st>>>(prm);
+    return launch_ok();
+}
+
+}  // namespace
+
+bool sliced_supported(const gpd_plan_s* plan) {
+    const gpd_shape& s = plan->shape;
+    const gpd_split& c = plan->split;
+    const int64_t K = s.N0 / c.n;
+    const int64_t M = s.N1 / c.m, N = s.B / c.d1;
+    const int nb_w = c.m * c.n, nb_x = c.n * c.d1;
+    auto ok_blk = [](int n) {
+        return n == 1 || n == 2 || n == 3 || n == 4 || n == 6 || n == 8 || n == 9 || n == 12 || n == 16;
+    };
+    if (K % 16 != 0 || !ok_blk(nb_w) || !ok_blk(nb_x)) return false;
+    // the scale pass evaluates the shares in FP32: the encoding coefficients must fit comfortably
+    for (double c : plan->coefW) if (!(std::fabs(c) < 1e30)) return false;
+    for (double c : plan->coefX) if (!(std::fabs(c) < 1e30)) return false;
+    // the sliced operands live in buffers sized for the FP64 shares they replace
+    return sliced_layout(plan->P, M, K).total_bytes <= 8 * (int64_t)plan->P * M * K &&
+           sliced_layout(plan->P, N, K).total_bytes <= 8 * (int64_t)plan->P * N * K;
+}
+
+SlicedLayout sliced_layout(int64_t P, int64_t rows, int64_t K) {
+    SlicedLayout l;
+    l.plane_bytes = P * rows * K;
+    l.expo_offset = (kSlices * l.plane_bytes + 255) / 256 * 256;
+    l.amax_offset = (l.expo_offset + P * rows * 4 + 255) / 256 * 256;
+    l.total_bytes = l.amax_offset + P * rows * 4;
+    return l;
+}
+
+gpd_status encode_sliced_launch(gpd_plan_s* plan, bool is_A, const float* src, void* dst, cudaStream_t st) {
+    gpd_status rc = ensure_device(plan);
+    if (rc != GPD_OK) return rc;
+    const gpd_shape& s = plan->shape;
+    const gpd_split& c = plan->split;
+    SliceParams prm{};
+    prm.src = src;
+    prm.P = plan->P;
+    int gr;
+    if (is_A) {                   // W: m x n blocks of (N1/m) x (N0/n); operand rows = share rows, K = N0/n
+        gr = c.m; prm.gc = c.n; prm.ld = s.N0; prm.br = s.N1 / c.m; prm.bc = s.N0 / c.n;
+        prm.coef = plan->dev.base + plan->dev.off_coefW;
+    } else {                      // X: n x d1 blocks of (N0/n) x (B/d1); operand rows = share columns, K = N0/n
+        gr = c.n; prm.gc = c.d1; prm.ld = s.B; prm.br = s.N0 / c.n; prm.bc = s.B / c.d1;
+        prm.coef = plan->dev.base + plan->dev.off_coefX;
+    }
+    prm.nblk = gr * prm.gc;
+    const SlicedLayout lay = is_A ? sliced_layout(plan->P, prm.br, prm.bc) : sliced_layout(plan->P, prm.bc, prm.br);
+    prm.planes = reinterpret_cast<int8_t*>(dst);
+    prm.expo = reinterpret_cast<int*>(reinterpret_cast<char*>(dst) + lay.expo_offset);
+    prm.amax = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(dst) + lay.amax_offset);
+#define GPD_SLICE_CASE(NB) case NB: return is_A ? launch_rows<NB>(prm, st) : launch_cols<NB>(prm, st)
+    switch (prm.nblk) {
+        GPD_SLICE_CASE(1); GPD_SLICE_CASE(2); GPD_SLICE_CASE(3); GPD_SLICE_CASE(4); GPD_SLICE_CASE(6);
+        GPD_SLICE_CASE(8); GPD_SLICE_CASE(9); GPD_SLICE_CASE(12); GPD_SLICE_CASE(16);
+        default: return GPD_ERR_UNSUPPORTED;
+    }
+#undef GPD_SLICE_CASE
+}
+
+}  // namespace gpd

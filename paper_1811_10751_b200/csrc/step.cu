@@ -24,6 +24,7 @@ extern "C" gpd_status coded_layer_step(gpd_plan_t plan, int32_t phases, void* W_
     if ((phases & ~(GPD_PHASE_FWD | GPD_PHASE_BWD | GPD_PHASE_UPD | GPD_PHASE_REGEN | GPD_PHASE_INJECT_SHARES)) ||
         !(phases & (GPD_PHASE_FWD | GPD_PHASE_BWD | GPD_PHASE_UPD)))
         return GPD_ERR_ARG;
+    if (plan->sliced && phases != GPD_PHASE_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward only
     cudaStream_t st = as_stream(stream);
     const gpd_shape& s = plan->shape;
     const gpd_split& c = plan->split;

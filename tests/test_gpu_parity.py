@@ -222,10 +222,10 @@ def test_config2_matvec_two_bitflips():
 # --------------------------------------------------------------------------------------------------
 # config 3 at reduced size: additive errors on random nodes, several seeds, failure included
 # --------------------------------------------------------------------------------------------------
-def _run_additive_case(cfg, seeds, check_against_full_oracle=True):
+def _run_additive_case(cfg, seeds, precision=g.GPD_PREC_AUTO):
     W, X = wl.matmul_inputs(cfg)
     code = make_code(cfg)
-    cp = CodedProduct(code)
+    cp = CodedProduct(code, precision=precision)
     assert cp.np_dtype == np.float64
     cp.encode_W(W)
     Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
@@ -253,9 +253,10 @@ def _run_additive_case(cfg, seeds, check_against_full_oracle=True):
     return outcomes
 
 
-def test_config3_scaled_additive_errors():
+@pytest.mark.parametrize("precision", [g.GPD_PREC_AUTO, g.GPD_PREC_FP64_SLICED])
+def test_config3_scaled_additive_errors(precision):
     cfg = wl.scaled_down(wl.CONFIG_3_MATMUL, 8)                         # 1024 x 1024 x 64, same code
-    outcomes = _run_additive_case(cfg, cfg.inject_seeds)
+    outcomes = _run_additive_case(cfg, cfg.inject_seeds, precision)
     assert CORRECTED in outcomes
 
 
@@ -401,7 +402,8 @@ def test_config4_full_size_layer():
 # (tests/golden/cfg3_full_expected.json, written by make_cfg3_expected.py from oracle/ alone),
 # sampled worker outputs and sampled rows of the decoded product against FP64 definitions
 # --------------------------------------------------------------------------------------------------
-def test_config3_full_size_against_oracle_decisions():
+@pytest.mark.parametrize("precision", [g.GPD_PREC_AUTO, g.GPD_PREC_FP64_SLICED])
+def test_config3_full_size_against_oracle_decisions(precision):
     import json
     import os
     gold = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "cfg3_full_expected.json")))
@@ -409,7 +411,7 @@ def test_config3_full_size_against_oracle_decisions():
     assert gold["config"] == cfg.name
     W, X = wl.matmul_inputs(cfg)
     code = make_code(cfg)
-    cp = CodedProduct(code)
+    cp = CodedProduct(code, precision=precision)
     assert cp.np_dtype == np.float64
     cp.encode_W(W)
     Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
@@ -417,7 +419,12 @@ def test_config3_full_size_against_oracle_decisions():
     pos = np.array(gold["sample_positions"])
     got = host(Z.reshape(cfg.P, L)[:, torch.from_numpy(pos).cuda()])
     want = np.array(gold["clean_outputs_at_samples"])
-    assert np.abs(got - want).max() <= 1e-12 * gold["scale"] * 8          # FP64 products, K = 2048
+    if precision == g.GPD_PREC_FP64_SLICED:
+        # digit planes: < 4e-13 of (row scale x column scale) per term, sqrt(K) = 45 terms deep, scales
+        # within 4.07 x 4.5 standard deviations of each operand (the bound is derived in test_gpu_sliced.py)
+        assert np.abs(got - want).max() <= 2e-9 * gold["scale"]
+    else:
+        assert np.abs(got - want).max() <= 1e-12 * gold["scale"] * 8      # FP64 products, K = 2048
     rows = np.arange(0, cfg.N1, cfg.N1 // 32)
     ref_rows = op.ref_forward(W[rows], X)
     for seed in cfg.inject_seeds:

@@ -1,0 +1,180 @@
+"""GPU parity of the integer-slice product path (GPD_PREC_FP64_SLICED) against the FP64 oracle.
+
+The shares are stored as six signed 7-bit digits per value under one power-of-two scale 2^e per
+operand row, chosen so that 2^e lies in (2.03, 4.07] times the row's largest magnitude.  Digit-plane
+products are exact, so a worker output differs from the exact product of the FP64 shares only by
+(i) the digits cut below 2^-43 of each scale and (ii) the 15 plane pairs of weight below 128^-7 that
+are not formed: per term of the contraction at most 2^-43 + 4096 * 5.03 * 128^-8 < 4e-13 of
+2^ea 2^eb.  The tests allow 6 sqrt(K) times that (signs of the per-term errors are independent),
+which a single missing plane pair of the kept set would exceed by an order of magnitude.
+"""
+
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+if not torch.cuda.is_available():
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+import paper_1811_10751_b200 as g                        # noqa: E402
+from oracle import product as op                         # noqa: E402
+from oracle.code import GPCode, FWD                      # noqa: E402
+from oracle.locate import NO_ERROR, CORRECTED, locate_subspace, tolerances_for   # noqa: E402
+from oracle import inject as oinj                        # noqa: E402
+from tests.gpu_pipeline import CodedProduct, dev, host   # noqa: E402
+
+PER_TERM = 4e-13
+SCALE_OVER_MAX = 4.07
+
+
+def _inputs(N1, N0, B, seed, w_scale=1.0, x_scale=1.0):
+    rng = np.random.default_rng(seed)
+    W = (rng.standard_normal((N1, N0)) / np.sqrt(N0) * w_scale).astype(np.float32)
+    X = (rng.standard_normal((N0, B)) * x_scale).astype(np.float32)
+    return W, X
+
+
+def _output_tolerance(Wsh, Xsh):
+    """Per-entry bound [P][M][N] from the oracle's FP64 shares (see the module docstring)."""
+    K = Wsh.shape[2]
+    row = SCALE_OVER_MAX * np.abs(Wsh).max(axis=2)         # [P][M]  >= 2^ea
+    col = SCALE_OVER_MAX * np.abs(Xsh).max(axis=1)         # [P][N]  >= 2^eb
+    return 6.0 * np.sqrt(K) * PER_TERM * row[:, :, None] * col[:, None, :]
+
+
+def _sliced_products(code, W, X):
+    cp = CodedProduct(code, precision=g.GPD_PREC_FP64_SLICED)
+    assert cp.plan.query(g.GPD_Q_PRECISION) == g.GPD_PREC_FP64_SLICED and cp.np_dtype == np.float64
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    assert g.gpd_device_status() == 0
+    return cp, Z
+
+
+@pytest.mark.parametrize("N1,N0,B,m,n,d1,P", [
+    (256, 256, 128, 2, 4, 2, 25),       # whole tiles
+    (400, 320, 144, 2, 4, 2, 25),       # ragged rows (200 = 128 + 72) and columns (72 = 64 + 8), K = 80
+    (384, 96, 66, 3, 2, 2, 20),         # 6 blocks per share of W, K = 48 (one partly filled k-block), odd column count
+    (130, 16, 4, 1, 1, 1, 4),           # K = 16, single block, two columns
+    (1024, 2048, 128, 2, 2, 1, 9),      # K = 1024: sixteen k-blocks, ring wraps five times
+    (512, 768, 96, 4, 4, 1, 40),        # 16 blocks per share of W, 40 nodes, threshold 19
+    (256, 256, 96, 2, 4, 3, 30),        # 12 blocks per share of X, threshold 27
+])
+def test_sliced_worker_products_match_oracle(N1, N0, B, m, n, d1, P):
+    W, X = _inputs(N1, N0, B, seed=N1 + N0 + B)
+    code = GPCode(N1, N0, B, m, n, d1, 1, P)
+    cp, Z = _sliced_products(code, W, X)
+    Wsh, Xsh = op.encode_W(W, code), op.encode_X(X, code)
+    Zo = op.worker_products(Wsh, Xsh)
+    got = cp.outputs_as_array(g.GPD_FWD, Z)
+    assert np.isfinite(got).all()
+    tol = _output_tolerance(Wsh, Xsh)
+    assert (np.abs(got - Zo) <= tol).all(), float((np.abs(got - Zo) / tol).max())
+    # and the bound is far below what FP32 shares could give: relative to the output scale
+    assert np.abs(got - Zo).max() < 1e-8 * np.sqrt(np.mean(Zo ** 2))
+
+
+def test_sliced_scales_zero_rows_and_tiny_values():
+    """Row / column scales: rows of zeros, columns of zeros and operands 1e-30 and 1e+20 times the
+    usual size decode to the same relative accuracy (the digits carry no absolute scale)."""
+    N1, N0, B, m, n, d1, P = 256, 128, 96, 2, 2, 2, 12
+    W, X = _inputs(N1, N0, B, seed=5, w_scale=1e-30, x_scale=1e20)
+    W[7, :] = 0.0                       # zero row in block 0
+    W[128 + 7, :] = 0.0                 # and the same row of block 1: share row 7 is zero on every node
+    X[:, 5] = 0.0
+    X[:, 48 + 5] = 0.0                  # share column 5 is zero on every node
+    code = GPCode(N1, N0, B, m, n, d1, 1, P)
+    cp, Z = _sliced_products(code, W, X)
+    Wsh, Xsh = op.encode_W(W, code), op.encode_X(X, code)
+    Zo = op.worker_products(Wsh, Xsh)
+    got = cp.outputs_as_array(g.GPD_FWD, Z)
+    assert (got[:, 7, :] == 0.0).all() and (got[:, :, 5] == 0.0).all()
+    assert (np.abs(got - Zo) <= _output_tolerance(Wsh, Xsh)).all()
+    r = cp.locate(g.GPD_FWD, Z)
+    assert r.outcome == NO_ERROR
+    S = cp.decode(g.GPD_FWD, Z)
+    assert op.rel_fro(S, op.ref_forward(W, X)) < 1e-4
+
+
+def test_sliced_pipeline_locates_and_decodes_like_the_oracle():
+    N1, N0, B, m, n, d1, P = 512, 512, 128, 2, 4, 2, 25
+    W, X = _inputs(N1, N0, B, seed=11)
+    code = GPCode(N1, N0, B, m, n, d1, 1, P)
+    cp, Z = _sliced_products(code, W, X)
+    Zo = op.worker_products(op.encode_W(W, code), op.encode_X(X, code))
+    scale = float(np.sqrt(np.mean(Zo ** 2)))
+    ref = op.ref_forward(W, X)
+    seen = set()
+    for seed in range(300, 306):
+        Zg = Z.clone()
+        g.gpd_inject(cp.plan, g.GPD_FWD, Zg, seed, g.GPD_INJECT_ADDITIVE, prob=0.1, scale=scale)
+        Zr = Zo.copy()
+        sel = oinj.inject_additive(Zr, seed, scale, prob=0.1)
+        ro = locate_subspace(Zr, code.points, code.Q_f, tolerances_for(np.float64))
+        r = cp.locate(g.GPD_FWD, Zg)
+        assert r.outcome == ro.outcome and np.array_equal(cp.flags(r), ro.flagged)
+        seen.add(r.outcome)
+        if r.outcome in (NO_ERROR, CORRECTED):
+            assert np.array_equal(ro.flagged, sel)
+            S = cp.decode(g.GPD_FWD, Zg)
+            assert op.rel_fro(S, ref) < 1e-4
+            assert op.rel_fro(S, op.decode(Zr, code, FWD, use=~ro.flagged)) < 1e-4
+    assert CORRECTED in seen
+
+
+def test_sliced_layer_step_forward_only():
+    N1, N0, B, m, n, d1, P = 256, 256, 64, 2, 2, 1, 9
+    W, X = _inputs(N1, N0, B, seed=21)
+    code = GPCode(N1, N0, B, m, n, d1, 1, P)
+    plan = g.gpd_plan((N1, N0, B), (m, n, d1, 1), P, points=code.points, precision=g.GPD_PREC_FP64_SLICED)
+    Wsh = plan.empty(g.GPD_Q_W_SHARE_ELEMS)
+    g.gpd_encode_A(plan, dev(W), Wsh)
+    S = torch.full((N1, B), float("nan"), dtype=torch.float32, device="cuda")
+    A = torch.full((N1, B), float("nan"), dtype=torch.float32, device="cuda")
+    res, ws = g.new_results(2), plan.workspace(step=True)
+    g.coded_layer_step(plan, g.GPD_PHASE_FWD, Wsh, X=dev(X), activation=g.GPD_ACT_RELU, inject_seed=70,
+                       inject_prob=0.2, inject_scale=1.0, S_out=S, Xnext_out=A, results=res, workspace=ws)
+    r = g.read_results(res)[0]
+    Zr = op.worker_products(op.encode_W(W, code), op.encode_X(X, code))
+    sel = oinj.inject_gauss(Zr, 70, 1.0, prob=0.2)
+    ro = locate_subspace(Zr, code.points, code.Q_f, tolerances_for(np.float64))
+    assert r.outcome == ro.outcome and np.array_equal(np.array(list(r.flagged)[:P], dtype=bool), ro.flagged)
+    assert sel.any() and ro.outcome == CORRECTED
+    ref = op.ref_forward(W, X)
+    assert op.rel_fro(host(S), ref) < 1e-4
+    assert op.rel_fro(host(A), np.maximum(ref, 0.0)) < 1e-4
+    # every other phase needs shares this storage cannot serve
+    for phases in (g.GPD_PHASE_FWD | g.GPD_PHASE_REGEN, g.GPD_PHASE_BWD, g.GPD_PHASE_UPD,
+                   g.GPD_PHASE_FWD | g.GPD_PHASE_BWD | g.GPD_PHASE_UPD):
+        with pytest.raises(g.GpdError) as ei:
+            g.coded_layer_step(plan, phases, Wsh, X=dev(X), Delta=dev(np.zeros((N1, B), np.float32)),
+                               DeltaT=dev(np.zeros((B, N1), np.float32)), S_out=S, Xnext_out=A,
+                               CT_out=torch.empty((B, N0), dtype=torch.float32, device="cuda"), results=res, workspace=ws)
+        assert ei.value.status == g.GPD_ERR_UNSUPPORTED
+
+
+def test_sliced_refuses_calls_on_other_shares():
+    N1, N0, B, m, n, d1, P = 128, 128, 32, 2, 2, 1, 9
+    code = GPCode(N1, N0, B, m, n, d1, 1, P)
+    cp = CodedProduct(code, precision=g.GPD_PREC_FP64_SLICED)
+    W, X = _inputs(N1, N0, B, seed=3)
+    cp.encode_W(W)
+    for operand, M in ((g.GPD_OPERAND_DELTAT_BWD, np.zeros((B, N1), np.float32)),
+                       (g.GPD_OPERAND_DELTA_UPD, np.zeros((N1, B), np.float32)),
+                       (g.GPD_OPERAND_X_UPD, X)):
+        with pytest.raises(g.GpdError) as ei:
+            cp.encode(operand, M)
+        assert ei.value.status == g.GPD_ERR_UNSUPPORTED
+    Xs = cp.encode(g.GPD_OPERAND_X_FWD, X)
+    out = cp.plan.empty(g.GPD_Q_OUT_ELEMS_BWD)
+    with pytest.raises(g.GpdError) as ei:
+        g.gpd_worker_gemm(cp.plan, g.GPD_BWD, cp.W_shares, Xs, out)
+    assert ei.value.status == g.GPD_ERR_UNSUPPORTED
+    with pytest.raises(g.GpdError) as ei:
+        g.gpd_locate_errors(cp.plan, g.GPD_AUDIT, cp.W_shares, cp.res, cp.ws)
+    assert ei.value.status == g.GPD_ERR_UNSUPPORTED
+    with pytest.raises(g.GpdError) as ei:
+        g.gpd_regenerate_shares(cp.plan, cp.W_shares, cp.res, cp.ws)
+    assert ei.value.status == g.GPD_ERR_UNSUPPORTED

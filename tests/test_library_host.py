@@ -95,6 +95,28 @@ def test_plan_error_codes():
     assert g.gpd_status_string(g.GPD_ERR_P_TOO_SMALL) == "fewer nodes than the recovery threshold"
 
 
+def test_sliced_precision_plans():
+    """Digit-plane storage: accepted when N0/n is a multiple of 16 and the block counts are ones the
+    encoder is built for; element size and buffer sizes are those of the FP64 plan it stands in for."""
+    c = wl.CONFIG_3_MATMUL
+    plan = g.gpd_plan((c.N1, c.N0, c.B), (c.m, c.n, c.d, 1), c.P, precision=g.GPD_PREC_FP64_SLICED)
+    ref = g.gpd_plan((c.N1, c.N0, c.B), (c.m, c.n, c.d, 1), c.P, precision=g.GPD_PREC_FP64)
+    assert plan.query(g.GPD_Q_PRECISION) == g.GPD_PREC_FP64_SLICED and plan.query(g.GPD_Q_ELEMENT_SIZE) == 8
+    for q in (g.GPD_Q_W_SHARE_ELEMS, g.GPD_Q_X_SHARE_ELEMS, g.GPD_Q_OUT_ELEMS_FWD, g.GPD_Q_THRESHOLD_FWD,
+              g.GPD_Q_STEP_WORKSPACE_BYTES):
+        assert plan.query(q) == ref.query(q)
+    plan.destroy(), ref.destroy()
+    for shape, split, P in (((64, 72, 8), (2, 2, 1, 1), 9),          # N0/n = 36
+                            ((64, 160, 8), (2, 5, 1, 1), 20),        # 10 blocks per share of W
+                            ((4, 32, 2), (1, 1, 1, 1), 2)):          # digit planes + scales would not fit
+        with pytest.raises(g.GpdError) as e:
+            g.gpd_plan(shape, split, P, precision=g.GPD_PREC_FP64_SLICED)
+        assert e.value.status == g.GPD_ERR_UNSUPPORTED
+    with pytest.raises(g.GpdError) as e:                              # coefficients up to 7e35: beyond the FP32 scale pass
+        g.gpd_plan((64, 64, 8), (2, 2, 1, 1), 9, points=np.linspace(1e11, 9e11, 9), precision=g.GPD_PREC_FP64_SLICED)
+    assert e.value.status == g.GPD_ERR_UNSUPPORTED
+
+
 def test_custom_points_are_kept():
     pts = np.linspace(-0.9, 0.9, 7)
     plan = g.gpd_plan((8, 8, 4), (2, 2, 1, 1), 7, points=pts)
