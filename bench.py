@@ -5,9 +5,12 @@ One "step" is one pass of the whole coded path over one batch of synthetic input
 encode W, encode X, the P worker products (one batched kernel), seeded error injection,
 error detection/location, interpolation decode.  Workload: the 8192 x 8192 x 512 coded
 matrix-matrix product (W split 2 x 4, X split 4 x 2, threshold 19, P = 25 nodes, additive
-errors on each node with probability 0.1), FP64 shares and products.
+errors on each node with probability 0.1).  Shares are evaluated in FP64; the worker products
+run either as exact int8 digit-plane contractions on the tcgen05 tensor cores with FP64
+recombination (--precision sliced, the default) or as FP64 mma (--precision fp64); worker
+outputs, location and decoding are FP64 in both.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--precision sliced|fp64]
 
 Prints one JSON line.  `value` is useful TFLOP/s = 2 N1 N0 B / time (the product the caller
 asked for); the coded path executes P/(m n d) = 1.5625 times those flops.  With --gpus N
@@ -35,10 +38,12 @@ METRIC = "coded matmul TFLOP/s (encode+workers+locate+decode)"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0        # dense, per GPU
 NOMINAL_FP64_TFLOPS = 37.0          # FP64 tensor, per GPU of an 8-GPU HGX B200 board (296 / 8)
+NOMINAL_INT8_TOPS = 4500.0          # dense int8, per GPU
 FALLBACK_BF16_SUSTAINED = 1400.0
 FALLBACK_HBM_GBS = 6650.0
 CPU_SAMPLE_ROWS = 1024              # rows of W in the CPU sample (1/8 of the workload)
 TRAFFIC_BYTES_PER_LAUNCH = None     # dram read+write bytes of the dominant kernel from ncu (see profiles/)
+TRAFFIC_BYTES_PER_LAUNCH_SLICED = None
 
 
 def load_peaks():
@@ -226,7 +231,9 @@ def run_ours(args, cfg):
     peaks = load_peaks()
 
     W, X = wl.matmul_inputs(cfg)
-    plan = g.gpd_plan((cfg.N1, cfg.N0, cfg.B), (cfg.m, cfg.n, cfg.d, 1), cfg.P)
+    sliced = args.precision == "sliced"
+    plan = g.gpd_plan((cfg.N1, cfg.N0, cfg.B), (cfg.m, cfg.n, cfg.d, 1), cfg.P,
+                      precision=g.GPD_PREC_FP64_SLICED if sliced else g.GPD_PREC_FP64)
     assert plan.query(g.GPD_Q_ELEMENT_SIZE) == 8
     stream = torch.cuda.Stream()
     Wh, Xh = torch.from_numpy(W).pin_memory(), torch.from_numpy(X).pin_memory()
@@ -241,8 +248,9 @@ def run_ours(args, cfg):
     seeds = cfg.inject_seeds
     exec_flops = 2.0 * cfg.P * (cfg.N1 // cfg.m) * (cfg.N0 // cfg.n) * (cfg.B // cfg.d)
     useful_flops = 2.0 * cfg.N1 * cfg.N0 * cfg.B
-    KERNELS_PER_STEP = 8                # encode W, encode X, products, inject, syndrome, locate finish,
-                                        # decode matrix, decode stream
+    # encode W, encode X, products, inject, syndrome, locate finish, decode matrix, decode stream;
+    # the digit-plane encoders take two kernels each (scales, then digits)
+    KERNELS_PER_STEP = 10 if sliced else 8
 
     def step(i, gemm_events=None, stage_events=None, Wd=Wd, Xd=Xd):
         def mark(name):
@@ -349,25 +357,42 @@ def run_ours(args, cfg):
     value = whole_job_tflops(useful_flops, args.steps, world, ms)
     e2e_value = whole_job_tflops(useful_flops, args.steps, world, e2e_ms)
 
-    # FP64 tensor peak: MEASURED_PEAKS.json has no FP64 figure, and scaling its power-capped bf16
-    # number by the nominal ratio gives a value below what the FP64 path delivers (FP64 does not
-    # reach the power cap).  So the denominator is measured here the same way the bf16 one was:
-    # torch.matmul (cuBLAS) FP64 8192^3, best of 10, CUDA events.
-    fp64_measured = measure_fp64_matmul_peak(torch)
-    fp64_from_ratio = peaks["bf16_sustained"] * NOMINAL_FP64_TFLOPS / NOMINAL_BF16_TFLOPS
-    achieved = exec_flops / (gemm_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "dgemm_mma_kernel (P worker products, FP64 tensor path)",
-                "achieved": achieved, "peak": fp64_measured, "unit": "TFLOP/s", "frac": achieved / fp64_measured,
-                "traffic": TRAFFIC_BYTES_PER_LAUNCH,
-                "peak_source": "measured here: torch.matmul FP64 8192^3, best of 10 (cuBLAS)",
-                "peak_nominal_fp64": NOMINAL_FP64_TFLOPS,
-                "peak_from_bf16_ratio": fp64_from_ratio,
-                "flops_per_launch": exec_flops, "ms_per_launch": gemm_ms}
+    if sliced:
+        # The dominant kernel multiplies int8 digit planes: 21 plane pairs per FP64-class product.
+        # Its peak is the measured bf16 figure times the nominal int8 : bf16 ratio of the part (2).
+        pairs = 21
+        int8_ops = pairs * exec_flops
+        peak = peaks["bf16_burst"] * NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS
+        achieved = int8_ops / (gemm_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "gemm_i8_sliced_kernel (P worker products, int8 digit planes, tcgen05)",
+                    "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": TRAFFIC_BYTES_PER_LAUNCH_SLICED if args.scale_down == 1 else None,
+                    "peak_source": f"of {peaks['source']}: bf16 burst {peaks['bf16_burst']} TFLOP/s x nominal int8:bf16 ratio "
+                                   f"{NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS:g}",
+                    "ops": "int8 multiply-adds counted as 2 operations; 21 digit-plane pairs per product",
+                    "ops_per_launch": int8_ops, "ms_per_launch": gemm_ms,
+                    "fp64_equivalent_tflops": exec_flops / (gemm_ms * 1e-3) / 1e12}
+    else:
+        # FP64 tensor peak: MEASURED_PEAKS.json has no FP64 figure, and scaling its power-capped bf16
+        # number by the nominal ratio gives a value below what the FP64 path delivers (FP64 does not
+        # reach the power cap).  So the denominator is measured here the same way the bf16 one was:
+        # torch.matmul (cuBLAS) FP64 8192^3, best of 10, CUDA events.
+        fp64_measured = measure_fp64_matmul_peak(torch)
+        fp64_from_ratio = peaks["bf16_sustained"] * NOMINAL_FP64_TFLOPS / NOMINAL_BF16_TFLOPS
+        achieved = exec_flops / (gemm_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "dgemm_mma_kernel (P worker products, FP64 tensor path)",
+                    "achieved": achieved, "peak": fp64_measured, "unit": "TFLOP/s", "frac": achieved / fp64_measured,
+                    "traffic": TRAFFIC_BYTES_PER_LAUNCH,
+                    "peak_source": "measured here: torch.matmul FP64 8192^3, best of 10 (cuBLAS)",
+                    "peak_nominal_fp64": NOMINAL_FP64_TFLOPS,
+                    "peak_from_bf16_ratio": fp64_from_ratio,
+                    "flops_per_launch": exec_flops, "ms_per_launch": gemm_ms}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(cfg),
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64 (products: int8 digit planes, exact int32 accumulation)" if sliced else "f64",
+        "data": "synthetic", "config": dict(workload_config(cfg), precision=args.precision),
         "executed_tflops": value * exec_flops / useful_flops,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(W.nbytes + X.nbytes),
                 "d2h_bytes_per_step": int(cfg.N1 * cfg.B * 4 + g.RESULT_BYTES), "ms_per_step": e2e_ms / args.steps},
@@ -502,6 +527,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-down", type=int, default=1,
                     help="profiling aid: same code on matrices this many times smaller per side")
+    ap.add_argument("--precision", default="sliced", choices=["sliced", "fp64"],
+                    help="worker products of the matmul workload: int8 digit planes on tcgen05 (default) or FP64 mma")
     ap.add_argument("--workload", default="matmul", choices=["matmul", "mlp_layer"],
                     help="matmul: the headline 8192 x 8192 x 512 coded product; mlp_layer: secondary, FP32 path")
     args = ap.parse_args()
