@@ -10,7 +10,7 @@ run either as exact int8 digit-plane contractions on the tcgen05 tensor cores wi
 recombination (--precision sliced, the default) or as FP64 mma (--precision fp64); worker
 outputs, location and decoding are FP64 in both.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--precision sliced|fp64]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--precision sliced|sliced40|fp64]
 
 Prints one JSON line.  `value` is useful TFLOP/s = 2 N1 N0 B / time (the product the caller
 asked for); the coded path executes P/(m n d) = 1.5625 times those flops.  With --gpus N
@@ -231,9 +231,11 @@ def run_ours(args, cfg):
     peaks = load_peaks()
 
     W, X = wl.matmul_inputs(cfg)
-    sliced = args.precision == "sliced"
+    sliced = args.precision in ("sliced", "sliced40")
+    planes = {"sliced": 6, "sliced40": 5}.get(args.precision, 0)
     plan = g.gpd_plan((cfg.N1, cfg.N0, cfg.B), (cfg.m, cfg.n, cfg.d, 1), cfg.P,
-                      precision=g.GPD_PREC_FP64_SLICED if sliced else g.GPD_PREC_FP64)
+                      precision={"sliced": g.GPD_PREC_FP64_SLICED, "sliced40": g.GPD_PREC_FP64_SLICED40,
+                                 "fp64": g.GPD_PREC_FP64}[args.precision])
     assert plan.query(g.GPD_Q_ELEMENT_SIZE) == 8
     stream = torch.cuda.Stream()
     Wh, Xh = torch.from_numpy(W).pin_memory(), torch.from_numpy(X).pin_memory()
@@ -358,9 +360,9 @@ def run_ours(args, cfg):
     e2e_value = whole_job_tflops(useful_flops, args.steps, world, e2e_ms)
 
     if sliced:
-        # The dominant kernel multiplies int8 digit planes: 21 plane pairs per FP64-class product.
+        # The dominant kernel multiplies int8 digit planes: 21 (15) plane pairs per FP64-class product.
         # Its peak is the measured bf16 figure times the nominal int8 : bf16 ratio of the part (2).
-        pairs = 21
+        pairs = planes * (planes + 1) // 2
         int8_ops = pairs * exec_flops
         peak = peaks["bf16_burst"] * NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS
         achieved = int8_ops / (gemm_ms * 1e-3) / 1e12
@@ -369,7 +371,7 @@ def run_ours(args, cfg):
                     "traffic": TRAFFIC_BYTES_PER_LAUNCH_SLICED if args.scale_down == 1 else None,
                     "peak_source": f"of {peaks['source']}: bf16 burst {peaks['bf16_burst']} TFLOP/s x nominal int8:bf16 ratio "
                                    f"{NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS:g}",
-                    "ops": "int8 multiply-adds counted as 2 operations; 21 digit-plane pairs per product",
+                    "ops": f"int8 multiply-adds counted as 2 operations; {pairs} digit-plane pairs per product",
                     "ops_per_launch": int8_ops, "ms_per_launch": gemm_ms,
                     "fp64_equivalent_tflops": exec_flops / (gemm_ms * 1e-3) / 1e12}
     else:
@@ -527,8 +529,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-down", type=int, default=1,
                     help="profiling aid: same code on matrices this many times smaller per side")
-    ap.add_argument("--precision", default="sliced", choices=["sliced", "fp64"],
-                    help="worker products of the matmul workload: int8 digit planes on tcgen05 (default) or FP64 mma")
+    ap.add_argument("--precision", default="sliced", choices=["sliced", "sliced40", "fp64"],
+                    help="worker products of the matmul workload: six (default) or five int8 digit planes on tcgen05, "
+                         "or FP64 mma")
     ap.add_argument("--workload", default="matmul", choices=["matmul", "mlp_layer"],
                     help="matmul: the headline 8192 x 8192 x 512 coded product; mlp_layer: secondary, FP32 path")
     args = ap.parse_args()

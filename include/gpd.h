@@ -78,19 +78,23 @@ typedef enum {
     GPD_PREC_AUTO = 0,          /* FP32 if every threshold of the plan is <= 9, else FP64 */
     GPD_PREC_FP32 = 1,          /* shares/outputs float; products in 3xTF32 (tensor cores) or FP32 FMA */
     GPD_PREC_FP64 = 2,          /* shares/outputs double; products in FP64 */
-    GPD_PREC_FP64_SLICED = 3    /* forward product only (gpd_encode_A, gpd_encode_B with GPD_OPERAND_X_FWD,
+    GPD_PREC_FP64_SLICED = 3,   /* forward product only (gpd_encode_A, gpd_encode_B with GPD_OPERAND_X_FWD,
                                    gpd_worker_gemm with GPD_FWD, then inject / locate / decode as for
                                    GPD_PREC_FP64).  The shares W~_p (Eq. 1), X~_p (Theorem 2) are evaluated in
-                                   FP64 and stored as six signed 7-bit digit planes plus one power-of-two
-                                   scale per row of W~_p / column of X~_p, in buffers of the same byte size as
-                                   the FP64 shares (opaque to the caller); the worker products are exact
-                                   int8 x int8 -> int32 tensor-core contractions of digit planes, recombined
-                                   in FP64 (terms below 2^-49 of row scale x column scale dropped); worker
-                                   outputs are double.  Needs N0/n divisible by 16 and finite inputs (a row
-                                   holding a non-finite value encodes as zeros).  Every other call that takes
-                                   shares returns GPD_ERR_UNSUPPORTED; gpd_plan returns it when the shapes
-                                   do not fit.  An implementation choice of this library: the paper
-                                   prescribes no arithmetic for the nodes' products. */
+                                   FP64 and stored as six signed 8-bit digit planes plus one power-of-two
+                                   scale per row of W~_p / column of X~_p (48 bits below the scale), in buffers
+                                   of the same byte size as the FP64 shares (opaque to the caller); the worker
+                                   products are exact int8 x int8 -> int32 tensor-core contractions of digit
+                                   planes, recombined in FP64 (plane pairs below 2^-50 of row scale x column
+                                   scale are not formed); worker outputs are double.  Needs N0/n divisible
+                                   by 16 and at most 16384, and finite inputs (a non-finite entry makes its
+                                   share row meaningless without being flagged).  Every other call that takes
+                                   shares returns GPD_ERR_UNSUPPORTED; gpd_plan returns it when the shapes do
+                                   not fit.  An implementation choice of this library: the paper prescribes
+                                   no arithmetic for the nodes' products. */
+    GPD_PREC_FP64_SLICED40 = 4  /* the same with five digit planes (40 bits below the scale, 15 plane pairs
+                                   instead of 21): worker outputs accurate to about 1e-10 of their scale,
+                                   enough for recovery thresholds up to about 20 */
 } gpd_precision;
 
 typedef enum {

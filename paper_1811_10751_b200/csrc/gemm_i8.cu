@@ -1,19 +1,19 @@
 // FP64-class forward worker products (step O1) on the integer tensor cores.
 //
-// Both operands arrive cut into six signed 7-bit digit planes (slice.cu):
-//     W~_p[i][k] = 2^ea[i] * sum_s A_s[i][k] 128^-(s+1),   X~_p[k][j] = 2^eb[j] * sum_t B_t[j][k] 128^-(t+1).
+// Both operands arrive cut into S = 6 (or 5) signed 8-bit digit planes (slice.cu):
+//     W~_p[i][k] = 2^ea[i] * sum_s A_s[i][k] 256^-(s+1),   X~_p[k][j] = 2^eb[j] * sum_t B_t[j][k] 256^-(t+1).
 // A digit-plane product A_s B_t^T is an int8 x int8 -> int32 contraction, exact on the tensor
-// cores (|digit| <= 64, so K up to 87381 cannot overflow six summed pairs).  Pairs with
-// s + t <= 5 (weight >= 128^-7) are kept: 21 of 36, the rest lie below 2^-49 of the row/column
-// scales.  Pairs of equal weight share one accumulator, so a 128 x 64 output tile owns six
-// 128 x 64 int32 accumulators in tensor memory (384 of 512 columns), group g = s + t at columns
-// 64 g.  For a fixed s the planes t = 0 .. 5-s are adjacent in shared memory and their
-// accumulators are adjacent in tensor memory, so one tcgen05.mma of N = 64 (6 - s) columns
-// (two when that exceeds 256) covers all pairs of plane s: 8 instructions per 32 elements of K.
+// cores (|digit| <= 128, so six summed pairs cannot overflow for K <= 21845).  Pairs with
+// s + t <= S - 1 (weight >= 256^-(S+1)) are kept: 21 of 36 (15 of 25), the rest lie below
+// 2^-(8 S + 2) of the row/column scales.  Pairs of equal weight share one accumulator, so a 128 x 64
+// output tile owns S 128 x 64 int32 accumulators in tensor memory, group g = s + t at columns
+// 64 g.  For a fixed s the planes t = 0 .. S-1-s are adjacent in shared memory and their
+// accumulators are adjacent in tensor memory, so one tcgen05.mma of N = 64 (S - s) columns
+// (two when that exceeds 256) covers all pairs of plane s: 8 (6) instructions per 32 elements of K.
 //
-// Warp roles: warp 0 one lane issues the TMA copies (12 per 64-element k-block, 3-stage ring),
+// Warp roles: warp 0 one lane issues the TMA copies (2 S per 64-element k-block, 3-stage ring),
 // warp 1 allocates tensor memory and one lane issues the MMAs, warps 2..5 read the accumulators
-// back, combine them in FP64 (sum_g acc_g 2^-7g, then the row and column powers of two) and store.
+// back, combine them in FP64 (sum_g acc_g 2^-8g, then the row and column powers of two) and store.
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains its copies,
 // frees its tensor memory and returns.
 #include <cuda.h>
@@ -28,9 +28,9 @@ constexpr int BM = 128, BN = 64, BK = 64, STAGES = 3;
 constexpr int UMMA_K = 32;                            // int8 elements per MMA along K
 constexpr int A_PLANE_BYTES = BM * BK;                // 8 KB, rows of 64 B
 constexpr int B_PLANE_BYTES = BN * BK;                // 4 KB
-constexpr int STAGE_BYTES = kSlices * (A_PLANE_BYTES + B_PLANE_BYTES);   // 72 KB
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
-constexpr int TMEM_COLS = 512;                        // 6 x 64 used; allocations are powers of two
+__host__ __device__ constexpr int stage_bytes(int S) { return S * (A_PLANE_BYTES + B_PLANE_BYTES); }   // 72 KB (60 KB)
+__host__ __device__ constexpr int smem_bytes(int S) { return STAGES * stage_bytes(S) + 1024; }
+constexpr int TMEM_COLS = 512;                        // S x 64 used; allocations are powers of two
 constexpr int kEpiWarps = 4;
 constexpr int kThreads = 64 + kEpiWarps * 32;
 constexpr long long kWaitCycles = 2000000000LL;       // about one second
@@ -111,9 +111,11 @@ struct I8Params {
     int P;
 };
 
+template <int S>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, I8Params prm,
                       int tiles_m, int tiles_n) {
+    constexpr int STAGE_BYTES = stage_bytes(S);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
@@ -152,7 +154,7 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     volatile int* abort_p = &abort_flag;
 
     auto A_plane = [&](int s, int t) { return smem + s * STAGE_BYTES + t * A_PLANE_BYTES; };
-    auto B_plane = [&](int s, int t) { return smem + s * STAGE_BYTES + kSlices * A_PLANE_BYTES + t * B_PLANE_BYTES; };
+    auto B_plane = [&](int s, int t) { return smem + s * STAGE_BYTES + S * A_PLANE_BYTES + t * B_PLANE_BYTES; };
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
@@ -164,7 +166,7 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) break;
                 mbar_expect_tx(&full_bar[s], STAGE_BYTES);
 #pragma unroll
-                for (int t = 0; t < kSlices; ++t) {
+                for (int t = 0; t < S; ++t) {
                     tma_load_3d(A_plane(s, t), &tmA, kb * BK, m0, t * prm.P + p, &full_bar[s]);
                     tma_load_3d(B_plane(s, t), &tmB, kb * BK, n0, t * prm.P + p, &full_bar[s]);
                 }
@@ -190,13 +192,13 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
                 for (int k = 0; k < BK / UMMA_K; ++k) {
 #pragma unroll
-                    for (int ta = 0; ta < kSlices; ++ta) {
-                        // planes tb = 0 .. 5-ta of B in one operand of 64 (6 - ta) rows, at most 256 per MMA;
+                    for (int ta = 0; ta < S; ++ta) {
+                        // planes tb = 0 .. S-1-ta of B in one operand of 64 (S - ta) rows, at most 256 per MMA;
                         // the pair (ta, tb) lands in accumulator group ta + tb = columns 64 (ta + tb)
                         const uint64_t da = desc_sw64(a0 + ta * A_PLANE_BYTES + k * UMMA_K);
-                        const int n_total = BN * (kSlices - ta);
+                        const int n_total = BN * (S - ta);
                         const int n_first = n_total > 256 ? 256 : n_total;
-                        // the plane-0 instruction of the first k-step overwrites all six groups
+                        // the plane-0 instruction of the first k-step overwrites every group
                         const uint32_t acc = (kb > 0 || k > 0 || ta > 0) ? 1u : 0u;
                         umma_i8(tmem_base + BN * ta, da, desc_sw64(b0 + k * UMMA_K), idesc_i8(n_first), acc);
                         if (n_total > 256)
@@ -224,7 +226,7 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = 0.0;
 #pragma unroll
-                for (int g = kSlices - 1; g >= 0; --g) {             // smallest weight first
+                for (int g = S - 1; g >= 0; --g) {             // smallest weight first
                     uint32_t r[32];
                     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(BN * g + c0);
                     asm volatile(
@@ -311,7 +313,8 @@ gpd_status gemm_sliced_launch(gpd_plan_s* plan, const void* W_sliced, const void
     I8Params prm{};
     prm.P = plan->P;
     prm.M = s.N1 / c.m; prm.K = s.N0 / c.n; prm.N = s.B / c.d1;
-    const SlicedLayout la = sliced_layout(prm.P, prm.M, prm.K), lb = sliced_layout(prm.P, prm.N, prm.K);
+    const int S = plan->slices;
+    const SlicedLayout la = sliced_layout(S, prm.P, prm.M, prm.K), lb = sliced_layout(S, prm.P, prm.N, prm.K);
     prm.ea = reinterpret_cast<const int*>(reinterpret_cast<const char*>(W_sliced) + la.expo_offset);
     prm.eb = reinterpret_cast<const int*>(reinterpret_cast<const char*>(X_sliced) + lb.expo_offset);
     prm.C = reinterpret_cast<double*>(out);
@@ -319,13 +322,14 @@ gpd_status gemm_sliced_launch(gpd_plan_s* plan, const void* W_sliced, const void
         reinterpret_cast<uintptr_t>(out) % 16)
         return GPD_ERR_ARG;
     CUtensorMap tmA, tmB;
-    if (!make_map(&tmA, W_sliced, (int64_t)kSlices * prm.P, prm.M, prm.K, BM)) return GPD_ERR_CUDA;
-    if (!make_map(&tmB, X_sliced, (int64_t)kSlices * prm.P, prm.N, prm.K, BN)) return GPD_ERR_CUDA;
-    if (cudaFuncSetAttribute(gemm_i8_sliced_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-        return GPD_ERR_CUDA;
+    if (!make_map(&tmA, W_sliced, (int64_t)S * prm.P, prm.M, prm.K, BM)) return GPD_ERR_CUDA;
+    if (!make_map(&tmB, X_sliced, (int64_t)S * prm.P, prm.N, prm.K, BN)) return GPD_ERR_CUDA;
+    auto kernel = S == 6 ? gemm_i8_sliced_kernel<6> : gemm_i8_sliced_kernel<5>;
+    const int smem = S == 6 ? smem_bytes(6) : smem_bytes(5);
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GPD_ERR_CUDA;
     const int tiles_n = (int)((prm.N + BN - 1) / BN), tiles_m = (int)((prm.M + BM - 1) / BM);
     const int64_t tiles = (int64_t)tiles_n * tiles_m * prm.P;
-    gemm_i8_sliced_kernel<<<(unsigned)tiles, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n);
+    kernel<<<(unsigned)tiles, kThreads, smem, st>>>(tmA, tmB, prm, tiles_m, tiles_n);
     return launch_ok();
 }
 

@@ -55,7 +55,8 @@ struct gpd_plan_s {
     int Qf = 0, Qb = 0, Qw = 0;  // thresholds under the plan's substitution
     gpd_precision prec = GPD_PREC_FP32;
     int elem_size = 4;
-    bool sliced = false;         // GPD_PREC_FP64_SLICED: shares are int8 digit planes, outputs double
+    bool sliced = false;         // GPD_PREC_FP64_SLICED / _SLICED40: shares are int8 digit planes, outputs double
+    int slices = 0;              // digit planes per operand (6 or 5) when sliced
     double tau_col = 0, tau_in = 0;
     std::vector<double> points;
     std::vector<double> coefW, coefX, coefDT, coefDup, coefXup;   // [P][blocks]

@@ -153,7 +153,7 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
     if (subst != GPD_SUBST_U_EQ_VN && subst != GPD_SUBST_V_EQ_UM) return GPD_ERR_ARG;
     const bool alt = subst == GPD_SUBST_V_EQ_UM;
     if (precision != GPD_PREC_AUTO && precision != GPD_PREC_FP32 && precision != GPD_PREC_FP64 &&
-        precision != GPD_PREC_FP64_SLICED)
+        precision != GPD_PREC_FP64_SLICED && precision != GPD_PREC_FP64_SLICED40)
         return GPD_ERR_ARG;
     const int m = split->m, n = split->n, d1 = split->d1, d2 = split->d2;
     if (shape->N1 <= 0 || shape->N0 <= 0 || shape->B <= 0 || m <= 0 || n <= 0 || d1 <= 0 || d2 <= 0)
@@ -197,7 +197,8 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
     plan->elem_size = plan->prec == GPD_PREC_FP32 ? 4 : 8;
     plan->tau_col = plan->prec == GPD_PREC_FP32 ? kTauColFp32 : kTauColFp64;
     plan->tau_in = plan->prec == GPD_PREC_FP32 ? kTauInFp32 : kTauInFp64;
-    plan->sliced = plan->prec == GPD_PREC_FP64_SLICED;
+    plan->sliced = plan->prec == GPD_PREC_FP64_SLICED || plan->prec == GPD_PREC_FP64_SLICED40;
+    plan->slices = plan->prec == GPD_PREC_FP64_SLICED ? 6 : plan->prec == GPD_PREC_FP64_SLICED40 ? 5 : 0;
 
     // powers up to the largest exponent used by any encoding
     const int max_exp = (int)std::max<int64_t>(std::max(Qf, Qb), Qw) + 1;

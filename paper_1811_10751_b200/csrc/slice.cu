@@ -1,13 +1,13 @@
-// Encoding for the integer-slice product path (GPD_PREC_FP64_SLICED).
+// Encoding for the integer-slice product paths (GPD_PREC_FP64_SLICED, GPD_PREC_FP64_SLICED40).
 //
 // The shares W~_p (Eq. 1) and X~_p (Theorem 2) are evaluated in FP64 exactly as in encode.cu, but
-// instead of being stored as doubles each value a is stored as six signed 7-bit digits:
-//     a = 2^e * sum_{t=1..6} q_t * 128^-t  (+ remainder below 2^(e-43)),   q_t in [-64, 64],
-// with one exponent e per row of W~_p (per column of X~_p) chosen so that |a| < 2^(e-1).  The
-// digits of one operand form six int8 planes; products of planes are exact in int32 on the tensor
+// instead of being stored as doubles each value a is stored as S = 6 (or 5) signed 8-bit digits:
+//     a = 2^e * sum_{t=0..S-1} d_t * 256^-(t+1)  (+ remainder below 2^(e - 8 S - 1)),   d_t in [-128, 127],
+// with one exponent e per row of W~_p (per column of X~_p) chosen so that |a| < 0.4923 * 2^e.  The
+// digits of one operand form S int8 planes; products of planes are exact in int32 on the tensor
 // cores (gemm_i8.cu), which gives FP64-class worker products at integer-tensor-core speed.
-// Both operands are written K-major: W planes [6][P][M][K], X planes [6][P][N][K] (transposed).
-// Layout of a sliced share buffer: planes, then the int32 exponents (256-byte aligned).
+// Both operands are written K-major: W planes [S][P][M][K], X planes [S][P][N][K] (transposed).
+// Layout of a sliced share buffer: planes, then the int32 exponents, then encoder scratch.
 #include <cmath>
 
 #include "gpd_internal.h"
@@ -20,7 +20,7 @@ namespace {
 struct SliceParams {
     const float* src;      // source matrix, row-major, leading dimension ld
     const double* coef;    // [P][nblk]
-    int8_t* planes;        // [kSlices][P][R][K]   (R = rows of the K-major operand)
+    int8_t* planes;        // [S][P][R][K]   (R = rows of the K-major operand)
     int* expo;             // [P][R]
     unsigned int* amax;    // [P][R] scratch of the X side: largest |value| per operand row (high word)
     int64_t ld;            // leading dimension of src
@@ -36,7 +36,7 @@ __device__ __forceinline__ unsigned int abs_hi_max4(const double (&a)[4]) {
 }
 
 // Exponent e such that every |a| <= amax has |a| 2^-e < 0.4923, which keeps the biased fixed-point
-// value of digits4() inside 42 bits; amax is given by its high word as above.  Magnitudes below
+// value of digits4() inside 8 S bits; amax is given by its high word as above.  Magnitudes below
 // 2^-900 (and non-finite ones) get the marker -1000: all digits zero.
 __device__ __forceinline__ int slice_exponent(unsigned int amax_hi) {
     if (amax_hi < 0x07B00000u || amax_hi >= 0x7FF00000u) return -1000;
@@ -45,36 +45,36 @@ __device__ __forceinline__ int slice_exponent(unsigned int amax_hi) {
     frexp(amax * 1.015625, &x);   // amax (1 + 1/64) = f 2^x, f in [0.5, 1)
     return x + 1;
 }
-// 2^(42 - e) as a double, 0 for the all-zero marker
+// 2^(8 S - e) as a double, 0 for the all-zero marker
+template <int S>
 __device__ __forceinline__ double slice_scale(int e) {
     if (e <= -1000) return 0.0;
-    return __longlong_as_double((long long)(42 - e + 1023) << 52);
+    return __longlong_as_double((long long)(8 * S - e + 1023) << 52);
 }
 
-// Digits of four values at once.  U = rint(a 2^(42-e)) + sum_i 64 * 128^i lies in [0, 2^42); its
-// 7-bit fields minus 64 are the digits (each in [-64, 63]), most significant first.  U is read
-// from the mantissa of a 2^(42-e) + 2^52 + bias (one FMA); the fields of the four values are
-// gathered bytewise; word[t] holds digit t of values 0..3 in bytes 0..3.
-__device__ __forceinline__ void digits4(const double (&a)[4], double scale, unsigned int (&word)[kSlices]) {
-    const double magic = 4503599627370496.0 + 2216338399296.0;   // 2^52 + 64 (128^6 - 1) / 127
+// Digits of four values at once.  U = rint(a 2^(8S-e)) + sum_i 128 * 256^i lies in [0, 2^(8S));
+// its bytes minus 128 (= bytes with the top bit flipped) are the digits, most significant first.
+// U is read from the mantissa of a 2^(8S-e) + 2^52 + bias (one FMA); word[t] holds digit t of
+// values 0..3 in bytes 0..3.  A zero scale gives zero digits for finite a.
+template <int S>
+__device__ __forceinline__ void digits4(const double (&a)[4], double scale, unsigned int (&word)[S]) {
+    // 2^52 + 128 (256^S - 1) / 255
+    const double magic = S == 6 ? 4503599627370496.0 + 141289400074368.0 : 4503599627370496.0 + 551911719040.0;
     unsigned int lo[4], hi[4];
 #pragma unroll
     for (int v = 0; v < 4; ++v) {
-        const double t = fma(scale != 0.0 ? a[v] : 0.0, scale, magic);
+        const double t = fma(a[v], scale, magic);
         lo[v] = (unsigned int)__double2loint(t);
         hi[v] = (unsigned int)__double2hiint(t);
     }
 #pragma unroll
-    for (int t = 0; t < kSlices; ++t) {
-        unsigned int x[4];
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            const int bit = kDigitBits * (kSlices - 1 - t);              // position of digit t in U
-            x[v] = bit == 0 ? lo[v] : bit < 28 ? lo[v] >> bit : bit == 28 ? __funnelshift_r(lo[v], hi[v], 28) : hi[v] >> (bit - 32);
-        }
-        const unsigned int p01 = __byte_perm(x[0], x[1], 0x0040), p23 = __byte_perm(x[2], x[3], 0x0040);
-        const unsigned int u = __byte_perm(p01, p23, 0x5410) & 0x7F7F7F7Fu;
-        word[t] = (u + 0x40404040u) ^ 0x80808080u;                        // bytewise u - 64
+    for (int t = 0; t < S; ++t) {
+        const int byte = S - 1 - t;                                   // position of digit t in U
+        const unsigned int sel = byte < 4 ? (unsigned int)(((4 + byte) << 4) | byte)
+                                          : (unsigned int)(((4 + byte - 4) << 4) | (byte - 4));
+        const unsigned int p01 = byte < 4 ? __byte_perm(lo[0], lo[1], sel) : __byte_perm(hi[0], hi[1], sel);
+        const unsigned int p23 = byte < 4 ? __byte_perm(lo[2], lo[3], sel) : __byte_perm(hi[2], hi[3], sel);
+        word[t] = __byte_perm(p01, p23, 0x5410) ^ 0x80808080u;
     }
 }
 
@@ -141,15 +141,15 @@ __global__ void __launch_bounds__(256) rowmax_kernel(SliceParams prm) {
     }
 }
 
-// Pass 2: one thread per 4 consecutive columns of a share row: recompute the share values, cut
-// them into digits with the row's exponent, store 4 digits (one 32-bit word) per plane.
-template <int NBLK>
+// Pass 2: one thread per 4 consecutive columns of a share row: recompute the share values in FP64,
+// cut them into digits with the row's exponent, store 4 digits (one 32-bit word) per plane.
+template <int NBLK, int S>
 __global__ void __launch_bounds__(256) rowslice_kernel(SliceParams prm) {
     extern __shared__ double s_coef[];
     for (int i = threadIdx.x; i < prm.P * NBLK; i += 256) s_coef[i] = prm.coef[i];
     __syncthreads();
     const int64_t bc4 = prm.bc >> 2, total = prm.br * bc4;
-    const int64_t plane_stride = (int64_t)prm.P * prm.br * prm.bc;
+    const int64_t plane_stride = (int64_t)prm.P * prm.br * prm.bc, node_stride = prm.br * prm.bc;
     for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < total; t += (int64_t)gridDim.x * 256) {
         const int64_t r = t / bc4, c = (t - r * bc4) << 2;
         double x[NBLK][4];                       // converted once, used by every node
@@ -159,8 +159,10 @@ __global__ void __launch_bounds__(256) rowslice_kernel(SliceParams prm) {
             const float4 v = __ldg(reinterpret_cast<const float4*>(prm.src + (gi * prm.br + r) * prm.ld + gj * prm.bc + c));
             x[b][0] = v.x; x[b][1] = v.y; x[b][2] = v.z; x[b][3] = v.w;
         }
+        int8_t* dst = prm.planes + r * prm.bc + c;
+        const int* ex = prm.expo + r;
 #pragma unroll 2
-        for (int p = 0; p < prm.P; ++p) {
+        for (int p = 0; p < prm.P; ++p, dst += node_stride, ex += prm.br) {
             const double* cf = s_coef + p * NBLK;
             double a[4] = {0, 0, 0, 0};
 #pragma unroll
@@ -169,11 +171,10 @@ __global__ void __launch_bounds__(256) rowslice_kernel(SliceParams prm) {
                 a[0] = fma(k, x[b][0], a[0]); a[1] = fma(k, x[b][1], a[1]);
                 a[2] = fma(k, x[b][2], a[2]); a[3] = fma(k, x[b][3], a[3]);
             }
-            unsigned int word[kSlices];
-            digits4(a, slice_scale(__ldg(prm.expo + (int64_t)p * prm.br + r)), word);
-            int8_t* dst = prm.planes + ((int64_t)p * prm.br + r) * prm.bc + c;
+            unsigned int word[S];
+            digits4<S>(a, slice_scale<S>(__ldg(ex)), word);
 #pragma unroll
-            for (int s = 0; s < kSlices; ++s)
+            for (int s = 0; s < S; ++s)
                 __stcs(reinterpret_cast<unsigned int*>(dst + s * plane_stride), word[s]);
         }
     }
@@ -183,12 +184,12 @@ __global__ void __launch_bounds__(256) rowslice_kernel(SliceParams prm) {
 // A CTA stages the source values of a tile (128 rows kk x 8 columns n of every block) in shared
 // memory, transposed, so that a thread owns 4 consecutive kk of one column (warp = column,
 // lane = kk / 4): it converts its values once and runs over the nodes.
-//   SLICE = false: largest |X~_p[kk][n]| over kk, met in amax[p][n] (high words, zeroed before the launch)
-//   SLICE = true : digits with the column's exponent, written K-major (128 bytes per warp and plane);
-//                  the CTAs of the first row slab also publish the exponents.
+//   S = 0    : largest |X~_p[kk][n]| over kk, met in amax[p][n] (high words, zeroed before the launch)
+//   S = 5, 6 : S digits with the column's exponent, written K-major (128 bytes per warp and plane);
+//              the CTAs of the first row slab also publish the exponents.
 constexpr int XT_K = 128, XT_N = 8, XT_PITCH = XT_K + 4;
 
-template <int NBLK, bool SLICE>
+template <int NBLK, int S>
 __global__ void __launch_bounds__(256) colpass_kernel(SliceParams prm) {
     extern __shared__ double s_coef[];                             // [P][NBLK], then the tile
     float* xs = reinterpret_cast<float*>(s_coef + prm.P * NBLK);   // [NBLK][XT_N][XT_PITCH]
@@ -233,47 +234,53 @@ __global__ void __launch_bounds__(256) colpass_kernel(SliceParams prm) {
             a[0] = fma(k, x[b][0], a[0]); a[1] = fma(k, x[b][1], a[1]);
             a[2] = fma(k, x[b][2], a[2]); a[3] = fma(k, x[b][3], a[3]);
         }
-        if (!SLICE) {
+        if (S == 0) {
             const unsigned int mx = __reduce_max_sync(0xffffffffu, abs_hi_max4(a));
             if (lane == 0) atomicMax(prm.amax + (int64_t)p * prm.bc + gn, mx);
         } else {
             const int e = slice_exponent(prm.amax[(int64_t)p * prm.bc + gn]);
             if (blockIdx.y == 0 && lane == 0) prm.expo[(int64_t)p * prm.bc + gn] = e;
-            unsigned int word[kSlices];
-            digits4(a, slice_scale(e), word);
+            constexpr int SS = S > 0 ? S : 1;
+            unsigned int word[SS];
+            digits4<SS>(a, slice_scale<SS>(e), word);
             if (gk < prm.br) {                                     // br is a multiple of 16: whole words
                 int8_t* dst = prm.planes + ((int64_t)p * prm.bc + gn) * prm.br + gk;
 #pragma unroll
-                for (int s = 0; s < kSlices; ++s) *reinterpret_cast<unsigned int*>(dst + s * plane_stride) = word[s];
+                for (int s = 0; s < SS; ++s) *reinterpret_cast<unsigned int*>(dst + s * plane_stride) = word[s];
             }
         }
     }
 }
 
 template <int NBLK>
-gpd_status launch_rows(const SliceParams& prm, cudaStream_t st) {
-    const size_t smem = sizeof(double) * prm.P * NBLK;
-    rowmax_kernel<NBLK><<<(unsigned)prm.br, 256, smem + sizeof(float) * prm.P * NBLK, st>>>(prm);
+gpd_status launch_rows(const SliceParams& prm, int slices, cudaStream_t st) {
+    rowmax_kernel<NBLK><<<(unsigned)prm.br, 256, (sizeof(double) + sizeof(float)) * prm.P * NBLK, st>>>(prm);
     if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
     const int64_t work = prm.br * (prm.bc / 4);
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, 148 * 16));
-    rowslice_kernel<NBLK><<<grid, 256, smem, st>>>(prm);
+    const size_t smem = sizeof(double) * prm.P * NBLK;
+    if (slices == 6) rowslice_kernel<NBLK, 6><<<grid, 256, smem, st>>>(prm);
+    else rowslice_kernel<NBLK, 5><<<grid, 256, smem, st>>>(prm);
+    return launch_ok();
+}
+
+template <int NBLK, int S>
+gpd_status launch_colpass(const SliceParams& prm, cudaStream_t st) {
+    const size_t smem = sizeof(double) * prm.P * NBLK + sizeof(float) * NBLK * XT_N * XT_PITCH;
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(colpass_kernel<NBLK, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return GPD_ERR_CUDA;
+    dim3 grid((unsigned)((prm.bc + XT_N - 1) / XT_N), (unsigned)((prm.br + XT_K - 1) / XT_K));
+    colpass_kernel<NBLK, S><<<grid, 256, smem, st>>>(prm);
     return launch_ok();
 }
 
 template <int NBLK>
-gpd_status launch_cols(const SliceParams& prm, cudaStream_t st) {
+gpd_status launch_cols(const SliceParams& prm, int slices, cudaStream_t st) {
     if (cudaMemsetAsync(prm.amax, 0, sizeof(unsigned int) * prm.P * prm.bc, st) != cudaSuccess) return GPD_ERR_CUDA;
-    const size_t smem = sizeof(double) * prm.P * NBLK + sizeof(float) * NBLK * XT_N * XT_PITCH;
-    if (smem > 48 * 1024 &&
-        (cudaFuncSetAttribute(colpass_kernel<NBLK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-         cudaFuncSetAttribute(colpass_kernel<NBLK, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess))
-        return GPD_ERR_CUDA;
-    dim3 grid((unsigned)((prm.bc + XT_N - 1) / XT_N), (unsigned)((prm.br + XT_K - 1) / XT_K));
-    colpass_kernel<NBLK, false><<<grid, 256, smem, st>>>(prm);
-    if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
-    colpass_kernel<NBLK, true><<<grid, 256, smem, st>>>(prm);
-    return launch_ok();
+    gpd_status rc = launch_colpass<NBLK, 0>(prm, st);
+    if (rc != GPD_OK) return rc;
+    return slices == 6 ? launch_colpass<NBLK, 6>(prm, st) : launch_colpass<NBLK, 5>(prm, st);
 }
 
 }  // namespace
@@ -287,19 +294,20 @@ bool sliced_supported(const gpd_plan_s* plan) {
     auto ok_blk = [](int n) {
         return n == 1 || n == 2 || n == 3 || n == 4 || n == 6 || n == 8 || n == 9 || n == 12 || n == 16;
     };
-    if (K % 16 != 0 || !ok_blk(nb_w) || !ok_blk(nb_x)) return false;
+    // int32 accumulation of up to 6 plane pairs of |digit| <= 128 over K terms
+    if (K % 16 != 0 || K > 16384 || !ok_blk(nb_w) || !ok_blk(nb_x)) return false;
     // the scale pass evaluates the shares in FP32: the encoding coefficients must fit comfortably
     for (double c : plan->coefW) if (!(std::fabs(c) < 1e30)) return false;
     for (double c : plan->coefX) if (!(std::fabs(c) < 1e30)) return false;
     // the sliced operands live in buffers sized for the FP64 shares they replace
-    return sliced_layout(plan->P, M, K).total_bytes <= 8 * (int64_t)plan->P * M * K &&
-           sliced_layout(plan->P, N, K).total_bytes <= 8 * (int64_t)plan->P * N * K;
+    return sliced_layout(plan->slices, plan->P, M, K).total_bytes <= 8 * (int64_t)plan->P * M * K &&
+           sliced_layout(plan->slices, plan->P, N, K).total_bytes <= 8 * (int64_t)plan->P * N * K;
 }
 
-SlicedLayout sliced_layout(int64_t P, int64_t rows, int64_t K) {
+SlicedLayout sliced_layout(int slices, int64_t P, int64_t rows, int64_t K) {
     SlicedLayout l;
     l.plane_bytes = P * rows * K;
-    l.expo_offset = (kSlices * l.plane_bytes + 255) / 256 * 256;
+    l.expo_offset = (slices * l.plane_bytes + 255) / 256 * 256;
     l.amax_offset = (l.expo_offset + P * rows * 4 + 255) / 256 * 256;
     l.total_bytes = l.amax_offset + P * rows * 4;
     return l;
@@ -322,11 +330,13 @@ gpd_status encode_sliced_launch(gpd_plan_s* plan, bool is_A, const float* src, v
         prm.coef = plan->dev.base + plan->dev.off_coefX;
     }
     prm.nblk = gr * prm.gc;
-    const SlicedLayout lay = is_A ? sliced_layout(plan->P, prm.br, prm.bc) : sliced_layout(plan->P, prm.bc, prm.br);
+    const SlicedLayout lay = is_A ? sliced_layout(plan->slices, plan->P, prm.br, prm.bc)
+                                  : sliced_layout(plan->slices, plan->P, prm.bc, prm.br);
     prm.planes = reinterpret_cast<int8_t*>(dst);
     prm.expo = reinterpret_cast<int*>(reinterpret_cast<char*>(dst) + lay.expo_offset);
     prm.amax = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(dst) + lay.amax_offset);
-#define GPD_SLICE_CASE(NB) case NB: return is_A ? launch_rows<NB>(prm, st) : launch_cols<NB>(prm, st)
+#define GPD_SLICE_CASE(NB) \
+    case NB: return is_A ? launch_rows<NB>(prm, plan->slices, st) : launch_cols<NB>(prm, plan->slices, st)
     switch (prm.nblk) {
         GPD_SLICE_CASE(1); GPD_SLICE_CASE(2); GPD_SLICE_CASE(3); GPD_SLICE_CASE(4); GPD_SLICE_CASE(6);
         GPD_SLICE_CASE(8); GPD_SLICE_CASE(9); GPD_SLICE_CASE(12); GPD_SLICE_CASE(16);

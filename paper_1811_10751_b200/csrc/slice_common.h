@@ -6,20 +6,20 @@
 
 namespace gpd {
 
-constexpr int kSlices = 6;        // signed 7-bit digits kept per value (42 bits below the row exponent)
-constexpr int kDigitBits = 7;
+constexpr int kMaxSlices = 6;      // signed 8-bit digits kept per value: 6 (48 bits below the row scale) or 5 (40 bits)
+constexpr int kDigitBits = 8;
 
 // A sliced operand with R rows of K contiguous elements per node:
-//   int8 planes [kSlices][P][R][K], then (256-byte aligned) int32 exponents [P][R], then
+//   int8 planes [S][P][R][K], then (256-byte aligned) int32 exponents [P][R], then
 //   (256-byte aligned) 4-byte encoder scratch [P][R].
-// value(p, r, k) = 2^expo[p][r] * sum_t planes[t][p][r][k] * 2^(-7 (t + 1))
+// value(p, r, k) = 2^expo[p][r] * sum_t planes[t][p][r][k] * 2^(-8 (t + 1))
 struct SlicedLayout {
     int64_t plane_bytes;   // P * R * K
     int64_t expo_offset;   // byte offset of the exponents
     int64_t amax_offset;   // byte offset of the encoder's scratch
     int64_t total_bytes;
 };
-SlicedLayout sliced_layout(int64_t P, int64_t rows, int64_t K);
+SlicedLayout sliced_layout(int slices, int64_t P, int64_t rows, int64_t K);
 
 // Whether the plan's shapes fit this path (K = N0/n a multiple of 16, block counts the encoder
 // is instantiated for, sliced buffers no larger than the FP64 share buffers they replace).

@@ -253,7 +253,7 @@ def _run_additive_case(cfg, seeds, precision=g.GPD_PREC_AUTO):
     return outcomes
 
 
-@pytest.mark.parametrize("precision", [g.GPD_PREC_AUTO, g.GPD_PREC_FP64_SLICED])
+@pytest.mark.parametrize("precision", [g.GPD_PREC_AUTO, g.GPD_PREC_FP64_SLICED, g.GPD_PREC_FP64_SLICED40])
 def test_config3_scaled_additive_errors(precision):
     cfg = wl.scaled_down(wl.CONFIG_3_MATMUL, 8)                         # 1024 x 1024 x 64, same code
     outcomes = _run_additive_case(cfg, cfg.inject_seeds, precision)
@@ -402,7 +402,7 @@ def test_config4_full_size_layer():
 # (tests/golden/cfg3_full_expected.json, written by make_cfg3_expected.py from oracle/ alone),
 # sampled worker outputs and sampled rows of the decoded product against FP64 definitions
 # --------------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("precision", [g.GPD_PREC_AUTO, g.GPD_PREC_FP64_SLICED])
+@pytest.mark.parametrize("precision", [g.GPD_PREC_AUTO, g.GPD_PREC_FP64_SLICED, g.GPD_PREC_FP64_SLICED40])
 def test_config3_full_size_against_oracle_decisions(precision):
     import json
     import os
@@ -419,10 +419,11 @@ def test_config3_full_size_against_oracle_decisions(precision):
     pos = np.array(gold["sample_positions"])
     got = host(Z.reshape(cfg.P, L)[:, torch.from_numpy(pos).cuda()])
     want = np.array(gold["clean_outputs_at_samples"])
-    if precision == g.GPD_PREC_FP64_SLICED:
-        # digit planes: < 4e-13 of (row scale x column scale) per term, sqrt(K) = 45 terms deep, scales
-        # within 4.07 x 4.5 standard deviations of each operand (the bound is derived in test_gpu_sliced.py)
-        assert np.abs(got - want).max() <= 2e-9 * gold["scale"]
+    if precision in (g.GPD_PREC_FP64_SLICED, g.GPD_PREC_FP64_SLICED40):
+        # digit planes: < 6e-15 (1.4e-12 with five planes) of (row scale x column scale) per term, sqrt(K) = 45
+        # terms deep, scales within 4.07 x 4.5 standard deviations of each operand (bound derived in
+        # test_gpu_sliced.py)
+        assert np.abs(got - want).max() <= (3e-11 if precision == g.GPD_PREC_FP64_SLICED else 7e-9) * gold["scale"]
     else:
         assert np.abs(got - want).max() <= 1e-12 * gold["scale"] * 8      # FP64 products, K = 2048
     rows = np.arange(0, cfg.N1, cfg.N1 // 32)

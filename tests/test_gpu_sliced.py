@@ -1,12 +1,16 @@
-"""GPU parity of the integer-slice product path (GPD_PREC_FP64_SLICED) against the FP64 oracle.
+"""GPU parity of the integer-slice product paths (GPD_PREC_FP64_SLICED, GPD_PREC_FP64_SLICED40)
+against the FP64 oracle.
 
-The shares are stored as six signed 7-bit digits per value under one power-of-two scale 2^e per
-operand row, chosen so that 2^e lies in (2.03, 4.07] times the row's largest magnitude.  Digit-plane
-products are exact, so a worker output differs from the exact product of the FP64 shares only by
-(i) the digits cut below 2^-43 of each scale and (ii) the 15 plane pairs of weight below 128^-7 that
-are not formed: per term of the contraction at most 2^-43 + 4096 * 5.03 * 128^-8 < 4e-13 of
-2^ea 2^eb.  The tests allow 6 sqrt(K) times that (signs of the per-term errors are independent),
-which a single missing plane pair of the kept set would exceed by an order of magnitude.
+The shares are stored as S = 6 (or 5) signed 8-bit digits per value under one power-of-two scale 2^e
+per operand row, chosen so that 2^e lies in (2.03, 4.07] times the row's largest magnitude.
+Digit-plane products are exact, so a worker output differs from the exact product of the FP64 shares
+only by (i) the digits cut below 2^-(8S+1) of each scale and (ii) the plane pairs of weight below
+256^-(S+1) that are not formed (S - 1 of them at the largest dropped weight, |digit| <= 128): per
+term of the contraction at most 2^-(8S+1) + (S - 1) * 1.004 * 2^14 * 256^-(S+2) of 2^ea 2^eb, which is
+6.5e-15 for S = 6 and 1.4e-12 for S = 5 (reached only with every digit at its largest value).  The
+tests allow 4 sqrt(K) times that (signs of the per-term errors are independent); a single missing
+plane pair of the kept set, 256 times heavier than the heaviest dropped one, exceeds it several
+times over.
 """
 
 import numpy as np
@@ -25,7 +29,8 @@ from oracle.locate import NO_ERROR, CORRECTED, locate_subspace, tolerances_for  
 from oracle import inject as oinj                        # noqa: E402
 from tests.gpu_pipeline import CodedProduct, dev, host   # noqa: E402
 
-PER_TERM = 4e-13
+PER_TERM = {6: 6.5e-15, 5: 1.4e-12}
+PRECISIONS = {6: g.GPD_PREC_FP64_SLICED, 5: g.GPD_PREC_FP64_SLICED40}
 SCALE_OVER_MAX = 4.07
 
 
@@ -36,17 +41,17 @@ def _inputs(N1, N0, B, seed, w_scale=1.0, x_scale=1.0):
     return W, X
 
 
-def _output_tolerance(Wsh, Xsh):
+def _output_tolerance(Wsh, Xsh, S=6):
     """Per-entry bound [P][M][N] from the oracle's FP64 shares (see the module docstring)."""
     K = Wsh.shape[2]
     row = SCALE_OVER_MAX * np.abs(Wsh).max(axis=2)         # [P][M]  >= 2^ea
     col = SCALE_OVER_MAX * np.abs(Xsh).max(axis=1)         # [P][N]  >= 2^eb
-    return 6.0 * np.sqrt(K) * PER_TERM * row[:, :, None] * col[:, None, :]
+    return 4.0 * np.sqrt(K) * PER_TERM[S] * row[:, :, None] * col[:, None, :]
 
 
-def _sliced_products(code, W, X):
-    cp = CodedProduct(code, precision=g.GPD_PREC_FP64_SLICED)
-    assert cp.plan.query(g.GPD_Q_PRECISION) == g.GPD_PREC_FP64_SLICED and cp.np_dtype == np.float64
+def _sliced_products(code, W, X, S=6):
+    cp = CodedProduct(code, precision=PRECISIONS[S])
+    assert cp.plan.query(g.GPD_Q_PRECISION) == PRECISIONS[S] and cp.np_dtype == np.float64
     cp.encode_W(W)
     Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
     assert g.gpd_device_status() == 0
@@ -62,18 +67,19 @@ def _sliced_products(code, W, X):
     (512, 768, 96, 4, 4, 1, 40),        # 16 blocks per share of W, 40 nodes, threshold 19
     (256, 256, 96, 2, 4, 3, 30),        # 12 blocks per share of X, threshold 27
 ])
-def test_sliced_worker_products_match_oracle(N1, N0, B, m, n, d1, P):
+@pytest.mark.parametrize("S", [6, 5])
+def test_sliced_worker_products_match_oracle(N1, N0, B, m, n, d1, P, S):
     W, X = _inputs(N1, N0, B, seed=N1 + N0 + B)
     code = GPCode(N1, N0, B, m, n, d1, 1, P)
-    cp, Z = _sliced_products(code, W, X)
+    cp, Z = _sliced_products(code, W, X, S)
     Wsh, Xsh = op.encode_W(W, code), op.encode_X(X, code)
     Zo = op.worker_products(Wsh, Xsh)
     got = cp.outputs_as_array(g.GPD_FWD, Z)
     assert np.isfinite(got).all()
-    tol = _output_tolerance(Wsh, Xsh)
+    tol = _output_tolerance(Wsh, Xsh, S)
     assert (np.abs(got - Zo) <= tol).all(), float((np.abs(got - Zo) / tol).max())
     # and the bound is far below what FP32 shares could give: relative to the output scale
-    assert np.abs(got - Zo).max() < 1e-8 * np.sqrt(np.mean(Zo ** 2))
+    assert np.abs(got - Zo).max() < (1e-10 if S == 6 else 2e-8) * np.sqrt(np.mean(Zo ** 2))
 
 
 def test_sliced_scales_zero_rows_and_tiny_values():
@@ -98,11 +104,12 @@ def test_sliced_scales_zero_rows_and_tiny_values():
     assert op.rel_fro(S, op.ref_forward(W, X)) < 1e-4
 
 
-def test_sliced_pipeline_locates_and_decodes_like_the_oracle():
+@pytest.mark.parametrize("S", [6, 5])
+def test_sliced_pipeline_locates_and_decodes_like_the_oracle(S):
     N1, N0, B, m, n, d1, P = 512, 512, 128, 2, 4, 2, 25
     W, X = _inputs(N1, N0, B, seed=11)
     code = GPCode(N1, N0, B, m, n, d1, 1, P)
-    cp, Z = _sliced_products(code, W, X)
+    cp, Z = _sliced_products(code, W, X, S)
     Zo = op.worker_products(op.encode_W(W, code), op.encode_X(X, code))
     scale = float(np.sqrt(np.mean(Zo ** 2)))
     ref = op.ref_forward(W, X)
