@@ -3,7 +3,8 @@
 // The shares W~_p (Eq. 1) and X~_p (Theorem 2) are evaluated in FP64 exactly as in encode.cu, but
 // instead of being stored as doubles each value a is stored as S = 6 (or 5) signed 8-bit digits:
 //     a = 2^e * sum_{t=0..S-1} d_t * 256^-(t+1)  (+ remainder below 2^(e - 8 S - 1)),   d_t in [-128, 127],
-// with one exponent e per row of W~_p (per column of X~_p) chosen so that |a| < 0.4923 * 2^e.  The
+// with one exponent e per row of W~_p (per column of X~_p) chosen so that |a| < 0.4923 * 2^e (from
+// a bound of the row's magnitudes for W~_p, from the column's largest magnitude for X~_p).  The
 // digits of one operand form S int8 planes; products of planes are exact in int32 on the tensor
 // cores (gemm_i8.cu), which gives FP64-class worker products at integer-tensor-core speed.
 // Both operands are written K-major: W planes [S][P][M][K], X planes [S][P][N][K] (transposed).
@@ -79,64 +80,39 @@ __device__ __forceinline__ void digits4(const double (&a)[4], double scale, unsi
 }
 
 // ---- W side: operand rows are rows of the share (K = block columns, contiguous in the source) ----
-// Pass 1: one CTA per share row r; an upper bound of max_c |W~_p[r][c]| for every p.  The share
-// values are evaluated in FP32 here (they only fix a power-of-two scale); the bound adds the
-// worst-case FP32 evaluation error (NBLK + 1) 2^-23 sum_b |coef_pb| max_c |W_b[r][c]|.
+// Pass 1: one CTA per share row r.  The scale of W~_p[r][:] comes from the bound
+//     max_c |W~_p[r][c]| <= sum_b |coef_pb| max_c |W_b[r][c]|,
+// which needs one streaming pass over W and no evaluation of the shares; it overestimates the true
+// maximum by the cancellation between blocks (a factor below the number of blocks, about 3 for
+// eight Gaussian blocks), i.e. it spends one to two of the 8 S bits.
 template <int NBLK>
-__global__ void __launch_bounds__(256) rowmax_kernel(SliceParams prm) {
-    __shared__ unsigned int sMax[kMaxNodes];     // bit patterns of non-negative floats order like integers
-    __shared__ unsigned int sBlk[NBLK];
-    extern __shared__ double s_coef[];           // [P][NBLK]
-    float* s_cf32 = reinterpret_cast<float*>(s_coef + prm.P * NBLK);
-    for (int i = threadIdx.x; i < prm.P * NBLK; i += 256) {
-        const double c = prm.coef[i];
-        s_coef[i] = c;
-        s_cf32[i] = (float)c;
-    }
-    if (threadIdx.x < kMaxNodes) sMax[threadIdx.x] = 0u;
+__global__ void __launch_bounds__(256) rowscale_kernel(SliceParams prm) {
+    __shared__ unsigned int sBlk[NBLK];          // bit patterns of non-negative floats order like integers
     if (threadIdx.x < NBLK) sBlk[threadIdx.x] = 0u;
     __syncthreads();
     const int64_t r = blockIdx.x;
     const int lane = threadIdx.x & 31;
-    // every lane of a warp runs the same number of rounds (the warp reductions need all 32)
-    for (int64_t c0 = 0; c0 < prm.bc; c0 += 1024) {
-        const int64_t c = c0 + (int64_t)threadIdx.x * 4;
-        float4 x[NBLK];
+    unsigned int m[NBLK];
+#pragma unroll
+    for (int b = 0; b < NBLK; ++b) m[b] = 0u;
+    for (int64_t c = (int64_t)threadIdx.x * 4; c < prm.bc; c += 1024) {
 #pragma unroll
         for (int b = 0; b < NBLK; ++b) {
             const int gi = b / prm.gc, gj = b - gi * prm.gc;
-            x[b] = c < prm.bc ? __ldg(reinterpret_cast<const float4*>(prm.src + (gi * prm.br + r) * prm.ld + gj * prm.bc + c))
-                              : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int b = 0; b < NBLK; ++b) {
-            const unsigned int m = max(max(__float_as_uint(fabsf(x[b].x)), __float_as_uint(fabsf(x[b].y))),
-                                       max(__float_as_uint(fabsf(x[b].z)), __float_as_uint(fabsf(x[b].w))));
-            const unsigned int w = __reduce_max_sync(0xffffffffu, m);
-            if (lane == 0) atomicMax(&sBlk[b], w);
-        }
-#pragma unroll 2
-        for (int p = 0; p < prm.P; ++p) {
-            const float* cf = s_cf32 + p * NBLK;
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-            for (int b = 0; b < NBLK; ++b) {
-                const float k = cf[b];
-                a0 = fmaf(k, x[b].x, a0); a1 = fmaf(k, x[b].y, a1);
-                a2 = fmaf(k, x[b].z, a2); a3 = fmaf(k, x[b].w, a3);
-            }
-            const unsigned int m = max(max(__float_as_uint(fabsf(a0)), __float_as_uint(fabsf(a1))),
-                                       max(__float_as_uint(fabsf(a2)), __float_as_uint(fabsf(a3))));
-            const unsigned int w = __reduce_max_sync(0xffffffffu, m);
-            if (lane == 0) atomicMax(&sMax[p], w);
+            const float4 v = __ldg(reinterpret_cast<const float4*>(prm.src + (gi * prm.br + r) * prm.ld + gj * prm.bc + c));
+            m[b] = max(m[b], max(max(__float_as_uint(fabsf(v.x)), __float_as_uint(fabsf(v.y))),
+                                 max(__float_as_uint(fabsf(v.z)), __float_as_uint(fabsf(v.w)))));
         }
     }
+#pragma unroll
+    for (int b = 0; b < NBLK; ++b) {             // all 32 lanes are here: the column loop has ended
+        const unsigned int w = __reduce_max_sync(0xffffffffu, m[b]);
+        if (lane == 0) atomicMax(&sBlk[b], w);
+    }
     __syncthreads();
-    if (threadIdx.x < prm.P) {
-        const int p = threadIdx.x;
-        double spread = 0.0;
-        for (int b = 0; b < NBLK; ++b) spread += fabs(s_coef[p * NBLK + b]) * (double)__uint_as_float(sBlk[b]);
-        const double bound = (double)__uint_as_float(sMax[p]) + (NBLK + 1) * 1.1920928955078125e-7 * spread;
+    for (int p = threadIdx.x; p < prm.P; p += 256) {
+        double bound = 0.0;
+        for (int b = 0; b < NBLK; ++b) bound += fabs(prm.coef[p * NBLK + b]) * (double)__uint_as_float(sBlk[b]);
         prm.expo[(int64_t)p * prm.br + r] = slice_exponent(abs_hi(bound));
     }
 }
@@ -254,7 +230,7 @@ __global__ void __launch_bounds__(256) colpass_kernel(SliceParams prm) {
 
 template <int NBLK>
 gpd_status launch_rows(const SliceParams& prm, int slices, cudaStream_t st) {
-    rowmax_kernel<NBLK><<<(unsigned)prm.br, 256, (sizeof(double) + sizeof(float)) * prm.P * NBLK, st>>>(prm);
+    rowscale_kernel<NBLK><<<(unsigned)prm.br, 256, 0, st>>>(prm);
     if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
     const int64_t work = prm.br * (prm.bc / 4);
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, 148 * 16));
@@ -296,7 +272,7 @@ bool sliced_supported(const gpd_plan_s* plan) {
     };
     // int32 accumulation of up to 6 plane pairs of |digit| <= 128 over K terms
     if (K % 16 != 0 || K > 16384 || !ok_blk(nb_w) || !ok_blk(nb_x)) return false;
-    // the scale pass evaluates the shares in FP32: the encoding coefficients must fit comfortably
+    // scales are tracked through FP32 magnitudes of the inputs times the coefficients
     for (double c : plan->coefW) if (!(std::fabs(c) < 1e30)) return false;
     for (double c : plan->coefX) if (!(std::fabs(c) < 1e30)) return false;
     // the sliced operands live in buffers sized for the FP64 shares they replace

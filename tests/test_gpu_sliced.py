@@ -2,7 +2,9 @@
 against the FP64 oracle.
 
 The shares are stored as S = 6 (or 5) signed 8-bit digits per value under one power-of-two scale 2^e
-per operand row, chosen so that 2^e lies in (2.03, 4.07] times the row's largest magnitude.
+per operand row.  For a column of X~_p, 2^e lies in (2.03, 4.07] times the column's largest magnitude;
+for a row of W~_p it lies in the same range times the bound sum_b |coef_pb| max_c |W_b[r][c]| of the
+row's magnitudes (W_b the blocks the share combines).
 Digit-plane products are exact, so a worker output differs from the exact product of the FP64 shares
 only by (i) the digits cut below 2^-(8S+1) of each scale and (ii) the plane pairs of weight below
 256^-(S+1) that are not formed (S - 1 of them at the largest dropped weight, |digit| <= 128): per
@@ -41,10 +43,19 @@ def _inputs(N1, N0, B, seed, w_scale=1.0, x_scale=1.0):
     return W, X
 
 
-def _output_tolerance(Wsh, Xsh, S=6):
-    """Per-entry bound [P][M][N] from the oracle's FP64 shares (see the module docstring)."""
+def _row_bound(W, code):
+    """sum_b |coef_pb| max_c |W_b[r][c]| for every node p and share row r: [P][M]."""
+    M, K = code.N1 // code.m, code.N0 // code.n
+    blkmax = np.abs(W.astype(np.float64)).reshape(code.m, M, code.n, K).max(axis=3)      # [m][M][n]
+    coef = np.abs(code.points)[:, None, None] ** code.exp_W()[None, :, :]                 # [P][m][n]
+    return np.einsum("pij,irj->pr", coef, blkmax)
+
+
+def _output_tolerance(W, code, Wsh, Xsh, S=6):
+    """Per-entry bound [P][M][N] from the inputs and the oracle's FP64 shares (see the module docstring)."""
     K = Wsh.shape[2]
-    row = SCALE_OVER_MAX * np.abs(Wsh).max(axis=2)         # [P][M]  >= 2^ea
+    row = SCALE_OVER_MAX * _row_bound(W, code)             # [P][M]  >= 2^ea
+    assert (row >= SCALE_OVER_MAX * np.abs(Wsh).max(axis=2) * (1 - 1e-12)).all()
     col = SCALE_OVER_MAX * np.abs(Xsh).max(axis=1)         # [P][N]  >= 2^eb
     return 4.0 * np.sqrt(K) * PER_TERM[S] * row[:, :, None] * col[:, None, :]
 
@@ -76,7 +87,7 @@ def test_sliced_worker_products_match_oracle(N1, N0, B, m, n, d1, P, S):
     Zo = op.worker_products(Wsh, Xsh)
     got = cp.outputs_as_array(g.GPD_FWD, Z)
     assert np.isfinite(got).all()
-    tol = _output_tolerance(Wsh, Xsh, S)
+    tol = _output_tolerance(W, code, Wsh, Xsh, S)
     assert (np.abs(got - Zo) <= tol).all(), float((np.abs(got - Zo) / tol).max())
     # and the bound is far below what FP32 shares could give: relative to the output scale
     assert np.abs(got - Zo).max() < (1e-10 if S == 6 else 2e-8) * np.sqrt(np.mean(Zo ** 2))
@@ -97,7 +108,7 @@ def test_sliced_scales_zero_rows_and_tiny_values():
     Zo = op.worker_products(Wsh, Xsh)
     got = cp.outputs_as_array(g.GPD_FWD, Z)
     assert (got[:, 7, :] == 0.0).all() and (got[:, :, 5] == 0.0).all()
-    assert (np.abs(got - Zo) <= _output_tolerance(Wsh, Xsh)).all()
+    assert (np.abs(got - Zo) <= _output_tolerance(W, code, Wsh, Xsh)).all()
     r = cp.locate(g.GPD_FWD, Z)
     assert r.outcome == NO_ERROR
     S = cp.decode(g.GPD_FWD, Z)
