@@ -11,12 +11,16 @@
 // accumulators are adjacent in tensor memory, so one tcgen05.mma of N = 64 (S - s) columns
 // (two when that exceeds 256) covers all pairs of plane s: 8 (6) instructions per 32 elements of K.
 //
-// Warp roles: warp 0 one lane issues the TMA copies (2 S per 64-element k-block, 3-stage ring),
-// warp 1 allocates tensor memory and one lane issues the MMAs, warps 2..5 read the accumulators
-// back, combine them in FP64 (sum_g acc_g 2^-8g, then the row and column powers of two) and store.
+// One CTA per SM walks the output tiles.  Warp roles: warp 0 one lane issues the TMA copies (2 S per
+// 64-element k-block, 3-stage ring that runs on across tiles), warp 1 allocates tensor memory and
+// one lane issues the MMAs, warps 2..9 read the accumulators back and combine them in FP64
+// (sum_g acc_g 2^-8g), release tensor memory to the next tile's MMAs, then apply the row and column
+// powers of two and store while that tile's main loop is already running.
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains its copies,
 // frees its tensor memory and returns.
 #include <cuda.h>
+
+#include <algorithm>
 
 #include "slice_common.h"
 
@@ -31,7 +35,7 @@ constexpr int B_PLANE_BYTES = BN * BK;                // 4 KB
 __host__ __device__ constexpr int stage_bytes(int S) { return S * (A_PLANE_BYTES + B_PLANE_BYTES); }   // 72 KB (60 KB)
 __host__ __device__ constexpr int smem_bytes(int S) { return STAGES * stage_bytes(S) + 1024; }
 constexpr int TMEM_COLS = 512;                        // S x 64 used; allocations are powers of two
-constexpr int kEpiWarps = 4;
+constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + kEpiWarps * 32;
 constexpr long long kWaitCycles = 2000000000LL;       // about one second
 
@@ -43,6 +47,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
@@ -114,20 +121,17 @@ struct I8Params {
 template <int S>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, I8Params prm,
-                      int tiles_m, int tiles_n) {
+                      int tiles_m, int tiles_n, int tiles) {
     constexpr int STAGE_BYTES = stage_bytes(S);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_bar;
+    // full/empty: operand ring (runs on across the tiles of this CTA); acc_full: a tile's accumulators
+    // are complete; acc_empty: the epilogue warps have read them, the next tile may overwrite them
+    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full, acc_empty;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ double col_scale[BN];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x;
-    const int tn = tile % tiles_n, tm = (tile / tiles_n) % tiles_m;
-    const int p = tile / (tiles_n * tiles_m);
-    const int m0 = tm * BM, n0 = tn * BN;
     const int num_kb = (int)((prm.K + BK - 1) / BK);
 
     if (threadIdx.x == 0) {
@@ -135,17 +139,14 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&acc_bar, 1);
+        mbar_init(&acc_full, 1);
+        mbar_init(&acc_empty, kEpiWarps);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + BN) {
-        const int j = threadIdx.x - 64;
-        col_scale[j] = (n0 + j < prm.N) ? exp2i(prm.eb[(int64_t)p * prm.N + n0 + j]) : 0.0;
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -155,108 +156,143 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 
     auto A_plane = [&](int s, int t) { return smem + s * STAGE_BYTES + t * A_PLANE_BYTES; };
     auto B_plane = [&](int s, int t) { return smem + s * STAGE_BYTES + S * A_PLANE_BYTES + t * B_PLANE_BYTES; };
+    // tile -> (node p, row tile, column tile); consecutive CTAs take consecutive tiles of one round
+    auto tile_origin = [&](int tile, int& p, int& m0, int& n0) {
+        const int tn = tile % tiles_n, tm = (tile / tiles_n) % tiles_m;
+        p = tile / (tiles_n * tiles_m);
+        m0 = tm * BM;
+        n0 = tn * BN;
+    };
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
-            int issued = 0;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (kb / STAGES) & 1;
-                if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) break;
-                mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+            int it = 0;                          // k-blocks issued so far, over all tiles
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+                int p, m0, n0;
+                tile_origin(tile, p, m0, n0);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) { ok = false; break; }
+                    mbar_expect_tx(&full_bar[s], STAGE_BYTES);
 #pragma unroll
-                for (int t = 0; t < S; ++t) {
-                    tma_load_3d(A_plane(s, t), &tmA, kb * BK, m0, t * prm.P + p, &full_bar[s]);
-                    tma_load_3d(B_plane(s, t), &tmB, kb * BK, n0, t * prm.P + p, &full_bar[s]);
+                    for (int t = 0; t < S; ++t) {
+                        tma_load_3d(A_plane(s, t), &tmA, kb * BK, m0, t * prm.P + p, &full_bar[s]);
+                        tma_load_3d(B_plane(s, t), &tmB, kb * BK, n0, t * prm.P + p, &full_bar[s]);
+                    }
                 }
-                ++issued;
             }
             if (*abort_p) {                      // let copies still in flight land before the CTA exits
-                for (int kb = issued > STAGES ? issued - STAGES : 0; kb < issued; ++kb) {
+                for (int j = it > STAGES ? it - STAGES : 0; j < it; ++j) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(&full_bar[kb % STAGES], (kb / STAGES) & 1) && clock64() - t0 < kWaitCycles) {}
+                    while (!mbar_try_wait(&full_bar[j % STAGES], (j / STAGES) & 1) && clock64() - t0 < kWaitCycles) {}
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
+            int it = 0, ti = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (kb / STAGES) & 1;
-                if (!mbar_wait(&full_bar[s], ph, abort_p)) { ok = false; break; }
+            for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++ti) {
+                // the previous tile's accumulators must have been read
+                if (!mbar_wait(&acc_empty, (ti & 1) ^ 1, abort_p)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a0 = smem_u32(A_plane(s, 0)), b0 = smem_u32(B_plane(s, 0));
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(&full_bar[s], ph, abort_p)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a0 = smem_u32(A_plane(s, 0)), b0 = smem_u32(B_plane(s, 0));
 #pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k) {
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
 #pragma unroll
-                    for (int ta = 0; ta < S; ++ta) {
-                        // planes tb = 0 .. S-1-ta of B in one operand of 64 (S - ta) rows, at most 256 per MMA;
-                        // the pair (ta, tb) lands in accumulator group ta + tb = columns 64 (ta + tb)
-                        const uint64_t da = desc_sw64(a0 + ta * A_PLANE_BYTES + k * UMMA_K);
-                        const int n_total = BN * (S - ta);
-                        const int n_first = n_total > 256 ? 256 : n_total;
-                        // the plane-0 instruction of the first k-step overwrites every group
-                        const uint32_t acc = (kb > 0 || k > 0 || ta > 0) ? 1u : 0u;
-                        umma_i8(tmem_base + BN * ta, da, desc_sw64(b0 + k * UMMA_K), idesc_i8(n_first), acc);
-                        if (n_total > 256)
-                            umma_i8(tmem_base + BN * ta + 256, da, desc_sw64(b0 + 4 * B_PLANE_BYTES + k * UMMA_K),
-                                    idesc_i8(n_total - 256), acc);
+                        for (int ta = 0; ta < S; ++ta) {
+                            // planes tb = 0 .. S-1-ta of B in one operand of 64 (S - ta) rows, at most 256 per MMA;
+                            // the pair (ta, tb) lands in accumulator group ta + tb = columns 64 (ta + tb)
+                            const uint64_t da = desc_sw64(a0 + ta * A_PLANE_BYTES + k * UMMA_K);
+                            const int n_total = BN * (S - ta);
+                            const int n_first = n_total > 256 ? 256 : n_total;
+                            // the plane-0 instruction of a tile's first k-step overwrites every group
+                            const uint32_t acc = (kb > 0 || k > 0 || ta > 0) ? 1u : 0u;
+                            umma_i8(tmem_base + BN * ta, da, desc_sw64(b0 + k * UMMA_K), idesc_i8(n_first), acc);
+                            if (n_total > 256)
+                                umma_i8(tmem_base + BN * ta + 256, da, desc_sw64(b0 + 4 * B_PLANE_BYTES + k * UMMA_K),
+                                        idesc_i8(n_total - 256), acc);
+                        }
                     }
+                    umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
                 }
-                umma_commit(&empty_bar[s]);          // stage reusable once these MMAs have read it
+                if (ok) umma_commit(&acc_full);      // this tile's accumulators complete
             }
-            if (ok) umma_commit(&acc_bar);           // accumulators complete
         }
     } else {
         // ------------------------------ epilogue ------------------------------
-        const bool acc_ready = mbar_wait(&acc_bar, 0, abort_p);
-        __syncwarp();
-        if (__all_sync(0xffffffffu, acc_ready)) {    // tcgen05.ld is warp-collective: all lanes or none
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int q = warp & 3;                  // this warp may touch TMEM lanes 32q .. 32q+31
+        const int q = warp & 3;                      // this warp may touch TMEM lanes 32q .. 32q+31
+        const int c0 = ((warp - 2) >> 2) * 32;       // two warps per lane quarter: 32 columns each
+        int ti = 0;
+        for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++ti) {
+            int p, m0, n0;
+            tile_origin(tile, p, m0, n0);
             const int64_t gm = (int64_t)m0 + q * 32 + lane;
+            const int64_t gn = (int64_t)n0 + c0 + lane;  // lane j keeps the scale of column c0 + j
             const double row_scale = gm < prm.M ? exp2i(prm.ea[(int64_t)p * prm.M + gm] - 2 * kDigitBits) : 0.0;
-            double* C = prm.C + (int64_t)p * prm.M * prm.N;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                double v[32];
+            const double col_scale = gn < prm.N ? exp2i(prm.eb[(int64_t)p * prm.N + gn]) : 0.0;
+            const bool acc_ready = mbar_wait(&acc_full, ti & 1, abort_p);
+            __syncwarp();
+            if (!__all_sync(0xffffffffu, acc_ready)) break;   // tcgen05.ld is warp-collective: all lanes or none
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            double v[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = 0.0;
+            for (int j = 0; j < 32; ++j) v[j] = 0.0;
+            // smallest weight first; two groups are in flight per wait (one for the odd one out)
+            auto tmem_ld32 = [&](uint32_t (&r)[32], int g) {
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(BN * g + c0);
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                    : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                      "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                      "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                      "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                    : "r"(taddr));
+            };
 #pragma unroll
-                for (int g = S - 1; g >= 0; --g) {             // smallest weight first
-                    uint32_t r[32];
-                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(BN * g + c0);
-                    asm volatile(
-                        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                        : "r"(taddr));
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    const double w = exp2i(-kDigitBits * g);
+            for (int g = S - 1; g >= 0; g -= 2) {
+                uint32_t r0[32], r1[32];
+                tmem_ld32(r0, g);
+                if (g >= 1) tmem_ld32(r1, g - 1);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const double w0 = exp2i(-kDigitBits * g);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = fma(i2d(r[j]), w, v[j]);
+                for (int j = 0; j < 32; ++j) v[j] = fma(i2d(r0[j]), w0, v[j]);
+                if (g >= 1) {
+                    const double w1 = exp2i(-kDigitBits * (g - 1));
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = fma(i2d(r1[j]), w1, v[j]);
                 }
+            }
+            // the accumulators are in registers: hand tensor memory back to the MMA warp, then scale
+            // and store while the next tile's main loop runs
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty);
+            double* crow = prm.C + (int64_t)p * prm.M * prm.N + gm * prm.N + n0 + c0;
+            const bool vec = (prm.N & 1) == 0 && n0 + c0 + 32 <= prm.N;
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                double2 o;                               // column scales come from the lanes that hold them
+                o.x = v[j] * row_scale * __shfl_sync(0xffffffffu, col_scale, j);
+                o.y = v[j + 1] * row_scale * __shfl_sync(0xffffffffu, col_scale, j + 1);
                 if (gm < prm.M) {
-                    double* crow = C + gm * prm.N + n0 + c0;
-                    if ((prm.N & 1) == 0 && n0 + c0 + 32 <= prm.N) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 2) {
-                            double2 o;
-                            o.x = v[j] * row_scale * col_scale[c0 + j];
-                            o.y = v[j + 1] * row_scale * col_scale[c0 + j + 1];
-                            __stcs(reinterpret_cast<double2*>(crow + j), o);
-                        }
+                    if (vec) {
+                        __stcs(reinterpret_cast<double2*>(crow + j), o);
                     } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (n0 + c0 + j < prm.N) crow[j] = v[j] * row_scale * col_scale[c0 + j];
+                        if (n0 + c0 + j < prm.N) crow[j] = o.x;
+                        if (n0 + c0 + j + 1 < prm.N) crow[j + 1] = o.y;
                     }
                 }
             }
@@ -329,7 +365,12 @@ gpd_status gemm_sliced_launch(gpd_plan_s* plan, const void* W_sliced, const void
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GPD_ERR_CUDA;
     const int tiles_n = (int)((prm.N + BN - 1) / BN), tiles_m = (int)((prm.M + BM - 1) / BM);
     const int64_t tiles = (int64_t)tiles_n * tiles_m * prm.P;
-    kernel<<<(unsigned)tiles, kThreads, smem, st>>>(tmA, tmB, prm, tiles_m, tiles_n);
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        sms <= 0)
+        sms = 148;
+    const unsigned grid = (unsigned)std::min<int64_t>(tiles, sms);      // persistent: one CTA per SM walks the tiles
+    kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, prm, tiles_m, tiles_n, (int)tiles);
     return launch_ok();
 }
 
