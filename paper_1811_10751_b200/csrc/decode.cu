@@ -2,7 +2,7 @@
 // keep the wanted coefficients (Theorem 2's proof; the Vandermonde system of the decoding
 // appendix).  Done as one small FP64 factorisation followed by a bandwidth-bound streaming pass:
 //
-//   1. decode_matrix_kernel (one warp): Householder QR of the |S| x Q Vandermonde matrix of the
+//   1. decode_matrix_kernel (one CTA): Householder QR of the |S| x Q Vandermonde matrix of the
 //      nodes in use; row w of D = e_w^T R^-1 Q^T is the linear functional that reads coefficient
 //      w of the least-squares polynomial off the node values.  Normal equations are never
 //      formed (the Vandermonde matrix is too ill-conditioned for that at thresholds near 30).
@@ -28,14 +28,25 @@ struct MatrixParams {
                                      // polynomial at the flagged nodes' points (share regeneration)
 };
 
-__global__ void __launch_bounds__(32) decode_matrix_kernel(MatrixParams prm) {
+constexpr int kMatrixThreads = 256;
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// One CTA of 8 warps.  Factorisation: every warp forms the column norm itself (lanes over rows),
+// thread c of the CTA then reflects column k + c.  Rows of the pseudo-inverse: one warp per wanted
+// coefficient, lanes over the entries of y (Q <= 32) and of x (rows <= 64, two per lane).
+__global__ void __launch_bounds__(kMatrixThreads) decode_matrix_kernel(MatrixParams prm) {
     __shared__ double A[kMaxNodes][kMaxQ + 1];       // Vandermonde rows of the nodes in use -> R
     __shared__ double Vh[kMaxNodes][kMaxQ + 1];      // Householder vectors (column k = reflector k)
     __shared__ int node_of[kMaxNodes];
     __shared__ int s_rows;
-    const int lane = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int P = prm.P, Q = prm.Q;
-    if (lane == 0) {
+    if (tid == 0) {
         int rows = 0;
         bool ok = true;
         if (prm.have_mask) {
@@ -50,11 +61,11 @@ __global__ void __launch_bounds__(32) decode_matrix_kernel(MatrixParams prm) {
         s_rows = ok ? rows : 0;
         prm.gate[0] = ok ? 1 : 0;
     }
-    __syncwarp();
+    __syncthreads();
     const int rows = s_rows;
-    for (int i = lane; i < prm.n_wanted * P; i += 32) prm.D[i] = 0.0;
+    for (int i = tid; i < prm.n_wanted * P; i += kMatrixThreads) prm.D[i] = 0.0;
     if (rows == 0) return;
-    for (int r = lane; r < rows; r += 32) {
+    for (int r = tid; r < rows; r += kMatrixThreads) {
         const double b = prm.points[node_of[r]];
         if (prm.regen) {
             // regeneration only needs the polynomial's values, not its monomial coefficients: the
@@ -66,53 +77,58 @@ __global__ void __launch_bounds__(32) decode_matrix_kernel(MatrixParams prm) {
             for (int c = 0; c < Q; ++c) { A[r][c] = acc; acc *= b; }
         }
     }
-    __syncwarp();
-    // Householder triangularisation; lane c owns column c
+    __syncthreads();
+    // Householder triangularisation
     for (int k = 0; k < Q; ++k) {
-        double sigma = 0.0;
-        for (int r = k; r < rows; ++r) sigma += A[r][k] * A[r][k];     // every lane, same value
+        double part = 0.0;
+        for (int r = k + lane; r < rows; r += 32) part += A[r][k] * A[r][k];
+        const double sigma = warp_sum(part);         // same value in every warp (same order of additions)
         const double akk = A[k][k];
         const double alpha = akk >= 0.0 ? -sqrt(sigma) : sqrt(sigma);
         const double vnorm = sqrt(fmax(sigma - 2.0 * alpha * akk + alpha * alpha, 1e-300));
-        __syncwarp();
-        for (int r = k + lane; r < rows; r += 32) Vh[r][k] = (A[r][k] - (r == k ? alpha : 0.0)) / vnorm;
-        __syncwarp();
-        if (lane >= k && lane < Q) {
-            double dot = 0.0;
-            for (int r = k; r < rows; ++r) dot += Vh[r][k] * A[r][lane];
-            for (int r = k; r < rows; ++r) A[r][lane] -= 2.0 * dot * Vh[r][k];
+        for (int r = k + tid; r < rows; r += kMatrixThreads) Vh[r][k] = (A[r][k] - (r == k ? alpha : 0.0)) / vnorm;
+        __syncthreads();
+        if (tid < Q - k) {
+            const int c = k + tid;
+            double d0 = 0.0, d1 = 0.0;
+            int r = k;
+            for (; r + 1 < rows; r += 2) { d0 += Vh[r][k] * A[r][c]; d1 += Vh[r + 1][k] * A[r + 1][c]; }
+            if (r < rows) d0 += Vh[r][k] * A[r][c];
+            const double dot2 = 2.0 * (d0 + d1);
+            for (r = k; r < rows; ++r) A[r][c] -= dot2 * Vh[r][k];
         }
-        __syncwarp();
+        __syncthreads();
     }
     // row w of the pseudo-inverse: solve R^T y = e_w, then x = H_0 H_1 ... H_{Q-1} [y; 0]
-    for (int wi = lane; wi < prm.n_wanted; wi += 32) {
+    for (int wi = warp; wi < prm.n_wanted; wi += kMatrixThreads / 32) {
         const int w = prm.wanted[wi];
-        double y[kMaxQ];
-        for (int i = 0; i < Q; ++i) {
-            double rhs = i == w ? 1.0 : 0.0;
-            for (int j = 0; j < i; ++j) rhs -= A[j][i] * y[j];
-            y[i] = rhs / A[i][i];
+        double y = 0.0;                              // lane i keeps y_i
+        for (int i = w; i < Q; ++i) {                // y_i = 0 for i < w
+            const double s = warp_sum(lane < i ? A[lane][i] * y : 0.0);
+            const double yi = ((i == w ? 1.0 : 0.0) - s) / A[i][i];
+            if (lane == i) y = yi;
         }
-        double x[kMaxNodes];
-        for (int r = 0; r < rows; ++r) x[r] = r < Q ? y[r] : 0.0;
+        double x0 = lane < Q ? y : 0.0, x1 = 0.0;    // x[lane], x[lane + 32]
+        const bool in0 = lane < rows, in1 = lane + 32 < rows;
         for (int k = Q - 1; k >= 0; --k) {
-            double dot = 0.0;
-            for (int r = k; r < rows; ++r) dot += Vh[r][k] * x[r];
-            for (int r = k; r < rows; ++r) x[r] -= 2.0 * dot * Vh[r][k];
+            const double v0 = (in0 && lane >= k) ? Vh[lane][k] : 0.0, v1 = in1 ? Vh[lane + 32][k] : 0.0;
+            const double dot2 = 2.0 * warp_sum(v0 * x0 + v1 * x1);
+            x0 -= dot2 * v0;
+            x1 -= dot2 * v1;
         }
-        for (int r = 0; r < rows; ++r) prm.D[wi * P + node_of[r]] = x[r];
+        if (in0) prm.D[wi * P + node_of[lane]] = x0;
+        if (in1) prm.D[wi * P + node_of[lane + 32]] = x1;
     }
     if (prm.regen) {
         // Regeneration (Section VI): node f's share is a polynomial of degree Q-1 evaluated at b_f.
         // With D[c][q] the functional giving its c-th Chebyshev coefficient from the clean nodes q,
         // share_f = sum_q (sum_c T_c(b_f) D[c][q]) share_q.  Needs n_wanted == Q, wanted[c] == c.
-        __syncwarp();
-        __threadfence_block();
+        __syncthreads();                             // D was written by other warps of this CTA
         int nf = 0;
         for (int f = 0; f < P; ++f) {
             if (!prm.result->flagged[f]) continue;
             const double b = prm.points[f];
-            for (int q = lane; q < P; q += 32) {
+            for (int q = tid; q < P; q += kMatrixThreads) {
                 double acc = 0.0, t0 = 1.0, t1 = b;
                 for (int c = 0; c < Q; ++c) {
                     acc = fma(t0, prm.D[c * P + q], acc);
@@ -122,7 +138,7 @@ __global__ void __launch_bounds__(32) decode_matrix_kernel(MatrixParams prm) {
             }
             ++nf;
         }
-        if (lane == 0) prm.gate[1] = nf;
+        if (tid == 0) prm.gate[1] = nf;
     }
 }
 
@@ -295,7 +311,7 @@ gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* output
     mp.have_mask = have_mask ? 1 : 0;
     mp.P = plan->P; mp.Q = pi.Q; mp.n_wanted = pi.grid_rows * pi.grid_cols;
     for (int i = 0; i < mp.n_wanted; ++i) mp.wanted[i] = pi.wanted[i];
-    decode_matrix_kernel<<<1, 32, 0, st>>>(mp);
+    decode_matrix_kernel<<<1, kMatrixThreads, 0, st>>>(mp);
     rc = launch_ok();
     if (rc != GPD_OK) return rc;
     StreamParams sp{};
@@ -374,7 +390,7 @@ gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_re
     mp.P = plan->P; mp.Q = pi.Q; mp.n_wanted = pi.Q;
     for (int c = 0; c < pi.Q; ++c) mp.wanted[c] = c;
     mp.regen = reinterpret_cast<double*>(ws + wl.off_regen);
-    decode_matrix_kernel<<<1, 32, 0, st>>>(mp);
+    decode_matrix_kernel<<<1, kMatrixThreads, 0, st>>>(mp);
     if ((rc = launch_ok()) != GPD_OK) return rc;
     RegenParams rp{};
     rp.shares = shares; rp.Rg = mp.regen; rp.gate = mp.gate; rp.result = result;

@@ -172,6 +172,8 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     __shared__ double Qa[kMaxR][kMaxR + 1];
     __shared__ double Hs[kMaxR][kMaxNodes];
     __shared__ double lam[kMaxR];
+    __shared__ double rot_c[kMaxR / 2 + 1], rot_s[kMaxR / 2 + 1];
+    __shared__ int rot_p[kMaxR / 2 + 1], rot_q[kMaxR / 2 + 1];
     __shared__ int order[kMaxR];
     __shared__ unsigned char inside[kMaxNodes];
     __shared__ double dist[kMaxNodes];
@@ -217,9 +219,13 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     unsigned long long flagged = forced;
     double max_in = 0.0, min_out = 1e300;
     if (n_active > 0ULL) {
-        // ---- cyclic Jacobi: G <- J^T G J, V <- V J --------------------------------------
+        // ---- Jacobi: G <- J^T G J, V <- V J ----------------------------------------------
         double tr = 0.0;
         for (int i = 0; i < R; ++i) tr += G[i][i];
+        // Rotations of one round act on disjoint index pairs (round-robin pairing of n = R or R + 1
+        // indices: n - 1 rounds of n / 2 pairs), so their angles are found side by side (lane = pair)
+        // and applied together: columns of G and V first, then rows of G.
+        const int n = (R + 1) & ~1, half = n >> 1;
         for (int sweep = 0; sweep < 40; ++sweep) {
             double off = 0.0;
             for (int i = lane; i < R * R; i += 32) {
@@ -229,33 +235,50 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
             if (off <= 1e-27 * tr * tr) break;          // off-diagonal mass at the FP64 rounding floor
-            for (int p = 0; p < R - 1; ++p) {
-                for (int q = p + 1; q < R; ++q) {
-                    const double gpq = G[p][q];
-                    const double gpp = G[p][p], gqq = G[q][q];
-                    __syncwarp();
-                    if (fabs(gpq) <= 1e-300 || fabs(gpq) <= 1e-20 * sqrt(fabs(gpp * gqq))) continue;
-                    const double th = (gqq - gpp) / (2.0 * gpq);
-                    const double t = (th >= 0.0 ? 1.0 : -1.0) / (fabs(th) + sqrt(th * th + 1.0));
-                    const double c = 1.0 / sqrt(t * t + 1.0), s = t * c;
-                    if (lane < R) {                          // G <- G J   (columns p, q)
-                        const double a = G[lane][p], b = G[lane][q];
-                        G[lane][p] = c * a - s * b;
-                        G[lane][q] = s * a + c * b;
-                        const double va = V[lane][p], vb = V[lane][q];
-                        V[lane][p] = c * va - s * vb;
-                        V[lane][q] = s * va + c * vb;
+            for (int rd = 0; rd < n - 1; ++rd) {
+                if (lane < half) {
+                    const int a = lane == 0 ? n - 1 : (rd + lane) % (n - 1);
+                    const int b = lane == 0 ? rd : (rd + n - 1 - lane) % (n - 1);
+                    const int p = min(a, b), q = max(a, b);
+                    double c = 1.0, sn = 0.0;
+                    if (q < R) {
+                        const double gpq = G[p][q], gpp = G[p][p], gqq = G[q][q];
+                        if (!(fabs(gpq) <= 1e-300 || fabs(gpq) <= 1e-20 * sqrt(fabs(gpp * gqq)))) {
+                            const double th = (gqq - gpp) / (2.0 * gpq);
+                            const double t = (th >= 0.0 ? 1.0 : -1.0) / (fabs(th) + sqrt(th * th + 1.0));
+                            c = 1.0 / sqrt(t * t + 1.0);
+                            sn = t * c;
+                        }
                     }
-                    __syncwarp();
-                    if (lane < R) {                          // G <- J^T G (rows p, q)
-                        const double a = G[p][lane], b = G[q][lane];
-                        G[p][lane] = c * a - s * b;
-                        G[q][lane] = s * a + c * b;
-                    }
-                    __syncwarp();
-                    if (lane == 0) { G[p][q] = 0.0; G[q][p] = 0.0; }
-                    __syncwarp();
+                    rot_c[lane] = c; rot_s[lane] = sn; rot_p[lane] = p; rot_q[lane] = q;
                 }
+                __syncwarp();
+                for (int it = lane; it < half * R; it += 32) {      // G <- G J, V <- V J (columns p, q)
+                    const int t = it / R, i = it - t * R, p = rot_p[t], q = rot_q[t];
+                    if (q >= R || rot_s[t] == 0.0) continue;
+                    const double c = rot_c[t], sn = rot_s[t];
+                    const double a = G[i][p], b = G[i][q];
+                    G[i][p] = c * a - sn * b;
+                    G[i][q] = sn * a + c * b;
+                    const double va = V[i][p], vb = V[i][q];
+                    V[i][p] = c * va - sn * vb;
+                    V[i][q] = sn * va + c * vb;
+                }
+                __syncwarp();
+                for (int it = lane; it < half * R; it += 32) {      // G <- J^T G (rows p, q)
+                    const int t = it / R, j = it - t * R, p = rot_p[t], q = rot_q[t];
+                    if (q >= R || rot_s[t] == 0.0) continue;
+                    const double c = rot_c[t], sn = rot_s[t];
+                    const double a = G[p][j], b = G[q][j];
+                    G[p][j] = c * a - sn * b;
+                    G[q][j] = sn * a + c * b;
+                }
+                __syncwarp();
+                if (lane < half && rot_q[lane] < R && rot_s[lane] != 0.0) {
+                    G[rot_p[lane]][rot_q[lane]] = 0.0;
+                    G[rot_q[lane]][rot_p[lane]] = 0.0;
+                }
+                __syncwarp();
             }
         }
         // ---- eigenvalues in descending order ---------------------------------------------
