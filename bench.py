@@ -43,7 +43,7 @@ FALLBACK_BF16_SUSTAINED = 1400.0
 FALLBACK_HBM_GBS = 6650.0
 CPU_SAMPLE_ROWS = 1024              # rows of W in the CPU sample (1/8 of the workload)
 TRAFFIC_BYTES_PER_LAUNCH = None     # dram read+write bytes of the dominant kernel from ncu (see profiles/)
-TRAFFIC_BYTES_PER_LAUNCH_SLICED = None   # set from ncu once the kernel is final (profiles/)
+TRAFFIC_BYTES_PER_LAUNCH_SLICED = 1545943568   # gemm_i8_sliced_kernel<6>: dram read 1.349930 GB + write 0.196014 GB (profiles/)
 
 
 def load_peaks():
