@@ -134,6 +134,20 @@ typedef struct {
     uint8_t forced[GPD_MAX_NODES];    /* 1 = erased by the caller or holding a non-finite value */
 } gpd_locate_result;
 
+/* Result of gpd_correct_positions; lives in device memory, copied back by the caller. */
+typedef struct {
+    int32_t outcome;            /* gpd_outcome: GPD_CORRECTED only if every failing position was repaired */
+    int32_t max_errors;         /* largest number of errors corrected in one position */
+    int32_t device_status;      /* 0 */
+    int32_t reserved;
+    int64_t n_active;           /* positions whose syndrome failed the zero test (non-finite ones included) */
+    int64_t n_corrected;        /* of those, repaired in place */
+    int64_t n_failed;           /* of those, left untouched: no support of size <= floor((P-Q)/2) explains the
+                                   syndrome, or the position holds a non-finite value */
+    int64_t n_entries;          /* worker-output entries changed */
+    uint8_t touched[GPD_MAX_NODES];   /* 1 = at least one entry of this node was changed */
+} gpd_position_result;
+
 /* What gpd_plan_query returns. */
 typedef enum {
     GPD_Q_THRESHOLD_FWD = 0,    /* mn d1 + n - 1   (Theorem 2)          or, alternate substitution, mn d1 + mn - m */
@@ -150,7 +164,8 @@ typedef enum {
     GPD_Q_WORKSPACE_BYTES = 11, /* bytes of workspace for gpd_locate_errors / gpd_decode */
     GPD_Q_STEP_WORKSPACE_BYTES = 12, /* bytes of workspace for coded_layer_step       */
     GPD_Q_PRECISION = 13,       /* resolved gpd_precision                            */
-    GPD_Q_NODES = 14
+    GPD_Q_NODES = 14,
+    GPD_Q_POSITION_WORKSPACE_BYTES = 15 /* bytes of workspace for gpd_correct_positions (any product) */
 } gpd_query;
 
 /* Host tables a test may read back with gpd_plan_table. */
@@ -247,6 +262,23 @@ gpd_status gpd_inject(gpd_plan_t plan, gpd_product which, void* outputs_dev, uin
 gpd_status gpd_locate_errors(gpd_plan_t plan, gpd_product which, const void* outputs_dev,
                              const uint8_t* erased_host, gpd_locate_result* result_dev,
                              void* workspace_dev, void* stream);
+
+/*
+ * gpd_correct_positions — error correction of every output position on its own under the
+ * adversarial model (lemma on real-number error correction under the adversarial model; section on
+ * decoding methods): a position is one codeword of P node values; when its syndrome H z is not
+ * zero, the solution of H e = H z with the fewest non-zeros, at most floor((P-Q)/2), is looked for
+ * (power-sum syndromes, error-locator polynomial, least-squares error values, acceptance by the
+ * zero test on what is left of the syndrome) and subtracted from outputs_dev IN PLACE.  Different
+ * positions may blame different nodes, so more than P-Q-1 nodes may be hit overall - the case
+ * gpd_locate_errors must give up on.  Afterwards gpd_decode with a use-mask of all nodes (or any
+ * Q of them) reads the repaired outputs.  Positions that cannot be repaired are left as they are
+ * and counted; the outcome is then GPD_DECODE_FAILURE.  Meant for small floor((P-Q)/2) (the
+ * locator is found in the monomial basis).
+ * result_dev: device gpd_position_result.  workspace_dev: GPD_Q_POSITION_WORKSPACE_BYTES bytes.
+ */
+gpd_status gpd_correct_positions(gpd_plan_t plan, gpd_product which, void* outputs_dev,
+                                 gpd_position_result* result_dev, void* workspace_dev, void* stream);
 
 /*
  * gpd_locate_errors_static — gpd_locate_errors for callers that must not allocate device memory.

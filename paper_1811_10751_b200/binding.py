@@ -35,7 +35,7 @@ GPD_PHASE_FWD, GPD_PHASE_BWD, GPD_PHASE_UPD, GPD_PHASE_REGEN, GPD_PHASE_INJECT_S
 (GPD_Q_THRESHOLD_FWD, GPD_Q_THRESHOLD_BWD, GPD_Q_THRESHOLD_AUDIT, GPD_Q_ELEMENT_SIZE,
  GPD_Q_W_SHARE_ELEMS, GPD_Q_X_SHARE_ELEMS, GPD_Q_DT_SHARE_ELEMS, GPD_Q_DHAT_ELEMS, GPD_Q_XHAT_ELEMS,
  GPD_Q_OUT_ELEMS_FWD, GPD_Q_OUT_ELEMS_BWD, GPD_Q_WORKSPACE_BYTES, GPD_Q_STEP_WORKSPACE_BYTES,
- GPD_Q_PRECISION, GPD_Q_NODES) = range(15)
+ GPD_Q_PRECISION, GPD_Q_NODES, GPD_Q_POSITION_WORKSPACE_BYTES) = range(16)
 (GPD_TABLE_POINTS, GPD_TABLE_PARITY_FWD, GPD_TABLE_PARITY_BWD, GPD_TABLE_PARITY_AUDIT,
  GPD_TABLE_COEF_W, GPD_TABLE_COEF_X, GPD_TABLE_COEF_DT) = range(7)
 GPD_MAX_NODES = 64
@@ -44,7 +44,7 @@ GPD_SUBST_U_EQ_VN, GPD_SUBST_V_EQ_UM = 0, 1
 EXPORTED = [
     "gpd_status_string", "gpd_plan", "gpd_plan_subst", "gpd_plan_destroy", "gpd_plan_query", "gpd_plan_table",
     "gpd_encode_A", "gpd_encode_B", "gpd_worker_gemm", "gpd_device_status", "gpd_update_shares", "gpd_inject",
-    "gpd_locate_errors", "gpd_locate_errors_static", "gpd_decode", "gpd_regenerate_shares", "gpd_activation", "gpd_softmax_xent_delta",
+    "gpd_locate_errors", "gpd_locate_errors_static", "gpd_correct_positions", "gpd_decode", "gpd_regenerate_shares", "gpd_activation", "gpd_softmax_xent_delta",
     "gpd_backprop_hadamard", "gpd_sae_output_delta", "gpd_sae_hidden_delta", "coded_layer_step",
 ]
 
@@ -66,6 +66,15 @@ class gpd_locate_result(C.Structure):
 
 RESULT_BYTES = C.sizeof(gpd_locate_result)
 
+
+class gpd_position_result(C.Structure):
+    _fields_ = [("outcome", C.c_int32), ("max_errors", C.c_int32), ("device_status", C.c_int32),
+                ("reserved", C.c_int32), ("n_active", C.c_int64), ("n_corrected", C.c_int64),
+                ("n_failed", C.c_int64), ("n_entries", C.c_int64), ("touched", C.c_uint8 * GPD_MAX_NODES)]
+
+
+POSITION_RESULT_BYTES = C.sizeof(gpd_position_result)
+
 _vp, _i32, _i64, _u64, _f, _d = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_float, C.c_double
 lib.gpd_status_string.restype = C.c_char_p
 lib.gpd_status_string.argtypes = [C.c_int]
@@ -84,6 +93,7 @@ lib.gpd_update_shares.argtypes = [_vp, _vp, _vp, _vp, _f, _f, _vp, _vp]
 lib.gpd_inject.argtypes = [_vp, C.c_int, _vp, _u64, C.c_int, _d, _u64, _i32, _d, _vp, _vp]
 lib.gpd_locate_errors.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp, _vp]
 lib.gpd_locate_errors_static.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp]
+lib.gpd_correct_positions.argtypes = [_vp, C.c_int, _vp, _vp, _vp, _vp]
 lib.gpd_decode.argtypes = [_vp, C.c_int, _vp, C.POINTER(C.c_uint8), _vp, _vp, _vp, C.c_int, _vp, _vp]
 lib.gpd_regenerate_shares.argtypes = [_vp, _vp, _vp, _vp, _vp]
 lib.gpd_activation.argtypes = [C.c_int, _vp, _vp, _i64, _vp]
@@ -258,6 +268,17 @@ def gpd_locate_errors_static(plan: Plan, which: int, outputs, result, erased=Non
     share that array, so keep them ordered on one stream."""
     _check(lib.gpd_locate_errors_static(plan.handle, which, _ptr(outputs), _mask(erased, plan.P), _ptr(result),
                                         _stream(stream)), "gpd_locate_errors_static")
+
+
+def gpd_correct_positions(plan: Plan, which: int, outputs, workspace=None, stream=None) -> gpd_position_result:
+    """Repairs every output position on its own (up to floor((P-Q)/2) errors each), in place; returns
+    the result struct copied back to the host (synchronises)."""
+    if workspace is None:
+        workspace = torch.empty(plan.query(GPD_Q_POSITION_WORKSPACE_BYTES), dtype=torch.uint8, device=outputs.device)
+    res = torch.zeros(POSITION_RESULT_BYTES, dtype=torch.uint8, device=outputs.device)
+    _check(lib.gpd_correct_positions(plan.handle, which, _ptr(outputs, plan.dtype), _ptr(res), _ptr(workspace),
+                                     _stream(stream)), "gpd_correct_positions")
+    return gpd_position_result.from_buffer_copy(res.cpu().numpy().tobytes())
 
 
 def gpd_decode(plan: Plan, which: int, outputs, out, workspace, result=None, use_mask=None, act_out=None,

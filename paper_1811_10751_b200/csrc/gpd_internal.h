@@ -34,8 +34,10 @@ struct ProductInfo {
     int64_t bc = 0;
     int wanted[kMaxWanted] = {0};   // exponent of block (r, c), row-major over the grid
     std::vector<double> H;          // R x P, orthonormal rows, H * Vandermonde(points, Q) = 0
+    std::vector<double> Hg;         // R x P, row j = w_p b_p^j (w the barycentric weights of the points,
+                                    // largest magnitude 1): the same null space in power-sum form
     // offsets (in doubles) into the device table buffer
-    int64_t off_H = 0;
+    int64_t off_H = 0, off_Hg = 0;
 };
 
 // Device-resident tables of a plan (one allocation).
@@ -104,6 +106,9 @@ gpd_status locate_static_launch(gpd_plan_s* plan, gpd_product which, const void*
                                 uint64_t erased_mask, gpd_locate_result* result, cudaStream_t st);
 gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_result* result, void* workspace,
                              cudaStream_t st);
+gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* outputs, gpd_position_result* result,
+                                    void* workspace, cudaStream_t st);
+int64_t position_workspace_bytes(const gpd_plan_s* plan);
 gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, bool have_mask,
                          uint64_t use_mask, const gpd_locate_result* result, float* out, float* act_out,
                          int activation, void* workspace, cudaStream_t st);

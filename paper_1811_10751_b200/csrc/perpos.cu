@@ -1,0 +1,264 @@
+// Per-codeword error correction under the adversarial model (lemma on real-number error correction:
+// a (P, Q) MDS code corrects t = floor((P - Q) / 2) errors of arbitrary value in one codeword;
+// section on decoding methods: find the solution of H e = H z with the fewest non-zeros).
+// Every output position is one codeword of P node values and is repaired on its own, so different
+// positions may blame different nodes.
+//
+//   1. position_scan_kernel: one thread per position; syndrome r = H z (orthonormal H in shared
+//      memory), zero test ||r||^2 <= tau^2 ||z||^2; positions that fail it are appended to a list.
+//   2. position_fix_kernel: one thread per listed position.  The code is a polynomial code, so the
+//      sparsest solution is found the Reed-Solomon way in real arithmetic: power-sum syndromes
+//      S_j = sum_p w_p b_p^j z_p (w the barycentric weights), and for nu = 1 .. t the locator
+//      x^nu + sum_i l_i x^i from the Hankel system sum_i l_i S_{j+i} = -S_{j+nu}; its nu smallest
+//      values over the points name the support A; the error values are the least-squares solution
+//      of H_A e = r; the support is accepted when what is left of r passes the zero test.  The
+//      accepted errors are subtracted in place.
+//   3. position_finish_kernel: outcome and counters into the result struct.
+#include "gpd_internal.h"
+
+namespace gpd {
+
+namespace {
+
+constexpr int kMaxT = kMaxR / 2;          // errors correctable per codeword
+
+struct PosParams {
+    void* Z;                              // [P][L]
+    const double* H;                      // [R][P] orthonormal parity check
+    const double* Hg;                     // [R][P] power-sum parity check
+    const double* points;                 // [P]
+    unsigned long long* counters;         // [0] listed, [1] active, [2] corrected, [3] failed, [4] entries,
+                                          // [5] largest support, [6] touched-node mask
+    unsigned int* list;                   // positions that failed the zero test
+    gpd_position_result* result;
+    int64_t L;
+    int P, R;
+    double tau2;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256) position_scan_kernel(PosParams prm) {
+    extern __shared__ double sH[];        // [R][P]
+    for (int i = threadIdx.x; i < prm.R * prm.P; i += 256) sH[i] = prm.H[i];
+    __syncthreads();
+    const T* Z = reinterpret_cast<const T*>(prm.Z);
+    for (int64_t pos = (int64_t)blockIdx.x * 256 + threadIdx.x; pos < prm.L; pos += (int64_t)gridDim.x * 256) {
+        double r[kMaxR];
+#pragma unroll
+        for (int j = 0; j < kMaxR; ++j) r[j] = 0.0;
+        double z2 = 0.0;
+        bool finite = true;
+        for (int p = 0; p < prm.P; ++p) {
+            const double z = (double)Z[(int64_t)p * prm.L + pos];
+            finite &= isfinite(z);
+            z2 = fma(z, z, z2);
+#pragma unroll
+            for (int j = 0; j < kMaxR; ++j)
+                if (j < prm.R) r[j] = fma(sH[j * prm.P + p], z, r[j]);
+        }
+        double r2 = 0.0;
+#pragma unroll
+        for (int j = 0; j < kMaxR; ++j) r2 = fma(r[j], r[j], r2);
+        if (!finite) {                    // reported as failed, left untouched
+            atomicAdd(&prm.counters[1], 1ULL);
+            atomicAdd(&prm.counters[3], 1ULL);
+        } else if (r2 > prm.tau2 * z2) {
+            atomicAdd(&prm.counters[1], 1ULL);
+            prm.list[atomicAdd(&prm.counters[0], 1ULL)] = (unsigned int)pos;
+        }
+    }
+}
+
+// Gaussian elimination with partial pivoting on the n x (n + 1) system held in a (row stride
+// kMaxT + 1); false when a pivot vanishes against the size of the matrix.
+__device__ bool solve_small(double (*a)[kMaxT + 1], int n, double* x) {
+    double amax = 0.0;
+    for (int i = 0; i < n; ++i)
+        for (int j = 0; j < n; ++j) amax = fmax(amax, fabs(a[i][j]));
+    if (!(amax > 0.0)) return false;
+    for (int k = 0; k < n; ++k) {
+        int piv = k;
+        for (int i = k + 1; i < n; ++i)
+            if (fabs(a[i][k]) > fabs(a[piv][k])) piv = i;
+        if (fabs(a[piv][k]) <= 1e-13 * amax) return false;
+        if (piv != k)
+            for (int j = k; j <= n; ++j) { const double t = a[k][j]; a[k][j] = a[piv][j]; a[piv][j] = t; }
+        const double inv = 1.0 / a[k][k];
+        for (int i = k + 1; i < n; ++i) {
+            const double f = a[i][k] * inv;
+            for (int j = k; j <= n; ++j) a[i][j] -= f * a[k][j];
+        }
+    }
+    for (int i = n - 1; i >= 0; --i) {
+        double s = a[i][n];
+        for (int j = i + 1; j < n; ++j) s -= a[i][j] * x[j];
+        x[i] = s / a[i][i];
+    }
+    return true;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128) position_fix_kernel(PosParams prm) {
+    extern __shared__ double sm[];        // H [R][P], Hg [R][P], points [P]
+    double* sH = sm;
+    double* sHg = sm + prm.R * prm.P;
+    double* sPts = sHg + prm.R * prm.P;
+    for (int i = threadIdx.x; i < prm.R * prm.P; i += 128) { sH[i] = prm.H[i]; sHg[i] = prm.Hg[i]; }
+    for (int i = threadIdx.x; i < prm.P; i += 128) sPts[i] = prm.points[i];
+    __syncthreads();
+    T* Z = reinterpret_cast<T*>(prm.Z);
+    const int P = prm.P, R = prm.R, t = R / 2;
+    const unsigned long long listed = prm.counters[0];
+    for (unsigned long long it = (unsigned long long)blockIdx.x * 128 + threadIdx.x; it < listed;
+         it += (unsigned long long)gridDim.x * 128) {
+        const int64_t pos = prm.list[it];
+        double r[kMaxR], S[kMaxR];
+        for (int j = 0; j < R; ++j) { r[j] = 0.0; S[j] = 0.0; }
+        double z2 = 0.0;
+        for (int p = 0; p < P; ++p) {
+            const double z = (double)Z[(int64_t)p * prm.L + pos];
+            z2 = fma(z, z, z2);
+            for (int j = 0; j < R; ++j) {
+                r[j] = fma(sH[j * P + p], z, r[j]);
+                S[j] = fma(sHg[j * P + p], z, S[j]);
+            }
+        }
+        const double limit = prm.tau2 * z2;
+        int accepted = 0;
+        int nodes[kMaxT];
+        double err[kMaxT];
+        for (int nu = 1; nu <= t && accepted == 0; ++nu) {
+            double a[kMaxT][kMaxT + 1], lam[kMaxT];
+            for (int j = 0; j < nu; ++j) {
+                for (int i = 0; i < nu; ++i) a[j][i] = S[j + i];
+                a[j][nu] = -S[j + nu];
+            }
+            if (!solve_small(a, nu, lam)) continue;
+            // the nu points where the locator is smallest
+            unsigned long long taken = 0ULL;
+            for (int k = 0; k < nu; ++k) {
+                int best = -1;
+                double best_v = 0.0;
+                for (int p = 0; p < P; ++p) {
+                    if ((taken >> p) & 1ULL) continue;
+                    const double x = sPts[p];
+                    double v = 1.0;
+                    for (int i = nu - 1; i >= 0; --i) v = fma(v, x, lam[i]);
+                    v = fabs(v);
+                    if (best < 0 || v < best_v) { best = p; best_v = v; }
+                }
+                nodes[k] = best;
+                taken |= 1ULL << best;
+            }
+            // least squares H_A e = r through the normal equations (H has orthonormal rows)
+            for (int i = 0; i < nu; ++i) {
+                for (int j = 0; j < nu; ++j) {
+                    double s = 0.0;
+                    for (int q = 0; q < R; ++q) s = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s);
+                    a[i][j] = s;
+                }
+                double s = 0.0;
+                for (int q = 0; q < R; ++q) s = fma(sH[q * P + nodes[i]], r[q], s);
+                a[i][nu] = s;
+            }
+            if (!solve_small(a, nu, err)) continue;
+            double left = 0.0;
+            for (int q = 0; q < R; ++q) {
+                double v = r[q];
+                for (int i = 0; i < nu; ++i) v = fma(-sH[q * P + nodes[i]], err[i], v);
+                left = fma(v, v, left);
+            }
+            if (left <= limit) accepted = nu;
+        }
+        if (accepted == 0) {
+            atomicAdd(&prm.counters[3], 1ULL);
+            continue;
+        }
+        unsigned long long mask = 0ULL;
+        for (int i = 0; i < accepted; ++i) {
+            T* cell = Z + (int64_t)nodes[i] * prm.L + pos;
+            *cell = (T)((double)*cell - err[i]);
+            mask |= 1ULL << nodes[i];
+        }
+        atomicAdd(&prm.counters[2], 1ULL);
+        atomicAdd(&prm.counters[4], (unsigned long long)accepted);
+        atomicMax(&prm.counters[5], (unsigned long long)accepted);
+        atomicOr(&prm.counters[6], mask);
+    }
+}
+
+__global__ void position_finish_kernel(PosParams prm) {
+    gpd_position_result* res = prm.result;
+    const unsigned long long active = prm.counters[1], failed = prm.counters[3];
+    if (threadIdx.x == 0) {
+        res->outcome = active == 0ULL ? GPD_NO_ERROR : (failed ? GPD_DECODE_FAILURE : GPD_CORRECTED);
+        res->max_errors = (int32_t)prm.counters[5];
+        res->device_status = 0;
+        res->reserved = 0;
+        res->n_active = (int64_t)active;
+        res->n_corrected = (int64_t)prm.counters[2];
+        res->n_failed = (int64_t)failed;
+        res->n_entries = (int64_t)prm.counters[4];
+    }
+    for (int p = threadIdx.x; p < kMaxNodes; p += blockDim.x)
+        res->touched[p] = (p < prm.P && ((prm.counters[6] >> p) & 1ULL)) ? 1 : 0;
+}
+
+constexpr int64_t kPosHeaderBytes = 256;  // counters
+
+}  // namespace
+
+int64_t position_workspace_bytes(const gpd_plan_s* plan) {
+    int64_t L = 0;
+    for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT})
+        if (plan->prod[w].Q > 0) L = std::max<int64_t>(L, plan->prod[w].br * plan->prod[w].bc);
+    return kPosHeaderBytes + (L * 4 + 255) / 256 * 256;
+}
+
+gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* outputs, gpd_position_result* result,
+                                    void* workspace, cudaStream_t st) {
+    if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
+    if (plan->sliced && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward product only
+    const ProductInfo& pi = plan->prod[which];
+    if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
+    const int64_t L = pi.br * pi.bc;
+    if (L >= (int64_t)1 << 32) return GPD_ERR_UNSUPPORTED;               // positions are listed as 32-bit indices
+    gpd_status rc = ensure_device(plan);
+    if (rc != GPD_OK) return rc;
+    PosParams prm{};
+    prm.Z = outputs;
+    prm.H = plan->dev.base + pi.off_H;
+    prm.Hg = plan->dev.base + pi.off_Hg;
+    prm.points = plan->dev.base + plan->dev.off_points;
+    prm.counters = reinterpret_cast<unsigned long long*>(workspace);
+    prm.list = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(workspace) + kPosHeaderBytes);
+    prm.result = result;
+    prm.L = L; prm.P = plan->P; prm.R = pi.R;
+    prm.tau2 = plan->tau_col * plan->tau_col;
+    if (cudaMemsetAsync(workspace, 0, kPosHeaderBytes, st) != cudaSuccess) return GPD_ERR_CUDA;
+    if (pi.R > 0) {
+        const size_t smem1 = sizeof(double) * pi.R * plan->P;
+        const int grid1 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 255) / 256, 148 * 8));
+        if (plan->elem_size == 4) position_scan_kernel<float><<<grid1, 256, smem1, st>>>(prm);
+        else position_scan_kernel<double><<<grid1, 256, smem1, st>>>(prm);
+        if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+        const size_t smem2 = sizeof(double) * (2 * pi.R * plan->P + plan->P);
+        const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 127) / 128, 148 * 4));
+        if (plan->elem_size == 4) position_fix_kernel<float><<<grid2, 128, smem2, st>>>(prm);
+        else position_fix_kernel<double><<<grid2, 128, smem2, st>>>(prm);
+        if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+    }
+    position_finish_kernel<<<1, 64, 0, st>>>(prm);
+    return launch_ok();
+}
+
+}  // namespace gpd
+
+using namespace gpd;
+
+extern "C" gpd_status gpd_correct_positions(gpd_plan_t plan, gpd_product which, void* outputs_dev,
+                                            gpd_position_result* result_dev, void* workspace_dev, void* stream) {
+    if (!plan || !outputs_dev || !result_dev) return GPD_ERR_ARG;
+    if (!workspace_dev) return GPD_ERR_WORKSPACE;
+    return correct_positions_launch(plan, which, outputs_dev, result_dev, workspace_dev, as_stream(stream));
+}

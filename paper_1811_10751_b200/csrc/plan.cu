@@ -72,6 +72,26 @@ std::vector<double> left_null_space(const std::vector<double>& b, int Q) {
 
 int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
 
+// Row j of the power-sum parity check: w_p b_p^j, j = 0 .. R-1, with w_p = 1 / prod_{q != p} (b_p - b_q)
+// scaled to largest magnitude 1.  sum_p w_p b_p^k f(b_p) is the divided difference of x^k f over all
+// P points and vanishes when deg(x^k f) <= P - 2, i.e. for every codeword and k <= R - 1.
+std::vector<double> power_sum_parity(const std::vector<double>& pts, int R) {
+    const int P = (int)pts.size();
+    std::vector<double> w(P, 1.0);
+    double wmax = 0.0;
+    for (int p = 0; p < P; ++p) {
+        for (int q = 0; q < P; ++q)
+            if (q != p) w[p] /= (pts[p] - pts[q]);
+        wmax = std::max(wmax, std::fabs(w[p]));
+    }
+    std::vector<double> Hg((size_t)R * P);
+    for (int p = 0; p < P; ++p) {
+        double acc = w[p] / wmax;
+        for (int j = 0; j < R; ++j) { Hg[(size_t)j * P + p] = acc; acc *= pts[p]; }
+    }
+    return Hg;
+}
+
 }  // namespace
 
 WorkspaceLayout workspace_layout() {
@@ -104,6 +124,7 @@ gpd_status ensure_device(gpd_plan_s* plan) {
     d.off_coefDup = push(plan->coefDup);
     d.off_coefXup = push(plan->coefXup);
     for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT}) plan->prod[w].off_H = push(plan->prod[w].H);
+    for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT}) plan->prod[w].off_Hg = push(plan->prod[w].Hg);
     d.n_doubles = (int64_t)host.size();
     if (cudaGetDevice(&plan->device) != cudaSuccess) return GPD_ERR_CUDA;
     if (cudaMalloc(&d.base, sizeof(double) * host.size()) != cudaSuccess) return GPD_ERR_CUDA;
@@ -232,6 +253,7 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
         for (int k = 0; k < d1; ++k)
             f.wanted[i * d1 + k] = alt ? i + m * (n - 1) + m * n * k : n * i + m * n * k + n - 1;
     f.H = left_null_space(plan->points, f.Q);
+    f.Hg = power_sum_parity(plan->points, f.R);
     ProductInfo& b = plan->prod[GPD_BWD];
     if (bwd_ok) {
         b.Q = (int)Qb; b.R = P - b.Q; b.grid_rows = d2; b.grid_cols = n;
@@ -240,6 +262,7 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
             for (int j = 0; j < n; ++j)
                 b.wanted[k * n + j] = alt ? m * n * k + (m - 1) + m * j : m * n * k + n * (m - 1) + j;
         b.H = left_null_space(plan->points, b.Q);
+        b.Hg = power_sum_parity(plan->points, b.R);
     }
     ProductInfo& a = plan->prod[GPD_AUDIT];
     if (audit_ok) {
@@ -248,6 +271,7 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
         for (int i = 0; i < m; ++i)
             for (int j = 0; j < n; ++j) a.wanted[i * n + j] = alt ? i + m * j : n * i + j;
         a.H = left_null_space(plan->points, a.Q);
+        a.Hg = power_sum_parity(plan->points, a.R);
     }
     if (plan->sliced && !sliced_supported(plan)) { delete plan; return GPD_ERR_UNSUPPORTED; }
     *out = plan;
@@ -289,6 +313,7 @@ extern "C" gpd_status gpd_plan_query(gpd_plan_t plan, gpd_query what, int64_t* v
             *value = workspace_layout().total + ((big * e + 255) / 256 + 2) * 256;
             break;
         }
+        case GPD_Q_POSITION_WORKSPACE_BYTES: *value = position_workspace_bytes(plan); break;
         case GPD_Q_PRECISION: *value = plan->prec; break;
         case GPD_Q_NODES: *value = P; break;
         default: return GPD_ERR_ARG;
