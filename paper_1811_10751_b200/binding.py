@@ -270,15 +270,20 @@ def gpd_locate_errors_static(plan: Plan, which: int, outputs, result, erased=Non
                                         _stream(stream)), "gpd_locate_errors_static")
 
 
-def gpd_correct_positions(plan: Plan, which: int, outputs, workspace=None, stream=None) -> gpd_position_result:
-    """Repairs every output position on its own (up to floor((P-Q)/2) errors each), in place; returns
-    the result struct copied back to the host (synchronises)."""
+def gpd_correct_positions(plan: Plan, which: int, outputs, workspace=None, result=None, stream=None):
+    """Repairs every output position on its own (up to floor((P-Q)/2) errors each), in place.  With
+    `result` (a device buffer of POSITION_RESULT_BYTES) the call only enqueues work; without it the
+    result struct is copied back to the host and returned (synchronises)."""
     if workspace is None:
         workspace = torch.empty(plan.query(GPD_Q_POSITION_WORKSPACE_BYTES), dtype=torch.uint8, device=outputs.device)
-    res = torch.zeros(POSITION_RESULT_BYTES, dtype=torch.uint8, device=outputs.device)
+    res = result if result is not None else torch.zeros(POSITION_RESULT_BYTES, dtype=torch.uint8, device=outputs.device)
     _check(lib.gpd_correct_positions(plan.handle, which, _ptr(outputs, plan.dtype), _ptr(res), _ptr(workspace),
                                      _stream(stream)), "gpd_correct_positions")
-    return gpd_position_result.from_buffer_copy(res.cpu().numpy().tobytes())
+    return None if result is not None else read_position_result(res)
+
+
+def read_position_result(buf: torch.Tensor) -> gpd_position_result:
+    return gpd_position_result.from_buffer_copy(buf.cpu().numpy().tobytes())
 
 
 def gpd_decode(plan: Plan, which: int, outputs, out, workspace, result=None, use_mask=None, act_out=None,

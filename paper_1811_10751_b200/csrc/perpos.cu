@@ -36,29 +36,29 @@ struct PosParams {
     double tau2;
 };
 
-template <typename T>
+template <typename T, int RT>                 // RT: parity checks rounded up to 8, 16 or 32
 __global__ void __launch_bounds__(256) position_scan_kernel(PosParams prm) {
-    extern __shared__ double sH[];        // [R][P]
-    for (int i = threadIdx.x; i < prm.R * prm.P; i += 256) sH[i] = prm.H[i];
+    extern __shared__ double sH[];        // [RT][P], zero rows past R
+    for (int i = threadIdx.x; i < RT * prm.P; i += 256) sH[i] = i < prm.R * prm.P ? prm.H[i] : 0.0;
     __syncthreads();
     const T* Z = reinterpret_cast<const T*>(prm.Z);
     for (int64_t pos = (int64_t)blockIdx.x * 256 + threadIdx.x; pos < prm.L; pos += (int64_t)gridDim.x * 256) {
-        double r[kMaxR];
+        double r[RT];
 #pragma unroll
-        for (int j = 0; j < kMaxR; ++j) r[j] = 0.0;
+        for (int j = 0; j < RT; ++j) r[j] = 0.0;
         double z2 = 0.0;
         bool finite = true;
+#pragma unroll 5
         for (int p = 0; p < prm.P; ++p) {
-            const double z = (double)Z[(int64_t)p * prm.L + pos];
+            const double z = (double)__ldcs(Z + (int64_t)p * prm.L + pos);
             finite &= isfinite(z);
             z2 = fma(z, z, z2);
 #pragma unroll
-            for (int j = 0; j < kMaxR; ++j)
-                if (j < prm.R) r[j] = fma(sH[j * prm.P + p], z, r[j]);
+            for (int j = 0; j < RT; ++j) r[j] = fma(sH[j * prm.P + p], z, r[j]);   // rows R .. RT-1 are zero
         }
         double r2 = 0.0;
 #pragma unroll
-        for (int j = 0; j < kMaxR; ++j) r2 = fma(r[j], r[j], r2);
+        for (int j = 0; j < RT; ++j) r2 = fma(r[j], r[j], r2);
         if (!finite) {                    // reported as failed, left untouched
             atomicAdd(&prm.counters[1], 1ULL);
             atomicAdd(&prm.counters[3], 1ULL);
@@ -98,19 +98,19 @@ __device__ bool solve_small(double (*a)[kMaxT + 1], int n, double* x) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(128) position_fix_kernel(PosParams prm) {
+__global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
     extern __shared__ double sm[];        // H [R][P], Hg [R][P], points [P]
     double* sH = sm;
     double* sHg = sm + prm.R * prm.P;
     double* sPts = sHg + prm.R * prm.P;
-    for (int i = threadIdx.x; i < prm.R * prm.P; i += 128) { sH[i] = prm.H[i]; sHg[i] = prm.Hg[i]; }
-    for (int i = threadIdx.x; i < prm.P; i += 128) sPts[i] = prm.points[i];
+    for (int i = threadIdx.x; i < prm.R * prm.P; i += 64) { sH[i] = prm.H[i]; sHg[i] = prm.Hg[i]; }
+    for (int i = threadIdx.x; i < prm.P; i += 64) sPts[i] = prm.points[i];
     __syncthreads();
     T* Z = reinterpret_cast<T*>(prm.Z);
     const int P = prm.P, R = prm.R, t = R / 2;
     const unsigned long long listed = prm.counters[0];
-    for (unsigned long long it = (unsigned long long)blockIdx.x * 128 + threadIdx.x; it < listed;
-         it += (unsigned long long)gridDim.x * 128) {
+    for (unsigned long long it = (unsigned long long)blockIdx.x * 64 + threadIdx.x; it < listed;
+         it += (unsigned long long)gridDim.x * 64) {
         const int64_t pos = prm.list[it];
         double r[kMaxR], S[kMaxR];
         for (int j = 0; j < R; ++j) { r[j] = 0.0; S[j] = 0.0; }
@@ -150,23 +150,39 @@ __global__ void __launch_bounds__(128) position_fix_kernel(PosParams prm) {
                 nodes[k] = best;
                 taken |= 1ULL << best;
             }
-            // least squares H_A e = r through the normal equations (H has orthonormal rows)
-            for (int i = 0; i < nu; ++i) {
-                for (int j = 0; j < nu; ++j) {
-                    double s = 0.0;
-                    for (int q = 0; q < R; ++q) s = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s);
-                    a[i][j] = s;
-                }
-                double s = 0.0;
-                for (int q = 0; q < R; ++q) s = fma(sH[q * P + nodes[i]], r[q], s);
-                a[i][nu] = s;
-            }
-            if (!solve_small(a, nu, err)) continue;
+            // least squares H_A e = r through the normal equations, then one step of refinement on the
+            // residual (neighbouring nodes make H_A ill-conditioned; the refinement brings the error
+            // values back to the accuracy of an orthogonal factorisation)
+            bool solved = true;
             double left = 0.0;
+            for (int i = 0; i < nu; ++i) err[i] = 0.0;
+            for (int pass = 0; pass < 2 && solved; ++pass) {
+                double v[kMaxR];
+                for (int q = 0; q < R; ++q) {
+                    double w = r[q];
+                    for (int i = 0; i < nu; ++i) w = fma(-sH[q * P + nodes[i]], err[i], w);
+                    v[q] = w;
+                }
+                for (int i = 0; i < nu; ++i) {
+                    for (int j = 0; j < nu; ++j) {
+                        double s = 0.0;
+                        for (int q = 0; q < R; ++q) s = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s);
+                        a[i][j] = s;
+                    }
+                    double s = 0.0;
+                    for (int q = 0; q < R; ++q) s = fma(sH[q * P + nodes[i]], v[q], s);
+                    a[i][nu] = s;
+                }
+                double delta[kMaxT];
+                solved = solve_small(a, nu, delta);
+                if (solved)
+                    for (int i = 0; i < nu; ++i) err[i] += delta[i];
+            }
+            if (!solved) continue;
             for (int q = 0; q < R; ++q) {
-                double v = r[q];
-                for (int i = 0; i < nu; ++i) v = fma(-sH[q * P + nodes[i]], err[i], v);
-                left = fma(v, v, left);
+                double w = r[q];
+                for (int i = 0; i < nu; ++i) w = fma(-sH[q * P + nodes[i]], err[i], w);
+                left = fma(w, w, left);
             }
             if (left <= limit) accepted = nu;
         }
@@ -237,15 +253,21 @@ gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* o
     prm.tau2 = plan->tau_col * plan->tau_col;
     if (cudaMemsetAsync(workspace, 0, kPosHeaderBytes, st) != cudaSuccess) return GPD_ERR_CUDA;
     if (pi.R > 0) {
-        const size_t smem1 = sizeof(double) * pi.R * plan->P;
+        const int RT = pi.R <= 8 ? 8 : pi.R <= 16 ? 16 : 32;
+        const size_t smem1 = sizeof(double) * RT * plan->P;
         const int grid1 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 255) / 256, 148 * 8));
-        if (plan->elem_size == 4) position_scan_kernel<float><<<grid1, 256, smem1, st>>>(prm);
-        else position_scan_kernel<double><<<grid1, 256, smem1, st>>>(prm);
+        const bool f32 = plan->elem_size == 4;
+        if (RT == 8) f32 ? position_scan_kernel<float, 8><<<grid1, 256, smem1, st>>>(prm)
+                         : position_scan_kernel<double, 8><<<grid1, 256, smem1, st>>>(prm);
+        else if (RT == 16) f32 ? position_scan_kernel<float, 16><<<grid1, 256, smem1, st>>>(prm)
+                               : position_scan_kernel<double, 16><<<grid1, 256, smem1, st>>>(prm);
+        else f32 ? position_scan_kernel<float, 32><<<grid1, 256, smem1, st>>>(prm)
+                 : position_scan_kernel<double, 32><<<grid1, 256, smem1, st>>>(prm);
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
         const size_t smem2 = sizeof(double) * (2 * pi.R * plan->P + plan->P);
-        const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 127) / 128, 148 * 4));
-        if (plan->elem_size == 4) position_fix_kernel<float><<<grid2, 128, smem2, st>>>(prm);
-        else position_fix_kernel<double><<<grid2, 128, smem2, st>>>(prm);
+        const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 63) / 64, 148 * 8));
+        if (f32) position_fix_kernel<float><<<grid2, 64, smem2, st>>>(prm);
+        else position_fix_kernel<double><<<grid2, 64, smem2, st>>>(prm);
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
     }
     position_finish_kernel<<<1, 64, 0, st>>>(prm);

@@ -121,3 +121,40 @@ def test_positions_backward_product():
            (CORRECTED, int((sizes > 0).sum()), int(sizes.sum()))
     CT = cp.decode(g.GPD_BWD, Zg, use_mask=[True] * P)
     assert op.rel_fro(CT, op.ref_backward(DT, W)) < 1e-4
+
+
+def test_positions_full_size_outputs_on_a_sample():
+    """The 8192 x 8192 x 512 product's outputs (P = 25, 1.05 M positions, digit-plane products) with
+    1-3 errors on 1 % of the positions, in the launch configuration the benchmark times.  The oracle
+    repairs a sample of 20 000 positions that holds every corrupted one; counters must match, and
+    the sampled outputs must come back as the oracle leaves them."""
+    import workloads as wl
+    cfg = wl.CONFIG_3_MATMUL
+    W, X = wl.matmul_inputs(cfg)
+    code = GPCode(cfg.N1, cfg.N0, cfg.B, cfg.m, cfg.n, cfg.d, 1, cfg.P)
+    cp = CodedProduct(code, precision=g.GPD_PREC_FP64_SLICED)
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    P, L = cfg.P, Z.numel() // cfg.P
+    rng = np.random.default_rng(99)
+    sample = np.sort(rng.choice(L, size=20000, replace=False))
+    hit = rng.choice(sample, size=L // 100, replace=False)
+    sizes = rng.integers(1, 4, size=hit.size)
+    pos = np.repeat(hit, sizes)
+    node = np.concatenate([rng.choice(P, size=k, replace=False) for k in sizes])
+    scale = float(Z.pow(2).mean().sqrt())
+    val = rng.choice([-1.0, 1.0], size=pos.size) * rng.uniform(0.25, 8.0, size=pos.size) * scale
+    Zv = Z.view(P, L)
+    Zv[torch.from_numpy(node).cuda(), torch.from_numpy(pos).cuda()] += torch.from_numpy(val).cuda()
+    smp = torch.from_numpy(sample).cuda()
+    bad_sample = host(Zv[:, smp])
+    ro = correct_positions(bad_sample, code.points, code.Q_f, tolerances_for(np.float64))
+    r = g.gpd_correct_positions(cp.plan, g.GPD_FWD, Z)
+    assert (r.outcome, r.n_active, r.n_corrected, r.n_failed, r.n_entries, r.max_errors) == \
+           (ro.outcome, ro.n_active, ro.n_corrected, ro.n_failed, ro.n_entries, ro.max_errors) == \
+           (CORRECTED, hit.size, hit.size, 0, int(sizes.sum()), 3)
+    assert np.array_equal(np.array(list(r.touched)[:P], dtype=bool), ro.touched)
+    assert np.abs(host(Zv[:, smp]) - ro.corrected).max() <= 1e-9 * scale
+    rows = np.arange(0, cfg.N1, cfg.N1 // 32)
+    S = cp.decode(g.GPD_FWD, Z, use_mask=[True] * P)
+    assert op.rel_fro(S[rows], op.ref_forward(W[rows], X)) < 1e-4
