@@ -3,13 +3,15 @@
 // shared memory by TMA, and 3xTF32 splitting so that the result keeps FP32-level accuracy:
 //     a = a_hi + a_lo (both exactly representable in TF32),   a*b ~ a_lo*b_hi + a_hi*b_lo + a_hi*b_hi.
 //
-// One CTA computes one 128 x 128 tile of one node's product (column strips of it for the tiles
-// left over after the last full round over the SMs).  Warp roles:
-//   warp 0      : TMA producer (one lane) - raw FP32 tiles of A and B into a 3-stage ring
-//   warp 1      : allocates tensor memory; one lane issues the MMAs and commits them to mbarriers
-//   warps 2..9  : split every landed tile in place into hi (overwrites the raw tile) and lo (second
-//                 tile), then, after the last k-block, read the accumulator back (tcgen05.ld) and
-//                 write the tile (plain store, or read-modify-write for the coded update)
+// One CTA per SM walks a list of 128 x 128 tiles of the nodes' products (column strips of them for
+// the tiles left over after the last full round over the SMs).  Two accumulators in tensor memory
+// alternate, so a tile's epilogue runs under the next tile's main loop.  Warp roles:
+//   warp 0       : TMA producer (one lane) - raw FP32 tiles of A and B into a 3-stage ring that
+//                  runs on across tiles
+//   warp 1       : allocates tensor memory; one lane issues the MMAs and commits them to mbarriers
+//   warps 2..9   : split every landed tile in place into hi (overwrites the raw tile) and lo (second tile)
+//   warps 10..13 : read a finished accumulator back (tcgen05.ld), hand it back to the MMA warp, and
+//                  write the tile (plain store, or read-modify-write for the coded update)
 // Operand tiles use the 128-byte swizzle; A is K-major; B is K-major for the update (X^_p is
 // [N][K]) and MN-major for the forward / backward products (X~_p, W~_p are [K][N]).
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains its copies,
@@ -28,10 +30,11 @@ constexpr int A_TILE_BYTES = BM * BK * 4;            // 16 KB, rows of 128 B
 constexpr int B_TILE_BYTES = BN * BK * 4;            // 16 KB
 constexpr int STAGE_BYTES = 2 * A_TILE_BYTES + 2 * B_TILE_BYTES;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
-constexpr int TMEM_COLS = 128;
-constexpr int kConvWarps = 8;                        // warps 2..9: split tiles, then drain tensor memory
+constexpr int TMEM_COLS = 256;                       // two 128-column accumulators: one fills while the other drains
+constexpr int kConvWarps = 8;                        // warps 2..9: split tiles
 constexpr int kConvThreads = kConvWarps * 32;
-constexpr int kThreads = 64 + kConvThreads;
+constexpr int kEpiWarps = 4;                         // warps 10..13: drain tensor memory, one per lane quarter
+constexpr int kThreads = 64 + kConvThreads + kEpiWarps * 32;
 constexpr long long kWaitCycles = 2000000000LL;      // about one second
 
 __device__ int g_tf32_status = 0;                    // GPD_ERR_TIMEOUT if a bounded wait expired
@@ -113,30 +116,35 @@ __device__ __forceinline__ float to_tf32(float x) {
 template <bool B_KMAJOR, bool UPDATE>
 __global__ void __launch_bounds__(kThreads, 1)
 sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams prm,
-                    int tiles_m, int tiles_n, int full_tiles, int split) {
+                    int tiles_m, int tiles_n, int full_tiles, int split, int n_virtual) {
     if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t full_bar[STAGES], conv_bar[STAGES], empty_bar[STAGES], acc_bar;
+    // full / conv / empty: operand ring, runs on across the tiles of this CTA; acc_full[b] / acc_empty[b]:
+    // accumulator b (tensor-memory columns 128 b ..) complete / read back
+    __shared__ __align__(8) uint64_t full_bar[STAGES], conv_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // Tile schedule: CTAs 0 .. full_tiles-1 take whole 128 x 128 tiles; the tiles left over after the
-    // last full round over the SMs are cut into `split` column strips, one per CTA, so that the
-    // final, partly filled round is short (128 x 32 strips when split = 4).
-    int tile = blockIdx.x, sub = 0, bn = BN;
-    if (tile >= full_tiles) {
-        const int piece = tile - full_tiles;
-        tile = full_tiles + piece / split;
-        sub = piece % split;
-        bn = BN / split;
-    }
-    const int tn = tile % tiles_n, tm = (tile / tiles_n) % tiles_m;
-    const int p = tile / (tiles_n * tiles_m);
-    const int m0 = tm * BM, n0 = tn * BN + sub * bn;
     const int num_kb = (int)((prm.K + BK - 1) / BK);
-    const int b_float4 = bn * BK / 4;                // 16-byte units of one B tile
+    // Virtual tile list: whole 128 x 128 tiles first; the tiles left over after the last full round
+    // over the SMs follow as `split` column strips each (128 x 32 strips when split = 4), so that
+    // the last, partly filled round is short.  CTA b takes virtual tiles b, b + grid, ...
+    auto decode = [&](int vt, int& p, int& m0, int& n0, int& bn) {
+        int tile = vt, sub = 0;
+        bn = BN;
+        if (vt >= full_tiles) {
+            const int piece = vt - full_tiles;
+            tile = full_tiles + piece / split;
+            sub = piece % split;
+            bn = BN / split;
+        }
+        const int tn = tile % tiles_n, tm = (tile / tiles_n) % tiles_m;
+        p = tile / (tiles_n * tiles_m);
+        m0 = tm * BM;
+        n0 = tn * BN + sub * bn;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -144,7 +152,10 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(&conv_bar[s], kConvWarps);
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&acc_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], kEpiWarps);
+        }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -166,102 +177,126 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
-            int issued = 0;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (kb / STAGES) & 1;
-                if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) break;
-                mbar_expect_tx(&full_bar[s], A_TILE_BYTES + bn * BK * 4);
-                tma_load_3d(A_hi(s), &tmA, kb * BK, m0, p, &full_bar[s]);
-                for (int c = 0; c < bn / 32; ++c) {      // B arrives in boxes of 32 columns (or 32 rows of X^_p)
-                    if (B_KMAJOR)
-                        tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, kb * BK, n0 + 32 * c, p, &full_bar[s]);
-                    else
-                        tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, n0 + 32 * c, kb * BK, p, &full_bar[s]);
+            int it = 0;                          // k-blocks issued so far, over all tiles
+            bool ok = true;
+            for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
+                int p, m0, n0, bn;
+                decode(vt, p, m0, n0, bn);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) { ok = false; break; }
+                    mbar_expect_tx(&full_bar[s], A_TILE_BYTES + bn * BK * 4);
+                    tma_load_3d(A_hi(s), &tmA, kb * BK, m0, p, &full_bar[s]);
+                    for (int c = 0; c < bn / 32; ++c) {      // B arrives in boxes of 32 columns (or 32 rows of X^_p)
+                        if (B_KMAJOR)
+                            tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, kb * BK, n0 + 32 * c, p, &full_bar[s]);
+                        else
+                            tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, n0 + 32 * c, kb * BK, p, &full_bar[s]);
+                    }
                 }
-                ++issued;
             }
             if (*abort_p) {                      // let copies still in flight land before the CTA exits
-                for (int kb = issued > STAGES ? issued - STAGES : 0; kb < issued; ++kb) {
+                for (int j = it > STAGES ? it - STAGES : 0; j < it; ++j) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(&full_bar[kb % STAGES], (kb / STAGES) & 1) && clock64() - t0 < kWaitCycles) {}
+                    while (!mbar_try_wait(&full_bar[j % STAGES], (j / STAGES) & 1) && clock64() - t0 < kWaitCycles) {}
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
-                                   ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            int it = 0, ti = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (kb / STAGES) & 1;
-                if (!mbar_wait(&conv_bar[s], ph, abort_p)) { ok = false; break; }
+            for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x, ++ti) {
+                int p, m0, n0, bn;
+                decode(vt, p, m0, n0, bn);
+                const int buf = ti & 1;
+                // the tile before last used this accumulator: it must have been read back
+                if (!mbar_wait(&acc_empty[buf], ((ti >> 1) & 1) ^ 1, abort_p)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_hi = smem_u32(A_hi(s)), a_lo = smem_u32(A_lo(s));
-                const uint32_t b_hi = smem_u32(B_hi(s)), b_lo = smem_u32(B_lo(s));
+                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
+                const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
+                                       ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    if (!mbar_wait(&conv_bar[s], ph, abort_p)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_hi = smem_u32(A_hi(s)), a_lo = smem_u32(A_lo(s));
+                    const uint32_t b_hi = smem_u32(B_hi(s)), b_lo = smem_u32(B_lo(s));
 #pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k) {
-                    // K-major: next 8 elements of K are 32 bytes further inside the swizzled row;
-                    // MN-major: next 8 k-rows are 8 * 128 bytes further in every 32-column chunk
-                    const uint32_t a_off = k * UMMA_K * 4;
-                    const uint32_t b_off = B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128;
-                    const uint64_t da_hi = desc_kmajor(a_hi + a_off);
-                    const uint64_t da_lo = desc_kmajor(a_lo + a_off);
-                    const uint64_t db_hi = B_KMAJOR ? desc_kmajor(b_hi + b_off) : desc_mnmajor(b_hi + b_off);
-                    const uint64_t db_lo = B_KMAJOR ? desc_kmajor(b_lo + b_off) : desc_mnmajor(b_lo + b_off);
-                    umma_tf32(tmem_base, da_lo, db_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);   // small terms first
-                    umma_tf32(tmem_base, da_hi, db_lo, idesc, 1u);
-                    umma_tf32(tmem_base, da_hi, db_hi, idesc, 1u);
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // K-major: next 8 elements of K are 32 bytes further inside the swizzled row;
+                        // MN-major: next 8 k-rows are 8 * 128 bytes further in every 32-column chunk
+                        const uint32_t a_off = k * UMMA_K * 4;
+                        const uint32_t b_off = B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128;
+                        const uint64_t da_hi = desc_kmajor(a_hi + a_off);
+                        const uint64_t da_lo = desc_kmajor(a_lo + a_off);
+                        const uint64_t db_hi = B_KMAJOR ? desc_kmajor(b_hi + b_off) : desc_mnmajor(b_hi + b_off);
+                        const uint64_t db_lo = B_KMAJOR ? desc_kmajor(b_lo + b_off) : desc_mnmajor(b_lo + b_off);
+                        umma_tf32(tmem_d, da_lo, db_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);   // small terms first
+                        umma_tf32(tmem_d, da_hi, db_lo, idesc, 1u);
+                        umma_tf32(tmem_d, da_hi, db_hi, idesc, 1u);
+                    }
+                    umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
                 }
-                umma_commit(&empty_bar[s]);          // stage reusable once these MMAs have read it
+                if (ok) umma_commit(&acc_full[buf]); // this tile's accumulator complete
             }
-            if (ok) umma_commit(&acc_bar);           // accumulator complete
+        }
+    } else if (warp < 2 + kConvWarps) {
+        // ------------------------------ split hi / lo ------------------------------
+        const int tc = threadIdx.x - 64;             // 0..kConvThreads-1
+        int it = 0;
+        bool ok = true;
+        for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
+            int p, m0, n0, bn;
+            decode(vt, p, m0, n0, bn);
+            const int b_float4 = bn * BK / 4;        // 16-byte units of one B tile
+            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                if (!mbar_wait(&full_bar[s], ph, abort_p)) { ok = false; break; }
+                float4* hi[2] = {reinterpret_cast<float4*>(A_hi(s)), reinterpret_cast<float4*>(B_hi(s))};
+                float4* lo[2] = {reinterpret_cast<float4*>(A_lo(s)), reinterpret_cast<float4*>(B_lo(s))};
+                const int count[2] = {A_TILE_BYTES / 16, b_float4};
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+#pragma unroll 4
+                    for (int idx = tc; idx < count[t]; idx += kConvThreads) {
+                        const float4 v = hi[t][idx];
+                        float4 h, l;
+                        h.x = to_tf32(v.x); h.y = to_tf32(v.y); h.z = to_tf32(v.z); h.w = to_tf32(v.w);
+                        l.x = to_tf32(v.x - h.x); l.y = to_tf32(v.y - h.y); l.z = to_tf32(v.z - h.z); l.w = to_tf32(v.w - h.w);
+                        hi[t][idx] = h;
+                        lo[t][idx] = l;
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the tiles visible to the MMA unit
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&conv_bar[s]);
+            }
         }
     } else {
-        // ------------------------------ split hi / lo, then epilogue ------------------------------
-        const int tc = threadIdx.x - 64;             // 0..kConvThreads-1
-        bool ok = true;
-        for (int kb = 0; kb < num_kb; ++kb) {
-            const int s = kb % STAGES;
-            const uint32_t ph = (kb / STAGES) & 1;
-            if (!mbar_wait(&full_bar[s], ph, abort_p)) { ok = false; break; }
-            float4* hi[2] = {reinterpret_cast<float4*>(A_hi(s)), reinterpret_cast<float4*>(B_hi(s))};
-            float4* lo[2] = {reinterpret_cast<float4*>(A_lo(s)), reinterpret_cast<float4*>(B_lo(s))};
-            const int count[2] = {A_TILE_BYTES / 16, b_float4};
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-#pragma unroll 4
-                for (int idx = tc; idx < count[t]; idx += kConvThreads) {
-                    const float4 v = hi[t][idx];
-                    float4 h, l;
-                    h.x = to_tf32(v.x); h.y = to_tf32(v.y); h.z = to_tf32(v.z); h.w = to_tf32(v.w);
-                    l.x = to_tf32(v.x - h.x); l.y = to_tf32(v.y - h.y); l.z = to_tf32(v.z - h.z); l.w = to_tf32(v.w - h.w);
-                    hi[t][idx] = h;
-                    lo[t][idx] = l;
-                }
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the tiles visible to the MMA unit
+        // ------------------------------ epilogue ------------------------------
+        const int q = warp & 3;                      // this warp may touch TMEM lanes 32q .. 32q+31
+        const float shrink = (float)prm.shrink, eta = (float)prm.eta;
+        const bool vec = (prm.N % 4 == 0);
+        int ti = 0;
+        for (int vt = blockIdx.x; vt < n_virtual; vt += gridDim.x, ++ti) {
+            int p, m0, n0, bn;
+            decode(vt, p, m0, n0, bn);
+            const int buf = ti & 1;
+            const bool acc_ready = mbar_wait(&acc_full[buf], (ti >> 1) & 1, abort_p);
             __syncwarp();
-            if (lane == 0) mbar_arrive(&conv_bar[s]);
-        }
-        const bool acc_ready = ok && mbar_wait(&acc_bar, 0, abort_p);
-        __syncwarp();
-        if (__all_sync(0xffffffffu, acc_ready)) {    // tcgen05.ld is warp-collective: all lanes or none
+            if (!__all_sync(0xffffffffu, acc_ready)) break;   // tcgen05.ld is warp-collective: all lanes or none
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int q = warp & 3;                  // this warp may touch TMEM lanes 32q .. 32q+31
-            const int half = (warp - 2) >> 2;        // two warps share a lane quarter: half the columns each
-            const int c_begin = bn >= 64 ? half * (bn / 2) : (half == 0 ? 0 : bn);
-            const int c_end = bn >= 64 ? (half + 1) * (bn / 2) : bn;
             const int64_t gm = (int64_t)m0 + q * 32 + lane;
             float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
-            const float shrink = (float)prm.shrink, eta = (float)prm.eta;
-            const bool vec = (prm.N % 4 == 0);
 #pragma unroll 1
-            for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+            for (int c0 = 0; c0 < bn; c0 += 32) {
                 uint32_t r[32];
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0;
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0);
                 asm volatile(
                     "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
                     "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -272,6 +307,11 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                       "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                     : "r"(taddr));
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (c0 + 32 >= bn) {                 // last read of this accumulator: hand it back
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                }
                 if (gm < prm.M) {
                     float* crow = C + gm * prm.N + n0 + c0;
                     if (vec && n0 + c0 + 32 <= prm.N) {
@@ -374,9 +414,10 @@ gpd_status launch(const GemmParams& prm, cudaStream_t st) {
     if (rem > 0 && rem * 4 <= sms) split = 4;
     else if (rem > 0 && rem * 2 <= sms) split = 2;
     const int full_tiles = (int)(tiles - (split > 1 ? rem : 0));
-    const int64_t ctas = full_tiles + (int64_t)(split > 1 ? rem : 0) * split;
-    sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<(unsigned)ctas, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n,
-                                                                                         full_tiles, split);
+    const int64_t n_virtual = full_tiles + (int64_t)(split > 1 ? rem : 0) * split;
+    const unsigned grid = (unsigned)std::min<int64_t>(n_virtual, sms);   // persistent: one CTA per SM walks the list
+    sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<grid, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n, full_tiles,
+                                                                              split, (int)n_virtual);
     return launch_ok();
 }
 
