@@ -36,6 +36,21 @@ def test_result_struct_layout_matches_header():
     assert g.gpd_locate_result.flagged.offset == 48 and g.gpd_locate_result.forced.offset == 112
 
 
+def test_position_result_layout_workspace_query_and_argument_checks():
+    import ctypes as C
+    # int32 x4, int64 x4, 64 bytes
+    assert g.POSITION_RESULT_BYTES == 16 + 32 + 64 and g.gpd_position_result.touched.offset == 48
+    c = wl.CONFIG_3_MATMUL
+    plan = g.gpd_plan((c.N1, c.N0, c.B), (c.m, c.n, c.d, 1), c.P)
+    L = (c.N1 // c.m) * max(c.B // c.d, c.N0 // c.n)             # largest product of the plan (audit: N1/m x N0/n)
+    assert plan.query(g.GPD_Q_POSITION_WORKSPACE_BYTES) == 256 + 4 * L
+    one = C.c_void_p(4096)                                        # never dereferenced: the checks come first
+    assert g.lib.gpd_correct_positions(plan.handle, g.GPD_FWD, one, one, None, None) == g.GPD_ERR_WORKSPACE
+    assert g.lib.gpd_correct_positions(plan.handle, g.GPD_FWD, None, one, one, None) == g.GPD_ERR_ARG
+    assert g.lib.gpd_correct_positions(None, g.GPD_FWD, one, one, one, None) == g.GPD_ERR_ARG
+    plan.destroy()
+
+
 @pytest.mark.parametrize("shape,split,P", [
     ((64, 64, 64), (2, 2, 2, 1), 11), ((4096, 4096, 1), (4, 2, 1, 1), 13),
     ((8192, 8192, 512), (2, 4, 2, 1), 25), ((4096, 4096, 256), (2, 2, 1, 1), 10),
