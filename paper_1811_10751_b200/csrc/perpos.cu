@@ -20,8 +20,6 @@ namespace gpd {
 
 namespace {
 
-constexpr int kMaxT = kMaxR / 2;          // errors correctable per codeword
-
 struct PosParams {
     void* Z;                              // [P][L]
     const double* H;                      // [R][P] orthonormal parity check
@@ -42,62 +40,99 @@ __global__ void __launch_bounds__(256) position_scan_kernel(PosParams prm) {
     for (int i = threadIdx.x; i < RT * prm.P; i += 256) sH[i] = i < prm.R * prm.P ? prm.H[i] : 0.0;
     __syncthreads();
     const T* Z = reinterpret_cast<const T*>(prm.Z);
-    for (int64_t pos = (int64_t)blockIdx.x * 256 + threadIdx.x; pos < prm.L; pos += (int64_t)gridDim.x * 256) {
+    const int lane = threadIdx.x & 31;
+    // all lanes of a warp run the same rounds (the counters are updated once per warp and round)
+    for (int64_t base = (int64_t)blockIdx.x * 256; base < prm.L; base += (int64_t)gridDim.x * 256) {
+        const int64_t pos = base + threadIdx.x;
+        const bool valid = pos < prm.L;
         double r[RT];
 #pragma unroll
         for (int j = 0; j < RT; ++j) r[j] = 0.0;
         double z2 = 0.0;
         bool finite = true;
+        if (valid) {
 #pragma unroll 5
-        for (int p = 0; p < prm.P; ++p) {
-            const double z = (double)__ldcs(Z + (int64_t)p * prm.L + pos);
-            finite &= isfinite(z);
-            z2 = fma(z, z, z2);
+            for (int p = 0; p < prm.P; ++p) {
+                const double z = (double)__ldcs(Z + (int64_t)p * prm.L + pos);
+                finite &= isfinite(z);
+                z2 = fma(z, z, z2);
 #pragma unroll
-            for (int j = 0; j < RT; ++j) r[j] = fma(sH[j * prm.P + p], z, r[j]);   // rows R .. RT-1 are zero
+                for (int j = 0; j < RT; ++j) r[j] = fma(sH[j * prm.P + p], z, r[j]);   // rows R .. RT-1 are zero
+            }
         }
         double r2 = 0.0;
 #pragma unroll
         for (int j = 0; j < RT; ++j) r2 = fma(r[j], r[j], r2);
-        if (!finite) {                    // reported as failed, left untouched
-            atomicAdd(&prm.counters[1], 1ULL);
-            atomicAdd(&prm.counters[3], 1ULL);
-        } else if (r2 > prm.tau2 * z2) {
-            atomicAdd(&prm.counters[1], 1ULL);
-            prm.list[atomicAdd(&prm.counters[0], 1ULL)] = (unsigned int)pos;
+        const bool bad = valid && !finite;                    // reported as failed, left untouched
+        const bool listed = valid && finite && r2 > prm.tau2 * z2;
+        const unsigned int m_bad = __ballot_sync(0xffffffffu, bad), m_list = __ballot_sync(0xffffffffu, listed);
+        if (m_bad | m_list) {
+            unsigned long long slot = 0ULL;
+            if (lane == 0) {
+                atomicAdd(&prm.counters[1], (unsigned long long)(__popc(m_bad) + __popc(m_list)));
+                if (m_bad) atomicAdd(&prm.counters[3], (unsigned long long)__popc(m_bad));
+                if (m_list) slot = atomicAdd(&prm.counters[0], (unsigned long long)__popc(m_list));
+            }
+            slot = __shfl_sync(0xffffffffu, slot, 0);
+            if (listed) prm.list[slot + __popc(m_list & ((1u << lane) - 1u))] = (unsigned int)pos;
         }
     }
 }
 
-// Gaussian elimination with partial pivoting on the n x (n + 1) system held in a (row stride
-// kMaxT + 1); false when a pivot vanishes against the size of the matrix.
-__device__ bool solve_small(double (*a)[kMaxT + 1], int n, double* x) {
+// Gaussian elimination with partial pivoting on the n x (n + 1) system held in a; false when a
+// pivot vanishes against the size of the matrix.  Every loop has the compile-time bound TT and
+// every index is static after unrolling, so that for small TT the system stays in registers.
+template <int TT>
+__device__ __forceinline__ bool solve_small(double (&a)[TT][TT + 1], int n, double (&x)[TT]) {
+    constexpr int UF = TT <= 4 ? 32 : 1;     // small systems: fully unrolled, register-resident
     double amax = 0.0;
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j) amax = fmax(amax, fabs(a[i][j]));
+#pragma unroll UF
+    for (int i = 0; i < TT; ++i)
+#pragma unroll UF
+        for (int j = 0; j < TT; ++j)
+            if (i < n && j < n) amax = fmax(amax, fabs(a[i][j]));
     if (!(amax > 0.0)) return false;
-    for (int k = 0; k < n; ++k) {
-        int piv = k;
-        for (int i = k + 1; i < n; ++i)
-            if (fabs(a[i][k]) > fabs(a[piv][k])) piv = i;
-        if (fabs(a[piv][k]) <= 1e-13 * amax) return false;
-        if (piv != k)
-            for (int j = k; j <= n; ++j) { const double t = a[k][j]; a[k][j] = a[piv][j]; a[piv][j] = t; }
-        const double inv = 1.0 / a[k][k];
-        for (int i = k + 1; i < n; ++i) {
-            const double f = a[i][k] * inv;
-            for (int j = k; j <= n; ++j) a[i][j] -= f * a[k][j];
+    bool ok = true;
+#pragma unroll UF
+    for (int k = 0; k < TT; ++k) {
+        if (k < n) {
+#pragma unroll UF
+            for (int i = k + 1; i < TT; ++i) {                   // bring the largest entry of column k up
+                if (i < n && fabs(a[i][k]) > fabs(a[k][k])) {
+#pragma unroll UF
+                    for (int j = 0; j <= TT; ++j) { const double t = a[k][j]; a[k][j] = a[i][j]; a[i][j] = t; }
+                }
+            }
+            if (fabs(a[k][k]) <= 1e-13 * amax) ok = false;
+            const double inv = 1.0 / a[k][k];
+#pragma unroll UF
+            for (int i = k + 1; i < TT; ++i) {
+                if (i < n) {
+                    const double f = a[i][k] * inv;
+#pragma unroll UF
+                    for (int j = 0; j <= TT; ++j)
+                        if (j >= k) a[i][j] -= f * a[k][j];
+                }
+            }
         }
     }
-    for (int i = n - 1; i >= 0; --i) {
-        double s = a[i][n];
-        for (int j = i + 1; j < n; ++j) s -= a[i][j] * x[j];
-        x[i] = s / a[i][i];
+    if (!ok) return false;
+#pragma unroll UF
+    for (int i = TT - 1; i >= 0; --i) {
+        if (i < n) {
+            double s = a[i][TT];
+#pragma unroll UF
+            for (int j = 0; j < TT; ++j)
+                if (j > i && j < n) s -= a[i][j] * x[j];
+            x[i] = s / a[i][i];
+        }
     }
     return true;
 }
 
-template <typename T>
+// RT: parity checks rounded up (8 or 32); TT: errors per codeword rounded up (4 or 16).  The
+// right-hand side of a system sits in column TT of its rows.
+template <typename T, int RT, int TT>
 __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
     extern __shared__ double sm[];        // H [R][P], Hg [R][P], points [P]
     double* sH = sm;
@@ -106,100 +141,179 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
     for (int i = threadIdx.x; i < prm.R * prm.P; i += 64) { sH[i] = prm.H[i]; sHg[i] = prm.Hg[i]; }
     for (int i = threadIdx.x; i < prm.P; i += 64) sPts[i] = prm.points[i];
     __syncthreads();
+    constexpr int UF = TT <= 4 ? 32 : 1;     // small codes: loops fully unrolled, everything in registers
     T* Z = reinterpret_cast<T*>(prm.Z);
     const int P = prm.P, R = prm.R, t = R / 2;
     const unsigned long long listed = prm.counters[0];
-    for (unsigned long long it = (unsigned long long)blockIdx.x * 64 + threadIdx.x; it < listed;
-         it += (unsigned long long)gridDim.x * 64) {
-        const int64_t pos = prm.list[it];
-        double r[kMaxR], S[kMaxR];
-        for (int j = 0; j < R; ++j) { r[j] = 0.0; S[j] = 0.0; }
+    // all lanes of a warp run the same rounds (the counters are updated once per warp and round)
+    for (unsigned long long base = (unsigned long long)blockIdx.x * 64; base < listed;
+         base += (unsigned long long)gridDim.x * 64) {
+        const unsigned long long it = base + threadIdx.x;
+        const bool valid = it < listed;
+        const int64_t pos = valid ? prm.list[it] : 0;
+        double r[RT], S[RT];
+#pragma unroll UF
+        for (int j = 0; j < RT; ++j) { r[j] = 0.0; S[j] = 0.0; }
         double z2 = 0.0;
         for (int p = 0; p < P; ++p) {
             const double z = (double)Z[(int64_t)p * prm.L + pos];
             z2 = fma(z, z, z2);
-            for (int j = 0; j < R; ++j) {
-                r[j] = fma(sH[j * P + p], z, r[j]);
-                S[j] = fma(sHg[j * P + p], z, S[j]);
+#pragma unroll UF
+            for (int j = 0; j < RT; ++j) {
+                if (j < R) {
+                    r[j] = fma(sH[j * P + p], z, r[j]);
+                    S[j] = fma(sHg[j * P + p], z, S[j]);
+                }
             }
         }
         const double limit = prm.tau2 * z2;
         int accepted = 0;
-        int nodes[kMaxT];
-        double err[kMaxT];
-        for (int nu = 1; nu <= t && accepted == 0; ++nu) {
-            double a[kMaxT][kMaxT + 1], lam[kMaxT];
-            for (int j = 0; j < nu; ++j) {
-                for (int i = 0; i < nu; ++i) a[j][i] = S[j + i];
-                a[j][nu] = -S[j + nu];
+        int nodes[TT];
+        double err[TT];
+#pragma unroll UF
+        for (int i = 0; i < TT; ++i) { nodes[i] = 0; err[i] = 0.0; }
+#pragma unroll 1
+        for (int nu = 1; valid && nu <= t && accepted == 0; ++nu) {
+            double a[TT][TT + 1], lam[TT];
+#pragma unroll UF
+            for (int j = 0; j < TT; ++j) {
+                lam[j] = 0.0;
+#pragma unroll UF
+                for (int i = 0; i <= TT; ++i) a[j][i] = 0.0;
             }
-            if (!solve_small(a, nu, lam)) continue;
+            // Hankel system of the locator: sum_i l_i S_{j+i} = -S_{j+nu}, j = 0 .. nu-1
+            if constexpr (TT <= 4) {                              // S_{j+i} without a dynamic index
+#pragma unroll
+                for (int j = 0; j < TT; ++j)
+#pragma unroll
+                    for (int i = 0; i < TT; ++i)
+                        if (j < nu && i < nu) {
+#pragma unroll
+                            for (int q = 0; q < RT; ++q)
+                                if (q == j + i) a[j][i] = S[q];
+                        }
+#pragma unroll
+                for (int j = 0; j < TT; ++j)
+                    if (j < nu) {
+#pragma unroll
+                        for (int q = 0; q < RT; ++q)
+                            if (q == j + nu) a[j][TT] = -S[q];
+                    }
+            } else {
+                for (int j = 0; j < nu; ++j) {
+                    for (int i = 0; i < nu; ++i) a[j][i] = S[j + i];
+                    a[j][TT] = -S[j + nu];
+                }
+            }
+            if (!solve_small<TT>(a, nu, lam)) continue;
             // the nu points where the locator is smallest
             unsigned long long taken = 0ULL;
-            for (int k = 0; k < nu; ++k) {
-                int best = -1;
-                double best_v = 0.0;
-                for (int p = 0; p < P; ++p) {
-                    if ((taken >> p) & 1ULL) continue;
-                    const double x = sPts[p];
-                    double v = 1.0;
-                    for (int i = nu - 1; i >= 0; --i) v = fma(v, x, lam[i]);
-                    v = fabs(v);
-                    if (best < 0 || v < best_v) { best = p; best_v = v; }
+#pragma unroll UF
+            for (int k = 0; k < TT; ++k) {
+                if (k < nu) {
+                    int best = -1;
+                    double best_v = 0.0;
+                    for (int p = 0; p < P; ++p) {
+                        if ((taken >> p) & 1ULL) continue;
+                        const double x = sPts[p];
+                        double v = 1.0;
+#pragma unroll UF
+                        for (int i = TT - 1; i >= 0; --i)
+                            if (i < nu) v = fma(v, x, lam[i]);
+                        v = fabs(v);
+                        if (best < 0 || v < best_v) { best = p; best_v = v; }
+                    }
+                    nodes[k] = best;
+                    taken |= 1ULL << best;
                 }
-                nodes[k] = best;
-                taken |= 1ULL << best;
             }
             // least squares H_A e = r through the normal equations, then one step of refinement on the
             // residual (neighbouring nodes make H_A ill-conditioned; the refinement brings the error
             // values back to the accuracy of an orthogonal factorisation)
             bool solved = true;
-            double left = 0.0;
-            for (int i = 0; i < nu; ++i) err[i] = 0.0;
+#pragma unroll UF
+            for (int i = 0; i < TT; ++i) err[i] = 0.0;
+#pragma unroll 1
             for (int pass = 0; pass < 2 && solved; ++pass) {
-                double v[kMaxR];
-                for (int q = 0; q < R; ++q) {
+                double v[RT];
+#pragma unroll UF
+                for (int q = 0; q < RT; ++q) {
                     double w = r[q];
-                    for (int i = 0; i < nu; ++i) w = fma(-sH[q * P + nodes[i]], err[i], w);
+                    if (q < R) {
+#pragma unroll UF
+                        for (int i = 0; i < TT; ++i)
+                            if (i < nu) w = fma(-sH[q * P + nodes[i]], err[i], w);
+                    }
                     v[q] = w;
                 }
-                for (int i = 0; i < nu; ++i) {
-                    for (int j = 0; j < nu; ++j) {
-                        double s = 0.0;
-                        for (int q = 0; q < R; ++q) s = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s);
-                        a[i][j] = s;
+#pragma unroll UF
+                for (int i = 0; i < TT; ++i) {
+#pragma unroll UF
+                    for (int j = 0; j <= TT; ++j) a[i][j] = 0.0;
+                    if (i < nu) {
+#pragma unroll UF
+                        for (int j = 0; j < TT; ++j) {
+                            if (j < nu) {
+                                double s2 = 0.0;
+                                for (int q = 0; q < R; ++q) s2 = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s2);
+                                a[i][j] = s2;
+                            }
+                        }
+                        double s2 = 0.0;
+#pragma unroll UF
+                        for (int q = 0; q < RT; ++q)
+                            if (q < R) s2 = fma(sH[q * P + nodes[i]], v[q], s2);
+                        a[i][TT] = s2;
                     }
-                    double s = 0.0;
-                    for (int q = 0; q < R; ++q) s = fma(sH[q * P + nodes[i]], v[q], s);
-                    a[i][nu] = s;
                 }
-                double delta[kMaxT];
-                solved = solve_small(a, nu, delta);
-                if (solved)
-                    for (int i = 0; i < nu; ++i) err[i] += delta[i];
+                double delta[TT];
+#pragma unroll UF
+                for (int i = 0; i < TT; ++i) delta[i] = 0.0;
+                solved = solve_small<TT>(a, nu, delta);
+                if (solved) {
+#pragma unroll UF
+                    for (int i = 0; i < TT; ++i)
+                        if (i < nu) err[i] += delta[i];
+                }
             }
             if (!solved) continue;
-            for (int q = 0; q < R; ++q) {
-                double w = r[q];
-                for (int i = 0; i < nu; ++i) w = fma(-sH[q * P + nodes[i]], err[i], w);
-                left = fma(w, w, left);
+            double left = 0.0;
+#pragma unroll UF
+            for (int q = 0; q < RT; ++q) {
+                if (q < R) {
+                    double w = r[q];
+#pragma unroll UF
+                    for (int i = 0; i < TT; ++i)
+                        if (i < nu) w = fma(-sH[q * P + nodes[i]], err[i], w);
+                    left = fma(w, w, left);
+                }
             }
             if (left <= limit) accepted = nu;
         }
-        if (accepted == 0) {
-            atomicAdd(&prm.counters[3], 1ULL);
-            continue;
-        }
         unsigned long long mask = 0ULL;
-        for (int i = 0; i < accepted; ++i) {
-            T* cell = Z + (int64_t)nodes[i] * prm.L + pos;
-            *cell = (T)((double)*cell - err[i]);
-            mask |= 1ULL << nodes[i];
+#pragma unroll UF
+        for (int i = 0; i < TT; ++i) {
+            if (i < accepted) {
+                T* cell = Z + (int64_t)nodes[i] * prm.L + pos;
+                *cell = (T)((double)*cell - err[i]);
+                mask |= 1ULL << nodes[i];
+            }
         }
-        atomicAdd(&prm.counters[2], 1ULL);
-        atomicAdd(&prm.counters[4], (unsigned long long)accepted);
-        atomicMax(&prm.counters[5], (unsigned long long)accepted);
-        atomicOr(&prm.counters[6], mask);
+        const unsigned int n_fixed = __popc(__ballot_sync(0xffffffffu, valid && accepted > 0));
+        const unsigned int n_lost = __popc(__ballot_sync(0xffffffffu, valid && accepted == 0));
+        const unsigned int n_ent = __reduce_add_sync(0xffffffffu, (unsigned int)accepted);
+        const unsigned int n_max = __reduce_max_sync(0xffffffffu, (unsigned int)accepted);
+        const unsigned int m_lo = __reduce_or_sync(0xffffffffu, (unsigned int)mask);
+        const unsigned int m_hi = __reduce_or_sync(0xffffffffu, (unsigned int)(mask >> 32));
+        if ((threadIdx.x & 31) == 0) {
+            if (n_fixed) atomicAdd(&prm.counters[2], (unsigned long long)n_fixed);
+            if (n_lost) atomicAdd(&prm.counters[3], (unsigned long long)n_lost);
+            if (n_ent) {
+                atomicAdd(&prm.counters[4], (unsigned long long)n_ent);
+                atomicMax(&prm.counters[5], (unsigned long long)n_max);
+                atomicOr(&prm.counters[6], ((unsigned long long)m_hi << 32) | m_lo);
+            }
+        }
     }
 }
 
@@ -266,8 +380,10 @@ gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* o
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
         const size_t smem2 = sizeof(double) * (2 * pi.R * plan->P + plan->P);
         const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 63) / 64, 148 * 8));
-        if (f32) position_fix_kernel<float><<<grid2, 64, smem2, st>>>(prm);
-        else position_fix_kernel<double><<<grid2, 64, smem2, st>>>(prm);
+        if (pi.R <= 8) f32 ? position_fix_kernel<float, 8, 4><<<grid2, 64, smem2, st>>>(prm)
+                           : position_fix_kernel<double, 8, 4><<<grid2, 64, smem2, st>>>(prm);
+        else f32 ? position_fix_kernel<float, 32, 16><<<grid2, 64, smem2, st>>>(prm)
+                 : position_fix_kernel<double, 32, 16><<<grid2, 64, smem2, st>>>(prm);
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
     }
     position_finish_kernel<<<1, 64, 0, st>>>(prm);

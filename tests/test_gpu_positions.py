@@ -38,6 +38,7 @@ def _scatter_errors(Z, t_max, frac, seed, scale):
     (256, 256, 64, 2, 2, 1, 9, g.GPD_PREC_FP32),             # Q = 5,  R = 4, t = 2, FP32 outputs
     (512, 512, 128, 2, 4, 2, 25, g.GPD_PREC_FP64_SLICED),    # Q = 19, R = 6, t = 3, digit-plane products
     (128, 128, 32, 2, 2, 1, 6, g.GPD_PREC_FP32),             # R = 1: nothing correctable, errors only detected
+    (128, 128, 32, 2, 2, 2, 20, g.GPD_PREC_FP64),            # Q = 9,  R = 11, t = 5: the general (not unrolled) form
 ])
 def test_positions_repaired_like_the_oracle(N1, N0, B, m, n, d1, P, prec):
     rng = np.random.default_rng(N1 + P)
