@@ -203,8 +203,13 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
     if (points_host) {
         for (int p = 0; p < P; ++p) plan->points[p] = points_host[p];
     } else {
+        // Chebyshev points of the first kind, mirrored so that b_{P-1-p} = -b_p holds exactly
         const double pi = 3.14159265358979323846;
-        for (int p = 0; p < P; ++p) plan->points[p] = std::cos((2.0 * p + 1.0) * pi / (2.0 * P));
+        for (int p = 0; p < (P + 1) / 2; ++p) {
+            const double c = (2 * p + 1 == P) ? 0.0 : std::cos((2.0 * p + 1.0) * pi / (2.0 * P));
+            plan->points[p] = c;
+            plan->points[P - 1 - p] = -c;
+        }
     }
     for (int p = 0; p < P; ++p) {
         if (!std::isfinite(plan->points[p])) { delete plan; return GPD_ERR_POINTS; }

@@ -93,6 +93,27 @@ def test_sliced_worker_products_match_oracle(N1, N0, B, m, n, d1, P, S):
     assert np.abs(got - Zo).max() < (1e-10 if S == 6 else 2e-8) * np.sqrt(np.mean(Zo ** 2))
 
 
+@pytest.mark.parametrize("N1,N0,B,m,n,d1,P,S", [(256, 512, 128, 2, 4, 2, 25, 6), (192, 96, 64, 3, 2, 2, 20, 5),
+                                                (256, 256, 64, 2, 2, 1, 8, 6)])
+def test_sliced_products_with_the_library_points(N1, N0, B, m, n, d1, P, S):
+    """The library's own evaluation points (Chebyshev, mirrored exactly: b_{P-1-p} = -b_p, 0 in the
+    middle for odd P) instead of the oracle's; the oracle is given the same points."""
+    plan0 = g.gpd_plan((N1, N0, B), (m, n, d1, 1), P)
+    pts = plan0.table(g.GPD_TABLE_POINTS)
+    plan0.destroy()
+    assert np.array_equal(pts, -pts[::-1]) and np.all(np.diff(pts) < 0)
+    W, X = _inputs(N1, N0, B, seed=N1 + P)
+    code = GPCode(N1, N0, B, m, n, d1, 1, P, points=pts)
+    cp, Z = _sliced_products(code, W, X, S)
+    Wsh, Xsh = op.encode_W(W, code), op.encode_X(X, code)
+    got = cp.outputs_as_array(g.GPD_FWD, Z)
+    tol = _output_tolerance(W, code, Wsh, Xsh, S)
+    assert (np.abs(got - op.worker_products(Wsh, Xsh)) <= tol).all()
+    r = cp.locate(g.GPD_FWD, Z)
+    assert r.outcome == NO_ERROR
+    assert op.rel_fro(cp.decode(g.GPD_FWD, Z), op.ref_forward(W, X)) < 1e-4
+
+
 def test_sliced_scales_zero_rows_and_tiny_values():
     """Row / column scales: rows of zeros, columns of zeros and operands 1e-30 and 1e+20 times the
     usual size decode to the same relative accuracy (the digits carry no absolute scale)."""
