@@ -386,6 +386,9 @@ def run_ours(args, cfg):
                     "ops": f"int8 multiply-adds counted as 2 operations; {pairs} digit-plane pairs per product",
                     "ops_per_launch": int8_ops, "ms_per_launch": gemm_ms,
                     "fp64_equivalent_tflops": exec_flops / (gemm_ms * 1e-3) / 1e12}
+        fp64_measured = measure_fp64_matmul_peak(torch)
+        roofline["fp64_peak_measured_here"] = fp64_measured       # torch.matmul FP64 8192^3, best of 10 (cuBLAS)
+        roofline["fp64_equivalent_over_fp64_peak"] = roofline["fp64_equivalent_tflops"] / fp64_measured
     else:
         # FP64 tensor peak: MEASURED_PEAKS.json has no FP64 figure, and scaling its power-capped bf16
         # number by the nominal ratio gives a value below what the FP64 path delivers (FP64 does not
@@ -401,6 +404,25 @@ def run_ours(args, cfg):
                     "peak_nominal_fp64": NOMINAL_FP64_TFLOPS,
                     "peak_from_bf16_ratio": fp64_from_ratio,
                     "flops_per_launch": exec_flops, "ms_per_launch": gemm_ms}
+    # Sum of the stage rooflines (the stages depend on each other, so their floors add): algorithmic
+    # bytes at the measured copy bandwidth, the products at the tensor peak of the arithmetic they run in.
+    hbm = peaks["hbm_gbs"] * 1e9
+    Lpos = (cfg.N1 // cfg.m) * (cfg.B // cfg.d)
+    e_s = float(planes) if sliced else 8.0               # bytes per stored share value
+    t_stage = {
+        "encode_A": (cfg.N1 * cfg.N0 * 4 + cfg.P * (cfg.N1 // cfg.m) * (cfg.N0 // cfg.n) * e_s) / hbm,
+        "encode_B": (cfg.N0 * cfg.B * 4 + cfg.P * (cfg.N0 // cfg.n) * (cfg.B // cfg.d) * e_s) / hbm,
+        "worker_gemm": max((roofline.get("ops_per_launch") or roofline.get("flops_per_launch")) / (roofline["peak"] * 1e12),
+                           (cfg.P * ((cfg.N1 // cfg.m) + (cfg.B // cfg.d)) * (cfg.N0 // cfg.n) * e_s + cfg.P * Lpos * 8) / hbm),
+        "inject": 2 * cfg.inject_prob * cfg.P * Lpos * 8 / hbm,
+        "locate": cfg.P * Lpos * 8 / hbm,
+        "decode": (cfg.P * Lpos * 8 + cfg.N1 * cfg.B * 4) / hbm,
+    }
+    path_roofline = {"stages_us": {k: round(v * 1e6, 1) for k, v in t_stage.items()},
+                     "sum_ms": sum(t_stage.values()) * 1e3,
+                     "frac": sum(t_stage.values()) * 1e3 / (ms / args.steps),
+                     "note": "sum of stage floors / measured ms_per_step; bytes at the measured copy bandwidth, "
+                             "products at the peak named in roofline.peak_source"}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -411,7 +433,7 @@ def run_ours(args, cfg):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(W.nbytes + X.nbytes),
                 "d2h_bytes_per_step": int(cfg.N1 * cfg.B * 4 + g.RESULT_BYTES), "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
-        "clocks": clocks, "roofline": roofline, "stage_ms": stage_ms, "check": check,
+        "clocks": clocks, "roofline": roofline, "path_roofline": path_roofline, "stage_ms": stage_ms, "check": check,
     }
     if rank == 0 and world == 1 and cfg.N1 >= CPU_SAMPLE_ROWS:
         Wsmp = np.ascontiguousarray(W[:CPU_SAMPLE_ROWS])
