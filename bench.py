@@ -473,35 +473,45 @@ def measure_tf32_matmul_peak(torch) -> float:
     return 2.0 * n ** 3 / (best * 1e-3) / 1e12
 
 
-def run_mlp_layer(args):
-    """Secondary workload (not the headline line): one hidden layer of the coded MLP step,
-    4096 x 4096 weights, batch 256, split 2 x 2, P = 10, FP32 shares, tensor-core 3xTF32 products;
-    step = coded forward + coded backward + coded update through coded_layer_step."""
+def run_layer(args, kind):
+    """Secondary workloads (not the headline line): the coded training step of one layer,
+    step = coded forward + coded backward + coded update through coded_layer_step.
+      mlp_layer: hidden layer of the MLP, 4096 x 4096 weights, batch 256, split 2 x 2, P = 10; thresholds
+                 5 / 6, so FP32 shares and tensor-core 3xTF32 products
+      sae_layer: encoder of the sparse autoencoder, 8192 x 1024 weights, batch 1024, split 4 x 4, P = 36;
+                 thresholds 19 / 28, so FP64 shares and FP64 mma products"""
     import torch
     import paper_1811_10751_b200 as g
     import workloads as wl
-    c4 = wl.CONFIG_4_MLP
-    N, B, P = c4.widths[1], c4.B, c4.P
+    if kind == "mlp_layer":
+        c = wl.CONFIG_4_MLP
+        N1, N0, B, m, n, P, prob, seed = c.widths[1], c.widths[1], c.B, c.m, c.n, c.P, c.inject_prob, c.seed
+        act, wname = g.GPD_ACT_RELU, "cfg4_mlp_hidden_layer_4096x4096_b256"
+    else:
+        c = wl.CONFIG_5_AUTOENCODER
+        N1, N0, B, m, n, P, prob, seed = c.n_hidden, c.n_visible, c.B, c.m, c.n, c.P, c.inject_prob, c.seed
+        act, wname = g.GPD_ACT_SIGMOID, "cfg5_autoencoder_encoder_8192x1024_b1024"
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-    gen = torch.Generator(device="cuda").manual_seed(c4.seed)
-    W = torch.randn((N, N), device="cuda", generator=gen) * (2.0 / N) ** 0.5
-    X = torch.randn((N, B), device="cuda", generator=gen).clamp_(min=0)
-    D = torch.randn((N, B), device="cuda", generator=gen) / B
+    gen = torch.Generator(device="cuda").manual_seed(seed)
+    W = torch.randn((N1, N0), device="cuda", generator=gen) * (2.0 / N0) ** 0.5
+    X = torch.randn((N0, B), device="cuda", generator=gen).clamp_(min=0)
+    D = torch.randn((N1, B), device="cuda", generator=gen) / B
     DT = D.t().contiguous()
-    plan = g.gpd_plan((N, N, B), (c4.m, c4.n, 1, 1), P)
+    plan = g.gpd_plan((N1, N0, B), (m, n, 1, 1), P)
+    f32 = plan.query(g.GPD_Q_ELEMENT_SIZE) == 4
     Wsh = plan.empty(g.GPD_Q_W_SHARE_ELEMS)
     g.gpd_encode_A(plan, W, Wsh)
     ws, res = plan.workspace(step=True), g.new_results(3)
-    S, Xn = torch.empty((N, B), device="cuda"), torch.empty((N, B), device="cuda")
-    CT = torch.empty((B, N), device="cuda")
+    S, Xn = torch.empty((N1, B), device="cuda"), torch.empty((N1, B), device="cuda")
+    CT = torch.empty((B, N0), device="cuda")
     stream = torch.cuda.Stream()
 
     def step(i):
-        g.coded_layer_step(plan, g.GPD_PHASE_FWD, Wsh, X=X, activation=g.GPD_ACT_RELU, inject_seed=1000 + 16 * i,
-                           inject_prob=c4.inject_prob, S_out=S, Xnext_out=Xn, CT_out=CT, results=res, workspace=ws,
+        g.coded_layer_step(plan, g.GPD_PHASE_FWD, Wsh, X=X, activation=act, inject_seed=1000 + 16 * i,
+                           inject_prob=prob, S_out=S, Xnext_out=Xn, CT_out=CT, results=res, workspace=ws,
                            stream=stream)
         g.coded_layer_step(plan, g.GPD_PHASE_BWD | g.GPD_PHASE_UPD, Wsh, X=X, Delta=D, DeltaT=DT, eta=1e-4,
-                           inject_seed=1000 + 16 * i, inject_prob=c4.inject_prob, S_out=S, Xnext_out=Xn, CT_out=CT,
+                           inject_seed=1000 + 16 * i, inject_prob=prob, S_out=S, Xnext_out=Xn, CT_out=CT,
                            results=res, workspace=ws, stream=stream)
 
     with torch.cuda.stream(stream):
@@ -538,20 +548,31 @@ def run_mlp_layer(args):
         torch.cuda.synchronize()
         kern[name] = a.elapsed_time(b) / args.steps
     status = g.gpd_device_status()
-    peak = measure_tf32_matmul_peak(torch) / 3.0
-    flops = 2.0 * P * (N // c4.m) * (N // c4.n) * B            # FP32-equivalent flops of one product
-    useful = 3 * 2.0 * N * N * B
+    outcomes = [int(r.outcome) for r in g.read_results(res)[:2]]
+    if f32:
+        peak = measure_tf32_matmul_peak(torch) / 3.0
+        kernel = "sgemm_3xtf32_kernel (forward products)"
+        src = "measured here: torch.matmul TF32 8192^3 best of 10, divided by 3 (3xTF32)"
+        dtype = "f32 (3xTF32 products, FP64 encode/locate/decode arithmetic)"
+    else:
+        peak = measure_fp64_matmul_peak(torch)
+        kernel = "dgemm_mma_kernel (forward products)"
+        src = "measured here: torch.matmul FP64 8192^3, best of 10 (cuBLAS)"
+        dtype = "f64"
+    flops = 2.0 * P * (N1 // m) * (N0 // n) * B               # flops of one product over all nodes
+    useful = 3 * 2.0 * N1 * N0 * B
     line = {"metric": METRIC, "value": useful / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32 (3xTF32 products, FP64 encode/locate/decode arithmetic)",
-            "data": "synthetic",
-            "config": {"workload": "cfg4_mlp_hidden_layer_4096x4096_b256", "split": [c4.m, c4.n, 1, 1], "nodes": P,
-                       "step": "coded forward + backward + update of one layer", "l2": "shares 168 MB > L2"},
-            "kernel_ms": kern, "device_status": status,
-            "roofline": {"bound": "tensor", "kernel": "sgemm_3xtf32_kernel (forward products)",
+            "vs_baseline": None, "dtype": dtype, "data": "synthetic",
+            "config": {"workload": wname, "split": [m, n, 1, 1], "nodes": P,
+                       "thresholds": [plan.query(g.GPD_Q_THRESHOLD_FWD), plan.query(g.GPD_Q_THRESHOLD_BWD)],
+                       "step": "coded forward + backward + update of one layer",
+                       "l2": f"shares {plan.query(g.GPD_Q_W_SHARE_ELEMS) * plan.query(g.GPD_Q_ELEMENT_SIZE) / 1e6:.0f} MB > L2"},
+            "kernel_ms": kern, "device_status": status, "last_outcomes_fwd_bwd": outcomes,
+            "roofline": {"bound": "tensor", "kernel": kernel,
                          "achieved": flops / (kern["forward"] * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
                          "frac": flops / (kern["forward"] * 1e-3) / 1e12 / peak, "traffic": None,
-                         "peak_source": "measured here: torch.matmul TF32 8192^3 best of 10, divided by 3 (3xTF32)"}}
+                         "peak_source": src}}
     print(json.dumps(line))
 
 
@@ -652,12 +673,13 @@ def main():
     ap.add_argument("--precision", default="sliced", choices=["sliced", "sliced40", "fp64"],
                     help="worker products of the matmul workload: six (default) or five int8 digit planes on tcgen05, "
                          "or FP64 mma")
-    ap.add_argument("--workload", default="matmul", choices=["matmul", "mlp_layer", "positions"],
-                    help="matmul: the headline 8192 x 8192 x 512 coded product; mlp_layer: secondary, FP32 path; "
-                         "positions: secondary, per-position correction of the same product's outputs")
+    ap.add_argument("--workload", default="matmul", choices=["matmul", "mlp_layer", "sae_layer", "positions"],
+                    help="matmul: the headline 8192 x 8192 x 512 coded product; mlp_layer / sae_layer: secondary, coded "
+                         "training step of one MLP layer (FP32 path) / of the autoencoder's encoder (FP64 path); "
+                         "positions: secondary, per-position correction of the headline product's outputs")
     args = ap.parse_args()
-    if args.workload == "mlp_layer" and args.impl == "ours":
-        run_mlp_layer(args)
+    if args.workload in ("mlp_layer", "sae_layer") and args.impl == "ours":
+        run_layer(args, args.workload)
         return
     if args.workload == "positions" and args.impl == "ours":
         run_positions(args)
