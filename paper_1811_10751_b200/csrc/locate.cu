@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(kThreads) syndrome_gram_kernel(SyndromeParams 
 #pragma unroll
                 for (int a = 0; a < NT; ++a)
 #pragma unroll
-                    for (int b = 0; b < NT; ++b) dmma_m8n8k4(acc[a][b][0], acc[a][b][1], f[a], f[b]);
+                    for (int b = a; b < NT; ++b) dmma_m8n8k4(acc[a][b][0], acc[a][b][1], f[a], f[b]);   // upper triangle
             }
             __syncwarp();
         }
@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(kThreads) syndrome_gram_kernel(SyndromeParams 
 #pragma unroll
     for (int a = 0; a < NT; ++a)
 #pragma unroll
-        for (int b = 0; b < NT; ++b) {
+        for (int b = a; b < NT; ++b) {
             const int r = 8 * a + (lane >> 2), c = 8 * b + 2 * (lane & 3);
             if (acc[a][b][0] != 0.0) atomicAdd(&sG[r * RT + c], acc[a][b][0]);
             if (acc[a][b][1] != 0.0) atomicAdd(&sG[r * RT + c + 1], acc[a][b][1]);
@@ -405,6 +405,7 @@ template <typename T>
 gpd_status dispatch_syndrome(const SyndromeParams& prm, cudaStream_t st) {
     if (prm.R <= 8) return launch_syndrome<T, 8>(prm, st);
     if (prm.R <= 16) return launch_syndrome<T, 16>(prm, st);
+    if (prm.R <= 24) return launch_syndrome<T, 24>(prm, st);
     return launch_syndrome<T, 32>(prm, st);
 }
 
