@@ -87,7 +87,8 @@ typedef enum {
                                    products are exact int8 x int8 -> int32 tensor-core contractions of digit
                                    planes, recombined in FP64 (plane pairs below 2^-50 of row scale x column
                                    scale are not formed); worker outputs are double.  Needs N0/n divisible
-                                   by 16 and at most 16384, and finite inputs (a non-finite entry makes its
+                                   by 16 and at most 16384, 16-byte aligned W, X and share buffers
+                                   (GPD_ERR_ARG otherwise), and finite inputs (a non-finite entry makes its
                                    share row meaningless without being flagged).  Every other call that takes
                                    shares returns GPD_ERR_UNSUPPORTED; gpd_plan returns it when the shapes do
                                    not fit.  An implementation choice of this library: the paper prescribes

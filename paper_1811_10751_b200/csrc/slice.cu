@@ -290,6 +290,8 @@ SlicedLayout sliced_layout(int slices, int64_t P, int64_t rows, int64_t K) {
 }
 
 gpd_status encode_sliced_launch(gpd_plan_s* plan, bool is_A, const float* src, void* dst, cudaStream_t st) {
+    // 16-byte loads of the source rows, word stores into the planes, aligned exponent tables
+    if (reinterpret_cast<uintptr_t>(src) % 16 != 0 || reinterpret_cast<uintptr_t>(dst) % 16 != 0) return GPD_ERR_ARG;
     gpd_status rc = ensure_device(plan);
     if (rc != GPD_OK) return rc;
     const gpd_shape& s = plan->shape;

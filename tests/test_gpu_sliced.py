@@ -207,6 +207,11 @@ def test_sliced_refuses_calls_on_other_shares():
             cp.encode(operand, M)
         assert ei.value.status == g.GPD_ERR_UNSUPPORTED
     Xs = cp.encode(g.GPD_OPERAND_X_FWD, X)
+    # a source matrix that does not start on a 16-byte boundary is refused, not read with vector loads
+    skew = torch.empty(N1 * N0 + 1, dtype=torch.float32, device="cuda")[1:].view(N1, N0)
+    with pytest.raises(g.GpdError) as ei:
+        g.gpd_encode_A(cp.plan, skew, cp.W_shares)
+    assert ei.value.status == g.GPD_ERR_ARG
     out = cp.plan.empty(g.GPD_Q_OUT_ELEMS_BWD)
     with pytest.raises(g.GpdError) as ei:
         g.gpd_worker_gemm(cp.plan, g.GPD_BWD, cp.W_shares, Xs, out)
