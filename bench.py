@@ -662,6 +662,17 @@ def run_positions(args):
     print(json.dumps(line))
 
 
+def ensure_library():
+    """Built artefacts are not tracked: on a clean checkout compile libgpd.so once (nvcc, sm_100a)."""
+    if os.path.exists(os.path.join(ROOT, "paper_1811_10751_b200", "libgpd.so")):
+        return
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("_gpd_build", os.path.join(ROOT, "paper_1811_10751_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.build(force=False)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -678,6 +689,15 @@ def main():
                          "training step of one MLP layer (FP32 path) / of the autoencoder's encoder (FP64 path); "
                          "positions: secondary, per-position correction of the headline product's outputs")
     args = ap.parse_args()
+    if args.impl == "ours":
+        if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+            ensure_library()
+        else:                                            # the other ranks of a node wait for rank 0's build
+            lib_path = os.path.join(ROOT, "paper_1811_10751_b200", "libgpd.so")
+            for _ in range(1200):
+                if os.path.exists(lib_path):
+                    break
+                time.sleep(0.5)
     if args.workload in ("mlp_layer", "sae_layer") and args.impl == "ours":
         run_layer(args, args.workload)
         return
