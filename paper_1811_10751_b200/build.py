@@ -65,7 +65,9 @@ def build(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
     with ThreadPoolExecutor(max_workers=min(8, max(1, len(jobs)))) as ex:
         list(ex.map(run, jobs))
     if jobs or force or not os.path.exists(LIB_PATH):
-        run([nvcc, "-shared", "-o", LIB_PATH, *objs, "-gencode", "arch=compute_100a,code=sm_100a"])
+        tmp = LIB_PATH + f".tmp{os.getpid()}"          # linked aside, then moved: readers never see half a file
+        run([nvcc, "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a"])
+        os.replace(tmp, LIB_PATH)
     return LIB_PATH
 
 
