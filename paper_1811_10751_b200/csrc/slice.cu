@@ -68,15 +68,17 @@ __device__ __forceinline__ void digits4(const double (&a)[4], double scale, unsi
         lo[v] = (unsigned int)__double2loint(t);
         hi[v] = (unsigned int)__double2hiint(t);
     }
+    // 4 x 4 byte transposes in two rounds of permutes: pairs of values first, then pairs of pairs
+    unsigned int byte_of[8];                                          // byte i of U for values 0..3
+    const unsigned int l01a = __byte_perm(lo[0], lo[1], 0x5140), l23a = __byte_perm(lo[2], lo[3], 0x5140);
+    const unsigned int l01b = __byte_perm(lo[0], lo[1], 0x7362), l23b = __byte_perm(lo[2], lo[3], 0x7362);
+    byte_of[0] = __byte_perm(l01a, l23a, 0x5410); byte_of[1] = __byte_perm(l01a, l23a, 0x7632);
+    byte_of[2] = __byte_perm(l01b, l23b, 0x5410); byte_of[3] = __byte_perm(l01b, l23b, 0x7632);
+    const unsigned int h01 = __byte_perm(hi[0], hi[1], 0x5140), h23 = __byte_perm(hi[2], hi[3], 0x5140);
+    byte_of[4] = __byte_perm(h01, h23, 0x5410); byte_of[5] = __byte_perm(h01, h23, 0x7632);
+    byte_of[6] = byte_of[7] = 0u;                                     // S <= 6
 #pragma unroll
-    for (int t = 0; t < S; ++t) {
-        const int byte = S - 1 - t;                                   // position of digit t in U
-        const unsigned int sel = byte < 4 ? (unsigned int)(((4 + byte) << 4) | byte)
-                                          : (unsigned int)(((4 + byte - 4) << 4) | (byte - 4));
-        const unsigned int p01 = byte < 4 ? __byte_perm(lo[0], lo[1], sel) : __byte_perm(hi[0], hi[1], sel);
-        const unsigned int p23 = byte < 4 ? __byte_perm(lo[2], lo[3], sel) : __byte_perm(hi[2], hi[3], sel);
-        word[t] = __byte_perm(p01, p23, 0x5410) ^ 0x80808080u;
-    }
+    for (int t = 0; t < S; ++t) word[t] = byte_of[S - 1 - t] ^ 0x80808080u;   // digit t sits in byte S-1-t
 }
 
 // ---- W side: operand rows are rows of the share (K = block columns, contiguous in the source) ----
@@ -156,6 +158,117 @@ __global__ void __launch_bounds__(256) rowslice_kernel(SliceParams prm) {
     }
 }
 
+// Both passes in one kernel, for share rows whose source values (NBLK block rows of bc floats) fit
+// in shared memory twice.  A persistent CTA walks share rows r; while it works on row r the source
+// values of its next row arrive through asynchronous 16-byte copies, so that no thread waits on
+// global memory inside the node loop and W is read from DRAM once.  Per row: block maxima from
+// shared memory -> the P exponents of the row (same bound as rowscale_kernel) -> digits.
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    const unsigned int s = (unsigned int)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;\n" ::: "memory"); }
+
+constexpr int kFusedMaxThreads = 512;
+// shared memory of the fused kernel: coefficients, per-node scales, block maxima (two sets), two row buffers
+inline size_t fused_smem_bytes(int P, int nblk, int64_t bc) {
+    const size_t head = (sizeof(double) * ((size_t)P * nblk + P) + sizeof(unsigned int) * 2 * nblk + 15) / 16 * 16;
+    return head + 2 * sizeof(float) * (size_t)nblk * (size_t)bc;
+}
+
+template <int NBLK, int S>
+__global__ void __launch_bounds__(kFusedMaxThreads, 1) rowslice_fused_kernel(SliceParams prm) {
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    const int P = prm.P, tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
+    double* s_cf = reinterpret_cast<double*>(s_raw);                       // [P][NBLK]
+    double* s_scale = s_cf + P * NBLK;                                     // [P]  2^(8S - e_p) of the current row
+    unsigned int* s_blk = reinterpret_cast<unsigned int*>(s_scale + P);    // [2][NBLK] largest |W_b[r][:]| as float bits
+    const int64_t bc = prm.bc;
+    const int bc4 = (int)(bc >> 2);
+    float* stage = reinterpret_cast<float*>(s_raw + (sizeof(double) * ((size_t)P * NBLK + P) +
+                                                     sizeof(unsigned int) * 2 * NBLK + 15) / 16 * 16);   // [2][NBLK][bc]
+    for (int i = tid; i < P * NBLK; i += nthr) s_cf[i] = prm.coef[i];
+    if (tid < 2 * NBLK) s_blk[tid] = 0u;
+
+    auto fetch = [&](int64_t r, int buf) {
+        float* d = stage + (size_t)buf * NBLK * bc;
+#pragma unroll
+        for (int b = 0; b < NBLK; ++b) {
+            const int gi = b / prm.gc, gj = b - gi * prm.gc;
+            const float* srow = prm.src + (gi * prm.br + r) * prm.ld + gj * bc;
+            for (int it = tid; it < bc4; it += nthr) cp_async16(d + b * bc + 4 * it, srow + 4 * it);
+        }
+    };
+    // 32-bit word offsets into the planes (the launcher checks that all S planes stay below 2^32 words)
+    unsigned int* planes_w = reinterpret_cast<unsigned int*>(prm.planes);
+    const unsigned int node_words = (unsigned int)((prm.br * bc) >> 2), plane_words = (unsigned int)P * node_words;
+    int64_t r = blockIdx.x;
+    if (r < prm.br) fetch(r, 0);
+    cp_async_commit();
+    for (int buf = 0; r < prm.br; r += gridDim.x, buf ^= 1) {
+        if (r + gridDim.x < prm.br) fetch(r + gridDim.x, buf ^ 1);
+        cp_async_commit();
+        cp_async_wait_all_but_one();                 // this thread's copies of row r have landed ...
+        __syncthreads();                             // ... and so have everyone else's
+        const float* xb = stage + (size_t)buf * NBLK * bc;
+        unsigned int* blk = s_blk + buf * NBLK;
+        {
+            unsigned int m[NBLK];
+#pragma unroll
+            for (int b = 0; b < NBLK; ++b) m[b] = 0u;
+            for (int it = tid; it < bc4; it += nthr) {
+#pragma unroll
+                for (int b = 0; b < NBLK; ++b) {
+                    const float4 v = *reinterpret_cast<const float4*>(xb + b * bc + 4 * it);
+                    m[b] = max(m[b], max(max(__float_as_uint(fabsf(v.x)), __float_as_uint(fabsf(v.y))),
+                                         max(__float_as_uint(fabsf(v.z)), __float_as_uint(fabsf(v.w)))));
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < NBLK; ++b) {         // every lane is here: the item loop has ended
+                const unsigned int w = __reduce_max_sync(0xffffffffu, m[b]);
+                if (lane == 0 && w) atomicMax(&blk[b], w);
+            }
+        }
+        __syncthreads();
+        for (int p = tid; p < P; p += nthr) {
+            double bound = 0.0;
+            for (int b = 0; b < NBLK; ++b) bound += fabs(s_cf[p * NBLK + b]) * (double)__uint_as_float(blk[b]);
+            const int e = slice_exponent(abs_hi(bound));
+            prm.expo[(int64_t)p * prm.br + r] = e;
+            s_scale[p] = slice_scale<S>(e);
+        }
+        __syncthreads();
+        if (tid < NBLK) blk[tid] = 0u;               // next read two rows from now, barriers in between
+        for (int it = tid; it < bc4; it += nthr) {
+            double x[NBLK][4];
+#pragma unroll
+            for (int b = 0; b < NBLK; ++b) {
+                const float4 v = *reinterpret_cast<const float4*>(xb + b * bc + 4 * it);
+                x[b][0] = v.x; x[b][1] = v.y; x[b][2] = v.z; x[b][3] = v.w;
+            }
+            unsigned int off = (unsigned int)((r * bc) >> 2) + (unsigned int)it;   // word offset inside plane 0, node 0
+#pragma unroll 2
+            for (int p = 0; p < P; ++p, off += node_words) {
+                const double* cf = s_cf + p * NBLK;
+                double a[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (int b = 0; b < NBLK; ++b) {
+                    const double k = cf[b];
+                    a[0] = fma(k, x[b][0], a[0]); a[1] = fma(k, x[b][1], a[1]);
+                    a[2] = fma(k, x[b][2], a[2]); a[3] = fma(k, x[b][3], a[3]);
+                }
+                unsigned int word[S];
+                digits4<S>(a, s_scale[p], word);
+#pragma unroll
+                for (int s = 0; s < S; ++s) __stcs(planes_w + (off + (unsigned int)s * plane_words), word[s]);
+            }
+        }
+        __syncthreads();                             // row buffer `buf` is refilled by the next trip's copies
+    }
+}
+
 // ---- X side: operand rows are columns of the share (K = block rows, strided in the source) ----
 // A CTA stages the source values of a tile (128 rows kk x 8 columns n of every block) in shared
 // memory, transposed, so that a thread owns 4 consecutive kk of one column (warp = column,
@@ -229,7 +342,29 @@ __global__ void __launch_bounds__(256) colpass_kernel(SliceParams prm) {
 }
 
 template <int NBLK>
+gpd_status launch_rows_fused(const SliceParams& prm, int slices, size_t smem, cudaStream_t st) {
+    // CTA size follows the row length (one thread per four columns, at most 512); shorter rows run
+    // more CTAs per SM on the same register and shared-memory budget
+    const int threads = (int)std::min<int64_t>(kFusedMaxThreads, ((prm.bc >> 2) + 31) / 32 * 32);
+    const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(kFusedMaxThreads / threads, (200 * 1024) / smem));
+    const int grid = (int)std::min<int64_t>(prm.br, (int64_t)148 * per_sm);
+    auto go = [&](auto kernel) -> gpd_status {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return GPD_ERR_CUDA;
+        kernel<<<grid, threads, smem, st>>>(prm);
+        return launch_ok();
+    };
+    return slices == 6 ? go(rowslice_fused_kernel<NBLK, 6>) : go(rowslice_fused_kernel<NBLK, 5>);
+}
+
+template <int NBLK>
 gpd_status launch_rows(const SliceParams& prm, int slices, cudaStream_t st) {
+    if constexpr (NBLK <= 8) {       // beyond eight blocks the fused kernel's source values spill
+        const size_t fused = fused_smem_bytes(prm.P, NBLK, prm.bc);
+        const bool small_offsets = (int64_t)kMaxSlices * prm.P * prm.br * prm.bc < (int64_t)4 << 32;
+        if (fused <= 200 * 1024 && small_offsets) return launch_rows_fused<NBLK>(prm, slices, fused, st);
+    }
+    // many blocks, or rows too long to stage: scale pass, then slice pass from global memory
     rowscale_kernel<NBLK><<<(unsigned)prm.br, 256, 0, st>>>(prm);
     if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
     const int64_t work = prm.br * (prm.bc / 4);

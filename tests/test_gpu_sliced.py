@@ -77,6 +77,7 @@ def _sliced_products(code, W, X, S=6):
     (1024, 2048, 128, 2, 2, 1, 9),      # K = 1024: sixteen k-blocks, ring wraps five times
     (512, 768, 96, 4, 4, 1, 40),        # 16 blocks per share of W, 40 nodes, threshold 19
     (256, 256, 96, 2, 4, 3, 30),        # 12 blocks per share of X, threshold 27
+    (128, 16384, 32, 2, 2, 1, 8),       # K = 8192: share rows too long for the encoder's shared-memory staging
 ])
 @pytest.mark.parametrize("S", [6, 5])
 def test_sliced_worker_products_match_oracle(N1, N0, B, m, n, d1, P, S):
