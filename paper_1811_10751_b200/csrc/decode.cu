@@ -176,63 +176,93 @@ template <> struct Vec<double> {
 };
 
 // NW wanted coefficients per pass over the inputs; VECTOR: 16-byte loads of N positions.
+// Shared memory: the columns of D of the nodes in use, compacted and transposed to [node][wanted]
+// (padded to a multiple of NW) so that a node's NW coefficients come with 16-byte loads, and the
+// nodes' element offsets into Z.
 template <typename T, int NW, bool VECTOR>
 __global__ void __launch_bounds__(256) decode_stream_kernel(StreamParams prm) {
     if (prm.gate[0] == 0) return;
-    extern __shared__ double sD[];                   // [n_wanted][P]
+    extern __shared__ __align__(16) double sD[];     // [n_used][WP]
+    __shared__ int64_t s_off[kMaxNodes];             // node * L for the nodes in use
     __shared__ int s_nodes[kMaxNodes];
     __shared__ int s_nused;
-    for (int i = threadIdx.x; i < prm.n_wanted * prm.P; i += blockDim.x) sD[i] = prm.D[i];
-    __syncthreads();
-    if (threadIdx.x == 0) {                          // nodes with an all-zero column are not read
+    const int64_t L = prm.br * prm.bc;
+    const int WP = (prm.n_wanted + NW - 1) / NW * NW;
+    if (threadIdx.x < 32) {                          // nodes with an all-zero column of D are not read
         int n = 0;
-        for (int p = 0; p < prm.P; ++p) {
+        for (int base = 0; base < prm.P; base += 32) {
+            const int p = base + (int)threadIdx.x;
             bool used = false;
-            for (int w = 0; w < prm.n_wanted; ++w) used |= sD[w * prm.P + p] != 0.0;
-            if (used) s_nodes[n++] = p;
+            if (p < prm.P)
+                for (int w = 0; w < prm.n_wanted; ++w) used |= prm.D[w * prm.P + p] != 0.0;
+            const unsigned int m = __ballot_sync(0xffffffffu, used);
+            if (used) {
+                const int slot = n + __popc(m & ((1u << threadIdx.x) - 1u));
+                s_nodes[slot] = p;
+                s_off[slot] = (int64_t)p * L;
+            }
+            n += __popc(m);
         }
-        s_nused = n;
+        if (threadIdx.x == 0) s_nused = n;
+    }
+    __syncthreads();
+    const int nused = s_nused;
+    for (int i = threadIdx.x; i < nused * WP; i += blockDim.x) {
+        const int node = i / WP, w = i - node * WP;
+        sD[i] = w < prm.n_wanted ? prm.D[w * prm.P + s_nodes[node]] : 0.0;
     }
     __syncthreads();
     constexpr int N = VECTOR ? Vec<T>::N : 1;
+    constexpr int U = 6;                             // nodes per trip, loads issued first
     const T* Z = reinterpret_cast<const T*>(prm.Z);
-    const int64_t L = prm.br * prm.bc;
     const int64_t groups = VECTOR ? L / N : L;
     for (int64_t gidx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; gidx < groups;
          gidx += (int64_t)gridDim.x * blockDim.x) {
         const int64_t pos = gidx * N;
         const int64_t row = pos / prm.bc, col = pos - row * prm.bc;
+        const T* zpos = Z + pos;
         for (int w0 = 0; w0 < prm.n_wanted; w0 += NW) {
             double acc[NW][N];
 #pragma unroll
             for (int w = 0; w < NW; ++w)
 #pragma unroll
                 for (int v = 0; v < N; ++v) acc[w][v] = 0.0;
-            constexpr int U = 6;                         // nodes per trip, loads issued first
-            for (int i0 = 0; i0 < s_nused; i0 += U) {
+            auto fetch = [&](int i, double (&z)[N]) {
+                if constexpr (VECTOR) Vec<T>::load(zpos + s_off[i], z);
+                else z[0] = (double)__ldcs(zpos + s_off[i]);
+            };
+            auto absorb = [&](int i, const double (&z)[N]) {
+                const double* d = sD + i * WP + w0;  // NW coefficients, 16-byte aligned (NW is even)
+#pragma unroll
+                for (int w = 0; w < NW; w += 2) {
+                    const double2 dv = *reinterpret_cast<const double2*>(d + w);
+#pragma unroll
+                    for (int v = 0; v < N; ++v) {
+                        acc[w][v] = fma(dv.x, z[v], acc[w][v]);
+                        acc[w + 1][v] = fma(dv.y, z[v], acc[w + 1][v]);
+                    }
+                }
+            };
+            int i0 = 0;
+            for (; i0 + U <= nused; i0 += U) {
                 double z[U][N];
-                int pn[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) fetch(i0 + u, z[u]);
+#pragma unroll
+                for (int u = 0; u < U; ++u) absorb(i0 + u, z[u]);
+            }
+            if (i0 < nused) {                        // the last n_used mod U nodes
+                double z[U][N];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const bool live = i0 + u < s_nused;
-                    pn[u] = s_nodes[live ? i0 + u : 0];
-                    if (live) {
-                        if constexpr (VECTOR) Vec<T>::load(Z + (int64_t)pn[u] * L + pos, z[u]);
-                        else z[u][0] = (double)__ldcs(Z + (int64_t)pn[u] * L + pos);
-                    } else {
+                    if (i0 + u < nused) fetch(i0 + u, z[u]);
+                    else
 #pragma unroll
                         for (int v = 0; v < N; ++v) z[u][v] = 0.0;
-                    }
                 }
 #pragma unroll
-                for (int u = 0; u < U; ++u) {
-#pragma unroll
-                    for (int w = 0; w < NW; ++w) {
-                        const double d = (w0 + w < prm.n_wanted) ? sD[(w0 + w) * prm.P + pn[u]] : 0.0;
-#pragma unroll
-                        for (int v = 0; v < N; ++v) acc[w][v] = fma(d, z[u][v], acc[w][v]);
-                    }
-                }
+                for (int u = 0; u < U; ++u)
+                    if (i0 + u < nused) absorb(i0 + u, z[u]);
             }
 #pragma unroll
             for (int w = 0; w < NW; ++w) {
@@ -267,7 +297,8 @@ void launch_stream(const StreamParams& prm, cudaStream_t st) {
     constexpr int N = VECTOR ? Vec<T>::N : 1;
     const int64_t groups = prm.br * prm.bc / N;
     const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((groups + 255) / 256, 148 * 4));
-    decode_stream_kernel<T, NW, VECTOR><<<grid, 256, sizeof(double) * prm.n_wanted * prm.P, st>>>(prm);
+    const int WP = (prm.n_wanted + NW - 1) / NW * NW;
+    decode_stream_kernel<T, NW, VECTOR><<<grid, 256, sizeof(double) * WP * prm.P, st>>>(prm);
 }
 
 template <typename T>

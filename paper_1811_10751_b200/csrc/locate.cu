@@ -39,13 +39,57 @@ __device__ __forceinline__ void dmma_m8n8k4(double& d0, double& d1, double a, do
                  : "d"(a), "d"(b));
 }
 
-// One thread per output position (codeword): P coalesced loads (issued eight at a time), the
-// syndrome in RT registers, the zero test.  The Gram matrix of the failing codewords is formed
+// Syndrome s = H z and squared norm of one codeword: P loads at stride L, issued eight at a time.
+// CHECKED = false is the plain form: no per-value tests, a non-finite value shows up as a non-finite
+// norm and the caller repeats the codeword with CHECKED = true, which zeroes non-finite values
+// and erased nodes and records the nodes that held a non-finite value.
+template <typename T, int RT, bool CHECKED>
+__device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P, const double* sH,
+                                                  unsigned long long erased, double (&s)[RT], double& nz,
+                                                  unsigned long long& bad) {
+    constexpr int U = 8;                                 // loads issued together: bytes in flight
+#pragma unroll
+    for (int r = 0; r < RT; ++r) s[r] = 0.0;
+    nz = 0.0;
+    auto absorb = [&](double zz, int pnode, const double* hcol) {
+        if (CHECKED) {
+            if (!isfinite(zz)) { bad |= 1ULL << pnode; zz = 0.0; }
+            if ((erased >> pnode) & 1ULL) zz = 0.0;
+        }
+        nz = fma(zz, zz, nz);
+        const double2* h = reinterpret_cast<const double2*>(hcol);
+#pragma unroll
+        for (int r = 0; r < RT / 2; ++r) {
+            const double2 hv = h[r];
+            s[2 * r] = fma(hv.x, zz, s[2 * r]);
+            s[2 * r + 1] = fma(hv.y, zz, s[2 * r + 1]);
+        }
+    };
+    int p0 = 0;
+    for (; p0 + U <= P; p0 += U, zp += U * L, sH += U * RT) {
+        double z[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) z[u] = (double)__ldcs(zp + u * L);
+#pragma unroll
+        for (int u = 0; u < U; ++u) absorb(z[u], p0 + u, sH + u * RT);
+    }
+    if (p0 < P) {                                        // the last P mod 8 nodes
+        double z[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) z[u] = (p0 + u < P) ? (double)__ldcs(zp + u * L) : 0.0;
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (p0 + u < P) absorb(z[u], p0 + u, sH + u * RT);
+    }
+}
+
+// One thread per output position (codeword): the syndrome in RT registers, the zero test.  The
+// Gram matrix of the failing codewords is formed
 // warp by warp on the FP64 tensor cores: the 32 scaled syndromes of a warp are staged in shared
 // memory and fed to mma.m8n8k4 as both operands (G += S S^T, four codewords per instruction), so
 // the accumulator costs two registers per 8 x 8 tile and the streaming loop needs no CTA barrier.
 template <typename T, int RT>
-__global__ void __launch_bounds__(kThreads) syndrome_gram_kernel(SyndromeParams prm) {
+__global__ void __launch_bounds__(kThreads, RT <= 8 ? 4 : 1) syndrome_gram_kernel(SyndromeParams prm) {
     constexpr int NT = RT / 8;                          // 8 x 8 tiles per side of the Gram matrix
     constexpr int LD = RT + 4;                          // row pitch of the staging buffer (bank spread)
     constexpr int kWarps = kThreads / 32;
@@ -74,35 +118,14 @@ __global__ void __launch_bounds__(kThreads) syndrome_gram_kernel(SyndromeParams 
     for (int64_t batch = blockIdx.x; batch < n_batches; batch += gridDim.x) {
         const int64_t l = batch * kThreads + threadIdx.x;
         double s[RT];
-#pragma unroll
-        for (int r = 0; r < RT; ++r) s[r] = 0.0;
         double nz = 0.0;
         if (l < prm.L) {
-            const T* zp = Z + l;
-            constexpr int U = 8;                         // loads issued together: bytes in flight
-            for (int p0 = 0; p0 < prm.P; p0 += U) {
-                double z[U];
+            if (prm.erased == 0ULL) codeword_syndrome<T, RT, false>(Z + l, prm.L, prm.P, sH, 0ULL, s, nz, bad_all);
+            if (prm.erased != 0ULL || !isfinite(nz))
+                codeword_syndrome<T, RT, true>(Z + l, prm.L, prm.P, sH, prm.erased, s, nz, bad_all);
+        } else {
 #pragma unroll
-                for (int u = 0; u < U; ++u)
-                    z[u] = (p0 + u < prm.P) ? (double)__ldcs(zp + (int64_t)(p0 + u) * prm.L) : 0.0;
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int pnode = p0 + u;
-                    if (pnode < prm.P) {
-                        double zz = z[u];
-                        if (!isfinite(zz)) { bad_all |= 1ULL << pnode; zz = 0.0; }
-                        if ((prm.erased >> pnode) & 1ULL) zz = 0.0;
-                        nz = fma(zz, zz, nz);
-                        const double2* h = reinterpret_cast<const double2*>(sH + pnode * RT);
-#pragma unroll
-                        for (int r = 0; r < RT / 2; ++r) {
-                            const double2 hv = h[r];
-                            s[2 * r] = fma(hv.x, zz, s[2 * r]);
-                            s[2 * r + 1] = fma(hv.y, zz, s[2 * r + 1]);
-                        }
-                    }
-                }
-            }
+            for (int r = 0; r < RT; ++r) s[r] = 0.0;
         }
         double ns = 0.0;
 #pragma unroll
