@@ -78,27 +78,36 @@ __global__ void __launch_bounds__(kMatrixThreads) decode_matrix_kernel(MatrixPar
         }
     }
     __syncthreads();
-    // Householder triangularisation
+    // Householder triangularisation.  Eight lanes share a column (column = k + tid / 8, rows strided
+    // by eight between them, partial sums met by three shuffles inside the group), so that a step
+    // costs rows / 8 dependent operations instead of rows.  Within a step column k is only read:
+    // its own group stores the unit reflector, and R's diagonal entry is put in after the barrier.
+    const int part = tid & 7, colg = tid >> 3;           // kMatrixThreads / 8 = 32 >= Q columns
     for (int k = 0; k < Q; ++k) {
-        double part = 0.0;
-        for (int r = k + lane; r < rows; r += 32) part += A[r][k] * A[r][k];
-        const double sigma = warp_sum(part);         // same value in every warp (same order of additions)
+        double sigma = 0.0;
+        for (int r = k + part; r < rows; r += 8) sigma += A[r][k] * A[r][k];
+        sigma += __shfl_xor_sync(0xffffffffu, sigma, 1);
+        sigma += __shfl_xor_sync(0xffffffffu, sigma, 2);
+        sigma += __shfl_xor_sync(0xffffffffu, sigma, 4);     // same value in every group (same order of additions)
         const double akk = A[k][k];
         const double alpha = akk >= 0.0 ? -sqrt(sigma) : sqrt(sigma);
-        const double vnorm = sqrt(fmax(sigma - 2.0 * alpha * akk + alpha * alpha, 1e-300));
-        for (int r = k + tid; r < rows; r += kMatrixThreads) Vh[r][k] = (A[r][k] - (r == k ? alpha : 0.0)) / vnorm;
-        __syncthreads();
-        if (tid < Q - k) {
-            const int c = k + tid;
-            double d0 = 0.0, d1 = 0.0;
-            int r = k;
-            for (; r + 1 < rows; r += 2) { d0 += Vh[r][k] * A[r][c]; d1 += Vh[r + 1][k] * A[r + 1][c]; }
-            if (r < rows) d0 += Vh[r][k] * A[r][c];
-            const double dot2 = 2.0 * (d0 + d1);
-            for (r = k; r < rows; ++r) A[r][c] -= dot2 * Vh[r][k];
+        const double inv_vnorm = rsqrt(fmax(sigma - 2.0 * alpha * akk + alpha * alpha, 1e-300));
+        const int c = k + colg;
+        if (colg == 0) {
+            for (int r = k + part; r < rows; r += 8) Vh[r][k] = (A[r][k] - (r == k ? alpha : 0.0)) * inv_vnorm;
+        } else if (c < Q) {
+            double dot = 0.0;
+            for (int r = k + part; r < rows; r += 8) dot += (A[r][k] - (r == k ? alpha : 0.0)) * A[r][c];
+            dot += __shfl_xor_sync(0xffu << (8 * (tid >> 3 & 3)), dot, 1);
+            dot += __shfl_xor_sync(0xffu << (8 * (tid >> 3 & 3)), dot, 2);
+            dot += __shfl_xor_sync(0xffu << (8 * (tid >> 3 & 3)), dot, 4);
+            const double f = 2.0 * dot * inv_vnorm * inv_vnorm;
+            for (int r = k + part; r < rows; r += 8) A[r][c] -= f * (A[r][k] - (r == k ? alpha : 0.0));
         }
         __syncthreads();
+        if (tid == 0) A[k][k] = alpha;               // R's diagonal; nothing below reads column k again
     }
+    __syncthreads();                                 // the last diagonal entry
     // row w of the pseudo-inverse: solve R^T y = e_w, then x = H_0 H_1 ... H_{Q-1} [y; 0]
     for (int wi = warp; wi < prm.n_wanted; wi += kMatrixThreads / 32) {
         const int w = prm.wanted[wi];
