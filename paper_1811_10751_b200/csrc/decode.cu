@@ -36,9 +36,9 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
-// One CTA of 8 warps.  Factorisation: every warp forms the column norm itself (lanes over rows),
-// thread c of the CTA then reflects column k + c.  Rows of the pseudo-inverse: one warp per wanted
-// coefficient, lanes over the entries of y (Q <= 32) and of x (rows <= 64, two per lane).
+// One CTA of 8 warps.  Factorisation: eight lanes per column (see the loop).  Rows of the
+// pseudo-inverse: one warp per wanted coefficient, lanes over the entries of y (Q <= 32) and of x
+// (rows <= 64, two per lane).
 __global__ void __launch_bounds__(kMatrixThreads) decode_matrix_kernel(MatrixParams prm) {
     __shared__ double A[kMaxNodes][kMaxQ + 1];       // Vandermonde rows of the nodes in use -> R
     __shared__ double Vh[kMaxNodes][kMaxQ + 1];      // Householder vectors (column k = reflector k)
@@ -46,20 +46,22 @@ __global__ void __launch_bounds__(kMatrixThreads) decode_matrix_kernel(MatrixPar
     __shared__ int s_rows;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int P = prm.P, Q = prm.Q;
-    if (tid == 0) {
+    if (tid < 32) {                                  // nodes in use, in increasing order (one warp, two ballots)
+        bool ok = prm.have_mask ? true : prm.result->outcome != GPD_DECODE_FAILURE;
         int rows = 0;
-        bool ok = true;
-        if (prm.have_mask) {
-            for (int p = 0; p < P; ++p)
-                if ((prm.use_mask >> p) & 1ULL) node_of[rows++] = p;
-        } else {
-            ok = prm.result->outcome != GPD_DECODE_FAILURE;
-            for (int p = 0; p < P; ++p)
-                if (!prm.result->flagged[p]) node_of[rows++] = p;
+        for (int base = 0; base < P; base += 32) {
+            const int p = base + tid;
+            bool use = false;
+            if (p < P) use = prm.have_mask ? ((prm.use_mask >> p) & 1ULL) != 0ULL : prm.result->flagged[p] == 0;
+            const unsigned int m = __ballot_sync(0xffffffffu, use);
+            if (use) node_of[rows + __popc(m & ((1u << tid) - 1u))] = p;
+            rows += __popc(m);
         }
         if (rows < Q) ok = false;                    // fewer clean nodes than the threshold
-        s_rows = ok ? rows : 0;
-        prm.gate[0] = ok ? 1 : 0;
+        if (tid == 0) {
+            s_rows = ok ? rows : 0;
+            prm.gate[0] = ok ? 1 : 0;
+        }
     }
     __syncthreads();
     const int rows = s_rows;
@@ -112,10 +114,10 @@ __global__ void __launch_bounds__(kMatrixThreads) decode_matrix_kernel(MatrixPar
     for (int wi = warp; wi < prm.n_wanted; wi += kMatrixThreads / 32) {
         const int w = prm.wanted[wi];
         double y = 0.0;                              // lane i keeps y_i
+        const double rdiag = lane < Q ? 1.0 / A[lane][lane] : 0.0;
         for (int i = w; i < Q; ++i) {                // y_i = 0 for i < w
             const double s = warp_sum(lane < i ? A[lane][i] * y : 0.0);
-            const double yi = ((i == w ? 1.0 : 0.0) - s) / A[i][i];
-            if (lane == i) y = yi;
+            if (lane == i) y = ((i == w ? 1.0 : 0.0) - s) * rdiag;
         }
         double x0 = lane < Q ? y : 0.0, x1 = 0.0;    // x[lane], x[lane + 32]
         const bool in0 = lane < rows, in1 = lane + 32 < rows;

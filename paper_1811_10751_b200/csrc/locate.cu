@@ -195,8 +195,8 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     __shared__ double Qa[kMaxR][kMaxR + 1];
     __shared__ double Hs[kMaxR][kMaxNodes];
     __shared__ double lam[kMaxR];
-    __shared__ double rot_c[kMaxR / 2 + 1], rot_s[kMaxR / 2 + 1];
-    __shared__ int rot_p[kMaxR / 2 + 1], rot_q[kMaxR / 2 + 1];
+    __shared__ double rot_c[kMaxR + 1], rot_s[kMaxR + 1];        // per index: row_i <- c row_i + s row_partner
+    __shared__ int partner[kMaxR + 1], pair_p[kMaxR / 2 + 1], pair_q[kMaxR / 2 + 1];
     __shared__ int order[kMaxR];
     __shared__ unsigned char inside[kMaxNodes];
     __shared__ double dist[kMaxNodes];
@@ -238,6 +238,7 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     }
     __syncwarp();
 
+    double (*Ga)[kMaxR + 1] = G, (*Gb)[kMaxR + 1] = Qa;          // current / next Gram matrix of the Jacobi rounds
     int rank = 0;
     unsigned long long flagged = forced;
     double max_in = 0.0, min_out = 1e300;
@@ -247,13 +248,15 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
         for (int i = 0; i < R; ++i) tr += G[i][i];
         // Rotations of one round act on disjoint index pairs (round-robin pairing of n = R or R + 1
         // indices: n - 1 rounds of n / 2 pairs), so their angles are found side by side (lane = pair)
-        // and applied together: columns of G and V first, then rows of G.
+        // and applied together: every index i gets its partner and the pair (c_i, s_i) with
+        // new row_i = c_i row_i + s_i row_partner, and G' = J^T G J is written entry by entry into
+        // the other of two buffers (Qa is free until the verification), V column pair by column pair.
         const int n = (R + 1) & ~1, half = n >> 1;
         for (int sweep = 0; sweep < 40; ++sweep) {
             double off = 0.0;
             for (int i = lane; i < R * R; i += 32) {
                 const int r = i / R, c = i % R;
-                if (r != c) off += G[r][c] * G[r][c];
+                if (r != c) off += Ga[r][c] * Ga[r][c];
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
@@ -265,48 +268,42 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
                     const int p = min(a, b), q = max(a, b);
                     double c = 1.0, sn = 0.0;
                     if (q < R) {
-                        const double gpq = G[p][q], gpp = G[p][p], gqq = G[q][q];
+                        const double gpq = Ga[p][q], gpp = Ga[p][p], gqq = Ga[q][q];
                         if (!(fabs(gpq) <= 1e-300 || fabs(gpq) <= 1e-20 * sqrt(fabs(gpp * gqq)))) {
-                            const double th = (gqq - gpp) / (2.0 * gpq);
-                            const double t = (th >= 0.0 ? 1.0 : -1.0) / (fabs(th) + sqrt(th * th + 1.0));
-                            c = 1.0 / sqrt(t * t + 1.0);
+                            // t = tan of the rotation angle, the root of smaller magnitude
+                            const double d = gqq - gpp, o2 = 2.0 * gpq;
+                            const double t = o2 / (d + copysign(sqrt(d * d + o2 * o2), d));
+                            c = rsqrt(t * t + 1.0);
                             sn = t * c;
                         }
+                        rot_c[q] = c; rot_s[q] = sn; partner[q] = p;
                     }
-                    rot_c[lane] = c; rot_s[lane] = sn; rot_p[lane] = p; rot_q[lane] = q;
+                    rot_c[p] = c; rot_s[p] = -sn; partner[p] = q < R ? q : p;
+                    pair_p[lane] = p; pair_q[lane] = q;
                 }
                 __syncwarp();
-                for (int it = lane; it < half * R; it += 32) {      // G <- G J, V <- V J (columns p, q)
-                    const int t = it / R, i = it - t * R, p = rot_p[t], q = rot_q[t];
-                    if (q >= R || rot_s[t] == 0.0) continue;
-                    const double c = rot_c[t], sn = rot_s[t];
-                    const double a = G[i][p], b = G[i][q];
-                    G[i][p] = c * a - sn * b;
-                    G[i][q] = sn * a + c * b;
+                for (int e = lane; e < R * R; e += 32) {           // G' = J^T G J
+                    const int i = e / R, jj = e - i * R, ip = partner[i], jp = partner[jj];
+                    const double ci = rot_c[i], si = rot_s[i], cj = rot_c[jj], sj = rot_s[jj];
+                    const double t0 = ci * Ga[i][jj] + si * Ga[ip][jj];
+                    const double t1 = ci * Ga[i][jp] + si * Ga[ip][jp];
+                    Gb[i][jj] = (jj == ip && si != 0.0) ? 0.0 : cj * t0 + sj * t1;   // the rotated pair's entry is zero by construction
+                }
+                for (int it = lane; it < half * R; it += 32) {      // V <- V J (columns p, q)
+                    const int t = it / R, i = it - t * R, p = pair_p[t], q = pair_q[t];
+                    if (q >= R || rot_s[q] == 0.0) continue;
+                    const double c = rot_c[q], sn = rot_s[q];
                     const double va = V[i][p], vb = V[i][q];
                     V[i][p] = c * va - sn * vb;
                     V[i][q] = sn * va + c * vb;
                 }
                 __syncwarp();
-                for (int it = lane; it < half * R; it += 32) {      // G <- J^T G (rows p, q)
-                    const int t = it / R, j = it - t * R, p = rot_p[t], q = rot_q[t];
-                    if (q >= R || rot_s[t] == 0.0) continue;
-                    const double c = rot_c[t], sn = rot_s[t];
-                    const double a = G[p][j], b = G[q][j];
-                    G[p][j] = c * a - sn * b;
-                    G[q][j] = sn * a + c * b;
-                }
-                __syncwarp();
-                if (lane < half && rot_q[lane] < R && rot_s[lane] != 0.0) {
-                    G[rot_p[lane]][rot_q[lane]] = 0.0;
-                    G[rot_q[lane]][rot_p[lane]] = 0.0;
-                }
-                __syncwarp();
+                double (*tmp)[kMaxR + 1] = Ga; Ga = Gb; Gb = tmp;
             }
         }
         // ---- eigenvalues in descending order ---------------------------------------------
         if (lane == 0) {
-            for (int i = 0; i < R; ++i) { lam[i] = G[i][i]; order[i] = i; }
+            for (int i = 0; i < R; ++i) { lam[i] = Ga[i][i]; order[i] = i; }
             for (int i = 1; i < R; ++i) {                    // insertion sort, R <= 32
                 const int oi = order[i];
                 int j = i - 1;
@@ -343,9 +340,20 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
         }
         __syncwarp();
         int n_inside = 0;
-        for (int p = 0; p < P; ++p) {
-            if (inside[p]) { ++n_inside; flagged |= 1ULL << p; max_in = fmax(max_in, dist[p]); }
-            else min_out = fmin(min_out, dist[p]);
+        for (int base = 0; base < P; base += 32) {       // lanes over nodes: support mask and the two extremes
+            const int p = base + lane;
+            const bool in = p < P && inside[p];
+            const unsigned int m = __ballot_sync(0xffffffffu, in);
+            n_inside += __popc(m);
+            flagged |= (unsigned long long)m << base;
+            double mi = in ? dist[p] : 0.0, mo = (p < P && !in) ? dist[p] : 1e300;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                mi = fmax(mi, __shfl_xor_sync(0xffffffffu, mi, o));
+                mo = fmin(mo, __shfl_xor_sync(0xffffffffu, mo, o));
+            }
+            max_in = fmax(max_in, mi);
+            min_out = fmin(min_out, mo);
         }
         if (lane == 0) { res->max_inside = max_in; res->min_outside = min_out; }
         if (n_inside != rank) {
@@ -383,22 +391,22 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     }
     double residual = 0.0;
     if (n_active > 0ULL) {
-        // tr((I-Pi) G (I-Pi)) = sum_i lambda_i ||(I-Pi) u_i||^2, every term non-negative
-        for (int i = 0; i < R; ++i) {
-            double u = lane < R ? V[lane][i] : 0.0;
+        // tr((I-Pi) G (I-Pi)) = sum_i lambda_i ||(I-Pi) u_i||^2, every term non-negative.
+        // Lane i projects eigenvector i (column i of V, in place: V is not needed afterwards).
+        if (lane < R) {
             for (int pass = 0; pass < 2; ++pass) {
                 for (int e = 0; e < na; ++e) {
-                    double part = lane < R ? Qa[lane][e] * u : 0.0;
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-                    if (lane < R) u -= part * Qa[lane][e];
+                    double dot = 0.0;
+                    for (int r = 0; r < R; ++r) dot += Qa[r][e] * V[r][lane];
+                    for (int r = 0; r < R; ++r) V[r][lane] -= dot * Qa[r][e];
                 }
             }
-            double un = u * u;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) un += __shfl_xor_sync(0xffffffffu, un, o);
-            residual += fmax(G[i][i], 0.0) * un;
+            double un = 0.0;
+            for (int r = 0; r < R; ++r) un += V[r][lane] * V[r][lane];
+            residual = fmax(lam[lane], 0.0) * un;
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) residual += __shfl_xor_sync(0xffffffffu, residual, o);
     }
     const double limit = prm.tau2 * (double)(n_active > 0ULL ? n_active : 1ULL);
     if (lane == 0) {
