@@ -252,6 +252,7 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
         // new row_i = c_i row_i + s_i row_partner, and G' = J^T G J is written entry by entry into
         // the other of two buffers (Qa is free until the verification), V column pair by column pair.
         const int n = (R + 1) & ~1, half = n >> 1;
+        const int lane_i = lane / R, lane_j = lane % R, step_i = 32 / R, step_j = 32 % R;   // entry e = lane + 32 k is (i, j)
         for (int sweep = 0; sweep < 40; ++sweep) {
             double off = 0.0;
             for (int i = lane; i < R * R; i += 32) {
@@ -270,11 +271,14 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
                     if (q < R) {
                         const double gpq = Ga[p][q], gpp = Ga[p][p], gqq = Ga[q][q];
                         if (!(fabs(gpq) <= 1e-300 || fabs(gpq) <= 1e-20 * sqrt(fabs(gpp * gqq)))) {
-                            // t = tan of the rotation angle, the root of smaller magnitude
-                            const double d = gqq - gpp, o2 = 2.0 * gpq;
-                            const double t = o2 / (d + copysign(sqrt(d * d + o2 * o2), d));
-                            c = rsqrt(t * t + 1.0);
-                            sn = t * c;
+                            // tan of the rotation angle (the root of smaller magnitude) is o2 / den with
+                            // den = d + sign(d) hypot(d, o2); cosine and sine follow from (den, o2)
+                            // normalised, which takes two reciprocal square roots and no division
+                            const double d = gqq - gpp, o2 = 2.0 * gpq, h2 = d * d + o2 * o2;
+                            const double den = d + copysign(h2 * rsqrt(h2), d);
+                            const double rn = rsqrt(den * den + o2 * o2);
+                            c = fabs(den) * rn;
+                            sn = copysign(o2, o2 * den) * rn;
                         }
                         rot_c[q] = c; rot_s[q] = sn; partner[q] = p;
                     }
@@ -282,8 +286,9 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
                     pair_p[lane] = p; pair_q[lane] = q;
                 }
                 __syncwarp();
-                for (int e = lane; e < R * R; e += 32) {           // G' = J^T G J
-                    const int i = e / R, jj = e - i * R, ip = partner[i], jp = partner[jj];
+                for (int e = lane, i = lane_i, jj = lane_j; e < R * R; e += 32, i += step_i, jj += step_j) {   // G' = J^T G J
+                    if (jj >= R) { jj -= R; ++i; }
+                    const int ip = partner[i], jp = partner[jj];
                     const double ci = rot_c[i], si = rot_s[i], cj = rot_c[jj], sj = rot_s[jj];
                     const double t0 = ci * Ga[i][jj] + si * Ga[ip][jj];
                     const double t1 = ci * Ga[i][jp] + si * Ga[ip][jp];
