@@ -253,8 +253,8 @@ def run_ours(args, cfg):
     exec_flops = 2.0 * cfg.P * (cfg.N1 // cfg.m) * (cfg.N0 // cfg.n) * (cfg.B // cfg.d)
     useful_flops = 2.0 * cfg.N1 * cfg.N0 * cfg.B
     # encode W, encode X, products, inject, syndrome, locate finish, decode matrix, decode stream;
-    # the digit-plane encoders take two kernels each (scales, then digits)
-    KERNELS_PER_STEP = 10 if sliced else 8
+    # the digit-plane encoder of X takes two kernels (scales, then digits), the one of W is fused
+    KERNELS_PER_STEP = 9 if sliced else 8
 
     def step(i, gemm_events=None, stage_events=None, Wd=Wd, Xd=Xd):
         def mark(name):
