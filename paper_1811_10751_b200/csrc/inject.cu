@@ -6,6 +6,8 @@
 //   mix64(z) = output function applied to z + GAMMA;  draw(key, ctr) = mix64(key + ctr*GAMMA);
 //   key(seed, tag, p) = mix64(mix64(seed ^ tag*TAGMUL) + p),
 // so every entry's error is a pure function of (seed, node, entry).
+#include <cmath>
+
 #include "gpd_internal.h"
 
 namespace gpd {
@@ -55,20 +57,40 @@ __host__ __device__ __forceinline__ bool node_selected(const InjectParams& prm, 
 
 __global__ void write_mask_kernel(unsigned long long* dst, unsigned long long value) { *dst = value; }
 
+// Per-node constants of the additive mode, evaluated on the host with the same generator.
+struct AdditiveNode {
+    unsigned long long phi_cut;   // entry l is hit when (draw(k_entry, l) >> 11) < phi_cut, i.e. unit(draw) < phi
+    unsigned long long first;     // the one entry that is always hit
+    unsigned long long k_entry, k_mag;
+};
+struct AdditiveParams {
+    AdditiveNode node[kMaxNodes];
+    unsigned char sel[kMaxNodes];
+    void* out;
+    int64_t L;
+    double scale;
+};
+
+inline AdditiveNode additive_node(unsigned long long seed, int p, int64_t L) {
+    AdditiveNode a;
+    const double phi = 1.0 - unit(draw(make_key(seed, TAG_PHI, 0), (unsigned long long)p));
+    // unit(r) < phi  <=>  (r >> 11) < ceil(phi 2^53): integers below 2^53 on both sides
+    a.phi_cut = (unsigned long long)std::ceil(phi * 9007199254740992.0);
+    a.first = draw(make_key(seed, TAG_FIRST, 0), (unsigned long long)p) % (unsigned long long)L;
+    a.k_entry = make_key(seed, TAG_ENTRY, (unsigned long long)p);
+    a.k_mag = make_key(seed, TAG_MAG, (unsigned long long)p);
+    return a;
+}
+
 template <typename T>
-__global__ void __launch_bounds__(256) inject_additive_kernel(InjectParams prm) {
-    const int p = prm.sel[blockIdx.y];
-    const double phi = 1.0 - unit(draw(make_key(prm.seed, TAG_PHI, 0), (unsigned long long)p));
-    const unsigned long long first = draw(make_key(prm.seed, TAG_FIRST, 0), (unsigned long long)p) %
-                                     (unsigned long long)prm.L;
-    const unsigned long long k_entry = make_key(prm.seed, TAG_ENTRY, (unsigned long long)p);
-    const unsigned long long k_mag = make_key(prm.seed, TAG_MAG, (unsigned long long)p);
-    T* out = reinterpret_cast<T*>(prm.out) + (int64_t)p * prm.L;
+__global__ void __launch_bounds__(256) inject_additive_kernel(const __grid_constant__ AdditiveParams prm) {
+    const AdditiveNode& nd = prm.node[blockIdx.y];
+    T* out = reinterpret_cast<T*>(prm.out) + (int64_t)prm.sel[blockIdx.y] * prm.L;
     for (int64_t l = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; l < prm.L;
          l += (int64_t)gridDim.x * blockDim.x) {
-        const bool hit = ((unsigned long long)l == first) || (unit(draw(k_entry, (unsigned long long)l)) < phi);
+        const bool hit = ((unsigned long long)l == nd.first) || ((draw(nd.k_entry, (unsigned long long)l) >> 11) < nd.phi_cut);
         if (!hit) continue;
-        const unsigned long long r = draw(k_mag, (unsigned long long)l);
+        const unsigned long long r = draw(nd.k_mag, (unsigned long long)l);
         const int k = -4 + (int)((r >> 53) % 12ULL);
         const double f = (double)(r & ((1ULL << 52) - 1ULL)) * (1.0 / 4503599627370496.0);   // 2^-52
         double mag = ldexp(1.0 + f, k) * prm.scale;
@@ -162,10 +184,17 @@ gpd_status inject_launch(gpd_plan_s* plan, gpd_product which, void* outputs, uin
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
     }
     if (prm.n_sel == 0) return GPD_OK;
-    dim3 grid((unsigned)std::min<int64_t>((prm.L + 1023) / 1024, 1024), (unsigned)prm.n_sel);
+    // one entry per thread up to 8192 CTAs per node: a single round trip to memory for most threads
+    dim3 grid((unsigned)std::min<int64_t>((prm.L + 255) / 256, 8192), (unsigned)prm.n_sel);
     if (mode == GPD_INJECT_ADDITIVE) {
-        if (f32) inject_additive_kernel<float><<<grid, 256, 0, st>>>(prm);
-        else inject_additive_kernel<double><<<grid, 256, 0, st>>>(prm);
+        AdditiveParams ap{};
+        for (int i = 0; i < prm.n_sel; ++i) {
+            ap.sel[i] = prm.sel[i];
+            ap.node[i] = additive_node(prm.seed, prm.sel[i], prm.L);
+        }
+        ap.out = prm.out; ap.L = prm.L; ap.scale = prm.scale;
+        if (f32) inject_additive_kernel<float><<<grid, 256, 0, st>>>(ap);
+        else inject_additive_kernel<double><<<grid, 256, 0, st>>>(ap);
     } else if (mode == GPD_INJECT_GAUSS) {
         if (f32) inject_gauss_kernel<float><<<grid, 256, 0, st>>>(prm);
         else inject_gauss_kernel<double><<<grid, 256, 0, st>>>(prm);

@@ -47,7 +47,7 @@ template <typename T, int RT, bool CHECKED>
 __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P, const double* sH,
                                                   unsigned long long erased, double (&s)[RT], double& nz,
                                                   unsigned long long& bad) {
-    constexpr int U = 8;                                 // loads issued together: bytes in flight
+    constexpr int U = RT <= 8 ? 8 : 4;                   // loads issued together (fewer where the syndrome fills the registers)
 #pragma unroll
     for (int r = 0; r < RT; ++r) s[r] = 0.0;
     nz = 0.0;
@@ -73,7 +73,7 @@ __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P,
 #pragma unroll
         for (int u = 0; u < U; ++u) absorb(z[u], p0 + u, sH + u * RT);
     }
-    if (p0 < P) {                                        // the last P mod 8 nodes
+    if (p0 < P) {                                        // the last P mod U nodes
         double z[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) z[u] = (p0 + u < P) ? (double)__ldcs(zp + u * L) : 0.0;
@@ -89,7 +89,7 @@ __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P,
 // memory and fed to mma.m8n8k4 as both operands (G += S S^T, four codewords per instruction), so
 // the accumulator costs two registers per 8 x 8 tile and the streaming loop needs no CTA barrier.
 template <typename T, int RT>
-__global__ void __launch_bounds__(kThreads, RT <= 8 ? 4 : 1) syndrome_gram_kernel(SyndromeParams prm) {
+__global__ void __launch_bounds__(kThreads, RT <= 8 ? 4 : (RT <= 24 ? 2 : 1)) syndrome_gram_kernel(SyndromeParams prm) {
     constexpr int NT = RT / 8;                          // 8 x 8 tiles per side of the Gram matrix
     constexpr int LD = RT + 4;                          // row pitch of the staging buffer (bank spread)
     constexpr int kWarps = kThreads / 32;
