@@ -8,7 +8,8 @@
 // CTA through a shared-memory SYRK and added to global memory with one atomic per entry.
 // Non-finite values and erased nodes count as zero and their node is flagged up front.
 //
-// Pass 2 (one warp): eigen-decomposition of G by cyclic Jacobi; numerical rank rho; the error
+// Pass 2 (one warp): eigen-decomposition of G (pivoted Cholesky down to its numerical rank, then
+// cyclic Jacobi on the small matrix L^T L); numerical rank rho; the error
 // support is the set of nodes whose parity-check column H_p lies in the span of the top-rho
 // eigenvectors (any P-Q columns of H are independent, so for at most P-Q-1 erroneous nodes no
 // other column does); the support is verified by the syndrome energy left outside span(H_A).
@@ -188,20 +189,38 @@ struct FinishParams {
     unsigned long long erased;
 };
 
-// One warp.  Shared: G[R][R], V[R][R] (eigenvectors in columns), Hs[R][P], Qa[R][R], lam[R].
+// Shared memory of the finish kernel for R parity checks and P nodes (doubles first, then ints, bytes).
+__host__ __device__ inline size_t finish_smem_bytes(int R, int P) {
+    const int ld = R | 1;
+    return sizeof(double) * ((size_t)5 * R * ld + (size_t)R * P + (size_t)R + 2 * (size_t)(R + 1) + (size_t)P) +
+           sizeof(int) * ((size_t)(R + 1) + 2 * (size_t)(R / 2 + 1) + (size_t)R) + (size_t)P;
+}
+
+// One warp.  The Gram matrix G of the failing codewords has rank = number of erroneous nodes (a
+// few) plus a noise floor far below the threshold, so its eigen-decomposition is done on a small
+// matrix: a diagonally pivoted Cholesky factorisation G = L L^T + (remainder below 2^-30 of the
+// eigenvalue threshold) gives k columns, the k x k matrix L^T L has the eigenvalues of L L^T, and
+// cyclic Jacobi runs on that.  The retained subspace is L w_i / sqrt(lambda_i) for the eigenpairs
+// above the threshold; the verification uses ||(I - Pi) L||_F^2 = tr((I - Pi) L L^T (I - Pi)).
 __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
-    __shared__ double G[kMaxR][kMaxR + 1];
-    __shared__ double V[kMaxR][kMaxR + 1];
-    __shared__ double Qa[kMaxR][kMaxR + 1];
-    __shared__ double Hs[kMaxR][kMaxNodes];
-    __shared__ double lam[kMaxR];
-    __shared__ double rot_c[kMaxR + 1], rot_s[kMaxR + 1];        // per index: row_i <- c row_i + s row_partner
-    __shared__ int partner[kMaxR + 1], pair_p[kMaxR / 2 + 1], pair_q[kMaxR / 2 + 1];
-    __shared__ int order[kMaxR];
-    __shared__ unsigned char inside[kMaxNodes];
-    __shared__ double dist[kMaxNodes];
+    extern __shared__ __align__(16) double fs[];
     const int lane = threadIdx.x;
-    const int R = prm.R, P = prm.P;
+    const int R = prm.R, P = prm.P, ld = R | 1;
+    double* A = fs;                          // [R][ld] G -> Schur complement; then the second Jacobi buffer
+    double* Lm = A + R * ld;                 // [R][ld] Cholesky columns
+    double* M = Lm + R * ld;                 // [R][ld] L^T L; after the eigen-decomposition: basis of span(H_A)
+    double* Wv = M + R * ld;                 // [R][ld] eigenvectors of L^T L in columns
+    double* U = Wv + R * ld;                 // [R][ld] orthonormal basis of the retained subspace in columns
+    double* Hs = U + R * ld;                 // [R][P]
+    double* lam = Hs + R * P;                // [R]
+    double* rot_c = lam + R;                 // [R + 1] per index: row_i <- c row_i + s row_partner
+    double* rot_s = rot_c + (R + 1);         // [R + 1]
+    double* dist = rot_s + (R + 1);          // [P]
+    int* partner = reinterpret_cast<int*>(dist + P);   // [R + 1]
+    int* pair_p = partner + (R + 1);         // [R / 2 + 1]
+    int* pair_q = pair_p + (R / 2 + 1);      // [R / 2 + 1]
+    int* order = pair_q + (R / 2 + 1);       // [R]
+    unsigned char* inside = reinterpret_cast<unsigned char*>(order + R);   // [P]
     gpd_locate_result* res = prm.result;
     const unsigned long long n_active = prm.counts[0];
     const unsigned long long forced = prm.counts[1] | prm.erased;
@@ -230,86 +249,134 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
         if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
         return;
     }
-    for (int i = lane; i < R * P; i += 32) Hs[i / P][i % P] = prm.H[i];
+    for (int i = lane; i < R * P; i += 32) Hs[i] = prm.H[i];
     for (int i = lane; i < R * R; i += 32) {
         const int r = i / R, c = i % R;
-        G[r][c] = prm.gram[r <= c ? r * R + c : c * R + r];
-        V[r][c] = r == c ? 1.0 : 0.0;
+        A[r * ld + c] = prm.gram[r <= c ? r * R + c : c * R + r];
     }
     __syncwarp();
+    const int lane_i = lane / R, lane_j = lane % R, step_i = 32 / R, step_j = 32 % R;   // entry lane + 32 k of an R x R matrix
 
-    double (*Ga)[kMaxR + 1] = G, (*Gb)[kMaxR + 1] = Qa;          // current / next Gram matrix of the Jacobi rounds
-    int rank = 0;
+    int rank = 0, nl = 0;
     unsigned long long flagged = forced;
-    double max_in = 0.0, min_out = 1e300;
+    double max_in = 0.0, min_out = 1e300, remainder = 0.0;
     if (n_active > 0ULL) {
-        // ---- Jacobi: G <- J^T G J, V <- V J ----------------------------------------------
-        double tr = 0.0;
-        for (int i = 0; i < R; ++i) tr += G[i][i];
-        // Rotations of one round act on disjoint index pairs (round-robin pairing of n = R or R + 1
-        // indices: n - 1 rounds of n / 2 pairs), so their angles are found side by side (lane = pair)
-        // and applied together: every index i gets its partner and the pair (c_i, s_i) with
-        // new row_i = c_i row_i + s_i row_partner, and G' = J^T G J is written entry by entry into
-        // the other of two buffers (Qa is free until the verification), V column pair by column pair.
-        const int n = (R + 1) & ~1, half = n >> 1;
-        const int lane_i = lane / R, lane_j = lane % R, step_i = 32 / R, step_j = 32 % R;   // entry e = lane + 32 k is (i, j)
-        for (int sweep = 0; sweep < 40; ++sweep) {
-            double off = 0.0;
-            for (int i = lane; i < R * R; i += 32) {
-                const int r = i / R, c = i % R;
-                if (r != c) off += Ga[r][c] * Ga[r][c];
-            }
+        const double theta = prm.tau2 * (double)n_active / (double)R;     // eigenvalue threshold
+        // ---- diagonally pivoted Cholesky: G = L L^T + remainder -------------------------------
+        const double stop = theta * 9.313225746154785e-10;                // 2^-30
+        unsigned int used = 0u;
+        for (int k = 0; k < R; ++k) {
+            const bool mine = lane < R && !((used >> lane) & 1u);
+            double v = mine ? A[lane * ld + lane] : -1.0;
+            int idx = lane;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
-            if (off <= 1e-27 * tr * tr) break;          // off-diagonal mass at the FP64 rounding floor
-            for (int rd = 0; rd < n - 1; ++rd) {
-                if (lane < half) {
-                    const int a = lane == 0 ? n - 1 : (rd + lane) % (n - 1);
-                    const int b = lane == 0 ? rd : (rd + n - 1 - lane) % (n - 1);
-                    const int p = min(a, b), q = max(a, b);
-                    double c = 1.0, sn = 0.0;
-                    if (q < R) {
-                        const double gpq = Ga[p][q], gpp = Ga[p][p], gqq = Ga[q][q];
-                        if (!(fabs(gpq) <= 1e-300 || fabs(gpq) <= 1e-20 * sqrt(fabs(gpp * gqq)))) {
-                            // tan of the rotation angle (the root of smaller magnitude) is o2 / den with
-                            // den = d + sign(d) hypot(d, o2); cosine and sine follow from (den, o2)
-                            // normalised, which takes two reciprocal square roots and no division
-                            const double d = gqq - gpp, o2 = 2.0 * gpq, h2 = d * d + o2 * o2;
-                            const double den = d + copysign(h2 * rsqrt(h2), d);
-                            const double rn = rsqrt(den * den + o2 * o2);
-                            c = fabs(den) * rn;
-                            sn = copysign(o2, o2 * den) * rn;
+            for (int o = 16; o > 0; o >>= 1) {
+                const double ov = __shfl_xor_sync(0xffffffffu, v, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+                if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+            }
+            if (!(v > stop)) break;
+            const double li = mine ? A[lane * ld + idx] * rsqrt(v) : 0.0;   // rows of earlier pivots are zero
+            if (lane < R) Lm[lane * ld + nl] = li;
+            __syncwarp();
+            for (int e = lane, i = lane_i, c = lane_j; e < R * R; e += 32, i += step_i, c += step_j) {
+                if (c >= R) { c -= R; ++i; }
+                A[i * ld + c] -= Lm[i * ld + nl] * Lm[c * ld + nl];
+            }
+            used |= 1u << idx;
+            ++nl;
+            __syncwarp();
+        }
+        {   // what the factorisation left: trace of the Schur complement (every eigenvalue of it is below `stop` R)
+            double d = (lane < R && !((used >> lane) & 1u)) ? fmax(A[lane * ld + lane], 0.0) : 0.0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+            remainder = d;
+        }
+        // ---- M = L^T L (nl x nl), W = I --------------------------------------------------------
+        for (int e = lane; e < nl * nl; e += 32) {
+            const int a = e / nl, b = e - a * nl;
+            double acc = 0.0;
+            for (int i = 0; i < R; ++i) acc = fma(Lm[i * ld + a], Lm[i * ld + b], acc);
+            M[a * ld + b] = acc;
+            Wv[a * ld + b] = a == b ? 1.0 : 0.0;
+        }
+        __syncwarp();
+        // ---- Jacobi on M: M <- J^T M J, W <- W J ----------------------------------------------
+        // Rotations of one round act on disjoint index pairs (round-robin pairing of n = nl or
+        // nl + 1 indices: n - 1 rounds of n / 2 pairs), so their angles are found side by side
+        // (lane = pair) and applied together: every index i gets its partner and the pair
+        // (c_i, s_i) with new row_i = c_i row_i + s_i row_partner, and J^T M J is written entry by
+        // entry into the other of two buffers (A is free by now), W column pair by column pair.
+        double* Ga = M;
+        double* Gb = A;
+        if (nl > 1) {
+            double tr = 0.0;
+            for (int i = 0; i < nl; ++i) tr += M[i * ld + i];
+            const int n = (nl + 1) & ~1, half = n >> 1;
+            const int ml_i = lane / nl, ml_j = lane % nl, ms_i = 32 / nl, ms_j = 32 % nl;
+            for (int sweep = 0; sweep < 40; ++sweep) {
+                double off = 0.0;
+                for (int e = lane, i = ml_i, c = ml_j; e < nl * nl; e += 32, i += ms_i, c += ms_j) {
+                    if (c >= nl) { c -= nl; ++i; }
+                    if (i != c) off += Ga[i * ld + c] * Ga[i * ld + c];
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
+                if (off <= 1e-27 * tr * tr) break;          // off-diagonal mass at the FP64 rounding floor
+                for (int rd = 0; rd < n - 1; ++rd) {
+                    if (lane < half) {
+                        int a = rd + lane, b = rd + n - 1 - lane;            // both below 2 (n - 1)
+                        if (a >= n - 1) a -= n - 1;
+                        if (b >= n - 1) b -= n - 1;
+                        if (lane == 0) { a = n - 1; b = rd; }
+                        const int p = min(a, b), q = max(a, b);
+                        double c = 1.0, sn = 0.0;
+                        if (q < nl) {
+                            const double gpq = Ga[p * ld + q], gpp = Ga[p * ld + p], gqq = Ga[q * ld + q];
+                            if (!(fabs(gpq) <= 1e-300 || gpq * gpq <= 1e-40 * fabs(gpp * gqq))) {
+                                // tan of the rotation angle (the root of smaller magnitude) is o2 / den with
+                                // den = d + sign(d) hypot(d, o2); cosine and sine follow from (den, o2)
+                                // normalised, which takes two reciprocal square roots and no division
+                                const double d = gqq - gpp, o2 = 2.0 * gpq, h2 = d * d + o2 * o2;
+                                const double den = d + copysign(h2 * rsqrt(h2), d);
+                                const double rn = rsqrt(den * den + o2 * o2);
+                                c = fabs(den) * rn;
+                                sn = copysign(o2, o2 * den) * rn;
+                            }
+                            rot_c[q] = c; rot_s[q] = sn; partner[q] = p;
                         }
-                        rot_c[q] = c; rot_s[q] = sn; partner[q] = p;
+                        rot_c[p] = c; rot_s[p] = -sn; partner[p] = q < nl ? q : p;
+                        pair_p[lane] = p; pair_q[lane] = q;
                     }
-                    rot_c[p] = c; rot_s[p] = -sn; partner[p] = q < R ? q : p;
-                    pair_p[lane] = p; pair_q[lane] = q;
+                    __syncwarp();
+                    for (int e = lane, i = ml_i, jj = ml_j; e < nl * nl; e += 32, i += ms_i, jj += ms_j) {
+                        if (jj >= nl) { jj -= nl; ++i; }
+                        const int ip = partner[i], jp = partner[jj];
+                        const double ci = rot_c[i], si = rot_s[i], cj = rot_c[jj], sj = rot_s[jj];
+                        const double t0 = ci * Ga[i * ld + jj] + si * Ga[ip * ld + jj];
+                        const double t1 = ci * Ga[i * ld + jp] + si * Ga[ip * ld + jp];
+                        Gb[i * ld + jj] = (jj == ip && si != 0.0) ? 0.0 : cj * t0 + sj * t1;   // the rotated pair's entry is zero by construction
+                    }
+                    for (int t = 0; t < half; ++t) {                 // W <- W J (columns p, q), lanes over rows
+                        const int pp = pair_p[t], q = pair_q[t];
+                        if (q >= nl || rot_s[q] == 0.0) continue;
+                        const double c = rot_c[q], sn = rot_s[q];
+                        for (int i = lane; i < nl; i += 32) {
+                            const double va = Wv[i * ld + pp], vb = Wv[i * ld + q];
+                            Wv[i * ld + pp] = c * va - sn * vb;
+                            Wv[i * ld + q] = sn * va + c * vb;
+                        }
+                    }
+                    __syncwarp();
+                    double* tmp = Ga; Ga = Gb; Gb = tmp;
                 }
-                __syncwarp();
-                for (int e = lane, i = lane_i, jj = lane_j; e < R * R; e += 32, i += step_i, jj += step_j) {   // G' = J^T G J
-                    if (jj >= R) { jj -= R; ++i; }
-                    const int ip = partner[i], jp = partner[jj];
-                    const double ci = rot_c[i], si = rot_s[i], cj = rot_c[jj], sj = rot_s[jj];
-                    const double t0 = ci * Ga[i][jj] + si * Ga[ip][jj];
-                    const double t1 = ci * Ga[i][jp] + si * Ga[ip][jp];
-                    Gb[i][jj] = (jj == ip && si != 0.0) ? 0.0 : cj * t0 + sj * t1;   // the rotated pair's entry is zero by construction
-                }
-                for (int it = lane; it < half * R; it += 32) {      // V <- V J (columns p, q)
-                    const int t = it / R, i = it - t * R, p = pair_p[t], q = pair_q[t];
-                    if (q >= R || rot_s[q] == 0.0) continue;
-                    const double c = rot_c[q], sn = rot_s[q];
-                    const double va = V[i][p], vb = V[i][q];
-                    V[i][p] = c * va - sn * vb;
-                    V[i][q] = sn * va + c * vb;
-                }
-                __syncwarp();
-                double (*tmp)[kMaxR + 1] = Ga; Ga = Gb; Gb = tmp;
             }
         }
         // ---- eigenvalues in descending order ---------------------------------------------
         if (lane == 0) {
-            for (int i = 0; i < R; ++i) { lam[i] = Ga[i][i]; order[i] = i; }
-            for (int i = 1; i < R; ++i) {                    // insertion sort, R <= 32
+            for (int i = 0; i < nl; ++i) { lam[i] = Ga[i * ld + i]; order[i] = i; }
+            for (int i = 1; i < nl; ++i) {                   // insertion sort, nl <= 32
                 const int oi = order[i];
                 int j = i - 1;
                 while (j >= 0 && lam[order[j]] < lam[oi]) { order[j + 1] = order[j]; --j; }
@@ -317,25 +384,45 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
             }
         }
         __syncwarp();
-        const double theta = prm.tau2 * (double)n_active / (double)R;
-        for (int i = 0; i < R; ++i) rank += lam[order[i]] > theta ? 1 : 0;
+        for (int i = 0; i < nl; ++i) rank += lam[order[i]] > theta ? 1 : 0;
         if (lane == 0) res->rank = rank;
         if (rank > budget) {
             if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
             return;
         }
-        // ---- distance of every H_p to span of the top-rank eigenvectors --------------------
+        // ---- retained subspace: u_e = L w_e / sqrt(lambda_e), then re-orthonormalised ---------
+        for (int e = 0; e < rank; ++e) {
+            const int col = order[e];
+            double u = 0.0;
+            if (lane < R) {
+                for (int a = 0; a < nl; ++a) u = fma(Lm[lane * ld + a], Wv[a * ld + col], u);
+                u *= rsqrt(lam[col]);
+            }
+            for (int pass = 0; pass < 2; ++pass) {
+                for (int f = 0; f < e; ++f) {
+                    double part = lane < R ? U[lane * ld + f] * u : 0.0;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                    if (lane < R) u -= part * U[lane * ld + f];
+                }
+            }
+            double nn = u * u;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(0xffffffffu, nn, o);
+            if (lane < R) U[lane * ld + e] = u * rsqrt(nn);
+            __syncwarp();
+        }
+        // ---- distance of every H_p to the retained subspace --------------------------------
         for (int p = lane; p < P; p += 32) {
             double hn = 0.0;
-            for (int r = 0; r < R; ++r) hn += Hs[r][p] * Hs[r][p];
+            for (int r = 0; r < R; ++r) hn += Hs[r * P + p] * Hs[r * P + p];
             double resid[kMaxR];
-            for (int r = 0; r < R; ++r) resid[r] = Hs[r][p];
+            for (int r = 0; r < R; ++r) resid[r] = Hs[r * P + p];
             for (int pass = 0; pass < 2; ++pass) {           // project twice (re-orthogonalisation)
                 for (int e = 0; e < rank; ++e) {
-                    const int col = order[e];
                     double dot = 0.0;
-                    for (int r = 0; r < R; ++r) dot += V[r][col] * resid[r];
-                    for (int r = 0; r < R; ++r) resid[r] -= dot * V[r][col];
+                    for (int r = 0; r < R; ++r) dot += U[r * ld + e] * resid[r];
+                    for (int r = 0; r < R; ++r) resid[r] -= dot * U[r * ld + e];
                 }
             }
             double rn = 0.0;
@@ -373,45 +460,45 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     }
     // ---- verification: syndrome energy outside span(H_A), A = flagged nodes ------------------
     // Orthonormal basis of span(H_A) by twice-applied modified Gram-Schmidt (columns of Qa).
+    double* Qa = M;
     int na = 0;
     for (int p = 0; p < P; ++p) {
         if (!((flagged >> p) & 1ULL)) continue;
-        if (lane < R) Qa[lane][na] = Hs[lane][p];
+        if (lane < R) Qa[lane * ld + na] = Hs[lane * P + p];
         __syncwarp();
         for (int pass = 0; pass < 2; ++pass) {
             for (int e = 0; e < na; ++e) {
-                double part = lane < R ? Qa[lane][e] * Qa[lane][na] : 0.0;
+                double part = lane < R ? Qa[lane * ld + e] * Qa[lane * ld + na] : 0.0;
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-                if (lane < R) Qa[lane][na] -= part * Qa[lane][e];
+                if (lane < R) Qa[lane * ld + na] -= part * Qa[lane * ld + e];
                 __syncwarp();
             }
         }
-        double nn = lane < R ? Qa[lane][na] * Qa[lane][na] : 0.0;
+        double nn = lane < R ? Qa[lane * ld + na] * Qa[lane * ld + na] : 0.0;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(0xffffffffu, nn, o);
-        if (lane < R) Qa[lane][na] *= rsqrt(nn);
+        if (lane < R) Qa[lane * ld + na] *= rsqrt(nn);
         __syncwarp();
         ++na;
     }
     double residual = 0.0;
     if (n_active > 0ULL) {
-        // tr((I-Pi) G (I-Pi)) = sum_i lambda_i ||(I-Pi) u_i||^2, every term non-negative.
-        // Lane i projects eigenvector i (column i of V, in place: V is not needed afterwards).
-        if (lane < R) {
+        // tr((I-Pi) G (I-Pi)) = ||(I-Pi) L||_F^2 + (what is left of the remainder: at most its trace).
+        // Lane k projects column k of L, in place.
+        if (lane < nl) {
             for (int pass = 0; pass < 2; ++pass) {
                 for (int e = 0; e < na; ++e) {
                     double dot = 0.0;
-                    for (int r = 0; r < R; ++r) dot += Qa[r][e] * V[r][lane];
-                    for (int r = 0; r < R; ++r) V[r][lane] -= dot * Qa[r][e];
+                    for (int r = 0; r < R; ++r) dot += Qa[r * ld + e] * Lm[r * ld + lane];
+                    for (int r = 0; r < R; ++r) Lm[r * ld + lane] -= dot * Qa[r * ld + e];
                 }
             }
-            double un = 0.0;
-            for (int r = 0; r < R; ++r) un += V[r][lane] * V[r][lane];
-            residual = fmax(lam[lane], 0.0) * un;
+            for (int r = 0; r < R; ++r) residual += Lm[r * ld + lane] * Lm[r * ld + lane];
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) residual += __shfl_xor_sync(0xffffffffu, residual, o);
+        residual += remainder;
     }
     const double limit = prm.tau2 * (double)(n_active > 0ULL ? n_active : 1ULL);
     if (lane == 0) {
@@ -421,6 +508,15 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     }
     if (residual <= limit)
         for (int p = lane; p < P; p += 32) res->flagged[p] = (flagged >> p) & 1ULL ? 1 : 0;
+}
+
+inline gpd_status launch_finish(const FinishParams& fp, cudaStream_t st) {
+    const size_t smem = finish_smem_bytes(fp.R, fp.P);
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(locate_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return GPD_ERR_CUDA;
+    locate_finish_kernel<<<1, 32, smem, st>>>(fp);
+    return launch_ok();
 }
 
 template <typename T, int RT>
@@ -475,8 +571,7 @@ gpd_status locate_launch(gpd_plan_s* plan, gpd_product which, const void* output
     fp.H = H; fp.gram = gram; fp.counts = counts; fp.result = result;
     fp.P = plan->P; fp.R = pi.R; fp.tau2 = plan->tau_col * plan->tau_col; fp.tau_in = plan->tau_in;
     fp.erased = erased_mask;
-    locate_finish_kernel<<<1, 32, 0, st>>>(fp);
-    return launch_ok();
+    return launch_finish(fp, st);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -547,8 +642,7 @@ gpd_status locate_static_launch(gpd_plan_s* plan, gpd_product which, const void*
     fp.H = H; fp.gram = gram; fp.counts = counts; fp.result = result;
     fp.P = plan->P; fp.R = pi.R; fp.tau2 = plan->tau_col * plan->tau_col; fp.tau_in = plan->tau_in;
     fp.erased = erased_mask;
-    locate_finish_kernel<<<1, 32, 0, st>>>(fp);
-    return launch_ok();
+    return launch_finish(fp, st);
 }
 
 }  // namespace gpd
