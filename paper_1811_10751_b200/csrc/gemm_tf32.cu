@@ -6,14 +6,18 @@
 // One CTA per SM walks a list of 128 x 128 tiles of the nodes' products (column strips of them for
 // the tiles left over after the last full round over the SMs).  Two accumulators in tensor memory
 // alternate, so a tile's epilogue runs under the next tile's main loop.  Warp roles:
-//   warp 0       : TMA producer (one lane) - raw FP32 tiles of A and B into a 3-stage ring that
+//   warp 0       : TMA producer (one lane) - raw FP32 tiles of A and B into a 4-stage ring that
 //                  runs on across tiles
 //   warp 1       : allocates tensor memory; one lane issues the MMAs and commits them to mbarriers
-//   warps 2..9   : split every landed tile in place into hi (overwrites the raw tile) and lo (second tile)
+//   warps 2..9   : split every landed pair of tiles: B in place in shared memory (hi overwrites the
+//                  raw tile, lo goes to a second tile); A row by row into tensor memory (hi and lo, 32
+//                  columns each per stage), from where the MMAs take it: the A operand then costs
+//                  shared-memory bandwidth once (its raw read) instead of four times
 //   warps 10..13 : read a finished accumulator back (tcgen05.ld), hand it back to the MMA warp, and
 //                  write the tile (plain store, or read-modify-write for the coded update)
 // Operand tiles use the 128-byte swizzle; A is K-major; B is K-major for the update (X^_p is
 // [N][K]) and MN-major for the forward / backward products (X~_p, W~_p are [K][N]).
+// Tensor memory (512 columns): accumulators in columns 0..255, the A stages behind them.
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains its copies,
 // frees its tensor memory and returns.
 #include <cuda.h>
@@ -24,13 +28,16 @@ namespace gpd {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 32, STAGES = 3;
+constexpr int BM = 128, BN = 128, BK = 32, STAGES = 4;
 constexpr int UMMA_K = 8;
 constexpr int A_TILE_BYTES = BM * BK * 4;            // 16 KB, rows of 128 B
 constexpr int B_TILE_BYTES = BN * BK * 4;            // 16 KB
-constexpr int STAGE_BYTES = 2 * A_TILE_BYTES + 2 * B_TILE_BYTES;
+constexpr int STAGE_BYTES = A_TILE_BYTES + 2 * B_TILE_BYTES;   // raw A, B hi, B lo
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
-constexpr int TMEM_COLS = 256;                       // two 128-column accumulators: one fills while the other drains
+constexpr int TMEM_ACC_COLS = 2 * BN;                // two 128-column accumulators: one fills while the other drains
+constexpr int TMEM_A_COLS = 2 * BK;                  // per stage: A hi (BK columns), A lo (BK columns); lane = row of the tile
+constexpr int TMEM_COLS = 512;
+static_assert(TMEM_ACC_COLS + STAGES * TMEM_A_COLS <= TMEM_COLS, "tensor memory budget");
 constexpr int kConvWarps = 8;                        // warps 2..9: split tiles
 constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kEpiWarps = 4;                         // warps 10..13: drain tensor memory, one per lane quarter
@@ -98,10 +105,19 @@ __device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) { return smem_des
 // MMA of K = 8); the next 32 columns start BK rows (BK * 128 bytes) further.
 __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) { return smem_desc(addr, BK * 128, 512, kLayoutSw128Base32); }
 
-__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// A operand from tensor memory (lane = row, one column per TF32 element)
+__device__ __forceinline__ void umma_tf32_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 16 consecutive columns of this thread's lane
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -169,10 +185,10 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t tmem_base = tmem_slot;
     volatile int* abort_p = &abort_flag;
 
-    auto A_hi = [&](int s) { return smem + s * STAGE_BYTES; };
-    auto A_lo = [&](int s) { return smem + s * STAGE_BYTES + A_TILE_BYTES; };
-    auto B_hi = [&](int s) { return smem + s * STAGE_BYTES + 2 * A_TILE_BYTES; };
-    auto B_lo = [&](int s) { return smem + s * STAGE_BYTES + 2 * A_TILE_BYTES + B_TILE_BYTES; };
+    auto A_raw = [&](int s) { return smem + s * STAGE_BYTES; };
+    auto B_hi = [&](int s) { return smem + s * STAGE_BYTES + A_TILE_BYTES; };
+    auto B_lo = [&](int s) { return smem + s * STAGE_BYTES + A_TILE_BYTES + B_TILE_BYTES; };
+    auto A_tmem = [&](int s) { return tmem_base + (uint32_t)(TMEM_ACC_COLS + s * TMEM_A_COLS); };   // hi; lo is BK columns further
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
@@ -187,7 +203,7 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) { ok = false; break; }
                     mbar_expect_tx(&full_bar[s], A_TILE_BYTES + bn * BK * 4);
-                    tma_load_3d(A_hi(s), &tmA, kb * BK, m0, p, &full_bar[s]);
+                    tma_load_3d(A_raw(s), &tmA, kb * BK, m0, p, &full_bar[s]);
                     for (int c = 0; c < bn / 32; ++c) {      // B arrives in boxes of 32 columns (or 32 rows of X^_p)
                         if (B_KMAJOR)
                             tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, kb * BK, n0 + 32 * c, p, &full_bar[s]);
@@ -223,21 +239,20 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(&conv_bar[s], ph, abort_p)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a_hi = smem_u32(A_hi(s)), a_lo = smem_u32(A_lo(s));
+                    const uint32_t a_hi = A_tmem(s), a_lo = A_tmem(s) + BK;
                     const uint32_t b_hi = smem_u32(B_hi(s)), b_lo = smem_u32(B_lo(s));
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // K-major: next 8 elements of K are 32 bytes further inside the swizzled row;
-                        // MN-major: next 8 k-rows are 8 * 128 bytes further in every 32-column chunk
-                        const uint32_t a_off = k * UMMA_K * 4;
+                        // A: the next 8 elements of K are 8 tensor-memory columns further.
+                        // B, K-major: 32 bytes further inside the swizzled row; MN-major: the next 8
+                        // k-rows are 8 * 128 bytes further in every 32-column chunk
+                        const uint32_t a_off = k * UMMA_K;
                         const uint32_t b_off = B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128;
-                        const uint64_t da_hi = desc_kmajor(a_hi + a_off);
-                        const uint64_t da_lo = desc_kmajor(a_lo + a_off);
                         const uint64_t db_hi = B_KMAJOR ? desc_kmajor(b_hi + b_off) : desc_mnmajor(b_hi + b_off);
                         const uint64_t db_lo = B_KMAJOR ? desc_kmajor(b_lo + b_off) : desc_mnmajor(b_lo + b_off);
-                        umma_tf32(tmem_d, da_lo, db_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);   // small terms first
-                        umma_tf32(tmem_d, da_hi, db_lo, idesc, 1u);
-                        umma_tf32(tmem_d, da_hi, db_hi, idesc, 1u);
+                        umma_tf32_ta(tmem_d, a_lo + a_off, db_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);   // small terms first
+                        umma_tf32_ta(tmem_d, a_hi + a_off, db_lo, idesc, 1u);
+                        umma_tf32_ta(tmem_d, a_hi + a_off, db_hi, idesc, 1u);
                     }
                     umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
                 }
@@ -247,6 +262,10 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else if (warp < 2 + kConvWarps) {
         // ------------------------------ split hi / lo ------------------------------
         const int tc = threadIdx.x - 64;             // 0..kConvThreads-1
+        // A: this warp may touch tensor-memory lanes 32 q .. 32 q + 31 (q = warp mod 4); the two warps
+        // of a quarter take 16 of the 32 k-columns each.  A thread owns one row of the tile.
+        const int q = warp & 3, khalf = (warp - 2) >> 2;
+        const int arow = q * 32 + lane;
         int it = 0;
         bool ok = true;
         for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
@@ -256,23 +275,41 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
                 const int s = it % STAGES;
                 const uint32_t ph = (it / STAGES) & 1;
-                if (!mbar_wait(&full_bar[s], ph, abort_p)) { ok = false; break; }
-                float4* hi[2] = {reinterpret_cast<float4*>(A_hi(s)), reinterpret_cast<float4*>(B_hi(s))};
-                float4* lo[2] = {reinterpret_cast<float4*>(A_lo(s)), reinterpret_cast<float4*>(B_lo(s))};
-                const int count[2] = {A_TILE_BYTES / 16, b_float4};
+                const bool landed = mbar_wait(&full_bar[s], ph, abort_p);
+                __syncwarp();
+                if (!__all_sync(0xffffffffu, landed)) { ok = false; break; }   // tcgen05.st is warp-collective: all lanes or none
+                {   // A row: four 16-byte chunks of the 128-byte swizzled row (chunk index xor row mod 8)
+                    const uint8_t* rowp = A_raw(s) + arow * 128;
+                    uint32_t hi[16], lo[16];
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
+                    for (int c = 0; c < 4; ++c) {
+                        const float4 v = *reinterpret_cast<const float4*>(rowp + (((khalf * 4 + c) ^ (arow & 7)) << 4));
+                        const float h0 = to_tf32(v.x), h1 = to_tf32(v.y), h2 = to_tf32(v.z), h3 = to_tf32(v.w);
+                        hi[4 * c] = __float_as_uint(h0); hi[4 * c + 1] = __float_as_uint(h1);
+                        hi[4 * c + 2] = __float_as_uint(h2); hi[4 * c + 3] = __float_as_uint(h3);
+                        lo[4 * c] = __float_as_uint(to_tf32(v.x - h0)); lo[4 * c + 1] = __float_as_uint(to_tf32(v.y - h1));
+                        lo[4 * c + 2] = __float_as_uint(to_tf32(v.z - h2)); lo[4 * c + 3] = __float_as_uint(to_tf32(v.w - h3));
+                    }
+                    const uint32_t taddr = A_tmem(s) + ((uint32_t)(q * 32) << 16) + (uint32_t)(khalf * 16);
+                    tmem_st16(taddr, hi);
+                    tmem_st16(taddr + BK, lo);
+                }
+                {   // B in place
+                    float4* hi = reinterpret_cast<float4*>(B_hi(s));
+                    float4* lo = reinterpret_cast<float4*>(B_lo(s));
 #pragma unroll 4
-                    for (int idx = tc; idx < count[t]; idx += kConvThreads) {
-                        const float4 v = hi[t][idx];
+                    for (int idx = tc; idx < b_float4; idx += kConvThreads) {
+                        const float4 v = hi[idx];
                         float4 h, l;
                         h.x = to_tf32(v.x); h.y = to_tf32(v.y); h.z = to_tf32(v.z); h.w = to_tf32(v.w);
                         l.x = to_tf32(v.x - h.x); l.y = to_tf32(v.y - h.y); l.z = to_tf32(v.z - h.z); l.w = to_tf32(v.w - h.w);
-                        hi[t][idx] = h;
-                        lo[t][idx] = l;
+                        hi[idx] = h;
+                        lo[idx] = l;
                     }
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the tiles visible to the MMA unit
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");       // A is in tensor memory
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");       // B tiles visible to the MMA unit
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&conv_bar[s]);
             }
