@@ -129,6 +129,9 @@ __device__ __forceinline__ float to_tf32(float x) {
     return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
 }
 
+// What the tensor core makes of a raw FP32 word in a TF32 operand: the 13 low mantissa bits dropped.
+__device__ __forceinline__ float trunc_tf32(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+
 template <bool B_KMAJOR, bool UPDATE>
 __global__ void __launch_bounds__(kThreads, 1)
 sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams prm,
@@ -300,10 +303,9 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll 4
                     for (int idx = tc; idx < b_float4; idx += kConvThreads) {
                         const float4 v = hi[idx];
-                        float4 h, l;
-                        h.x = to_tf32(v.x); h.y = to_tf32(v.y); h.z = to_tf32(v.z); h.w = to_tf32(v.w);
-                        l.x = to_tf32(v.x - h.x); l.y = to_tf32(v.y - h.y); l.z = to_tf32(v.z - h.z); l.w = to_tf32(v.w - h.w);
-                        hi[idx] = h;
+                        float4 l;
+                        l.x = to_tf32(v.x - trunc_tf32(v.x)); l.y = to_tf32(v.y - trunc_tf32(v.y));
+                        l.z = to_tf32(v.z - trunc_tf32(v.z)); l.w = to_tf32(v.w - trunc_tf32(v.w));
                         lo[idx] = l;
                     }
                 }
