@@ -242,20 +242,24 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(&conv_bar[s], ph, abort_p)) { ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    // One thread issues everything, so its instruction count per k-block is on the
+                    // critical path: the two B descriptors are built once per stage, a k-step only
+                    // adds its offset to their address field (16-byte units, no carry out of 14 bits:
+                    // a stage lies inside the 227 KB window).
                     const uint32_t a_hi = A_tmem(s), a_lo = A_tmem(s) + BK;
-                    const uint32_t b_hi = smem_u32(B_hi(s)), b_lo = smem_u32(B_lo(s));
+                    const uint64_t db_hi0 = B_KMAJOR ? desc_kmajor(smem_u32(B_hi(s))) : desc_mnmajor(smem_u32(B_hi(s)));
+                    const uint64_t db_lo0 = db_hi0 + (uint64_t)(B_TILE_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         // A: the next 8 elements of K are 8 tensor-memory columns further.
                         // B, K-major: 32 bytes further inside the swizzled row; MN-major: the next 8
                         // k-rows are 8 * 128 bytes further in every 32-column chunk
                         const uint32_t a_off = k * UMMA_K;
-                        const uint32_t b_off = B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128;
-                        const uint64_t db_hi = B_KMAJOR ? desc_kmajor(b_hi + b_off) : desc_mnmajor(b_hi + b_off);
-                        const uint64_t db_lo = B_KMAJOR ? desc_kmajor(b_lo + b_off) : desc_mnmajor(b_lo + b_off);
-                        umma_tf32_ta(tmem_d, a_lo + a_off, db_hi, idesc, (kb > 0 || k > 0) ? 1u : 0u);   // small terms first
-                        umma_tf32_ta(tmem_d, a_hi + a_off, db_lo, idesc, 1u);
-                        umma_tf32_ta(tmem_d, a_hi + a_off, db_hi, idesc, 1u);
+                        const uint64_t b_off = (uint64_t)((B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128) >> 4);
+                        const uint32_t first = (kb > 0 || k > 0) ? 1u : 0u;
+                        umma_tf32_ta(tmem_d, a_lo + a_off, db_hi0 + b_off, idesc, first);   // small terms first
+                        umma_tf32_ta(tmem_d, a_hi + a_off, db_lo0 + b_off, idesc, 1u);
+                        umma_tf32_ta(tmem_d, a_hi + a_off, db_hi0 + b_off, idesc, 1u);
                     }
                     umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
                 }
