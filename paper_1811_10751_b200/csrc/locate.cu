@@ -40,7 +40,7 @@ __device__ __forceinline__ void dmma_m8n8k4(double& d0, double& d1, double a, do
                  : "d"(a), "d"(b));
 }
 
-// Syndrome s = H z and squared norm of one codeword: P loads at stride L, issued eight at a time.
+// Syndrome s = H z and squared norm of one codeword: P loads at stride L, issued in equal groups of up to nine.
 // CHECKED = false is the plain form: no per-value tests, a non-finite value shows up as a non-finite
 // norm and the caller repeats the codeword with CHECKED = true, which zeroes non-finite values
 // and erased nodes and records the nodes that held a non-finite value.
@@ -48,7 +48,7 @@ template <typename T, int RT, bool CHECKED>
 __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P, const double* sH,
                                                   unsigned long long erased, double (&s)[RT], double& nz,
                                                   unsigned long long& bad) {
-    constexpr int U = RT <= 8 ? 8 : 4;                   // loads issued together (fewer where the syndrome fills the registers)
+    constexpr int U = RT <= 8 ? 9 : 4;                   // most loads issued together (fewer where the syndrome fills the registers)
 #pragma unroll
     for (int r = 0; r < RT; ++r) s[r] = 0.0;
     nz = 0.0;
@@ -66,27 +66,20 @@ __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P,
             s[2 * r + 1] = fma(hv.y, zz, s[2 * r + 1]);
         }
     };
-    int p0 = 0;
-    for (; p0 + U <= P; p0 += U, zp += U * L, sH += U * RT) {
+    // groups of equal size (no short last group: every group costs one trip to memory)
+    const int n_groups = (P + U - 1) / U, gs = (P + n_groups - 1) / n_groups;
+    for (int p0 = 0; p0 < P; p0 += gs, zp += gs * L, sH += gs * RT) {
         double z[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) z[u] = (double)__ldcs(zp + u * L);
-#pragma unroll
-        for (int u = 0; u < U; ++u) absorb(z[u], p0 + u, sH + u * RT);
-    }
-    if (p0 < P) {                                        // the last P mod U nodes
-        double z[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) z[u] = (p0 + u < P) ? (double)__ldcs(zp + u * L) : 0.0;
+        for (int u = 0; u < U; ++u) z[u] = (u < gs && p0 + u < P) ? (double)__ldcs(zp + u * L) : 0.0;
 #pragma unroll
         for (int u = 0; u < U; ++u)
-            if (p0 + u < P) absorb(z[u], p0 + u, sH + u * RT);
+            if (u < gs && p0 + u < P) absorb(z[u], p0 + u, sH + u * RT);
     }
 }
 
 // One thread per output position (codeword): the syndrome in RT registers, the zero test.  The
-// Gram matrix of the failing codewords is formed
-// warp by warp on the FP64 tensor cores: the 32 scaled syndromes of a warp are staged in shared
+// Gram matrix of the failing codewords is formed warp by warp on the FP64 tensor cores: the 32 scaled syndromes of a warp are staged in shared
 // memory and fed to mma.m8n8k4 as both operands (G += S S^T, four codewords per instruction), so
 // the accumulator costs two registers per 8 x 8 tile and the streaming loop needs no CTA barrier.
 template <typename T, int RT>
