@@ -35,12 +35,17 @@ struct PosParams {
 };
 
 template <typename T, int RT>                 // RT: parity checks rounded up to 8, 16 or 32
-__global__ void __launch_bounds__(256) position_scan_kernel(PosParams prm) {
-    extern __shared__ double sH[];        // [RT][P], zero rows past R
-    for (int i = threadIdx.x; i < RT * prm.P; i += 256) sH[i] = i < prm.R * prm.P ? prm.H[i] : 0.0;
+__global__ void __launch_bounds__(256, RT <= 8 ? 4 : 1) position_scan_kernel(PosParams prm) {
+    extern __shared__ __align__(16) double sH[];   // [P][RT] node-major, zero past row R
+    for (int i = threadIdx.x; i < RT * prm.P; i += 256) {
+        const int pnode = i / RT, j = i - pnode * RT;
+        sH[i] = j < prm.R ? prm.H[j * prm.P + pnode] : 0.0;
+    }
     __syncthreads();
     const T* Z = reinterpret_cast<const T*>(prm.Z);
     const int lane = threadIdx.x & 31;
+    constexpr int U = RT <= 8 ? 9 : 4;            // loads issued together, in groups of equal size
+    const int n_groups = (prm.P + U - 1) / U, gs = (prm.P + n_groups - 1) / n_groups;
     // all lanes of a warp run the same rounds (the counters are updated once per warp and round)
     for (int64_t base = (int64_t)blockIdx.x * 256; base < prm.L; base += (int64_t)gridDim.x * 256) {
         const int64_t pos = base + threadIdx.x;
@@ -51,13 +56,29 @@ __global__ void __launch_bounds__(256) position_scan_kernel(PosParams prm) {
         double z2 = 0.0;
         bool finite = true;
         if (valid) {
-#pragma unroll 5
-            for (int p = 0; p < prm.P; ++p) {
-                const double z = (double)__ldcs(Z + (int64_t)p * prm.L + pos);
-                finite &= isfinite(z);
-                z2 = fma(z, z, z2);
+            const T* zp = Z + pos;
+            const double* h = sH;
+            for (int p0 = 0; p0 < prm.P; p0 += gs, zp += gs * prm.L, h += gs * RT) {
+                double z[U];
 #pragma unroll
-                for (int j = 0; j < RT; ++j) r[j] = fma(sH[j * prm.P + p], z, r[j]);   // rows R .. RT-1 are zero
+                for (int u = 0; u < U; ++u) z[u] = (u < gs && p0 + u < prm.P) ? (double)__ldcs(zp + u * prm.L) : 0.0;
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (u < gs && p0 + u < prm.P) {
+                        z2 = fma(z[u], z[u], z2);
+                        const double2* hv = reinterpret_cast<const double2*>(h + u * RT);
+#pragma unroll
+                        for (int j = 0; j < RT / 2; ++j) {
+                            const double2 hh = hv[j];
+                            r[2 * j] = fma(hh.x, z[u], r[2 * j]);
+                            r[2 * j + 1] = fma(hh.y, z[u], r[2 * j + 1]);
+                        }
+                    }
+                }
+            }
+            if (!isfinite(z2)) {                  // rare: a non-finite value, or finite ones whose squares overflow
+                zp = Z + pos;
+                for (int p = 0; p < prm.P; ++p, zp += prm.L) finite &= isfinite((double)__ldcs(zp));
             }
         }
         double r2 = 0.0;
