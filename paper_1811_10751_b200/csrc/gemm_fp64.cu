@@ -3,7 +3,9 @@
 // FP32-level noise beyond the 1e-4 accuracy target (thresholds above 9), so shares, products
 // and outputs stay in FP64.  tcgen05 has no FP64 kind; this is the chip's native FP64 matrix path.
 //
-// CTA tile 128 x 128, K step 16, 8 warps (2 x 4), warp tile 64 x 32 = 8 x 4 MMA tiles.
+// CTA tile 64 x 128, K step 16, 4 warps side by side, warp tile 64 x 32 = 8 x 4 MMA tiles, two
+// CTAs per SM: the prologue and the epilogue of one CTA run under the other's main loop (the
+// kernel also builds as one 128 x 128 CTA of 8 warps per SM, WM = 2, which is 3 to 7 % slower).
 // Operands are staged with 16-byte cp.async into a 3-stage ring; rows are padded by 4 doubles
 // so that the 64-bit fragment loads of each half-warp hit 16 distinct bank pairs.
 #include "gemm_common.h"
@@ -12,11 +14,10 @@ namespace gpd {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 16, STAGES = 3;
+constexpr int BN = 128, BK = 16, STAGES = 3;        // BM = 64 WM, WM = warps along M (1 or 2)
 constexpr int A_LD = BK + 4;                  // A tile  [BM][A_LD]
 constexpr int BK_LD = BK + 4;                 // B tile, K-major source: [BN][BK_LD]
 constexpr int BN_LD = BN + 4;                 // B tile, N-major source: [BK][BN_LD]
-constexpr int A_STAGE = BM * A_LD;
 constexpr int B_STAGE_KMAJOR = BN * BK_LD;
 constexpr int B_STAGE_NMAJOR = BK * BN_LD;
 
@@ -35,10 +36,11 @@ __device__ __forceinline__ void dmma(double& d0, double& d1, double a, double b)
                  : "d"(a), "d"(b));
 }
 
-template <bool B_KMAJOR, bool UPDATE>
-__global__ void __launch_bounds__(256, 1) dgemm_mma_kernel(GemmParams prm) {
+template <bool B_KMAJOR, bool UPDATE, int WM>
+__global__ void __launch_bounds__(128 * WM, WM == 1 ? 2 : 1) dgemm_mma_kernel(GemmParams prm) {
     if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
     extern __shared__ __align__(16) double smem[];
+    constexpr int BM = 64 * WM, NT = 128 * WM, A_STAGE = BM * A_LD;
     constexpr int B_STAGE = B_KMAJOR ? B_STAGE_KMAJOR : B_STAGE_NMAJOR;
     double* sA = smem;
     double* sB = smem + STAGES * A_STAGE;
@@ -55,10 +57,10 @@ __global__ void __launch_bounds__(256, 1) dgemm_mma_kernel(GemmParams prm) {
     auto load_stage = [&](int stage, int64_t k0) {
         double* a = sA + stage * A_STAGE;
         double* b = sB + stage * B_STAGE;
-        // A tile: 128 rows x 8 chunks of 2 doubles
+        // A tile: BM rows x 8 chunks of 2 doubles
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int c = tid + i * 256;
+        for (int i = 0; i < BM * 8 / NT; ++i) {
+            const int c = tid + i * NT;
             const int row = c >> 3, ch = c & 7;
             const int64_t gm = m0 + row, gk = k0 + ch * 2;
             const bool ok = gm < prm.M && gk < prm.K;
@@ -66,8 +68,8 @@ __global__ void __launch_bounds__(256, 1) dgemm_mma_kernel(GemmParams prm) {
         }
         if (B_KMAJOR) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int c = tid + i * 256;
+            for (int i = 0; i < BN * 8 / NT; ++i) {
+                const int c = tid + i * NT;
                 const int row = c >> 3, ch = c & 7;
                 const int64_t gn = n0 + row, gk = k0 + ch * 2;
                 const bool ok = gn < prm.N && gk < prm.K;
@@ -75,8 +77,8 @@ __global__ void __launch_bounds__(256, 1) dgemm_mma_kernel(GemmParams prm) {
             }
         } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int c = tid + i * 256;
+            for (int i = 0; i < BK * 64 / NT; ++i) {
+                const int c = tid + i * NT;
                 const int kr = c >> 6, ch = c & 63;
                 const int64_t gk = k0 + kr, gn = n0 + ch * 2;
                 const bool ok = gk < prm.K && gn < prm.N;
@@ -154,20 +156,26 @@ __global__ void __launch_bounds__(256, 1) dgemm_mma_kernel(GemmParams prm) {
     }
 }
 
-template <bool B_KMAJOR, bool UPDATE>
-gpd_status launch(const GemmParams& prm, cudaStream_t st) {
+template <bool B_KMAJOR, bool UPDATE, int WM>
+gpd_status launch_tile(const GemmParams& prm, cudaStream_t st) {
+    constexpr int BM = 64 * WM;
     constexpr int B_STAGE = B_KMAJOR ? B_STAGE_KMAJOR : B_STAGE_NMAJOR;
-    constexpr size_t smem = sizeof(double) * STAGES * (A_STAGE + B_STAGE);
+    constexpr size_t smem = sizeof(double) * STAGES * (BM * A_LD + B_STAGE);
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(dgemm_mma_kernel<B_KMAJOR, UPDATE>,
+        if (cudaFuncSetAttribute(dgemm_mma_kernel<B_KMAJOR, UPDATE, WM>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return GPD_ERR_CUDA;
         configured = true;
     }
     dim3 grid((unsigned)((prm.N + BN - 1) / BN), (unsigned)((prm.M + BM - 1) / BM), (unsigned)prm.P);
-    dgemm_mma_kernel<B_KMAJOR, UPDATE><<<grid, 256, smem, st>>>(prm);
+    dgemm_mma_kernel<B_KMAJOR, UPDATE, WM><<<grid, 128 * WM, smem, st>>>(prm);
     return launch_ok();
+}
+
+template <bool B_KMAJOR, bool UPDATE>
+gpd_status launch(const GemmParams& prm, cudaStream_t st) {
+    return launch_tile<B_KMAJOR, UPDATE, 1>(prm, st);
 }
 
 }  // namespace
