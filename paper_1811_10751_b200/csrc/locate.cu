@@ -186,7 +186,7 @@ struct FinishParams {
 __host__ __device__ inline size_t finish_smem_bytes(int R, int P) {
     const int ld = R | 1;
     return sizeof(double) * ((size_t)5 * R * ld + (size_t)R * P + (size_t)R + 2 * (size_t)(R + 1) + (size_t)P) +
-           sizeof(int) * ((size_t)(R + 1) + 2 * (size_t)(R / 2 + 1) + (size_t)R) + (size_t)P;
+           sizeof(int) * ((size_t)(R + 1) + (size_t)R) + (size_t)P;
 }
 
 // One warp.  The Gram matrix G of the failing codewords has rank = number of erroneous nodes (a
@@ -210,9 +210,7 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     double* rot_s = rot_c + (R + 1);         // [R + 1]
     double* dist = rot_s + (R + 1);          // [P]
     int* partner = reinterpret_cast<int*>(dist + P);   // [R + 1]
-    int* pair_p = partner + (R + 1);         // [R / 2 + 1]
-    int* pair_q = pair_p + (R / 2 + 1);      // [R / 2 + 1]
-    int* order = pair_q + (R / 2 + 1);       // [R]
+    int* order = partner + (R + 1);          // [R]
     unsigned char* inside = reinterpret_cast<unsigned char*>(order + R);   // [P]
     gpd_locate_result* res = prm.result;
     const unsigned long long n_active = prm.counts[0];
@@ -300,9 +298,11 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
         // nl + 1 indices: n - 1 rounds of n / 2 pairs), so their angles are found side by side
         // (lane = pair) and applied together: every index i gets its partner and the pair
         // (c_i, s_i) with new row_i = c_i row_i + s_i row_partner, and J^T M J is written entry by
-        // entry into the other of two buffers (A is free by now), W column pair by column pair.
+        // entry into the other of two buffers (A is free by now), and so is W J (second buffer: U).
         double* Ga = M;
         double* Gb = A;
+        double* Wa = Wv;                     // eigenvectors, second buffer: U (not in use before the sweeps end)
+        double* Wb = U;
         if (nl > 1) {
             double tr = 0.0;
             for (int i = 0; i < nl; ++i) tr += M[i * ld + i];
@@ -340,7 +340,6 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
                             rot_c[q] = c; rot_s[q] = sn; partner[q] = p;
                         }
                         rot_c[p] = c; rot_s[p] = -sn; partner[p] = q < nl ? q : p;
-                        pair_p[lane] = p; pair_q[lane] = q;
                     }
                     __syncwarp();
                     for (int e = lane, i = ml_i, jj = ml_j; e < nl * nl; e += 32, i += ms_i, jj += ms_j) {
@@ -350,21 +349,17 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
                         const double t0 = ci * Ga[i * ld + jj] + si * Ga[ip * ld + jj];
                         const double t1 = ci * Ga[i * ld + jp] + si * Ga[ip * ld + jp];
                         Gb[i * ld + jj] = (jj == ip && si != 0.0) ? 0.0 : cj * t0 + sj * t1;   // the rotated pair's entry is zero by construction
-                    }
-                    for (int t = 0; t < half; ++t) {                 // W <- W J (columns p, q), lanes over rows
-                        const int pp = pair_p[t], q = pair_q[t];
-                        if (q >= nl || rot_s[q] == 0.0) continue;
-                        const double c = rot_c[q], sn = rot_s[q];
-                        for (int i = lane; i < nl; i += 32) {
-                            const double va = Wv[i * ld + pp], vb = Wv[i * ld + q];
-                            Wv[i * ld + pp] = c * va - sn * vb;
-                            Wv[i * ld + q] = sn * va + c * vb;
-                        }
+                        Wb[i * ld + jj] = cj * Wa[i * ld + jj] + sj * Wa[i * ld + jp];          // W J: columns rotate like those of M
                     }
                     __syncwarp();
                     double* tmp = Ga; Ga = Gb; Gb = tmp;
+                    tmp = Wa; Wa = Wb; Wb = tmp;
                 }
             }
+        }
+        if (Wa != Wv) {                      // the last round left the eigenvectors in U's storage
+            for (int e = lane; e < nl * ld; e += 32) Wv[e] = Wa[e];
+            __syncwarp();
         }
         // ---- eigenvalues in descending order ---------------------------------------------
         if (lane == 0) {
