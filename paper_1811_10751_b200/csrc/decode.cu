@@ -83,28 +83,55 @@ __global__ void __launch_bounds__(kMatrixThreads) decode_matrix_kernel(MatrixPar
     // Householder triangularisation.  Eight lanes share a column (column = k + tid / 8, rows strided
     // by eight between them, partial sums met by three shuffles inside the group), so that a step
     // costs rows / 8 dependent operations instead of rows.  Within a step column k is only read:
-    // its own group stores the unit reflector, and R's diagonal entry is put in after the barrier.
+    // the last warp stores the unit reflector (its own columns k + 28 .. k + 31 rarely exist, and
+    // the first warp, which holds the columns every step has, is left with one branch), and R's
+    // diagonal entry is put in after the barrier.  Row loops are unrolled to the largest trip
+    // count (64 rows / 8 lanes) so that their loads go out together.
     const int part = tid & 7, colg = tid >> 3;           // kMatrixThreads / 8 = 32 >= Q columns
+    constexpr int kTrips = kMaxNodes / 8;
     for (int k = 0; k < Q; ++k) {
+        double vk[kTrips];                               // this lane's entries of column k (rows k + part + 8 j)
         double sigma = 0.0;
-        for (int r = k + part; r < rows; r += 8) sigma += A[r][k] * A[r][k];
+#pragma unroll
+        for (int j = 0; j < kTrips; ++j) {
+            const int r = k + part + 8 * j;
+            vk[j] = r < rows ? A[r][k] : 0.0;
+            sigma = fma(vk[j], vk[j], sigma);
+        }
         sigma += __shfl_xor_sync(0xffffffffu, sigma, 1);
         sigma += __shfl_xor_sync(0xffffffffu, sigma, 2);
         sigma += __shfl_xor_sync(0xffffffffu, sigma, 4);     // same value in every group (same order of additions)
         const double akk = A[k][k];
         const double alpha = akk >= 0.0 ? -sqrt(sigma) : sqrt(sigma);
         const double inv_vnorm = rsqrt(fmax(sigma - 2.0 * alpha * akk + alpha * alpha, 1e-300));
+        if (part == 0) vk[0] -= alpha;                   // v = a_k - alpha e_k (row k sits in lane 0, trip 0)
         const int c = k + colg;
-        if (colg == 0) {
-            for (int r = k + part; r < rows; r += 8) Vh[r][k] = (A[r][k] - (r == k ? alpha : 0.0)) * inv_vnorm;
-        } else if (c < Q) {
+        if (colg > 0 && c < Q) {
+            double ac[kTrips];
             double dot = 0.0;
-            for (int r = k + part; r < rows; r += 8) dot += (A[r][k] - (r == k ? alpha : 0.0)) * A[r][c];
-            dot += __shfl_xor_sync(0xffu << (8 * (tid >> 3 & 3)), dot, 1);
-            dot += __shfl_xor_sync(0xffu << (8 * (tid >> 3 & 3)), dot, 2);
-            dot += __shfl_xor_sync(0xffu << (8 * (tid >> 3 & 3)), dot, 4);
+#pragma unroll
+            for (int j = 0; j < kTrips; ++j) {
+                const int r = k + part + 8 * j;
+                ac[j] = r < rows ? A[r][c] : 0.0;
+                dot = fma(vk[j], ac[j], dot);
+            }
+            const unsigned int gmask = 0xffu << (8 * (colg & 3));
+            dot += __shfl_xor_sync(gmask, dot, 1);
+            dot += __shfl_xor_sync(gmask, dot, 2);
+            dot += __shfl_xor_sync(gmask, dot, 4);
             const double f = 2.0 * dot * inv_vnorm * inv_vnorm;
-            for (int r = k + part; r < rows; r += 8) A[r][c] -= f * (A[r][k] - (r == k ? alpha : 0.0));
+#pragma unroll
+            for (int j = 0; j < kTrips; ++j) {
+                const int r = k + part + 8 * j;
+                if (r < rows) A[r][c] = fma(-f, vk[j], ac[j]);
+            }
+        }
+        if (warp == kMatrixThreads / 32 - 1) {           // unit reflector, 32 lanes over the rows
+#pragma unroll
+            for (int j = 0; j < kMaxNodes / 32; ++j) {
+                const int r = k + lane + 32 * j;
+                if (r < rows) Vh[r][k] = (A[r][k] - (r == k ? alpha : 0.0)) * inv_vnorm;
+            }
         }
         __syncthreads();
         if (tid == 0) A[k][k] = alpha;               // R's diagonal; nothing below reads column k again
