@@ -33,7 +33,9 @@ constexpr int UMMA_K = 8;
 constexpr int A_TILE_BYTES = BM * BK * 4;            // 16 KB, rows of 128 B
 constexpr int B_TILE_BYTES = BN * BK * 4;            // 16 KB
 constexpr int STAGE_BYTES = A_TILE_BYTES + 2 * B_TILE_BYTES;   // raw A, B hi, B lo
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;
+constexpr int EPI_PITCH = 36;                        // floats per staged row: 16-byte aligned, conflict-free for 16-byte accesses
+constexpr int EPI_STAGE_BYTES = 4 * 32 * EPI_PITCH * 4;   // one 32 x 32 chunk per epilogue warp
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_STAGE_BYTES + 1024;
 constexpr int TMEM_ACC_COLS = 2 * BN;                // two 128-column accumulators: one fills while the other drains
 constexpr int TMEM_A_COLS = 2 * BK;                  // per stage: A hi (BK columns), A lo (BK columns); lane = row of the tile
 constexpr int TMEM_COLS = 512;
@@ -338,6 +340,17 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
 #pragma unroll 1
             for (int c0 = 0; c0 < bn; c0 += 32) {
+                const bool whole = vec && n0 + c0 + 32 <= prm.N;     // the chunk leaves as 128-byte row segments
+                const int col4 = (lane & 7) * 4, rsub = lane >> 3;   // this lane's part of a staged chunk
+                float4 old[8];                                       // the stored share, asked for before the accumulator is read
+                if (UPDATE && whole) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int64_t grow = (int64_t)m0 + q * 32 + 4 * i + rsub;
+                        old[i] = grow < prm.M ? *reinterpret_cast<const float4*>(C + grow * prm.N + n0 + c0 + col4)
+                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0);
                 asm volatile(
@@ -355,28 +368,41 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 }
-                if (gm < prm.M) {
-                    float* crow = C + gm * prm.N + n0 + c0;
-                    if (vec && n0 + c0 + 32 <= prm.N) {
+                if (whole) {
+                    // A thread holds 32 columns of one row; written as they are, a store would touch 32
+                    // rows with 16 bytes each.  The chunk goes through shared memory instead and
+                    // leaves as whole 128-byte row segments (eight lanes per row, four rows per store).
+                    float* st = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES) + (warp - 2 - kConvWarps) * (32 * EPI_PITCH);
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                                   __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<float4*>(st + lane * EPI_PITCH + j) =
+                            make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                        __uint_as_float(r[j + 3]));
+                    __syncwarp();
+#pragma unroll
+                    for (int rr = 0; rr < 32; rr += 4) {
+                        const int row = rr + rsub;
+                        const int64_t grow = (int64_t)m0 + q * 32 + row;
+                        float4 v = *reinterpret_cast<const float4*>(st + row * EPI_PITCH + col4);
+                        if (grow < prm.M) {
+                            float* cp = C + grow * prm.N + n0 + c0 + col4;
                             if (UPDATE) {
-                                const float4 o = *reinterpret_cast<const float4*>(crow + j);
+                                const float4 o = old[rr / 4];
                                 v.x = shrink * o.x + eta * v.x; v.y = shrink * o.y + eta * v.y;
                                 v.z = shrink * o.z + eta * v.z; v.w = shrink * o.w + eta * v.w;
                             }
-                            *reinterpret_cast<float4*>(crow + j) = v;
+                            *reinterpret_cast<float4*>(cp) = v;
                         }
-                    } else {
+                    }
+                    __syncwarp();                        // the next chunk reuses the staging rows
+                } else if (gm < prm.M) {
+                    float* crow = C + gm * prm.N + n0 + c0;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (n0 + c0 + j < prm.N) {
-                                float v = __uint_as_float(r[j]);
-                                if (UPDATE) v = shrink * crow[j] + eta * v;
-                                crow[j] = v;
-                            }
+                    for (int j = 0; j < 32; ++j) {
+                        if (n0 + c0 + j < prm.N) {
+                            float v = __uint_as_float(r[j]);
+                            if (UPDATE) v = shrink * crow[j] + eta * v;
+                            crow[j] = v;
                         }
                     }
                 }
