@@ -92,9 +92,11 @@ __global__ void __launch_bounds__(256) inject_additive_kernel(const __grid_const
         if (!hit) continue;
         const unsigned long long r = draw(nd.k_mag, (unsigned long long)l);
         const int k = -4 + (int)((r >> 53) % 12ULL);
-        const double f = (double)(r & ((1ULL << 52) - 1ULL)) * (1.0 / 4503599627370496.0);   // 2^-52
-        double mag = ldexp(1.0 + f, k) * prm.scale;
-        if ((r >> 52) & 1ULL) mag = -mag;
+        // (1 + f) 2^k with f = the low 52 bits of r as a fraction: those bits are the mantissa, k the
+        // exponent, bit 52 the sign
+        const unsigned long long bits = (((r >> 52) & 1ULL) << 63) | ((unsigned long long)(1023 + k) << 52) |
+                                        (r & ((1ULL << 52) - 1ULL));
+        const double mag = __longlong_as_double((long long)bits) * prm.scale;
         out[l] = (T)((double)out[l] + mag);
     }
 }
