@@ -20,15 +20,24 @@ independent (MDS property), for |A| <= P-Q-1 and an error matrix of full row ran
 (probability 1 under Error Model 2) the column space of Sigma equals span(H_A) and
 no other column of H lies in it, so A = {p : H_p in range(Sigma)}.
 
-Readings where the paper is silent: the zero tolerances; non-finite values and
-caller-declared erasures are replaced by zero and their node flagged up front (an
-erasure is an error of known location and counts against the P-Q-1 budget); a
-rank-deficient error matrix makes the subspace form declare a decoding failure.
+When the error matrix is rank deficient (errors of several nodes confined to fewer
+codewords than nodes, e.g. two bit flips at one output position) fewer columns of H
+lie in range(Sigma) than its rank; those that do still belong to A, so the subspace
+form then falls back to Algorithm 1's search restricted to supersets of them, by
+increasing size, as long as the number of supports tried stays within
+``MAX_FALLBACK_SUPPORTS``.
+
+Readings where the paper is silent: the zero tolerances; non-finite values, values of
+magnitude >= ``HUGE`` (their squares leave the FP64 range, so no norm test can be
+applied to them) and caller-declared erasures are replaced by zero and their node
+flagged up front (an erasure is an error of known location and counts against the
+P-Q-1 budget); the bound on the fallback search.
 """
 
 from __future__ import annotations
 
 import itertools
+import math
 from dataclasses import dataclass, field
 from typing import List, Optional, Sequence
 
@@ -37,6 +46,8 @@ import numpy as np
 from .code import parity_check
 
 NO_ERROR, CORRECTED, DECODE_FAILURE = 0, 1, 2
+HUGE = 2.0 ** 500                 # |value| >= HUGE is handled like a non-finite value
+MAX_FALLBACK_SUPPORTS = 4096      # supports the fallback search of the subspace form may try
 
 
 @dataclass(frozen=True)
@@ -80,7 +91,8 @@ def syndrome_gram(outputs: np.ndarray, H: np.ndarray, tol: Tolerances,
     P = outputs.shape[0]
     Z = np.asarray(outputs, dtype=np.float64).reshape(P, -1).copy()
     er = np.zeros(P, dtype=bool) if erased is None else np.asarray(erased, dtype=bool)
-    finite = np.isfinite(Z)
+    with np.errstate(invalid="ignore"):
+        finite = np.abs(Z) < HUGE     # False for NaN, Inf and for values whose square overflows
     forced = er | ~finite.all(axis=1)
     Z[~finite] = 0.0          # a non-finite value is replaced by zero, its node flagged
     Z[er, :] = 0.0            # an erased node contributes nothing
@@ -130,6 +142,32 @@ def locate_exhaustive(outputs: np.ndarray, points: np.ndarray, Q: int, tol: Tole
     return LocateResult(DECODE_FAILURE, flagged, n_active, 0, 0.0, forced)
 
 
+def _superset_search(G: np.ndarray, H: np.ndarray, base: np.ndarray, budget: int, n_active: int,
+                     rank: int, tol: Tolerances, forced: np.ndarray) -> LocateResult:
+    """Algorithm 1's search over the supports that contain ``base`` (nodes already known to be
+    erroneous): sizes in increasing order, lexicographic within a size, the first support whose
+    residual passes is taken.  A size is searched only while the running number of supports
+    stays within MAX_FALLBACK_SUPPORTS; otherwise a decoding failure is declared."""
+    P = H.shape[1]
+    base_idx = [int(p) for p in np.flatnonzero(base)]
+    free = [p for p in range(P) if not base[p]]
+    limit = tol.tau_col ** 2 * max(n_active, 1)
+    tried = 0
+    for size in range(len(base_idx), budget + 1):
+        extra_n = size - len(base_idx)
+        tried += math.comb(len(free), extra_n)
+        if tried > MAX_FALLBACK_SUPPORTS:
+            break
+        for extra in itertools.combinations(free, extra_n):
+            nodes = sorted(base_idx + list(extra))
+            r = _residual(G, H, nodes)
+            if r <= limit:
+                flagged = np.zeros(P, dtype=bool)
+                flagged[nodes] = True
+                return LocateResult(CORRECTED, flagged, n_active, rank, r / max(n_active, 1), forced)
+    return LocateResult(DECODE_FAILURE, forced.copy(), n_active, rank, 0.0, forced)
+
+
 def locate_subspace(outputs: np.ndarray, points: np.ndarray, Q: int, tol: Tolerances,
                     erased: Optional[Sequence[bool]] = None) -> LocateResult:
     """Polynomial-time form: eigen-decompose the syndrome Gram matrix, read the support off
@@ -156,9 +194,9 @@ def locate_subspace(outputs: np.ndarray, points: np.ndarray, Q: int, tol: Tolera
         resid = H - Ur @ (Ur.T @ H)                        # component of each H_p outside range(G)
         dist = np.linalg.norm(resid, axis=0) / np.linalg.norm(H, axis=0)
         inside = dist <= tol.tau_in
-        if int(inside.sum()) != rank:                      # rank-deficient or ambiguous pattern
-            return LocateResult(DECODE_FAILURE, forced.copy(), n_active, rank, 0.0, forced)
         flagged |= inside
+        if int(inside.sum()) != rank:                      # rank-deficient error matrix
+            return _superset_search(G, H, flagged, budget, n_active, rank, tol, forced)
     if flagged.sum() > budget:
         return LocateResult(DECODE_FAILURE, forced.copy(), n_active, rank, 0.0, forced)
     r = _residual(G, H, np.flatnonzero(flagged))

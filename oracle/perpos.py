@@ -16,7 +16,8 @@ the error values are the least-squares solution of H_A e_A = H z, and they are s
 
 Readings where the paper is silent: the zero tolerance (the same relative test as locate.py,
 ||r||^2 <= tau_col^2 ||z||^2 with r the syndrome, resp. the part of it outside span(H_A)); a
-position holding a non-finite value is reported as failed and left untouched; a position that no
+position holding a non-finite value, or one of magnitude >= 2^500 (its square leaves the FP64 range),
+is reported as failed and left untouched; a position that no
 support of size <= t explains is reported as failed and left untouched.
 """
 
@@ -28,7 +29,7 @@ from dataclasses import dataclass
 import numpy as np
 
 from .code import parity_check
-from .locate import CORRECTED, DECODE_FAILURE, NO_ERROR, Tolerances
+from .locate import CORRECTED, DECODE_FAILURE, HUGE, NO_ERROR, Tolerances
 
 
 @dataclass
@@ -51,7 +52,8 @@ def correct_positions(outputs: np.ndarray, points: np.ndarray, Q: int, tol: Tole
     H = parity_check(np.asarray(points, dtype=np.float64), Q)        # [R, P], orthonormal rows
     R = H.shape[0]
     t = R // 2
-    finite = np.isfinite(Z).all(axis=0)
+    with np.errstate(invalid="ignore"):
+        finite = (np.abs(Z) < HUGE).all(axis=0)   # NaN, Inf and values whose square overflows FP64
     Zf = np.where(finite[None, :], Z, 0.0)
     S = H @ Zf                                                        # syndromes, one column per position
     z2 = (Zf ** 2).sum(axis=0)

@@ -38,6 +38,25 @@ def test_worked_example_printed_numbers():
     assert m * (2 * n - 1) * d == g["unaligned_coefficients"][0]
 
 
+def test_chebyshev_points_are_the_roots_of_T_P():
+    """Evaluation points of the workloads: the P roots of the first-kind Chebyshev polynomial,
+    in decreasing order (closed forms for P = 1, 2, 3; T_P(b_p) = 0 through numpy's Chebyshev
+    series evaluation; the extrema of T_P, the second-kind points, would fail every line)."""
+    assert np.allclose(chebyshev_points(1), [0.0], atol=1e-16)
+    assert np.allclose(chebyshev_points(2), [np.sqrt(0.5), -np.sqrt(0.5)], rtol=0, atol=1e-15)
+    assert np.allclose(chebyshev_points(3), [np.sqrt(3) / 2, 0.0, -np.sqrt(3) / 2], rtol=0, atol=1e-15)
+    for P in (2, 3, 10, 11, 13, 25, 36, 40, 64):
+        b = chebyshev_points(P)
+        assert b.shape == (P,) and np.all(np.diff(b) < 0) and np.all(np.abs(b) < 1)
+        T_P = np.zeros(P + 1)
+        T_P[P] = 1.0
+        assert np.abs(np.polynomial.chebyshev.chebval(b, T_P)).max() < 1e-13 * P
+        assert np.allclose(b, -b[::-1], rtol=0, atol=1e-15)          # symmetric about zero
+        # the P roots of the degree-P monic polynomial 2^(1-P) T_P: their product is its constant term
+        if P % 2 == 0:
+            assert np.isclose(np.prod(b), (-1) ** (P // 2) * 2.0 ** (1 - P), rtol=1e-12)
+
+
 def test_printed_thresholds():
     for line in open(os.path.join(GOLDEN, "printed_thresholds.txt")):
         line = line.split("#")[0].strip()

@@ -70,9 +70,9 @@ def test_detection_for_any_number_of_errors():
 
 
 def test_adversarial_bound_single_codeword():
-    """One codeword (L = 1): floor((P-Q)/2) errors of arbitrary value are located by the exhaustive
-    form (adversarial-model lemma); the subspace form needs a full-rank error matrix and must
-    fall back to a declared failure rather than a wrong answer."""
+    """One codeword (L = 1): floor((P-Q)/2) errors of arbitrary value are located (adversarial-model
+    lemma).  The error matrix then has rank 1 < number of errors, so the subspace form finds no
+    column of H in the syndrome's range and must get there through its superset search."""
     P, Q = 9, 5
     Z0, b = _codewords(P, Q, 1, seed=4)
     for nodes in [(0, 5), (2, 3), (7, 8)]:
@@ -81,13 +81,107 @@ def test_adversarial_bound_single_codeword():
         ex = locate_exhaustive(Z, b, Q, TOL_FP64)
         assert ex.outcome == CORRECTED and sorted(np.flatnonzero(ex.flagged)) == list(nodes)
         sb = locate_subspace(Z, b, Q, TOL_FP64)
-        assert sb.outcome == DECODE_FAILURE
+        assert sb.outcome == CORRECTED and np.array_equal(sb.flagged, ex.flagged) and sb.rank == 1
     # a single error in a single codeword is fine for both
     Z = Z0.copy()
     Z[4, 0] += 0.75
     for fn in (locate_exhaustive, locate_subspace):
         r = fn(Z, b, Q, TOL_FP64)
         assert r.outcome == CORRECTED and list(np.flatnonzero(r.flagged)) == [4]
+
+
+@pytest.mark.parametrize("P,Q,L", [(7, 4, 1), (8, 4, 1), (9, 5, 2), (8, 4, 2)])
+def test_rank_deficient_patterns_subspace_equals_exhaustive(P, Q, L):
+    """Few codewords (L = 1, 2) and every support of size 0..P-Q: the error matrix has rank
+    min(size, L), below the number of erroneous nodes for most patterns.  Theorem 3 (claims 2, 3)
+    holds per codeword, so up to P-Q-1 errors are still corrected, more are a declared failure,
+    and the subspace form (through its superset search) takes the exhaustive form's decision."""
+    Z0, b = _codewords(P, Q, L, seed=7 * P + Q + L)
+    rng = np.random.default_rng(P * 1000 + Q * 10 + L)
+    for size in range(0, P - Q + 1):
+        for nodes in itertools.combinations(range(P), size):
+            Z = Z0.copy()
+            Z[list(nodes), :] += rng.uniform(0.5, 2.0, (size, L)) * rng.choice([-1.0, 1.0], (size, L))
+            ex = locate_exhaustive(Z, b, Q, TOL_FP64)
+            sb = locate_subspace(Z, b, Q, TOL_FP64)
+            assert ex.outcome == sb.outcome, (nodes, ex.outcome, sb.outcome)
+            assert np.array_equal(ex.flagged, sb.flagged), nodes
+            if size == 0:
+                assert ex.outcome == NO_ERROR
+            elif size <= P - Q - 1:
+                assert ex.outcome == CORRECTED and sorted(np.flatnonzero(ex.flagged)) == list(nodes)
+            else:
+                assert ex.outcome == DECODE_FAILURE
+
+
+def test_partly_rank_deficient_pattern_keeps_the_nodes_already_inside():
+    """Three erroneous nodes, two of which err in one codeword only (the same one): rank 2 < 3.  The
+    third node's column of H lies in the syndromes' range and is kept; the search adds the others."""
+    P, Q, L = 12, 6, 40
+    Z0, b = _codewords(P, Q, L, seed=21)
+    Z = _corrupt(Z0, (4,), seed=22)
+    Z[[1, 9], 17] += np.array([3.0, -1.25])
+    for fn in (locate_exhaustive, locate_subspace):
+        r = fn(Z, b, Q, TOL_FP64)
+        assert r.outcome == CORRECTED and list(np.flatnonzero(r.flagged)) == [1, 4, 9]
+    assert locate_subspace(Z, b, Q, TOL_FP64).rank == 2
+
+
+def test_fallback_search_is_bounded():
+    """The superset search gives up (declared failure) once the supports to try exceed the bound:
+    P = 40, one codeword with 6 errors would need C(40,1) + ... + C(40,6) supports."""
+    from oracle.locate import MAX_FALLBACK_SUPPORTS
+    P, Q = 40, 20
+    Z0, b = _codewords(P, Q, 1, seed=23)
+    Z = Z0.copy()
+    Z[[0, 1], 0] += np.array([1.0, 2.0])
+    assert 40 + 780 <= MAX_FALLBACK_SUPPORTS < 40 + 780 + 9880
+    r = locate_subspace(Z, b, Q, TOL_FP64)
+    assert r.outcome == CORRECTED and list(np.flatnonzero(r.flagged)) == [0, 1]
+    Z[[5, 6, 7, 8], 0] += np.array([1.0, -1.0, 2.0, 0.5])
+    assert locate_subspace(Z, b, Q, TOL_FP64).outcome == DECODE_FAILURE
+
+
+def test_values_whose_square_overflows_are_located():
+    """A finite value above about 1e154 has an infinite square; the zero test ||Hz|| <= tau ||z||
+    would compare inf with inf and pass.  Such a value (for instance an FP64 exponent-bit flip:
+    x * 2^1000) is handled like a non-finite one: its node is flagged up front."""
+    P, Q = 10, 6
+    Z0, b = _codewords(P, Q, 20, seed=24)
+    Z = Z0.copy()
+    Z[3, 7] *= 2.0 ** 1000
+    assert np.isfinite(Z).all()
+    for fn in (locate_exhaustive, locate_subspace):
+        r = fn(Z, b, Q, TOL_FP64)
+        assert r.outcome == CORRECTED and list(np.flatnonzero(r.flagged)) == [3] and r.forced[3]
+    Z[5, 2] = -2.0 ** 499.5                                   # still squares inside the FP64 range
+    r = locate_subspace(Z, b, Q, TOL_FP64)
+    assert r.outcome == CORRECTED and list(np.flatnonzero(r.flagged)) == [3, 5] and not r.forced[5]
+    # the flip itself, through the injector's bit arithmetic: bit 62 of a value below 1
+    w = np.array([[0.75]])
+    w.view(np.uint64)[0, 0] ^= np.uint64(1 << 62)
+    assert np.isfinite(w[0, 0]) and abs(w[0, 0]) > 2.0 ** 900
+
+
+def test_bitflip_changes_exactly_one_bit_of_one_entry_per_hit_node():
+    rng = np.random.default_rng(25)
+    for dtype, itype, nbits in ((np.float32, np.uint32, 32), (np.float64, np.uint64, 64)):
+        Z0 = rng.standard_normal((9, 6, 5)).astype(dtype)
+        for seed in range(30):
+            for count in (1, 2, 4, 9, 12):
+                Z = Z0.copy()
+                hit = inj.inject_bitflip(Z, seed, count, scale=1.0)
+                assert hit.sum() == min(count, 9)
+                diff = (Z.view(itype) ^ Z0.view(itype)).reshape(9, -1)
+                for p in range(9):
+                    changed = np.flatnonzero(diff[p])
+                    if not hit[p]:
+                        assert changed.size == 0
+                        continue
+                    assert changed.size == 1                                   # one entry
+                    assert bin(int(diff[p, changed[0]])).count("1") == 1       # one bit
+                    new, old = Z.reshape(9, -1)[p, changed[0]], Z0.reshape(9, -1)[p, changed[0]]
+                    assert (not np.isfinite(new)) or abs(float(new) - float(old)) >= 2.0 ** -6
 
 
 def test_replication_special_case():
@@ -140,12 +234,16 @@ def test_fp32_outputs_clean_floor_and_bitflips():
         assert list(changed) == list(np.flatnonzero(hit))
         r = locate_subspace(Z, b, Q, TOL_FP32)
         e = locate_exhaustive(Z, b, Q, TOL_FP32)
-        assert r.outcome == e.outcome and np.array_equal(r.flagged, e.flagged)
-        if r.outcome == CORRECTED:
-            assert np.array_equal(r.flagged, hit)
-        else:                                                # both flips in the same codeword: rank 1
-            cols = [np.flatnonzero(Z.view(np.uint32)[p] != Z32.view(np.uint32)[p])[0] for p in changed]
-            assert cols[0] == cols[1]
+        assert r.outcome == e.outcome == CORRECTED and np.array_equal(r.flagged, e.flagged)
+        assert np.array_equal(r.flagged, hit)
+    # both flips in the same codeword (rank 1, two erroneous nodes): floor((13-9)/2) = 2 errors in
+    # one codeword are correctable (adversarial-model lemma), through the superset search
+    Z = Z32.copy()
+    Z.view(np.uint32)[2, 100] ^= np.uint32(1 << 27)
+    Z.view(np.uint32)[11, 100] ^= np.uint32(1 << 22)
+    for fn in (locate_exhaustive, locate_subspace):
+        r = fn(Z, b, Q, TOL_FP32)
+        assert r.outcome == CORRECTED and list(np.flatnonzero(r.flagged)) == [2, 11]
 
 
 def test_full_pipeline_with_additive_errors_decodes_correctly():
