@@ -20,6 +20,8 @@ struct GemmParams {
     int update;
     double shrink, eta;
     const gpd_locate_result* gate;
+    int max_threshold;      // largest recovery threshold the result will be decoded with (0: unknown);
+                            // the FP32 tensor-core path shortens its accumulation chains for large ones
 };
 
 gpd_status gemm_generic_launch(const GemmParams& prm, int elem_size, cudaStream_t st);

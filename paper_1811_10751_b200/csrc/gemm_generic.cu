@@ -158,6 +158,7 @@ gpd_status worker_gemm_launch(gpd_plan_s* plan, gpd_product which, const void* W
     } else {
         return GPD_ERR_ARG;
     }
+    prm.max_threshold = plan->prod[which].Q;
     if (prm.N == 1) return gemv_launch(prm, plan->elem_size, st);
     if (plan->elem_size == 8 && dgemm_mma_supported(prm)) return dgemm_mma_launch(prm, st);
     if (plan->elem_size == 4 && sgemm_3xtf32_supported(prm)) return sgemm_3xtf32_launch(prm, st);

@@ -4,8 +4,16 @@
 //     a = a_hi + a_lo (both exactly representable in TF32),   a*b ~ a_lo*b_hi + a_hi*b_lo + a_hi*b_hi.
 //
 // One CTA per SM walks a list of 128 x 128 tiles of the nodes' products (column strips of them for
-// the tiles left over after the last full round over the SMs).  Two accumulators in tensor memory
-// alternate, so a tile's epilogue runs under the next tile's main loop.  Warp roles:
+// the tiles left over after the last full round over the SMs).
+//
+// Accumulation.  The tensor cores add into their FP32 accumulator with truncation, so a long chain
+// of MMAs loses up to one ulp of the running sum per step, always towards zero: over K = 2048
+// (768 steps) that is 1.4e-5 of the output's rms, which a threshold-9 decoder amplifies beyond
+// the 1e-4 bar.  The chain is therefore kept short: tensor memory only holds the partial sum of
+// group_kb k-blocks (one k-block: K = 32, 12 steps); the epilogue warps pull every finished partial sum into
+// FP32 registers, where the groups are added with round-to-nearest, and two accumulators in
+// tensor memory alternate so that one group drains while the next one is being multiplied.
+// Warp roles:
 //   warp 0       : TMA producer (one lane) - raw FP32 tiles of A and B into a 4-stage ring that
 //                  runs on across tiles
 //   warp 1       : allocates tensor memory; one lane issues the MMAs and commits them to mbarriers
@@ -13,8 +21,10 @@
 //                  raw tile, lo goes to a second tile); A row by row into tensor memory (hi and lo, 32
 //                  columns each per stage), from where the MMAs take it: the A operand then costs
 //                  shared-memory bandwidth once (its raw read) instead of four times
-//   warps 10..13 : read a finished accumulator back (tcgen05.ld), hand it back to the MMA warp, and
-//                  write the tile (plain store, or read-modify-write for the coded update)
+//   warps 10..17 : read every finished group's partial sum back (tcgen05.ld; a warp owns one lane
+//                  quarter and one half of the columns), hand the accumulator back to the MMA warp,
+//                  add the partial sums up in registers and write the tile at its end (plain
+//                  store, or read-modify-write for the coded update)
 // Operand tiles use the 128-byte swizzle; A is K-major; B is K-major for the update (X^_p is
 // [N][K]) and MN-major for the forward / backward products (X~_p, W~_p are [K][N]).
 // Tensor memory (512 columns): accumulators in columns 0..255, the A stages behind them.
@@ -33,16 +43,28 @@ constexpr int UMMA_K = 8;
 constexpr int A_TILE_BYTES = BM * BK * 4;            // 16 KB, rows of 128 B
 constexpr int B_TILE_BYTES = BN * BK * 4;            // 16 KB
 constexpr int STAGE_BYTES = A_TILE_BYTES + 2 * B_TILE_BYTES;   // raw A, B hi, B lo
-constexpr int EPI_PITCH = 36;                        // floats per staged row: 16-byte aligned, conflict-free for 16-byte accesses
-constexpr int EPI_STAGE_BYTES = 4 * 32 * EPI_PITCH * 4;   // one 32 x 32 chunk per epilogue warp
+// k-blocks whose products are summed in tensor memory before they move to registers.  Measured error
+// of a product (K = 2048, against an FP64 product of the same shares, relative to the output's rms):
+// 2.8e-7 for groups of one k-block, 4.7e-7 for two, 9.1e-7 for four, 1.8e-6 for eight, 1.4e-5 with no
+// cut at all.  Decoding amplifies it: at threshold 9 the worst threshold-sized subset of 11 nodes
+// turns 2.8e-7 into 2.7e-5 of relative Frobenius error (an ideal FP32 product: 2e-5).  Products
+// decoded with a threshold of 7 or more use groups of one k-block, smaller thresholds two.  The
+// update contracts over the mini-batch only and its result is a small increment of the share, so
+// one chain of up to 256 elements is accurate enough there and keeps a whole tile of lead for the
+// read-modify-write.
+constexpr int kGroupKbProduct = 2, kGroupKbProductLarge = 1, kGroupKbUpdate = 8;
+constexpr int kEpiWarps = 8;                         // warps 10..17: lane quarter = warp mod 4, column half = (warp - 10) / 4
+constexpr int EPI_COLS = 16;                         // columns of a staged chunk
+constexpr int EPI_PITCH = 20;                        // floats per staged row: 16-byte aligned, conflict-free for 16-byte accesses
+constexpr int EPI_STAGE_BYTES = kEpiWarps * 32 * EPI_PITCH * 4;   // one 32 x 16 chunk per epilogue warp
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_STAGE_BYTES + 1024;
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr int TMEM_ACC_COLS = 2 * BN;                // two 128-column accumulators: one fills while the other drains
 constexpr int TMEM_A_COLS = 2 * BK;                  // per stage: A hi (BK columns), A lo (BK columns); lane = row of the tile
 constexpr int TMEM_COLS = 512;
 static_assert(TMEM_ACC_COLS + STAGES * TMEM_A_COLS <= TMEM_COLS, "tensor memory budget");
 constexpr int kConvWarps = 8;                        // warps 2..9: split tiles
 constexpr int kConvThreads = kConvWarps * 32;
-constexpr int kEpiWarps = 4;                         // warps 10..13: drain tensor memory, one per lane quarter
 constexpr int kThreads = 64 + kConvThreads + kEpiWarps * 32;
 constexpr long long kWaitCycles = 2000000000LL;      // about one second
 
@@ -137,7 +159,7 @@ __device__ __forceinline__ float trunc_tf32(float x) { return __uint_as_float(__
 template <bool B_KMAJOR, bool UPDATE>
 __global__ void __launch_bounds__(kThreads, 1)
 sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams prm,
-                    int tiles_m, int tiles_n, int full_tiles, int split, int n_virtual) {
+                    int tiles_m, int tiles_n, int full_tiles, int split, int n_virtual, int group_kb) {
     if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -227,19 +249,21 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            int it = 0, ti = 0;
+            int it = 0, gi = 0;                   // k-blocks / accumulation groups issued so far, over all tiles
             bool ok = true;
-            for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x, ++ti) {
+            for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
                 int p, m0, n0, bn;
                 decode(vt, p, m0, n0, bn);
-                const int buf = ti & 1;
-                // the tile before last used this accumulator: it must have been read back
-                if (!mbar_wait(&acc_empty[buf], ((ti >> 1) & 1) ^ 1, abort_p)) { ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
                 const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
                                        ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int buf = gi & 1, kg = kb % group_kb;
+                    if (kg == 0) {
+                        // the group before last used this accumulator: it must have been read back
+                        if (!mbar_wait(&acc_empty[buf], ((gi >> 1) & 1) ^ 1, abort_p)) { ok = false; break; }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    }
+                    const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(&conv_bar[s], ph, abort_p)) { ok = false; break; }
@@ -258,14 +282,17 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         // k-rows are 8 * 128 bytes further in every 32-column chunk
                         const uint32_t a_off = k * UMMA_K;
                         const uint64_t b_off = (uint64_t)((B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128) >> 4);
-                        const uint32_t first = (kb > 0 || k > 0) ? 1u : 0u;
+                        const uint32_t first = (kg > 0 || k > 0) ? 1u : 0u;    // a group starts from zero
                         umma_tf32_ta(tmem_d, a_lo + a_off, db_hi0 + b_off, idesc, first);   // small terms first
                         umma_tf32_ta(tmem_d, a_hi + a_off, db_lo0 + b_off, idesc, 1u);
                         umma_tf32_ta(tmem_d, a_hi + a_off, db_hi0 + b_off, idesc, 1u);
                     }
                     umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
+                    if (kg == group_kb - 1 || kb == num_kb - 1) {
+                        umma_commit(&acc_full[buf]); // this group's partial sum complete
+                        ++gi;
+                    }
                 }
-                if (ok) umma_commit(&acc_full[buf]); // this tile's accumulator complete
             }
         }
     } else if (warp < 2 + kConvWarps) {
@@ -324,83 +351,96 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
     } else {
         // ------------------------------ epilogue ------------------------------
+        const int ew = warp - (2 + kConvWarps);      // 0..7
         const int q = warp & 3;                      // this warp may touch TMEM lanes 32q .. 32q+31
+        const int ch = (ew >> 2) * (BN / 2);         // first of this warp's 64 columns of the tile
         const float shrink = (float)prm.shrink, eta = (float)prm.eta;
         const bool vec = (prm.N % 4 == 0);
-        int ti = 0;
-        for (int vt = blockIdx.x; vt < n_virtual; vt += gridDim.x, ++ti) {
+        const int n_groups = (num_kb + group_kb - 1) / group_kb;
+        float* st = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES) + ew * (32 * EPI_PITCH);
+        const int col4 = (lane & 3) * 4, rsub = lane >> 2;    // this lane's part of a staged 32 x 16 chunk
+        int gi = 0;
+        bool ok = true;
+        for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
             int p, m0, n0, bn;
             decode(vt, p, m0, n0, bn);
-            const int buf = ti & 1;
-            const bool acc_ready = mbar_wait(&acc_full[buf], (ti >> 1) & 1, abort_p);
-            __syncwarp();
-            if (!__all_sync(0xffffffffu, acc_ready)) break;   // tcgen05.ld is warp-collective: all lanes or none
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int64_t gm = (int64_t)m0 + q * 32 + lane;
-            float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
-#pragma unroll 1
-            for (int c0 = 0; c0 < bn; c0 += 32) {
-                const bool whole = vec && n0 + c0 + 32 <= prm.N;     // the chunk leaves as 128-byte row segments
-                const int col4 = (lane & 7) * 4, rsub = lane >> 3;   // this lane's part of a staged chunk
-                float4 old[8];                                       // the stored share, asked for before the accumulator is read
-                if (UPDATE && whole) {
+            float acc[BN / 2];                       // this thread's row, this warp's columns
+            for (int g = 0; g < n_groups; ++g, ++gi) {
+                const int buf = gi & 1;
+                const bool acc_ready = mbar_wait(&acc_full[buf], (gi >> 1) & 1, abort_p);
+                __syncwarp();
+                if (!__all_sync(0xffffffffu, acc_ready)) { ok = false; break; }   // tcgen05.ld is warp-collective: all lanes or none
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const int64_t grow = (int64_t)m0 + q * 32 + 4 * i + rsub;
-                        old[i] = grow < prm.M ? *reinterpret_cast<const float4*>(C + grow * prm.N + n0 + c0 + col4)
-                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int c = 0; c < BN / 2; c += 16) {
+                    if (ch + c < bn) {               // strips are 64 or 32 columns wide
+                        uint32_t r[16];
+                        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + ch + c);
+                        asm volatile(
+                            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                              "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                            : "r"(taddr));
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            acc[c + j] = g == 0 ? __uint_as_float(r[j]) : acc[c + j] + __uint_as_float(r[j]);
                     }
                 }
-                uint32_t r[32];
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0);
-                asm volatile(
-                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                    : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                      "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                      "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                      "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                    : "r"(taddr));
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (c0 + 32 >= bn) {                 // last read of this accumulator: hand it back
-                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
-                }
+                // this group's partial sum is in registers: hand the accumulator back
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            }
+            if (!ok) break;
+            const int64_t gm = (int64_t)m0 + q * 32 + lane;
+            float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
+#pragma unroll
+            for (int c0 = 0; c0 < BN / 2; c0 += EPI_COLS) {
+                if (ch + c0 >= bn) break;
+                const int64_t gc = (int64_t)n0 + ch + c0;           // first global column of the chunk
+                const bool whole = vec && gc + EPI_COLS <= prm.N;
                 if (whole) {
-                    // A thread holds 32 columns of one row; written as they are, a store would touch 32
-                    // rows with 16 bytes each.  The chunk goes through shared memory instead and
-                    // leaves as whole 128-byte row segments (eight lanes per row, four rows per store).
-                    float* st = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES) + (warp - 2 - kConvWarps) * (32 * EPI_PITCH);
+                    // A thread holds the columns of one row; written as they are, a store would touch 32
+                    // rows with 16 bytes each.  A 32 x 16 chunk goes through shared memory instead and
+                    // leaves as 64-byte row segments (four lanes per row, eight rows per store).  The
+                    // update asks for the stored share before it stages the chunk.
+                    float4 old[4];
+                    if (UPDATE) {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4)
+                        for (int i = 0; i < 4; ++i) {
+                            const int64_t grow = (int64_t)m0 + q * 32 + 8 * i + rsub;
+                            old[i] = grow < prm.M ? *reinterpret_cast<const float4*>(C + grow * prm.N + gc + col4)
+                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < EPI_COLS; j += 4)
                         *reinterpret_cast<float4*>(st + lane * EPI_PITCH + j) =
-                            make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                                        __uint_as_float(r[j + 3]));
+                            make_float4(acc[c0 + j], acc[c0 + j + 1], acc[c0 + j + 2], acc[c0 + j + 3]);
                     __syncwarp();
 #pragma unroll
-                    for (int rr = 0; rr < 32; rr += 4) {
-                        const int row = rr + rsub;
+                    for (int i = 0; i < 4; ++i) {
+                        const int row = 8 * i + rsub;
                         const int64_t grow = (int64_t)m0 + q * 32 + row;
                         float4 v = *reinterpret_cast<const float4*>(st + row * EPI_PITCH + col4);
                         if (grow < prm.M) {
-                            float* cp = C + grow * prm.N + n0 + c0 + col4;
                             if (UPDATE) {
-                                const float4 o = old[rr / 4];
+                                const float4 o = old[i];
                                 v.x = shrink * o.x + eta * v.x; v.y = shrink * o.y + eta * v.y;
                                 v.z = shrink * o.z + eta * v.z; v.w = shrink * o.w + eta * v.w;
                             }
-                            *reinterpret_cast<float4*>(cp) = v;
+                            *reinterpret_cast<float4*>(C + grow * prm.N + gc + col4) = v;
                         }
                     }
                     __syncwarp();                        // the next chunk reuses the staging rows
                 } else if (gm < prm.M) {
-                    float* crow = C + gm * prm.N + n0 + c0;
+                    float* crow = C + gm * prm.N + gc;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        if (n0 + c0 + j < prm.N) {
-                            float v = __uint_as_float(r[j]);
+                    for (int j = 0; j < EPI_COLS; ++j) {
+                        if (gc + j < prm.N) {
+                            float v = acc[c0 + j];
                             if (UPDATE) v = shrink * crow[j] + eta * v;
                             crow[j] = v;
                         }
@@ -485,8 +525,9 @@ gpd_status launch(const GemmParams& prm, cudaStream_t st) {
     const int full_tiles = (int)(tiles - (split > 1 ? rem : 0));
     const int64_t n_virtual = full_tiles + (int64_t)(split > 1 ? rem : 0) * split;
     const unsigned grid = (unsigned)std::min<int64_t>(n_virtual, sms);   // persistent: one CTA per SM walks the list
+    const int group_kb = UPDATE ? kGroupKbUpdate : (prm.max_threshold >= 7 ? kGroupKbProductLarge : kGroupKbProduct);
     sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<grid, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n, full_tiles,
-                                                                              split, (int)n_virtual);
+                                                                              split, (int)n_virtual, group_kb);
     return launch_ok();
 }
 

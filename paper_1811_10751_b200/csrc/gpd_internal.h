@@ -24,6 +24,11 @@ constexpr double kTauInFp32 = 3.0517578125e-5;           // 2^-15
 constexpr double kTauColFp64 = 9.5367431640625e-7;       // 2^-20
 constexpr double kTauInFp64 = 9.313225746154785e-10;     // 2^-30
 
+// A worker output of magnitude >= kHuge is handled like a non-finite one (zeroed, its node flagged):
+// the squared norms of the zero test stay inside the FP64 range for up to 64 values below it.
+constexpr double kHuge = 3.273390607896142e150;          // 2^500
+constexpr double kHugeSquared = 1.0715086071862673e301;  // 2^1000
+
 // Geometry of one decodable product (forward, backward or audit).
 struct ProductInfo {
     int Q = 0;             // recovery threshold = number of polynomial coefficients

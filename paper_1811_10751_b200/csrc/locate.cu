@@ -13,8 +13,10 @@
 // support is the set of nodes whose parity-check column H_p lies in the span of the top-rho
 // eigenvectors (any P-Q columns of H are independent, so for at most P-Q-1 erroneous nodes no
 // other column does); the support is verified by the syndrome energy left outside span(H_A).
-// More than P-Q-1 nodes, a rank-deficient error matrix or an ambiguous geometry end in a
-// declared decoding failure (Theorem 3, third claim).
+// A rank-deficient error matrix (fewer columns of H in that span than its rank) is handled by
+// Algorithm 1's search over the supersets of the columns found, bounded in the number of supports.
+// More than P-Q-1 nodes or an ambiguous geometry end in a declared decoding failure (Theorem 3,
+// third claim).
 #include "gpd_internal.h"
 
 namespace gpd {
@@ -22,6 +24,7 @@ namespace gpd {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr long long kMaxFallbackSupports = 4096;   // supports the superset search of the finish kernel may try
 
 struct SyndromeParams {
     const void* Z;              // [P][L]
@@ -41,9 +44,10 @@ __device__ __forceinline__ void dmma_m8n8k4(double& d0, double& d1, double a, do
 }
 
 // Syndrome s = H z and squared norm of one codeword: P loads at stride L, issued in equal groups of up to nine.
-// CHECKED = false is the plain form: no per-value tests, a non-finite value shows up as a non-finite
-// norm and the caller repeats the codeword with CHECKED = true, which zeroes non-finite values
-// and erased nodes and records the nodes that held a non-finite value.
+// CHECKED = false is the plain form: no per-value tests; a non-finite value, or one of magnitude
+// >= kHuge (its square would leave the FP64 range and turn the zero test into inf > inf), shows up
+// as a norm >= kHugeSquared and the caller repeats the codeword with CHECKED = true, which zeroes
+// such values and erased nodes and records the nodes that held one.
 template <typename T, int RT, bool CHECKED>
 __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P, const double* sH,
                                                   unsigned long long erased, double (&s)[RT], double& nz,
@@ -54,7 +58,7 @@ __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P,
     nz = 0.0;
     auto absorb = [&](double zz, int pnode, const double* hcol) {
         if (CHECKED) {
-            if (!isfinite(zz)) { bad |= 1ULL << pnode; zz = 0.0; }
+            if (!(fabs(zz) < kHuge)) { bad |= 1ULL << pnode; zz = 0.0; }   // NaN, Inf, or a square outside the FP64 range
             if ((erased >> pnode) & 1ULL) zz = 0.0;
         }
         nz = fma(zz, zz, nz);
@@ -115,7 +119,7 @@ __global__ void __launch_bounds__(kThreads, RT <= 8 ? 4 : (RT <= 24 ? 2 : 1)) sy
         double nz = 0.0;
         if (l < prm.L) {
             if (prm.erased == 0ULL) codeword_syndrome<T, RT, false>(Z + l, prm.L, prm.P, sH, 0ULL, s, nz, bad_all);
-            if (prm.erased != 0ULL || !isfinite(nz))
+            if (prm.erased != 0ULL || !(nz < kHugeSquared))
                 codeword_syndrome<T, RT, true>(Z + l, prm.L, prm.P, sH, prm.erased, s, nz, bad_all);
         } else {
 #pragma unroll
@@ -185,8 +189,8 @@ struct FinishParams {
 // Shared memory of the finish kernel for R parity checks and P nodes (doubles first, then ints, bytes).
 __host__ __device__ inline size_t finish_smem_bytes(int R, int P) {
     const int ld = R | 1;
-    return sizeof(double) * ((size_t)5 * R * ld + (size_t)R * P + (size_t)R + 2 * (size_t)(R + 1) + (size_t)P) +
-           sizeof(int) * ((size_t)(R + 1) + (size_t)R) + (size_t)P;
+    return sizeof(double) * ((size_t)5 * R * ld + 2 * (size_t)R * P + (size_t)R + 2 * (size_t)(R + 1) + (size_t)P) +
+           sizeof(int) * ((size_t)(R + 1) + (size_t)R + (size_t)P + (size_t)R) + (size_t)P;
 }
 
 // One warp.  The Gram matrix G of the failing codewords has rank = number of erroneous nodes (a
@@ -205,13 +209,16 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     double* Wv = M + R * ld;                 // [R][ld] eigenvectors of L^T L in columns
     double* U = Wv + R * ld;                 // [R][ld] orthonormal basis of the retained subspace in columns
     double* Hs = U + R * ld;                 // [R][P]
-    double* lam = Hs + R * P;                // [R]
+    double* Hp = Hs + R * P;                 // [R][P] fallback search: H with span(H_base) projected out
+    double* lam = Hp + R * P;                // [R]
     double* rot_c = lam + R;                 // [R + 1] per index: row_i <- c row_i + s row_partner
     double* rot_s = rot_c + (R + 1);         // [R + 1]
     double* dist = rot_s + (R + 1);          // [P]
     int* partner = reinterpret_cast<int*>(dist + P);   // [R + 1]
     int* order = partner + (R + 1);          // [R]
-    unsigned char* inside = reinterpret_cast<unsigned char*>(order + R);   // [P]
+    int* free_nodes = order + R;             // [P] fallback search: nodes outside the base set, increasing
+    int* comb = free_nodes + P;              // [R] fallback search: current combination (indices into free_nodes)
+    unsigned char* inside = reinterpret_cast<unsigned char*>(comb + R);   // [P]
     gpd_locate_result* res = prm.result;
     const unsigned long long n_active = prm.counts[0];
     const unsigned long long forced = prm.counts[1] | prm.erased;
@@ -437,8 +444,140 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
         }
         if (lane == 0) { res->max_inside = max_in; res->min_outside = min_out; }
         if (n_inside != rank) {
-            if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
-            return;
+            // Rank-deficient error matrix (errors of several nodes confined to fewer codewords than
+            // nodes): fewer columns of H lie in the syndromes' range than its rank.  Those that do
+            // are erroneous all the same, so Algorithm 1's search is run over the supports that
+            // contain them: by increasing size, lexicographic within a size, the first support
+            // that leaves no syndrome energy outside its span is taken.  A size is only searched
+            // while the running number of supports stays within kMaxFallbackSupports.
+            const int nb = __popcll(flagged);
+            bool found = false;
+            if (nb <= budget) {
+                const double limit_fb = prm.tau2 * (double)n_active;
+                // orthonormal basis of span(H_base) in the columns of M (twice-applied Gram-Schmidt)
+                int na0 = 0;
+                for (int p = 0; p < P; ++p) {
+                    if (!((flagged >> p) & 1ULL)) continue;
+                    double v = lane < R ? Hs[lane * P + p] : 0.0;
+                    for (int pass = 0; pass < 2; ++pass)
+                        for (int e = 0; e < na0; ++e) {
+                            const double qe = lane < R ? M[lane * ld + e] : 0.0;
+                            double part = qe * v;
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                            v -= part * qe;
+                        }
+                    double nn = v * v;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(0xffffffffu, nn, o);
+                    if (lane < R) M[lane * ld + na0] = v * rsqrt(nn);
+                    __syncwarp();
+                    ++na0;
+                }
+                // A <- (I - Pi_base) L (column k of the Cholesky factor, lane = row); Hp <- (I - Pi_base) H
+                double base_res = 0.0;
+                for (int k = 0; k < nl; ++k) {
+                    double v = lane < R ? Lm[lane * ld + k] : 0.0;
+                    for (int pass = 0; pass < 2; ++pass)
+                        for (int e = 0; e < na0; ++e) {
+                            const double qe = lane < R ? M[lane * ld + e] : 0.0;
+                            double part = qe * v;
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                            v -= part * qe;
+                        }
+                    if (lane < R) A[lane * ld + k] = v;
+                    base_res = fma(v, v, base_res);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) base_res += __shfl_xor_sync(0xffffffffu, base_res, o);
+                int n_free = 0;
+                for (int p = 0; p < P; ++p) {
+                    if ((flagged >> p) & 1ULL) continue;
+                    double v = lane < R ? Hs[lane * P + p] : 0.0;
+                    for (int pass = 0; pass < 2; ++pass)
+                        for (int e = 0; e < na0; ++e) {
+                            const double qe = lane < R ? M[lane * ld + e] : 0.0;
+                            double part = qe * v;
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                            v -= part * qe;
+                        }
+                    if (lane < R) Hp[lane * P + p] = v;
+                    if (lane == 0) free_nodes[n_free] = p;
+                    ++n_free;
+                }
+                __syncwarp();
+                long long tried = 1;                                     // the base set itself
+                if (base_res + remainder <= limit_fb) found = true;
+                for (int ex = 1; !found && nb + ex <= budget && ex <= n_free; ++ex) {
+                    // number of supports of this size: C(n_free, ex), computed exactly while it stays small
+                    long long cnt = 1;
+                    for (int i = 1; i <= ex; ++i) {
+                        cnt = cnt * (n_free - ex + i) / i;
+                        if (cnt > 4LL * kMaxFallbackSupports * 64) break;   // far beyond the bound: stop before it can overflow
+                    }
+                    tried += cnt;
+                    if (tried > kMaxFallbackSupports) break;
+                    if (lane < ex) comb[lane] = lane;
+                    __syncwarp();
+                    int redo = 0;                                        // columns U[.][redo ..] must be rebuilt
+                    while (true) {
+                        // orthonormalise the projected columns of this combination (columns of U)
+                        for (int j = redo; j < ex; ++j) {
+                            double v = lane < R ? Hp[lane * P + free_nodes[comb[j]]] : 0.0;
+                            for (int pass = 0; pass < 2; ++pass)
+                                for (int e = 0; e < j; ++e) {
+                                    const double qe = lane < R ? U[lane * ld + e] : 0.0;
+                                    double part = qe * v;
+#pragma unroll
+                                    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                                    v -= part * qe;
+                                }
+                            double nn = v * v;
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) nn += __shfl_xor_sync(0xffffffffu, nn, o);
+                            if (lane < R) U[lane * ld + j] = nn > 0.0 ? v * rsqrt(nn) : 0.0;
+                            __syncwarp();
+                        }
+                        // syndrome energy outside span(H_base, H_combination)
+                        double rr = 0.0;
+                        for (int k = 0; k < nl; ++k) {
+                            double v = lane < R ? A[lane * ld + k] : 0.0;
+                            for (int e = 0; e < ex; ++e) {
+                                const double qe = lane < R ? U[lane * ld + e] : 0.0;
+                                double part = qe * v;
+#pragma unroll
+                                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+                                v -= part * qe;
+                            }
+                            rr = fma(v, v, rr);
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) rr += __shfl_xor_sync(0xffffffffu, rr, o);
+                        if (rr + remainder <= limit_fb) {
+                            for (int j = 0; j < ex; ++j) flagged |= 1ULL << free_nodes[comb[j]];
+                            found = true;
+                            break;
+                        }
+                        // next combination in lexicographic order (every lane takes the same steps)
+                        int j = ex - 1;
+                        while (j >= 0 && comb[j] == n_free - ex + j) --j;
+                        if (j < 0) break;
+                        __syncwarp();
+                        if (lane == 0) {
+                            ++comb[j];
+                            for (int i = j + 1; i < ex; ++i) comb[i] = comb[i - 1] + 1;
+                        }
+                        redo = j;
+                        __syncwarp();
+                    }
+                }
+            }
+            if (!found) {
+                if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
+                return;
+            }
         }
     }
     const int n_flagged = __popcll(flagged);

@@ -76,9 +76,9 @@ __global__ void __launch_bounds__(256, RT <= 8 ? 4 : 1) position_scan_kernel(Pos
                     }
                 }
             }
-            if (!isfinite(z2)) {                  // rare: a non-finite value, or finite ones whose squares overflow
+            if (!(z2 < kHugeSquared)) {           // rare: a non-finite value, or a finite one whose square leaves the FP64 range
                 zp = Z + pos;
-                for (int p = 0; p < prm.P; ++p, zp += prm.L) finite &= isfinite((double)__ldcs(zp));
+                for (int p = 0; p < prm.P; ++p, zp += prm.L) finite &= fabs((double)__ldcs(zp)) < kHuge;
             }
         }
         double r2 = 0.0;
