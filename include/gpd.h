@@ -18,7 +18,7 @@
  *     errors only.  Data-dependent outcomes (no error / corrected / decoding failure) are
  *     written to a gpd_locate_result in device memory.
  *   - The library allocates device memory only for the plan's small coefficient tables
- *     (uploaded on the plan's first compute call, freed by gpd_plan_destroy).
+ *     (uploaded by gpd_plan_upload or on the plan's first compute call, freed by gpd_plan_destroy).
  *   - Storage type of shares and worker outputs: float (GPD_PREC_FP32) or double
  *     (GPD_PREC_FP64); inputs W, X, Delta and decoded results are always float.
  *   - A plan is immutable after creation; concurrent calls on different streams need distinct
@@ -104,7 +104,7 @@ typedef enum {
     GPD_INJECT_GAUSS = 2        /* selected nodes: scale * N(0,1) added to every entry (Error Model 2) */
 } gpd_inject_mode;
 
-/* Garbage-alignment substitution (Section VI, "we use one of the substitutions ..."; Tables I, III). */
+/* Garbage-alignment substitution (Section VI; Tables I, III; proofs of Theorems 4 and 6). */
 typedef enum {
     GPD_SUBST_U_EQ_VN = 0,      /* u = v^n, w = v^(mn): Q_f = mn d1 + n - 1,      Q_b = mn d2 + mn - n  */
     GPD_SUBST_V_EQ_UM = 1       /* v = u^m, w = u^(mn): Q_f = mn d1 + mn - m,     Q_b = mn d2 + m - 1   */
@@ -166,7 +166,8 @@ typedef enum {
     GPD_Q_STEP_WORKSPACE_BYTES = 12, /* bytes of workspace for coded_layer_step       */
     GPD_Q_PRECISION = 13,       /* resolved gpd_precision                            */
     GPD_Q_NODES = 14,
-    GPD_Q_POSITION_WORKSPACE_BYTES = 15 /* bytes of workspace for gpd_correct_positions (any product) */
+    GPD_Q_POSITION_WORKSPACE_BYTES = 15, /* bytes of workspace for gpd_correct_positions (any product) */
+    GPD_Q_TABLES_ON_DEVICE = 16 /* 1 once the plan's tables have been uploaded (device memory allocated), else 0 */
 } gpd_query;
 
 /* Host tables a test may read back with gpd_plan_table. */
@@ -187,7 +188,10 @@ const char* gpd_status_string(gpd_status s);
  * points; Section V-A: parity-check matrix H with H G^T = 0 for the Vandermonde generator).
  * points_host: P distinct finite doubles, or NULL for the roots of the first-kind Chebyshev
  * polynomial T_P on [-1,1].  Host only: needs no GPU.  Errors: GPD_ERR_SHAPE, GPD_ERR_POINTS,
- * GPD_ERR_P_TOO_SMALL (P below max(Q_f, Q_b)), GPD_ERR_Q_TOO_LARGE.
+ * GPD_ERR_P_TOO_SMALL (P below the forward threshold Q_f), GPD_ERR_Q_TOO_LARGE.
+ * A plan with Q_f <= P < Q_b (or a backward threshold above GPD_MAX_THRESHOLD) is a forward-only
+ * plan: every call on its backward product returns GPD_ERR_P_TOO_SMALL, and coded_layer_step
+ * checks that before it enqueues anything.  GPD_Q_THRESHOLD_BWD still reports Q_b.
  */
 gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, int32_t P,
                     const double* points_host, gpd_precision precision, gpd_plan_t* out);
@@ -197,6 +201,10 @@ gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, int32_t P,
  * u^(mn k + m-1-i), update operands Delta_i at u^i and X_j at u^(m j). */
 gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* split, gpd_substitution subst, int32_t P,
                           const double* points_host, gpd_precision precision, gpd_plan_t* out);
+/* Uploads the plan's coefficient tables to the current device now (one cudaMalloc and one synchronous
+ * copy of a few KB) instead of at the plan's first compute call; a second call does nothing.  Lets a
+ * caller keep allocation and synchronisation out of its timed or captured region. */
+gpd_status gpd_plan_upload(gpd_plan_t plan);
 gpd_status gpd_plan_destroy(gpd_plan_t plan);
 gpd_status gpd_plan_query(gpd_plan_t plan, gpd_query what, int64_t* value);
 /* Copies a host table into host_out (capacity in doubles); *count receives its length. */
@@ -231,6 +239,15 @@ gpd_status gpd_worker_gemm(gpd_plan_t plan, gpd_product which, const void* W_sha
  * synchronises the device, returns that word in *status_host (0, or GPD_ERR_TIMEOUT) and clears it.
  */
 gpd_status gpd_device_status(int32_t* status_host);
+
+/*
+ * gpd_selftest_bounded_wait - exercises the bounded-wait mechanism of the tensor-core kernels without
+ * touching them: one small CTA waits on a hardware barrier that nothing ever arrives at, gives up
+ * after `limit_cycles` clock cycles (clamped to [1e3, 1e8]), raises the same status word and
+ * returns.  Afterwards gpd_device_status reports GPD_ERR_TIMEOUT once, and the context stays usable.
+ * (No counterpart in the paper: a check of this library's failure reporting.)
+ */
+gpd_status gpd_selftest_bounded_wait(int64_t limit_cycles, void* stream);
 
 /*
  * gpd_update_shares — coded update (step O3, Eq. 10 and its weight-decay form):
@@ -299,7 +316,10 @@ gpd_status gpd_correct_positions(gpd_plan_t plan, gpd_product which, void* outpu
  * Limit: products with P - Q <= GPD_STATIC_MAX_PARITY (16); beyond that the call returns
  * GPD_ERR_STATIC_LIMIT and does nothing.
  * Set-up: the first call on a device looks up the array's device address (with that device
- * current); make that first call outside any stream capture.
+ * current); make that first call outside any stream capture.  The address is kept for the life of
+ * the process's context on that device (a cudaDeviceReset invalidates it).
+ * Lifetime: every call enqueues an asynchronous copy of the parity-check matrix out of the plan's
+ * host tables, so the plan must stay alive until the enqueued work has completed.
  * Sharing: every call on a GPU uses the same array.  It is cleared by the call itself, but two
  * calls whose work overlaps on the GPU (different streams, different threads) race on it: keep
  * calls to this entry point ordered on one stream per GPU.

@@ -35,14 +35,14 @@ GPD_PHASE_FWD, GPD_PHASE_BWD, GPD_PHASE_UPD, GPD_PHASE_REGEN, GPD_PHASE_INJECT_S
 (GPD_Q_THRESHOLD_FWD, GPD_Q_THRESHOLD_BWD, GPD_Q_THRESHOLD_AUDIT, GPD_Q_ELEMENT_SIZE,
  GPD_Q_W_SHARE_ELEMS, GPD_Q_X_SHARE_ELEMS, GPD_Q_DT_SHARE_ELEMS, GPD_Q_DHAT_ELEMS, GPD_Q_XHAT_ELEMS,
  GPD_Q_OUT_ELEMS_FWD, GPD_Q_OUT_ELEMS_BWD, GPD_Q_WORKSPACE_BYTES, GPD_Q_STEP_WORKSPACE_BYTES,
- GPD_Q_PRECISION, GPD_Q_NODES, GPD_Q_POSITION_WORKSPACE_BYTES) = range(16)
+ GPD_Q_PRECISION, GPD_Q_NODES, GPD_Q_POSITION_WORKSPACE_BYTES, GPD_Q_TABLES_ON_DEVICE) = range(17)
 (GPD_TABLE_POINTS, GPD_TABLE_PARITY_FWD, GPD_TABLE_PARITY_BWD, GPD_TABLE_PARITY_AUDIT,
  GPD_TABLE_COEF_W, GPD_TABLE_COEF_X, GPD_TABLE_COEF_DT) = range(7)
 GPD_MAX_NODES = 64
 GPD_SUBST_U_EQ_VN, GPD_SUBST_V_EQ_UM = 0, 1
 
 EXPORTED = [
-    "gpd_status_string", "gpd_plan", "gpd_plan_subst", "gpd_plan_destroy", "gpd_plan_query", "gpd_plan_table",
+    "gpd_status_string", "gpd_plan", "gpd_plan_subst", "gpd_plan_upload", "gpd_selftest_bounded_wait", "gpd_plan_destroy", "gpd_plan_query", "gpd_plan_table",
     "gpd_encode_A", "gpd_encode_B", "gpd_worker_gemm", "gpd_device_status", "gpd_update_shares", "gpd_inject",
     "gpd_locate_errors", "gpd_locate_errors_static", "gpd_correct_positions", "gpd_decode", "gpd_regenerate_shares", "gpd_activation", "gpd_softmax_xent_delta",
     "gpd_backprop_hadamard", "gpd_sae_output_delta", "gpd_sae_hidden_delta", "coded_layer_step",
@@ -83,6 +83,8 @@ lib.gpd_plan.argtypes = [C.POINTER(gpd_shape), C.POINTER(gpd_split), _i32, C.POI
 lib.gpd_plan_subst.argtypes = [C.POINTER(gpd_shape), C.POINTER(gpd_split), C.c_int, _i32, C.POINTER(C.c_double),
                                C.c_int, C.POINTER(_vp)]
 lib.gpd_plan_destroy.argtypes = [_vp]
+lib.gpd_plan_upload.argtypes = [_vp]
+lib.gpd_selftest_bounded_wait.argtypes = [_i64, _vp]
 lib.gpd_plan_query.argtypes = [_vp, C.c_int, C.POINTER(_i64)]
 lib.gpd_plan_table.argtypes = [_vp, C.c_int, C.POINTER(C.c_double), _i64, C.POINTER(_i64)]
 lib.gpd_encode_A.argtypes = [_vp, _vp, _vp, _vp]
@@ -223,6 +225,17 @@ def gpd_plan_subst(shape, split, subst: int, P: int, points=None, precision: int
 
 def gpd_plan_destroy(plan: Plan):
     plan.destroy()
+
+
+def gpd_plan_upload(plan: Plan):
+    """Uploads the plan's tables to the current device now instead of at the first compute call."""
+    _check(lib.gpd_plan_upload(plan.handle), "gpd_plan_upload")
+
+
+def gpd_selftest_bounded_wait(limit_cycles: int = 100000, stream=None):
+    """Launches a one-CTA kernel whose barrier wait must run out; gpd_device_status() then reports
+    GPD_ERR_TIMEOUT once."""
+    _check(lib.gpd_selftest_bounded_wait(int(limit_cycles), _stream(stream)), "gpd_selftest_bounded_wait")
 
 
 def gpd_encode_A(plan: Plan, W, W_shares, stream=None):

@@ -334,7 +334,7 @@ template <typename T, int NW, bool VECTOR>
 void launch_stream(const StreamParams& prm, cudaStream_t st) {
     constexpr int N = VECTOR ? Vec<T>::N : 1;
     const int64_t groups = prm.br * prm.bc / N;
-    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((groups + 255) / 256, 148 * 4));
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((groups + 255) / 256, sm_count() * 4));
     const int WP = (prm.n_wanted + NW - 1) / NW * NW;
     decode_stream_kernel<T, NW, VECTOR><<<grid, 256, sizeof(double) * WP * prm.P, st>>>(prm);
 }
@@ -464,7 +464,7 @@ gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_re
     RegenParams rp{};
     rp.shares = shares; rp.Rg = mp.regen; rp.gate = mp.gate; rp.result = result;
     rp.L = pi.br * pi.bc; rp.P = plan->P;
-    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((rp.L + 255) / 256, 148 * 8));
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((rp.L + 255) / 256, sm_count() * 8));
     const size_t smem = sizeof(double) * (size_t)plan->P * plan->P;
     if (plan->elem_size == 4) regen_stream_kernel<float><<<grid, 256, smem, st>>>(rp);
     else regen_stream_kernel<double><<<grid, 256, smem, st>>>(rp);

@@ -188,7 +188,7 @@ extern "C" gpd_status gpd_activation(gpd_activation_kind kind, const float* S_de
                                      int64_t count, void* stream) {
     if (!S_dev || !X_next_dev || count < 0) return GPD_ERR_ARG;
     if (count == 0) return GPD_OK;
-    const int grid = (int)std::min<int64_t>((count + 255) / 256, 148 * 8);
+    const int grid = (int)std::min<int64_t>((count + 255) / 256, sm_count() * 8);
     activation_kernel<<<grid, 256, 0, as_stream(stream)>>>(S_dev, X_next_dev, count, (int)kind);
     return launch_ok();
 }

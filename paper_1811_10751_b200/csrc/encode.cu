@@ -105,7 +105,7 @@ gpd_status dispatch(const EncodeParams& prm, cudaStream_t st) {
                         (reinterpret_cast<uintptr_t>(prm.src) % 16 == 0) &&
                         (reinterpret_cast<uintptr_t>(prm.dst) % 16 == 0);
     const int64_t work = vec_ok ? prm.br * (prm.bc / 4) : prm.br * prm.bc;
-    int grid = (int)std::min<int64_t>((work + 255) / 256, 148 * 16);
+    int grid = (int)std::min<int64_t>((work + 255) / 256, sm_count() * 16);
     if (grid < 1) grid = 1;
     if (vec_ok) {
         switch (prm.nblk) {

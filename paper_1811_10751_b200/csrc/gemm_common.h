@@ -30,6 +30,7 @@ bool dgemm_mma_supported(const GemmParams& prm);
 gpd_status dgemm_mma_launch(const GemmParams& prm, cudaStream_t st);
 bool sgemm_3xtf32_supported(const GemmParams& prm);
 gpd_status sgemm_3xtf32_launch(const GemmParams& prm, cudaStream_t st);
+gpd_status bounded_wait_selftest_launch(long long limit_cycles, cudaStream_t st);
 int tf32_device_status_fetch_and_clear();   // synchronous read of the tensor-path status word
 
 }  // namespace gpd

@@ -127,7 +127,7 @@ gpd_status gemm_generic_launch(const GemmParams& prm, int elem_size, cudaStream_
 
 gpd_status gemv_launch(const GemmParams& prm, int elem_size, cudaStream_t st) {
     const int64_t warps_needed = prm.M;
-    int blocks = (int)std::min<int64_t>((warps_needed + 7) / 8, 148 * 8 / std::max(1, std::min(prm.P, 8)));
+    int blocks = (int)std::min<int64_t>((warps_needed + 7) / 8, sm_count() * 8 / std::max(1, std::min(prm.P, 8)));
     if (blocks < 1) blocks = 1;
     dim3 grid((unsigned)blocks, (unsigned)prm.P);
     if (elem_size == 4)
@@ -199,6 +199,11 @@ extern "C" gpd_status gpd_update_shares(gpd_plan_t plan, void* W_shares_dev, con
                                         const gpd_locate_result* gate_dev, void* stream) {
     if (!plan || !W_shares_dev || !Dhat_dev || !Xhat_dev) return GPD_ERR_ARG;
     return update_launch(plan, W_shares_dev, Dhat_dev, Xhat_dev, eta, lambda, gate_dev, as_stream(stream));
+}
+
+extern "C" gpd_status gpd_selftest_bounded_wait(int64_t limit_cycles, void* stream) {
+    const long long limit = std::max<long long>(1000, std::min<long long>(limit_cycles, 100000000LL));
+    return bounded_wait_selftest_launch(limit, as_stream(stream));
 }
 
 extern "C" gpd_status gpd_device_status(int32_t* status_host) {

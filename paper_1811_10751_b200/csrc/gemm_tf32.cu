@@ -33,6 +33,7 @@
 #include <cuda.h>
 
 #include "gemm_common.h"
+#include "tc_common.h"
 
 namespace gpd {
 
@@ -66,47 +67,19 @@ static_assert(TMEM_ACC_COLS + STAGES * TMEM_A_COLS <= TMEM_COLS, "tensor memory 
 constexpr int kConvWarps = 8;                        // warps 2..9: split tiles
 constexpr int kConvThreads = kConvWarps * 32;
 constexpr int kThreads = 64 + kConvThreads + kEpiWarps * 32;
-constexpr long long kWaitCycles = 2000000000LL;      // about one second
 
 __device__ int g_tf32_status = 0;                    // GPD_ERR_TIMEOUT if a bounded wait expired
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false if the phase did not complete within about a second or the CTA is aborting.
+using tc::kWaitCycles;
+using tc::mbar_arrive;
+using tc::mbar_expect_tx;
+using tc::mbar_init;
+using tc::mbar_try_wait;
+using tc::smem_u32;
+using tc::tma_load_3d;
+using tc::umma_commit;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            *abort_flag = 1;
-            atomicExch(&g_tf32_status, (int)GPD_ERR_TIMEOUT);
-            return false;
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+    return tc::mbar_wait(bar, parity, abort_flag, &g_tf32_status);
 }
 
 // Shared-memory matrix descriptor: start address, leading / stride byte offsets in 16-byte units,
@@ -142,9 +115,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
         "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
         ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
 // Round to the nearest TF32 value (10 explicit mantissa bits) with integer arithmetic: add half
@@ -459,48 +429,11 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 }
 
 // ---- host side -------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
 // 3-D FP32 tensor [batch][rows][cols] (cols contiguous), box {box_cols, box_rows, 1}, given
 // 128-byte swizzle flavour, out-of-range elements read as zero.
 bool make_map(CUtensorMap* map, const void* base, int64_t batch, int64_t rows, int64_t cols, int box_cols, int box_rows,
               CUtensorMapSwizzle swizzle) {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
-    cuuint64_t strides[2] = {(cuuint64_t)cols * 4, (cuuint64_t)rows * (cuuint64_t)cols * 4};
-    cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
+    return tc::make_map_3d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, batch, rows, cols, box_cols, box_rows, swizzle);
 }
 
 template <bool B_KMAJOR, bool UPDATE>
@@ -538,12 +471,31 @@ bool sgemm_3xtf32_supported(const GemmParams& prm) {
     const bool aligned = reinterpret_cast<uintptr_t>(prm.A) % 16 == 0 && reinterpret_cast<uintptr_t>(prm.B) % 16 == 0 &&
                          reinterpret_cast<uintptr_t>(prm.C) % 16 == 0;
     const bool pitches = (prm.K % 4 == 0) && (prm.b_kmajor || prm.N % 4 == 0);
-    return aligned && pitches && prm.M >= 64 && prm.N >= 64 && prm.K >= 32 && encode_tiled_fn() != nullptr;
+    return aligned && pitches && prm.M >= 64 && prm.N >= 64 && prm.K >= 32 && tc::encode_tiled_fn() != nullptr;
 }
 
 gpd_status sgemm_3xtf32_launch(const GemmParams& prm, cudaStream_t st) {
     if (prm.b_kmajor) return prm.update ? launch<true, true>(prm, st) : launch<true, false>(prm, st);
     return prm.update ? launch<false, true>(prm, st) : launch<false, false>(prm, st);
+}
+
+namespace {
+// One warp's lane 0 waits on a barrier nobody arrives at; the wait gives up after `limit` cycles.
+__global__ void bounded_wait_selftest_kernel(long long limit) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tc::mbar_wait(&bar, 0, &abort_flag, &g_tf32_status, limit);
+    }
+}
+}  // namespace
+
+gpd_status bounded_wait_selftest_launch(long long limit, cudaStream_t st) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(limit);
+    return launch_ok();
 }
 
 int tf32_device_status_fetch_and_clear() {

@@ -82,6 +82,19 @@ inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s
 // Uploads the plan's tables on first use (cudaMalloc + cudaMemcpy on the current device).
 gpd_status ensure_device(gpd_plan_s* plan);
 
+// Number of SMs of the current device (cached per device; 148 if the query fails).
+inline int sm_count() {
+    static int cache[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cache[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cache[dev] = n;
+    }
+    return cache[dev];
+}
+
 inline gpd_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? GPD_OK : GPD_ERR_CUDA; }
 inline gpd_status launch_ok() { return cuda_ok(cudaGetLastError()); }
 

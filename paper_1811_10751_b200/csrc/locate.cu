@@ -655,7 +655,7 @@ gpd_status launch_syndrome(const SyndromeParams& prm, cudaStream_t st) {
             return GPD_ERR_CUDA;
     }
     const int64_t batches = (prm.L + kThreads - 1) / kThreads;
-    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(batches, 148 * 4));
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(batches, sm_count() * 4));
     syndrome_gram_kernel<T, RT><<<grid, kThreads, smem, st>>>(prm);
     return launch_ok();
 }

@@ -390,7 +390,7 @@ gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* o
     if (pi.R > 0) {
         const int RT = pi.R <= 8 ? 8 : pi.R <= 16 ? 16 : 32;
         const size_t smem1 = sizeof(double) * RT * plan->P;
-        const int grid1 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 255) / 256, 148 * 8));
+        const int grid1 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 255) / 256, sm_count() * 8));
         const bool f32 = plan->elem_size == 4;
         if (RT == 8) f32 ? position_scan_kernel<float, 8><<<grid1, 256, smem1, st>>>(prm)
                          : position_scan_kernel<double, 8><<<grid1, 256, smem1, st>>>(prm);
@@ -400,7 +400,7 @@ gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* o
                  : position_scan_kernel<double, 32><<<grid1, 256, smem1, st>>>(prm);
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
         const size_t smem2 = sizeof(double) * (2 * pi.R * plan->P + plan->P);
-        const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 63) / 64, 148 * 8));
+        const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 63) / 64, sm_count() * 8));
         if (pi.R <= 8) f32 ? position_fix_kernel<float, 8, 4><<<grid2, 64, smem2, st>>>(prm)
                            : position_fix_kernel<double, 8, 4><<<grid2, 64, smem2, st>>>(prm);
         else f32 ? position_fix_kernel<float, 32, 16><<<grid2, 64, smem2, st>>>(prm)

@@ -283,6 +283,11 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
     return GPD_OK;
 }
 
+extern "C" gpd_status gpd_plan_upload(gpd_plan_t plan) {
+    if (!plan) return GPD_ERR_ARG;
+    return ensure_device(plan);
+}
+
 extern "C" gpd_status gpd_plan_destroy(gpd_plan_t plan) {
     if (!plan) return GPD_ERR_ARG;
     if (plan->uploaded && plan->dev.base) cudaFree(plan->dev.base);
@@ -321,6 +326,11 @@ extern "C" gpd_status gpd_plan_query(gpd_plan_t plan, gpd_query what, int64_t* v
         case GPD_Q_POSITION_WORKSPACE_BYTES: *value = position_workspace_bytes(plan); break;
         case GPD_Q_PRECISION: *value = plan->prec; break;
         case GPD_Q_NODES: *value = P; break;
+        case GPD_Q_TABLES_ON_DEVICE: {
+            std::lock_guard<std::mutex> lock(plan->mu);
+            *value = plan->uploaded ? 1 : 0;
+            break;
+        }
         default: return GPD_ERR_ARG;
     }
     return GPD_OK;

@@ -347,7 +347,7 @@ gpd_status launch_rows_fused(const SliceParams& prm, int slices, size_t smem, cu
     // more CTAs per SM on the same register and shared-memory budget
     const int threads = (int)std::min<int64_t>(kFusedMaxThreads, ((prm.bc >> 2) + 31) / 32 * 32);
     const int per_sm = (int)std::max<size_t>(1, std::min<size_t>(kFusedMaxThreads / threads, (200 * 1024) / smem));
-    const int grid = (int)std::min<int64_t>(prm.br, (int64_t)148 * per_sm);
+    const int grid = (int)std::min<int64_t>(prm.br, (int64_t)sm_count() * per_sm);
     auto go = [&](auto kernel) -> gpd_status {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return GPD_ERR_CUDA;
@@ -368,7 +368,7 @@ gpd_status launch_rows(const SliceParams& prm, int slices, cudaStream_t st) {
     rowscale_kernel<NBLK><<<(unsigned)prm.br, 256, 0, st>>>(prm);
     if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
     const int64_t work = prm.br * (prm.bc / 4);
-    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, 148 * 16));
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((work + 255) / 256, sm_count() * 16));
     const size_t smem = sizeof(double) * prm.P * NBLK;
     if (slices == 6) rowslice_kernel<NBLK, 6><<<grid, 256, smem, st>>>(prm);
     else rowslice_kernel<NBLK, 5><<<grid, 256, smem, st>>>(prm);

@@ -25,6 +25,12 @@ extern "C" gpd_status coded_layer_step(gpd_plan_t plan, int32_t phases, void* W_
         !(phases & (GPD_PHASE_FWD | GPD_PHASE_BWD | GPD_PHASE_UPD)))
         return GPD_ERR_ARG;
     if (plan->sliced && phases != GPD_PHASE_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward only
+    // every requested phase is checked before anything is enqueued
+    if ((phases & GPD_PHASE_FWD) && (!X_dev || !S_out_dev)) return GPD_ERR_ARG;
+    if ((phases & GPD_PHASE_BWD) && (!DeltaT_dev || !CT_out_dev)) return GPD_ERR_ARG;
+    if ((phases & GPD_PHASE_UPD) && (!Delta_dev || !X_dev)) return GPD_ERR_ARG;
+    if ((phases & GPD_PHASE_BWD) && plan->prod[GPD_BWD].Q == 0) return GPD_ERR_P_TOO_SMALL;   // forward-only plan
+    if ((phases & GPD_PHASE_REGEN) && plan->prod[GPD_AUDIT].Q == 0) return GPD_ERR_UNSUPPORTED;
     cudaStream_t st = as_stream(stream);
     const gpd_shape& s = plan->shape;
     const gpd_split& c = plan->split;

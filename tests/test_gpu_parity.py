@@ -692,3 +692,40 @@ def test_tiny_and_skinny_shapes():
     Zb = cp.products(g.GPD_BWD, cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT))
     assert cp.locate(g.GPD_BWD, Zb).outcome == NO_ERROR
     assert op.rel_fro(cp.decode(g.GPD_BWD, Zb), op.ref_backward(DT, W)) < REL_TOL
+
+
+def test_bounded_wait_reports_timeout_and_leaves_the_context_usable():
+    """A barrier wait that nothing ever satisfies gives up after its cycle limit: the status word reads
+    GPD_ERR_TIMEOUT once, is cleared by the read, and later work runs normally."""
+    assert g.gpd_device_status() == 0
+    g.gpd_selftest_bounded_wait(100000)
+    assert g.gpd_device_status() == g.GPD_ERR_TIMEOUT
+    assert g.gpd_device_status() == 0
+    code = GPCode(512, 512, 256, 2, 2, 1, 1, 10)
+    cp = CodedProduct(code)
+    W, X = rand((512, 512), 95), rand((512, 256), 96)
+    cp.encode_W(W)
+    Z = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))      # tensor-core path, bounded waits inside
+    assert cp.locate(g.GPD_FWD, Z).outcome == NO_ERROR
+    assert op.rel_fro(cp.decode(g.GPD_FWD, Z), op.ref_forward(W, X)) < REL_TOL
+    assert g.gpd_device_status() == 0
+
+
+def test_plan_upload_and_forward_only_plan():
+    plan = g.gpd_plan((96, 60, 6), (3, 2, 2, 3), 20)                    # Q_f = 13 <= 20 < Q_b = 22
+    assert plan.query(g.GPD_Q_TABLES_ON_DEVICE) == 0
+    g.gpd_plan_upload(plan)
+    assert plan.query(g.GPD_Q_TABLES_ON_DEVICE) == 1
+    g.gpd_plan_upload(plan)                                            # idempotent
+    # a layer step that asks for the backward product is refused before anything is enqueued
+    Wsh = plan.empty(g.GPD_Q_W_SHARE_ELEMS).zero_()
+    X = torch.zeros((60, 6), device="cuda")
+    DT = torch.zeros((6, 96), device="cuda")
+    S = torch.full((96, 6), 5.0, device="cuda")
+    CT = torch.zeros((6, 60), device="cuda")
+    with pytest.raises(g.GpdError) as e:
+        g.coded_layer_step(plan, g.GPD_PHASE_FWD | g.GPD_PHASE_BWD, Wsh, X=X, DeltaT=DT, S_out=S, CT_out=CT,
+                           results=g.new_results(3), workspace=plan.workspace(step=True))
+    assert e.value.status == g.GPD_ERR_P_TOO_SMALL
+    torch.cuda.synchronize()
+    assert (S == 5.0).all()                                            # the forward phase did not run

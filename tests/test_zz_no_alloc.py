@@ -6,8 +6,9 @@ acceptable.  For them the library offers one entry point whose scratch space is 
 compiled into the library.  This test calls it through the C ABI, twice in a row (the array
 keeps the previous call's contents and must be cleared by the call itself), on a plan that has
 never been used by any other call, and checks every field of its result against the regular
-gpd_locate_errors.  It is collected last so that a run stopping at the first failure has
-already been through all other tests.
+gpd_locate_errors, the decision (outcome and flag vector) against the CPU oracle as well, and
+that the plan it ran on still owns no device memory afterwards.  It is collected last so that a
+run stopping at the first failure has already been through all other tests.
 """
 
 import numpy as np
@@ -20,7 +21,9 @@ if not torch.cuda.is_available():
     pytest.skip("needs a CUDA device", allow_module_level=True)
 
 import paper_1811_10751_b200 as g            # noqa: E402
+from oracle import inject as oinj            # noqa: E402
 from oracle.code import GPCode, powers       # noqa: E402
+from oracle.locate import locate_subspace, tolerances_for   # noqa: E402
 
 
 def _codewords(code, Q, L, seed, dtype):
@@ -54,12 +57,21 @@ def test_static_scratch_variant_matches_regular_entry_point_twice_in_a_row(prec,
         Z = torch.from_numpy(Z0).cuda().reshape(-1)
         if mask:
             g.gpd_inject(plan_regular, g.GPD_FWD, Z, 77, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=mask, scale=1.0)
+        # the oracle's decision on its own copy of the same seeded data
+        Zr = Z0.copy()
+        if mask:
+            oinj.inject_gauss(Zr, 77, 1.0, nodes=[(mask >> p) & 1 == 1 for p in range(P)])
+        ro = locate_subspace(Zr, code.points, code.Q_f, tolerances_for(dtype), erased=erased)
         for _ in range(2):                                         # two calls in a row
             g.gpd_locate_errors_static(plan_static, g.GPD_FWD, Z, res_static, erased=erased)
             a = g.read_results(res_static)[0]
             g.gpd_locate_errors(plan_regular, g.GPD_FWD, Z, res_regular, ws, erased=erased)
             b = g.read_results(res_regular)[0]
             assert _fields(a, P) == _fields(b, P)
+            assert a.outcome == ro.outcome and np.array_equal(np.array(a.flagged[:P], dtype=bool), ro.flagged)
+            # nothing on the static path uploads the plan's tables (the library's only device allocation)
+            assert plan_static.query(g.GPD_Q_TABLES_ON_DEVICE) == 0
+            assert plan_regular.query(g.GPD_Q_TABLES_ON_DEVICE) == 1
             for x, y in ((a.residual, b.residual), (a.max_inside, b.max_inside), (a.min_outside, b.min_outside)):
                 assert abs(x - y) <= 1e-9 * max(1.0, abs(y))
         outcomes.append(a.outcome)
