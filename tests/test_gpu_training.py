@@ -62,7 +62,20 @@ def _flags(r, P):
 
 @pytest.mark.parametrize("prob,step_seed", [(0.0, 0), (0.05, 4321)])
 def test_mlp_step_matches_oracle(prob, step_seed):
-    cfg = wl.scaled_down(wl.CONFIG_4_MLP, 16)                  # 256-256-256-256-10, batch 16
+    _run_mlp_step(wl.scaled_down(wl.CONFIG_4_MLP, 16), prob, step_seed)   # 256-256-256-256-10, batch 16
+
+
+def test_config4_full_size_step():
+    """The MLP workload as stated: 4096-4096-4096-4096-10, batch 256, split 2 x 2, P = 10, one SGD step
+    with every layer's forward product, backward product and update coded and node errors of
+    probability 0.05 (the last layer's W has 5-row blocks: the small-block kernels)."""
+    cfg = wl.CONFIG_4_MLP
+    assert cfg.widths == (4096, 4096, 4096, 4096, 10) and cfg.B == 256 and cfg.P == 10
+    _run_mlp_step(cfg, cfg.inject_prob, 4321)
+    assert g.gpd_device_status() == 0
+
+
+def _run_mlp_step(cfg, prob, step_seed):
     Ws, X1, labels = wl.mlp_inputs(cfg)
     L = len(Ws)
     # oracle: coded step (FP32 storage of worker outputs, same seeds) and uncoded FP64 step
@@ -283,7 +296,18 @@ def test_training_with_share_errors_and_regeneration():
 def test_config5_full_size_two_steps():
     """The sparse-autoencoder workload at full size (1024 <-> 8192, batch 1024, split 4 x 4, P = 36,
     thresholds 19 / 28 / 16, FP64 path), two coded SGD steps with Gaussian node errors."""
-    cfg = wl.CONFIG_5_AUTOENCODER
+    _run_autoencoder(wl.CONFIG_5_AUTOENCODER, 2)
+
+
+def test_config5_ten_steps_half_size():
+    """All ten SGD steps of the workload, at half the width and batch (512 <-> 4096, batch 512; same
+    split, node count, thresholds and error probability): the oracle's ten full-size steps take minutes."""
+    cfg = wl.scaled_down(wl.CONFIG_5_AUTOENCODER, 2)
+    assert cfg.steps == 10 and cfg.P == 36
+    _run_autoencoder(cfg, cfg.steps)
+
+
+def _run_autoencoder(cfg, n_steps):
     W1, W2, X = wl.autoencoder_inputs(cfg)
     enc_o = odnn.CodedLayer.from_weights(W1, GPCode(cfg.n_hidden, cfg.n_visible, cfg.B, cfg.m, cfg.n, 1, 1, cfg.P),
                                          inject_mode="gauss", inject_prob=cfg.inject_prob)
@@ -298,7 +322,7 @@ def test_config5_full_size_two_steps():
     D1, D1T = torch.empty((cfg.n_hidden, cfg.B), **f32), torch.empty((cfg.B, cfg.n_hidden), **f32)
     mse, kl = torch.zeros(1, **f32), torch.zeros(1, **f32)
     n_corrected = 0
-    for s in range(2):
+    for s in range(n_steps):
         seed = 8800 + 100 * s
         o = odnn.autoencoder_step_coded(enc_o, dec_o, X, cfg.lr, cfg.rho, cfg.beta, step_seed=seed)
         assert o is not None
