@@ -93,9 +93,19 @@ typedef enum {
                                    shares returns GPD_ERR_UNSUPPORTED; gpd_plan returns it when the shapes do
                                    not fit.  An implementation choice of this library: the paper prescribes
                                    no arithmetic for the nodes' products. */
-    GPD_PREC_FP64_SLICED40 = 4  /* the same with five digit planes (40 bits below the scale, 15 plane pairs
+    GPD_PREC_FP64_SLICED40 = 4, /* the same with five digit planes (40 bits below the scale, 15 plane pairs
                                    instead of 21): worker outputs accurate to about 1e-10 of their scale,
                                    enough for recovery thresholds up to about 20 */
+    GPD_PREC_FP64_SLICED_TRAIN = 5 /* digit-plane products (six planes) for every stage of the coded training
+                                   step (Sections VI, VIII): forward and backward products and the update of
+                                   Eq. 10 run as int8 tensor-core contractions; audit, regeneration and
+                                   share-error injection work on FP64 shares.  The share buffer of W
+                                   (GPD_Q_W_SHARE_ELEMS doubles, opaque, 16-byte aligned) holds the FP64
+                                   shares [P][N1/m][N0/n] first, then two sliced copies (rows of W~_p for the
+                                   forward product, columns for the backward product), re-cut by every call
+                                   that changes the FP64 shares; the other operands' buffers keep the sizes
+                                   of FP64 shares.  Needs N0/n, N1/m, B/d1, B/d2 and B divisible by 16 and at
+                                   most 16384, finite inputs. */
 } gpd_precision;
 
 typedef enum {
@@ -155,7 +165,7 @@ typedef enum {
     GPD_Q_THRESHOLD_BWD = 1,    /* mn (d2 + 1) - n (proof of Theorem 6) or, alternate substitution, mn d2 + m - 1  */
     GPD_Q_THRESHOLD_AUDIT = 2,  /* mn                                               */
     GPD_Q_ELEMENT_SIZE = 3,     /* bytes per share / worker-output element (4 or 8) */
-    GPD_Q_W_SHARE_ELEMS = 4,    /* P * (N1/m) * (N0/n)                              */
+    GPD_Q_W_SHARE_ELEMS = 4,    /* P * (N1/m) * (N0/n); GPD_PREC_FP64_SLICED_TRAIN: that plus the two sliced copies */
     GPD_Q_X_SHARE_ELEMS = 5,    /* P * (N0/n) * (B/d1)                              */
     GPD_Q_DT_SHARE_ELEMS = 6,   /* P * (B/d2) * (N1/m)                              */
     GPD_Q_DHAT_ELEMS = 7,       /* P * (N1/m) * B                                   */

@@ -29,6 +29,7 @@ GPD_NO_ERROR, GPD_CORRECTED, GPD_DECODE_FAILURE = 0, 1, 2
 GPD_FWD, GPD_BWD, GPD_UPD, GPD_AUDIT = 0, 1, 2, 3
 GPD_OPERAND_X_FWD, GPD_OPERAND_DELTAT_BWD, GPD_OPERAND_DELTA_UPD, GPD_OPERAND_X_UPD = 0, 1, 2, 3
 GPD_PREC_AUTO, GPD_PREC_FP32, GPD_PREC_FP64, GPD_PREC_FP64_SLICED, GPD_PREC_FP64_SLICED40 = 0, 1, 2, 3, 4
+GPD_PREC_FP64_SLICED_TRAIN = 5
 GPD_INJECT_BITFLIP, GPD_INJECT_ADDITIVE, GPD_INJECT_GAUSS = 0, 1, 2
 GPD_ACT_IDENTITY, GPD_ACT_RELU, GPD_ACT_SIGMOID = 0, 1, 2
 GPD_PHASE_FWD, GPD_PHASE_BWD, GPD_PHASE_UPD, GPD_PHASE_REGEN, GPD_PHASE_INJECT_SHARES = 1, 2, 4, 8, 16

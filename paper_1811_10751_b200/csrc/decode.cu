@@ -10,6 +10,7 @@
 //      read once with 16-byte loads, FP64 accumulation, FP32 store into the right block of the
 //      result; optional fused activation (step C1).
 #include "gpd_internal.h"
+#include "slice_common.h"
 
 namespace gpd {
 
@@ -364,7 +365,9 @@ gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* output
                          uint64_t use_mask, const gpd_locate_result* result, float* out, float* act_out,
                          int activation, void* workspace, cudaStream_t st) {
     if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
-    if (plan->sliced && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward product only
+    // digit-plane shares: forward product only, except in the training mode (its backward outputs and the
+    // FP64 shares that lead W's buffer are plain doubles)
+    if (plan->sliced && !plan->train && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;
     const ProductInfo& pi = plan->prod[which];
     if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
     gpd_status rc = ensure_device(plan);
@@ -445,7 +448,7 @@ __global__ void __launch_bounds__(256) regen_stream_kernel(RegenParams prm) {
 gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_result* result, void* workspace,
                              cudaStream_t st) {
     const ProductInfo& pi = plan->prod[GPD_AUDIT];
-    if (pi.Q == 0 || plan->sliced) return GPD_ERR_UNSUPPORTED;
+    if (pi.Q == 0 || (plan->sliced && !plan->train)) return GPD_ERR_UNSUPPORTED;
     gpd_status rc = ensure_device(plan);
     if (rc != GPD_OK) return rc;
     const WorkspaceLayout wl = workspace_layout();
@@ -468,7 +471,9 @@ gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_re
     const size_t smem = sizeof(double) * (size_t)plan->P * plan->P;
     if (plan->elem_size == 4) regen_stream_kernel<float><<<grid, 256, smem, st>>>(rp);
     else regen_stream_kernel<double><<<grid, 256, smem, st>>>(rp);
-    return launch_ok();
+    if ((rc = launch_ok()) != GPD_OK) return rc;
+    // training mode: the regenerated FP64 shares lead the buffer; the sliced copies follow them
+    return plan->train ? reslice_launch(plan, shares, st) : GPD_OK;
 }
 
 }  // namespace gpd

@@ -129,11 +129,9 @@ gpd_status dispatch(const EncodeParams& prm, cudaStream_t st) {
 
 gpd_status encode_launch(gpd_plan_s* plan, int operand_or_A, const float* src, void* dst,
                          cudaStream_t st) {
-    if (plan->sliced) {
-        if (operand_or_A == -1) return encode_sliced_launch(plan, true, src, dst, st);
-        if (operand_or_A == GPD_OPERAND_X_FWD) return encode_sliced_launch(plan, false, src, dst, st);
-        return GPD_ERR_UNSUPPORTED;
-    }
+    // digit-plane modes: operands are cut into planes by slice.cu; in the training mode W's shares are
+    // first evaluated to FP64 at the start of their buffer (below), then both sliced copies are cut
+    if (plan->sliced && !(plan->train && operand_or_A == -1)) return encode_sliced_launch(plan, operand_or_A, src, dst, st);
     gpd_status rc = ensure_device(plan);
     if (rc != GPD_OK) return rc;
     const gpd_shape& s = plan->shape;
@@ -162,7 +160,9 @@ gpd_status encode_launch(gpd_plan_s* plan, int operand_or_A, const float* src, v
         default: return GPD_ERR_ARG;
     }
     prm.nblk = gr * prm.gc;
-    return plan->elem_size == 4 ? dispatch<float>(prm, st) : dispatch<double>(prm, st);
+    rc = plan->elem_size == 4 ? dispatch<float>(prm, st) : dispatch<double>(prm, st);
+    if (rc == GPD_OK && plan->train && operand_or_A == -1) rc = reslice_launch(plan, dst, st);
+    return rc;
 }
 
 }  // namespace gpd

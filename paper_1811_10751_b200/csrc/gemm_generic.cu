@@ -141,8 +141,7 @@ gpd_status worker_gemm_launch(gpd_plan_s* plan, gpd_product which, const void* W
                               void* out, cudaStream_t st) {
     const gpd_shape& s = plan->shape;
     const gpd_split& c = plan->split;
-    if (plan->sliced)
-        return which == GPD_FWD ? gemm_sliced_launch(plan, W_sh, other, out, st) : GPD_ERR_UNSUPPORTED;
+    if (plan->sliced) return gemm_sliced_launch(plan, which, W_sh, other, out, st);
     GemmParams prm{};
     prm.P = plan->P;
     prm.C = out;
@@ -169,7 +168,8 @@ gpd_status update_launch(gpd_plan_s* plan, void* W_sh, const void* Dhat, const v
                          float lambda, const gpd_locate_result* gate, cudaStream_t st) {
     const gpd_shape& s = plan->shape;
     const gpd_split& c = plan->split;
-    if (plan->sliced) return GPD_ERR_UNSUPPORTED;
+    if (plan->sliced)
+        return update_sliced_launch(plan, W_sh, Dhat, Xhat, 1.0 - (double)eta * (double)lambda, (double)eta, gate, st);
     GemmParams prm{};
     prm.P = plan->P;
     prm.A = Dhat; prm.B = Xhat; prm.C = W_sh;

@@ -1,4 +1,7 @@
-// FP64-class forward worker products (step O1) on the integer tensor cores.
+// FP64-class worker products (steps O1, O2) and the coded update (O3, Eq. 10) on the integer tensor
+// cores.  The kernel multiplies two sliced operands, C[p] = A[p] B[p]^T; the forward product takes
+// A = W~_p (rows), B = X~_p^T, the backward product A = Delta~^T_p, B = W~_p^T (the column-sliced
+// copy of the shares), the update A = Delta^_p, B = X^_p and adds into the FP64 shares.
 //
 // Both operands arrive cut into S = 6 (or 5) signed 8-bit digit planes (slice.cu):
 //     W~_p[i][k] = 2^ea[i] * sum_s A_s[i][k] 256^-(s+1),   X~_p[k][j] = 2^eb[j] * sum_t B_t[j][k] 256^-(t+1).
@@ -89,12 +92,15 @@ struct I8Params {
     double* C;         // [P][M][N]
     int64_t M, N, K;
     int P;
+    double shrink, eta;                  // update: C <- shrink * C + eta * A B^T
+    const gpd_locate_result* gate;       // update: skipped when this reports a decoding failure
 };
 
-template <int S>
+template <int S, bool UPDATE>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, I8Params prm,
                       int tiles_m, int tiles_n, int tiles) {
+    if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
     constexpr int STAGE_BYTES = stage_bytes(S);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -255,6 +261,11 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             if (lane == 0) mbar_arrive(&acc_empty);
             double* crow = prm.C + (int64_t)p * prm.M * prm.N + gm * prm.N + n0 + c0;
             const bool vec = (prm.N & 1) == 0 && n0 + c0 + 32 <= prm.N;
+            double2 old[16];                             // update: the stored shares this thread adds into
+            if (UPDATE && vec && gm < prm.M) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) old[j] = *reinterpret_cast<const double2*>(crow + 2 * j);
+            }
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
                 double2 o;                               // column scales come from the lanes that hold them
@@ -262,10 +273,17 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 o.y = v[j + 1] * row_scale * __shfl_sync(0xffffffffu, col_scale, j + 1);
                 if (gm < prm.M) {
                     if (vec) {
-                        __stcs(reinterpret_cast<double2*>(crow + j), o);
+                        if (UPDATE) {
+                            o.x = fma(prm.eta, o.x, prm.shrink * old[j >> 1].x);
+                            o.y = fma(prm.eta, o.y, prm.shrink * old[j >> 1].y);
+                            *reinterpret_cast<double2*>(crow + j) = o;      // read again soon: no streaming hint
+                        } else {
+                            __stcs(reinterpret_cast<double2*>(crow + j), o);
+                        }
                     } else {
-                        if (n0 + c0 + j < prm.N) crow[j] = o.x;
-                        if (n0 + c0 + j + 1 < prm.N) crow[j + 1] = o.y;
+                        if (n0 + c0 + j < prm.N) crow[j] = UPDATE ? fma(prm.eta, o.x, prm.shrink * crow[j]) : o.x;
+                        if (n0 + c0 + j + 1 < prm.N)
+                            crow[j + 1] = UPDATE ? fma(prm.eta, o.y, prm.shrink * crow[j + 1]) : o.y;
                     }
                 }
             }
@@ -290,33 +308,90 @@ bool make_map(CUtensorMap* map, const void* base, int64_t batch, int64_t rows, i
 
 }  // namespace
 
-gpd_status gemm_sliced_launch(gpd_plan_s* plan, const void* W_sliced, const void* X_sliced, void* out,
-                              cudaStream_t st) {
-    const gpd_shape& s = plan->shape;
-    const gpd_split& c = plan->split;
-    I8Params prm{};
-    prm.P = plan->P;
-    prm.M = s.N1 / c.m; prm.K = s.N0 / c.n; prm.N = s.B / c.d1;
-    const int S = plan->slices;
-    const SlicedLayout la = sliced_layout(S, prm.P, prm.M, prm.K), lb = sliced_layout(S, prm.P, prm.N, prm.K);
-    prm.ea = reinterpret_cast<const int*>(reinterpret_cast<const char*>(W_sliced) + la.expo_offset);
-    prm.eb = reinterpret_cast<const int*>(reinterpret_cast<const char*>(X_sliced) + lb.expo_offset);
-    prm.C = reinterpret_cast<double*>(out);
-    if (reinterpret_cast<uintptr_t>(W_sliced) % 16 || reinterpret_cast<uintptr_t>(X_sliced) % 16 ||
-        reinterpret_cast<uintptr_t>(out) % 16)
+gpd_status gemm_i8_launch(const I8Gemm& g, cudaStream_t st) {
+    if (g.K % 16 != 0 || g.K > 16384 || (g.slices != 5 && g.slices != 6)) return GPD_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(g.A) % 16 || reinterpret_cast<uintptr_t>(g.B) % 16 ||
+        reinterpret_cast<uintptr_t>(g.C) % 16)
         return GPD_ERR_ARG;
+    I8Params prm{};
+    prm.P = g.P; prm.M = g.M; prm.N = g.N; prm.K = g.K;
+    prm.ea = g.ea; prm.eb = g.eb; prm.C = g.C;
+    prm.shrink = g.shrink; prm.eta = g.eta; prm.gate = g.gate;
+    const int S = g.slices;
     CUtensorMap tmA, tmB;
-    if (!make_map(&tmA, W_sliced, (int64_t)S * prm.P, prm.M, prm.K, BM)) return GPD_ERR_CUDA;
-    if (!make_map(&tmB, X_sliced, (int64_t)S * prm.P, prm.N, prm.K, BN)) return GPD_ERR_CUDA;
-    auto kernel = S == 6 ? gemm_i8_sliced_kernel<6> : gemm_i8_sliced_kernel<5>;
+    if (!make_map(&tmA, g.A, (int64_t)S * g.P, g.M, g.K, BM)) return GPD_ERR_CUDA;
+    if (!make_map(&tmB, g.B, (int64_t)S * g.P, g.N, g.K, BN)) return GPD_ERR_CUDA;
+    auto kernel = g.update ? gemm_i8_sliced_kernel<6, true>
+                           : (S == 6 ? gemm_i8_sliced_kernel<6, false> : gemm_i8_sliced_kernel<5, false>);
+    if (g.update && S != 6) return GPD_ERR_UNSUPPORTED;
     const int smem = S == 6 ? smem_bytes(6) : smem_bytes(5);
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GPD_ERR_CUDA;
-    const int tiles_n = (int)((prm.N + BN - 1) / BN), tiles_m = (int)((prm.M + BM - 1) / BM);
-    const int64_t tiles = (int64_t)tiles_n * tiles_m * prm.P;
-    const int sms = sm_count();
-    const unsigned grid = (unsigned)std::min<int64_t>(tiles, sms);      // persistent: one CTA per SM walks the tiles
+    const int tiles_n = (int)((g.N + BN - 1) / BN), tiles_m = (int)((g.M + BM - 1) / BM);
+    const int64_t tiles = (int64_t)tiles_n * tiles_m * g.P;
+    const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());     // persistent: one CTA per SM walks the tiles
     kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, prm, tiles_m, tiles_n, (int)tiles);
     return launch_ok();
+}
+
+gpd_status gemm_sliced_launch(gpd_plan_s* plan, gpd_product which, const void* W_shares, const void* other_sliced,
+                              void* out, cudaStream_t st) {
+    const gpd_shape& s = plan->shape;
+    const gpd_split& c = plan->split;
+    const int S = plan->slices;
+    const char* wbase = reinterpret_cast<const char*>(W_shares);
+    const char* obase = reinterpret_cast<const char*>(other_sliced);
+    I8Gemm g{};
+    g.slices = S; g.P = plan->P; g.C = reinterpret_cast<double*>(out);
+    g.update = false; g.shrink = 0.0; g.eta = 1.0; g.gate = nullptr;
+    if (which == GPD_FWD) {                       // S~_p = W~_p X~_p: A = rows of W~_p, B = columns of X~_p
+        g.M = s.N1 / c.m; g.K = s.N0 / c.n; g.N = s.B / c.d1;
+        const SlicedLayout lb = sliced_layout(S, g.P, g.N, g.K);
+        if (plan->train) {
+            const TrainLayout tl = train_layout(plan);
+            g.A = wbase + tl.rows_offset;
+            g.ea = reinterpret_cast<const int*>(wbase + tl.rows_offset + tl.rows.expo_offset);
+        } else {
+            const SlicedLayout la = sliced_layout(S, g.P, g.M, g.K);
+            g.A = wbase;
+            g.ea = reinterpret_cast<const int*>(wbase + la.expo_offset);
+        }
+        g.B = obase;
+        g.eb = reinterpret_cast<const int*>(obase + lb.expo_offset);
+    } else if (which == GPD_BWD) {                // C~^T_p = Delta~^T_p W~_p: A = rows of Delta~^T_p, B = columns of W~_p
+        if (!plan->train) return GPD_ERR_UNSUPPORTED;
+        if (plan->prod[GPD_BWD].Q == 0) return GPD_ERR_P_TOO_SMALL;
+        g.M = s.B / c.d2; g.K = s.N1 / c.m; g.N = s.N0 / c.n;
+        const TrainLayout tl = train_layout(plan);
+        const SlicedLayout la = sliced_layout(S, g.P, g.M, g.K);
+        g.A = obase;
+        g.ea = reinterpret_cast<const int*>(obase + la.expo_offset);
+        g.B = wbase + tl.cols_offset;
+        g.eb = reinterpret_cast<const int*>(wbase + tl.cols_offset + tl.cols.expo_offset);
+    } else {
+        return GPD_ERR_ARG;
+    }
+    return gemm_i8_launch(g, st);
+}
+
+gpd_status update_sliced_launch(gpd_plan_s* plan, void* W_shares, const void* Dhat_sliced, const void* Xhat_sliced,
+                                double shrink, double eta, const gpd_locate_result* gate, cudaStream_t st) {
+    if (!plan->train) return GPD_ERR_UNSUPPORTED;
+    const gpd_shape& s = plan->shape;
+    const gpd_split& c = plan->split;
+    const int S = plan->slices;
+    I8Gemm g{};
+    g.slices = S; g.P = plan->P;
+    g.M = s.N1 / c.m; g.N = s.N0 / c.n; g.K = s.B;                 // Delta^_p (M x B) X^_p^T (B x N)
+    const SlicedLayout la = sliced_layout(S, g.P, g.M, g.K), lb = sliced_layout(S, g.P, g.N, g.K);
+    g.A = Dhat_sliced;
+    g.ea = reinterpret_cast<const int*>(reinterpret_cast<const char*>(Dhat_sliced) + la.expo_offset);
+    g.B = Xhat_sliced;
+    g.eb = reinterpret_cast<const int*>(reinterpret_cast<const char*>(Xhat_sliced) + lb.expo_offset);
+    g.C = reinterpret_cast<double*>(W_shares);                     // the FP64 shares lead the buffer
+    g.update = true; g.shrink = shrink; g.eta = eta; g.gate = gate;
+    gpd_status rc = gemm_i8_launch(g, st);
+    if (rc != GPD_OK) return rc;
+    return reslice_launch(plan, W_shares, st);
 }
 
 int i8_device_status_fetch_and_clear() {

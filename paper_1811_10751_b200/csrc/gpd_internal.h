@@ -64,6 +64,7 @@ struct gpd_plan_s {
     int elem_size = 4;
     bool sliced = false;         // GPD_PREC_FP64_SLICED / _SLICED40: shares are int8 digit planes, outputs double
     int slices = 0;              // digit planes per operand (6 or 5) when sliced
+    bool train = false;          // GPD_PREC_FP64_SLICED_TRAIN: W's buffer holds FP64 shares and two sliced copies
     double tau_col = 0, tau_in = 0;
     std::vector<double> points;
     std::vector<double> coefW, coefX, coefDT, coefDup, coefXup;   // [P][blocks]

@@ -9,6 +9,7 @@
 #include <cmath>
 
 #include "gpd_internal.h"
+#include "slice_common.h"
 
 namespace gpd {
 
@@ -154,7 +155,9 @@ gpd_status inject_launch(gpd_plan_s* plan, gpd_product which, void* outputs, uin
                          double prob, uint64_t node_mask, int count, double scale, uint64_t* hit_mask,
                          cudaStream_t st) {
     if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
-    if (plan->sliced && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward product only
+    // digit-plane shares: forward product only, except in the training mode (its backward outputs and the
+    // FP64 shares that lead W's buffer are plain doubles)
+    if (plan->sliced && !plan->train && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;
     const ProductInfo& pi = plan->prod[which];
     if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
     InjectParams prm{};
@@ -169,11 +172,15 @@ gpd_status inject_launch(gpd_plan_s* plan, gpd_product which, void* outputs, uin
     prm.scale = scale;
     prm.hit_mask = reinterpret_cast<unsigned long long*>(hit_mask);
     const bool f32 = plan->elem_size == 4;
+    // training mode, errors written into the stored shares: they land in the FP64 shares, from which the
+    // sliced copies that the products read are then cut again
+    const bool recut = plan->train && which == GPD_AUDIT;
     if (mode == GPD_INJECT_BITFLIP) {
         if (count < 0) return GPD_ERR_ARG;
         if (f32) inject_bitflip_kernel<float, unsigned int><<<1, 32, 0, st>>>(prm);
         else inject_bitflip_kernel<double, unsigned long long><<<1, 32, 0, st>>>(prm);
-        return launch_ok();
+        if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+        return recut ? reslice_launch(plan, outputs, st) : GPD_OK;
     }
     if (mode != GPD_INJECT_ADDITIVE && mode != GPD_INJECT_GAUSS) return GPD_ERR_ARG;
     // Which nodes are hit is a pure function of (seed, node): evaluated here with the same
@@ -203,7 +210,8 @@ gpd_status inject_launch(gpd_plan_s* plan, gpd_product which, void* outputs, uin
     } else {
         return GPD_ERR_ARG;
     }
-    return launch_ok();
+    if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+    return recut ? reslice_launch(plan, outputs, st) : GPD_OK;
 }
 
 }  // namespace gpd

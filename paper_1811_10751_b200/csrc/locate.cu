@@ -673,7 +673,9 @@ gpd_status dispatch_syndrome(const SyndromeParams& prm, cudaStream_t st) {
 gpd_status locate_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, uint64_t erased_mask,
                          gpd_locate_result* result, void* workspace, cudaStream_t st) {
     if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
-    if (plan->sliced && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward product only
+    // digit-plane shares: forward product only, except in the training mode (its backward outputs and the
+    // FP64 shares that lead W's buffer are plain doubles)
+    if (plan->sliced && !plan->train && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;
     const ProductInfo& pi = plan->prod[which];
     if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
     gpd_status rc = ensure_device(plan);
@@ -739,7 +741,9 @@ gpd_status static_scratch(unsigned char** out) {
 gpd_status locate_static_launch(gpd_plan_s* plan, gpd_product which, const void* outputs,
                                 uint64_t erased_mask, gpd_locate_result* result, cudaStream_t st) {
     if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
-    if (plan->sliced && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward product only
+    // digit-plane shares: forward product only, except in the training mode (its backward outputs and the
+    // FP64 shares that lead W's buffer are plain doubles)
+    if (plan->sliced && !plan->train && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;
     const ProductInfo& pi = plan->prod[which];
     if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
     if (pi.R > kStaticMaxR) return GPD_ERR_STATIC_LIMIT;

@@ -369,7 +369,9 @@ int64_t position_workspace_bytes(const gpd_plan_s* plan) {
 gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* outputs, gpd_position_result* result,
                                     void* workspace, cudaStream_t st) {
     if (which != GPD_FWD && which != GPD_BWD && which != GPD_AUDIT) return GPD_ERR_ARG;
-    if (plan->sliced && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward product only
+    // digit-plane shares: forward product only, except in the training mode (its backward outputs and the
+    // FP64 shares that lead W's buffer are plain doubles)
+    if (plan->sliced && !plan->train && which != GPD_FWD) return GPD_ERR_UNSUPPORTED;
     const ProductInfo& pi = plan->prod[which];
     if (pi.Q == 0) return GPD_ERR_P_TOO_SMALL;
     const int64_t L = pi.br * pi.bc;

@@ -174,7 +174,8 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
     if (subst != GPD_SUBST_U_EQ_VN && subst != GPD_SUBST_V_EQ_UM) return GPD_ERR_ARG;
     const bool alt = subst == GPD_SUBST_V_EQ_UM;
     if (precision != GPD_PREC_AUTO && precision != GPD_PREC_FP32 && precision != GPD_PREC_FP64 &&
-        precision != GPD_PREC_FP64_SLICED && precision != GPD_PREC_FP64_SLICED40)
+        precision != GPD_PREC_FP64_SLICED && precision != GPD_PREC_FP64_SLICED40 &&
+        precision != GPD_PREC_FP64_SLICED_TRAIN)
         return GPD_ERR_ARG;
     const int m = split->m, n = split->n, d1 = split->d1, d2 = split->d2;
     if (shape->N1 <= 0 || shape->N0 <= 0 || shape->B <= 0 || m <= 0 || n <= 0 || d1 <= 0 || d2 <= 0)
@@ -223,8 +224,9 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
     plan->elem_size = plan->prec == GPD_PREC_FP32 ? 4 : 8;
     plan->tau_col = plan->prec == GPD_PREC_FP32 ? kTauColFp32 : kTauColFp64;
     plan->tau_in = plan->prec == GPD_PREC_FP32 ? kTauInFp32 : kTauInFp64;
-    plan->sliced = plan->prec == GPD_PREC_FP64_SLICED || plan->prec == GPD_PREC_FP64_SLICED40;
-    plan->slices = plan->prec == GPD_PREC_FP64_SLICED ? 6 : plan->prec == GPD_PREC_FP64_SLICED40 ? 5 : 0;
+    plan->train = plan->prec == GPD_PREC_FP64_SLICED_TRAIN;
+    plan->sliced = plan->prec == GPD_PREC_FP64_SLICED || plan->prec == GPD_PREC_FP64_SLICED40 || plan->train;
+    plan->slices = plan->prec == GPD_PREC_FP64_SLICED40 ? 5 : plan->sliced ? 6 : 0;
 
     // powers up to the largest exponent used by any encoding
     const int max_exp = (int)std::max<int64_t>(std::max(Qf, Qb), Qw) + 1;
@@ -305,7 +307,9 @@ extern "C" gpd_status gpd_plan_query(gpd_plan_t plan, gpd_query what, int64_t* v
         case GPD_Q_THRESHOLD_BWD: *value = plan->Qb; break;
         case GPD_Q_THRESHOLD_AUDIT: *value = plan->Qw; break;
         case GPD_Q_ELEMENT_SIZE: *value = plan->elem_size; break;
-        case GPD_Q_W_SHARE_ELEMS: *value = P * (s.N1 / c.m) * (s.N0 / c.n); break;
+        case GPD_Q_W_SHARE_ELEMS:
+            *value = plan->train ? (train_layout(plan).total_bytes + 7) / 8 : P * (s.N1 / c.m) * (s.N0 / c.n);
+            break;
         case GPD_Q_X_SHARE_ELEMS: *value = P * (s.N0 / c.n) * (s.B / c.d1); break;
         case GPD_Q_DT_SHARE_ELEMS: *value = P * (s.B / c.d2) * (s.N1 / c.m); break;
         case GPD_Q_DHAT_ELEMS: *value = P * (s.N1 / c.m) * s.B; break;

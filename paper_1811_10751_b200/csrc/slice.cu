@@ -341,6 +341,86 @@ __global__ void __launch_bounds__(256) colpass_kernel(SliceParams prm) {
     }
 }
 
+// ---- training mode: the sliced copies of W's shares, cut from the FP64 shares ----------------------
+// Rows: one warp per row (node p, share row r) of K doubles: largest magnitude (exact), exponent,
+// digits; a lane owns four consecutive values per trip, so a warp reads 1 KB and writes 128 bytes
+// per plane at a time.
+template <int S>
+__global__ void __launch_bounds__(256) reslice_rows_kernel(const double* __restrict__ master, int8_t* planes, int* expo,
+                                                          int64_t n_rows, int64_t K, int64_t plane_stride) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= n_rows) return;                                     // whole warp
+    const double* src = master + row * K;
+    unsigned int mx = 0u;
+    for (int64_t k = 4 * lane; k < K; k += 128) {
+        const double2 v0 = *reinterpret_cast<const double2*>(src + k), v1 = *reinterpret_cast<const double2*>(src + k + 2);
+        mx = max(mx, max(max(abs_hi(v0.x), abs_hi(v0.y)), max(abs_hi(v1.x), abs_hi(v1.y))));
+    }
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    const int e = slice_exponent(mx);
+    if (lane == 0) expo[row] = e;
+    const double scale = slice_scale<S>(e);
+    int8_t* dst = planes + row * K;
+    for (int64_t k = 4 * lane; k < K; k += 128) {                  // second read of the row: from L1 / L2
+        const double2 v0 = *reinterpret_cast<const double2*>(src + k), v1 = *reinterpret_cast<const double2*>(src + k + 2);
+        const double a[4] = {v0.x, v0.y, v1.x, v1.y};
+        unsigned int word[S];
+        digits4<S>(a, scale, word);
+#pragma unroll
+        for (int t = 0; t < S; ++t) *reinterpret_cast<unsigned int*>(dst + t * plane_stride + k) = word[t];
+    }
+}
+
+// Columns, pass 1: largest magnitude of every column of every node's share (M x K), met in
+// amax[p][c] (high words, zeroed before the launch).  Thread = column, CTA = slab of 64 rows.
+__global__ void __launch_bounds__(256) colmax_kernel(const double* __restrict__ master, unsigned int* amax, int64_t M, int64_t K) {
+    const int64_t c = (int64_t)blockIdx.x * 256 + threadIdx.x, r0 = (int64_t)blockIdx.y * 64, p = blockIdx.z;
+    if (c >= K) return;
+    const double* src = master + (p * M + r0) * K + c;
+    const int64_t rows = min((int64_t)64, M - r0);
+    unsigned int mx = 0u;
+    for (int64_t r = 0; r < rows; ++r) mx = max(mx, abs_hi(src[r * K]));
+    if (mx) atomicMax(amax + p * K + c, mx);
+}
+
+// Columns, pass 2: a CTA stages a tile of 128 rows x 32 columns of one node's share in shared memory
+// (read along the rows of the share, 256-byte segments), then every thread takes four consecutive
+// rows of one column (warp = column, four columns per warp in turn), cuts them into digits with the
+// column's exponent and writes them with the share's row index contiguous: [S][P][K][M].
+constexpr int RC_ROWS = 128, RC_COLS = 32, RC_PITCH = RC_ROWS + 1;
+template <int S>
+__global__ void __launch_bounds__(256) reslice_cols_kernel(const double* __restrict__ master, const unsigned int* amax,
+                                                          int8_t* planes, int* expo, int64_t M, int64_t K,
+                                                          int64_t plane_stride) {
+    __shared__ double xs[RC_COLS * RC_PITCH];
+    const int64_t c0 = (int64_t)blockIdx.x * RC_COLS, r0 = (int64_t)blockIdx.y * RC_ROWS, p = blockIdx.z;
+    const double* src = master + p * M * K;
+    for (int idx = threadIdx.x; idx < RC_ROWS * RC_COLS; idx += 256) {
+        const int cc = idx % RC_COLS, rr = idx / RC_COLS;
+        const int64_t gr = r0 + rr, gc = c0 + cc;
+        xs[cc * RC_PITCH + rr] = (gr < M && gc < K) ? src[gr * K + gc] : 0.0;
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t gr = r0 + 4 * lane;
+    for (int cc = warp; cc < RC_COLS; cc += 8) {
+        const int64_t gc = c0 + cc;
+        if (gc >= K) break;
+        const int e = slice_exponent(amax[p * K + gc]);
+        if (blockIdx.y == 0 && lane == 0) expo[p * K + gc] = e;
+        const double* col = xs + cc * RC_PITCH + 4 * lane;
+        const double a[4] = {col[0], col[1], col[2], col[3]};
+        unsigned int word[S];
+        digits4<S>(a, slice_scale<S>(e), word);
+        if (gr < M) {                                              // M is a multiple of 16: whole words
+            int8_t* dst = planes + (p * K + gc) * M + gr;
+#pragma unroll
+            for (int t = 0; t < S; ++t) *reinterpret_cast<unsigned int*>(dst + t * plane_stride) = word[t];
+        }
+    }
+}
+
 template <int NBLK>
 gpd_status launch_rows_fused(const SliceParams& prm, int slices, size_t smem, cudaStream_t st) {
     // CTA size follows the row length (one thread per four columns, at most 512); shorter rows run
@@ -405,14 +485,39 @@ bool sliced_supported(const gpd_plan_s* plan) {
     auto ok_blk = [](int n) {
         return n == 1 || n == 2 || n == 3 || n == 4 || n == 6 || n == 8 || n == 9 || n == 12 || n == 16;
     };
-    // int32 accumulation of up to 6 plane pairs of |digit| <= 128 over K terms
-    if (K % 16 != 0 || K > 16384 || !ok_blk(nb_w) || !ok_blk(nb_x)) return false;
+    auto ok_k = [](int64_t k) { return k % 16 == 0 && k <= 16384; };   // TMA rows of whole 16 bytes; int32 accumulation of
+                                                                        // up to 6 plane pairs of |digit| <= 128 over K terms
+    if (!ok_k(K) || !ok_blk(nb_w) || !ok_blk(nb_x)) return false;
     // scales are tracked through FP32 magnitudes of the inputs times the coefficients
     for (double c : plan->coefW) if (!(std::fabs(c) < 1e30)) return false;
     for (double c : plan->coefX) if (!(std::fabs(c) < 1e30)) return false;
     // the sliced operands live in buffers sized for the FP64 shares they replace
-    return sliced_layout(plan->slices, plan->P, M, K).total_bytes <= 8 * (int64_t)plan->P * M * K &&
-           sliced_layout(plan->slices, plan->P, N, K).total_bytes <= 8 * (int64_t)plan->P * N * K;
+    auto fits = [&](int64_t rows, int64_t k) {
+        return sliced_layout(plan->slices, plan->P, rows, k).total_bytes <= 8 * (int64_t)plan->P * rows * k;
+    };
+    if (!fits(M, K) || !fits(N, K)) return false;
+    if (plan->train) {
+        // backward product: contraction over N1/m, Delta~^T_p rows of B/d2; update: contraction over B
+        if (plan->prod[GPD_BWD].Q == 0 || plan->prod[GPD_AUDIT].Q == 0) return false;
+        if (!ok_k(M) || !ok_k(s.B) || !ok_k(s.B / c.d2) || !ok_k(N) || !ok_blk(c.d2 * c.m) || !ok_blk(c.m) || !ok_blk(c.n))
+            return false;
+        for (double c : plan->coefDT) if (!(std::fabs(c) < 1e30)) return false;
+        if (!fits(s.B / c.d2, M) || !fits(M, s.B) || !fits(K, s.B) || !fits(K, M)) return false;
+    }
+    return true;
+}
+
+TrainLayout train_layout(const gpd_plan_s* plan) {
+    const gpd_shape& s = plan->shape;
+    const gpd_split& c = plan->split;
+    const int64_t M = s.N1 / c.m, K = s.N0 / c.n, P = plan->P;
+    TrainLayout t;
+    t.rows = sliced_layout(plan->slices, P, M, K);
+    t.cols = sliced_layout(plan->slices, P, K, M);
+    t.rows_offset = (8 * P * M * K + 255) / 256 * 256;
+    t.cols_offset = (t.rows_offset + t.rows.total_bytes + 255) / 256 * 256;
+    t.total_bytes = t.cols_offset + t.cols.total_bytes;
+    return t;
 }
 
 SlicedLayout sliced_layout(int slices, int64_t P, int64_t rows, int64_t K) {
@@ -424,7 +529,35 @@ SlicedLayout sliced_layout(int slices, int64_t P, int64_t rows, int64_t K) {
     return l;
 }
 
-gpd_status encode_sliced_launch(gpd_plan_s* plan, bool is_A, const float* src, void* dst, cudaStream_t st) {
+gpd_status reslice_launch(gpd_plan_s* plan, void* W_shares, cudaStream_t st) {
+    if (!plan->train) return GPD_ERR_UNSUPPORTED;
+    const gpd_shape& s = plan->shape;
+    const gpd_split& c = plan->split;
+    const int64_t M = s.N1 / c.m, K = s.N0 / c.n, P = plan->P;
+    const TrainLayout tl = train_layout(plan);
+    char* base = reinterpret_cast<char*>(W_shares);
+    const double* master = reinterpret_cast<const double*>(base);
+    {   // rows of the shares
+        int8_t* planes = reinterpret_cast<int8_t*>(base + tl.rows_offset);
+        int* expo = reinterpret_cast<int*>(base + tl.rows_offset + tl.rows.expo_offset);
+        const int64_t n_rows = P * M;
+        reslice_rows_kernel<6><<<(unsigned)((n_rows + 7) / 8), 256, 0, st>>>(master, planes, expo, n_rows, K, P * M * K);
+        if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+    }
+    {   // columns of the shares
+        int8_t* planes = reinterpret_cast<int8_t*>(base + tl.cols_offset);
+        int* expo = reinterpret_cast<int*>(base + tl.cols_offset + tl.cols.expo_offset);
+        unsigned int* amax = reinterpret_cast<unsigned int*>(base + tl.cols_offset + tl.cols.amax_offset);
+        if (cudaMemsetAsync(amax, 0, sizeof(unsigned int) * P * K, st) != cudaSuccess) return GPD_ERR_CUDA;
+        colmax_kernel<<<dim3((unsigned)((K + 255) / 256), (unsigned)((M + 63) / 64), (unsigned)P), 256, 0, st>>>(master, amax, M, K);
+        if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+        reslice_cols_kernel<6><<<dim3((unsigned)((K + RC_COLS - 1) / RC_COLS), (unsigned)((M + RC_ROWS - 1) / RC_ROWS), (unsigned)P),
+                                 256, 0, st>>>(master, amax, planes, expo, M, K, P * M * K);
+    }
+    return launch_ok();
+}
+
+gpd_status encode_sliced_launch(gpd_plan_s* plan, int operand, const float* src, void* dst, cudaStream_t st) {
     // 16-byte loads of the source rows, word stores into the planes, aligned exponent tables
     if (reinterpret_cast<uintptr_t>(src) % 16 != 0 || reinterpret_cast<uintptr_t>(dst) % 16 != 0) return GPD_ERR_ARG;
     gpd_status rc = ensure_device(plan);
@@ -435,21 +568,34 @@ gpd_status encode_sliced_launch(gpd_plan_s* plan, bool is_A, const float* src, v
     prm.src = src;
     prm.P = plan->P;
     int gr;
-    if (is_A) {                   // W: m x n blocks of (N1/m) x (N0/n); operand rows = share rows, K = N0/n
-        gr = c.m; prm.gc = c.n; prm.ld = s.N0; prm.br = s.N1 / c.m; prm.bc = s.N0 / c.n;
-        prm.coef = plan->dev.base + plan->dev.off_coefW;
-    } else {                      // X: n x d1 blocks of (N0/n) x (B/d1); operand rows = share columns, K = N0/n
-        gr = c.n; prm.gc = c.d1; prm.ld = s.B; prm.br = s.N0 / c.n; prm.bc = s.B / c.d1;
-        prm.coef = plan->dev.base + plan->dev.off_coefX;
+    bool by_rows = true;          // operand rows = rows of the share (else: its columns, written transposed)
+    switch (operand) {
+        case -1:                  // W: m x n blocks of (N1/m) x (N0/n); operand rows = share rows, K = N0/n
+            gr = c.m; prm.gc = c.n; prm.ld = s.N0; prm.br = s.N1 / c.m; prm.bc = s.N0 / c.n;
+            prm.coef = plan->dev.base + plan->dev.off_coefW; break;
+        case GPD_OPERAND_X_FWD:   // X: n x d1 blocks of (N0/n) x (B/d1); operand rows = share columns, K = N0/n
+            gr = c.n; prm.gc = c.d1; prm.ld = s.B; prm.br = s.N0 / c.n; prm.bc = s.B / c.d1;
+            prm.coef = plan->dev.base + plan->dev.off_coefX; by_rows = false; break;
+        case GPD_OPERAND_DELTAT_BWD:   // Delta^T: d2 x m blocks of (B/d2) x (N1/m); operand rows = share rows, K = N1/m
+            gr = c.d2; prm.gc = c.m; prm.ld = s.N1; prm.br = s.B / c.d2; prm.bc = s.N1 / c.m;
+            prm.coef = plan->dev.base + plan->dev.off_coefDT; break;
+        case GPD_OPERAND_DELTA_UPD:    // Delta: m x 1 blocks of (N1/m) x B; operand rows = share rows, K = B
+            gr = c.m; prm.gc = 1; prm.ld = s.B; prm.br = s.N1 / c.m; prm.bc = s.B;
+            prm.coef = plan->dev.base + plan->dev.off_coefDup; break;
+        case GPD_OPERAND_X_UPD:        // X: n x 1 blocks of (N0/n) x B; operand rows = share rows, K = B
+            gr = c.n; prm.gc = 1; prm.ld = s.B; prm.br = s.N0 / c.n; prm.bc = s.B;
+            prm.coef = plan->dev.base + plan->dev.off_coefXup; break;
+        default: return GPD_ERR_ARG;
     }
+    if (operand != -1 && operand != GPD_OPERAND_X_FWD && !plan->train) return GPD_ERR_UNSUPPORTED;
     prm.nblk = gr * prm.gc;
-    const SlicedLayout lay = is_A ? sliced_layout(plan->slices, plan->P, prm.br, prm.bc)
-                                  : sliced_layout(plan->slices, plan->P, prm.bc, prm.br);
+    const SlicedLayout lay = by_rows ? sliced_layout(plan->slices, plan->P, prm.br, prm.bc)
+                                     : sliced_layout(plan->slices, plan->P, prm.bc, prm.br);
     prm.planes = reinterpret_cast<int8_t*>(dst);
     prm.expo = reinterpret_cast<int*>(reinterpret_cast<char*>(dst) + lay.expo_offset);
     prm.amax = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(dst) + lay.amax_offset);
 #define GPD_SLICE_CASE(NB) \
-    case NB: return is_A ? launch_rows<NB>(prm, plan->slices, st) : launch_cols<NB>(prm, plan->slices, st)
+    case NB: return by_rows ? launch_rows<NB>(prm, plan->slices, st) : launch_cols<NB>(prm, plan->slices, st)
     switch (prm.nblk) {
         GPD_SLICE_CASE(1); GPD_SLICE_CASE(2); GPD_SLICE_CASE(3); GPD_SLICE_CASE(4); GPD_SLICE_CASE(6);
         GPD_SLICE_CASE(8); GPD_SLICE_CASE(9); GPD_SLICE_CASE(12); GPD_SLICE_CASE(16);

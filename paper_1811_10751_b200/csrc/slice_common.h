@@ -1,5 +1,6 @@
-// Integer-slice product path (GPD_PREC_FP64_SLICED): layout of a sliced share buffer and the
-// entry points of its encoder (slice.cu) and of its tensor-core product (gemm_i8.cu).
+// Integer-slice product paths (GPD_PREC_FP64_SLICED, _SLICED40, _SLICED_TRAIN): layout of the sliced
+// share buffers and the entry points of their encoders (slice.cu) and of the tensor-core products
+// (gemm_i8.cu).
 #pragma once
 
 #include "gpd_internal.h"
@@ -21,16 +22,51 @@ struct SlicedLayout {
 };
 SlicedLayout sliced_layout(int slices, int64_t P, int64_t rows, int64_t K);
 
-// Whether the plan's shapes fit this path (K = N0/n a multiple of 16, block counts the encoder
-// is instantiated for, sliced buffers no larger than the FP64 share buffers they replace).
+// Share buffer of W in the training mode (GPD_PREC_FP64_SLICED_TRAIN), M = N1/m, K = N0/n:
+//   [0, rows_offset)            FP64 shares [P][M][K]: what the update accumulates into and what audit,
+//                               regeneration and share-error injection read and write
+//   [rows_offset, cols_offset)  the same values as a sliced operand with rows = share rows (K contiguous):
+//                               left operand of the forward product
+//   [cols_offset, total)        and as a sliced operand with rows = share columns (M contiguous): right
+//                               operand of the backward product
+// The two sliced copies are cut anew from the FP64 shares whenever those change.
+struct TrainLayout {
+    int64_t rows_offset, cols_offset, total_bytes;
+    SlicedLayout rows, cols;
+};
+TrainLayout train_layout(const gpd_plan_s* plan);
+
+// Whether the plan's shapes fit this path (contraction lengths multiples of 16 and at most 16384, block
+// counts the encoders are instantiated for, sliced buffers no larger than the FP64 buffers they replace).
 bool sliced_supported(const gpd_plan_s* plan);
 
-// W~_p (is_A) or X~_p -> sliced operand (W: rows of the share; X: columns of the share).
-gpd_status encode_sliced_launch(gpd_plan_s* plan, bool is_A, const float* src, void* dst, cudaStream_t st);
+// Encoders.  operand: -1 = W (gpd_encode_A), else a gpd_operand.  dst: the caller's share buffer.
+gpd_status encode_sliced_launch(gpd_plan_s* plan, int operand, const float* src, void* dst, cudaStream_t st);
+// Training mode: cut both sliced copies of W's shares from the FP64 shares at the start of the buffer.
+gpd_status reslice_launch(gpd_plan_s* plan, void* W_shares, cudaStream_t st);
 
-// S~_p = W~_p X~_p for all p from the two sliced operands, FP64 output [P][M][N].
-gpd_status gemm_sliced_launch(gpd_plan_s* plan, const void* W_sliced, const void* X_sliced, void* out,
-                              cudaStream_t st);
+// One batched int8 digit-plane product with FP64 recombination:
+//   C[p] (M x N, FP64, row-major) = A[p] (M x K) * B[p] (N x K)^T      for p = 0 .. P-1,
+// both operands sliced with K contiguous; update: C[p] <- shrink * C[p] + eta * A[p] B[p]^T, skipped
+// when gate reports a decoding failure.
+struct I8Gemm {
+    int slices, P;
+    const void* A; const int* ea; int64_t M;
+    const void* B; const int* eb; int64_t N;
+    int64_t K;
+    double* C;
+    bool update;
+    double shrink, eta;
+    const gpd_locate_result* gate;
+};
+gpd_status gemm_i8_launch(const I8Gemm& g, cudaStream_t st);
+
+// S~_p = W~_p X~_p (GPD_FWD) or C~^T_p = Delta~^T_p W~_p (GPD_BWD, training mode) from sliced operands.
+gpd_status gemm_sliced_launch(gpd_plan_s* plan, gpd_product which, const void* W_shares, const void* other_sliced,
+                              void* out, cudaStream_t st);
+// Training mode: FP64 shares <- shrink * shares + eta * Delta^_p X^_p^T, then both sliced copies re-cut.
+gpd_status update_sliced_launch(gpd_plan_s* plan, void* W_shares, const void* Dhat_sliced, const void* Xhat_sliced,
+                                double shrink, double eta, const gpd_locate_result* gate, cudaStream_t st);
 int i8_device_status_fetch_and_clear();
 
 }  // namespace gpd

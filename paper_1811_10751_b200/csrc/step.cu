@@ -24,7 +24,7 @@ extern "C" gpd_status coded_layer_step(gpd_plan_t plan, int32_t phases, void* W_
     if ((phases & ~(GPD_PHASE_FWD | GPD_PHASE_BWD | GPD_PHASE_UPD | GPD_PHASE_REGEN | GPD_PHASE_INJECT_SHARES)) ||
         !(phases & (GPD_PHASE_FWD | GPD_PHASE_BWD | GPD_PHASE_UPD)))
         return GPD_ERR_ARG;
-    if (plan->sliced && phases != GPD_PHASE_FWD) return GPD_ERR_UNSUPPORTED;   // digit-plane shares: forward only
+    if (plan->sliced && !plan->train && phases != GPD_PHASE_FWD) return GPD_ERR_UNSUPPORTED;   // forward-only digit-plane modes
     // every requested phase is checked before anything is enqueued
     if ((phases & GPD_PHASE_FWD) && (!X_dev || !S_out_dev)) return GPD_ERR_ARG;
     if ((phases & GPD_PHASE_BWD) && (!DeltaT_dev || !CT_out_dev)) return GPD_ERR_ARG;

@@ -1,5 +1,5 @@
-"""GPU parity of the integer-slice product paths (GPD_PREC_FP64_SLICED, GPD_PREC_FP64_SLICED40)
-against the FP64 oracle.
+"""GPU parity of the integer-slice product paths (GPD_PREC_FP64_SLICED, GPD_PREC_FP64_SLICED40,
+GPD_PREC_FP64_SLICED_TRAIN) against the FP64 oracle.
 
 The shares are stored as S = 6 (or 5) signed 8-bit digits per value under one power-of-two scale 2^e
 per operand row.  For a column of X~_p, 2^e lies in (2.03, 4.07] times the column's largest magnitude;
@@ -26,7 +26,7 @@ if not torch.cuda.is_available():
 
 import paper_1811_10751_b200 as g                        # noqa: E402
 from oracle import product as op                         # noqa: E402
-from oracle.code import GPCode, FWD                      # noqa: E402
+from oracle.code import GPCode, FWD, BWD                 # noqa: E402
 from oracle.locate import NO_ERROR, CORRECTED, locate_subspace, tolerances_for   # noqa: E402
 from oracle import inject as oinj                        # noqa: E402
 from tests.gpu_pipeline import CodedProduct, dev, host   # noqa: E402
@@ -223,3 +223,109 @@ def test_sliced_refuses_calls_on_other_shares():
     with pytest.raises(g.GpdError) as ei:
         g.gpd_regenerate_shares(cp.plan, cp.W_shares, cp.res, cp.ws)
     assert ei.value.status == g.GPD_ERR_UNSUPPORTED
+
+
+# --------------------------------------------------------------------------------------------------
+# training mode: every product of the coded step on digit planes, FP64 shares kept beside them
+# --------------------------------------------------------------------------------------------------
+def _pair_tolerance(rowmax_a, rowmax_b, K, slack_a=1.0, slack_b=1.0):
+    """Per-entry bound for A B^T from the largest magnitudes of A's and B's operand rows (scales lie
+    within 4.07 times those, times `slack` where the scale comes from a bound instead)."""
+    return 4.0 * np.sqrt(K) * PER_TERM[6] * (SCALE_OVER_MAX * slack_a * rowmax_a)[:, :, None] * \
+        (SCALE_OVER_MAX * slack_b * rowmax_b)[:, None, :]
+
+
+@pytest.mark.parametrize("N1,N0,B,m,n,P", [
+    (512, 256, 128, 2, 2, 10),          # whole tiles; thresholds 5 / 6 / 4
+    (416, 320, 48, 2, 4, 14),           # ragged tiles: 208-row and 80-column shares, batch 48; thresholds 11 / 12 / 8
+    (256, 128, 64, 4, 4, 36),           # the autoencoder's code: thresholds 19 / 28 / 16
+])
+def test_training_mode_products_update_and_audit_match_oracle(N1, N0, B, m, n, P):
+    rng = np.random.default_rng(N1 + N0 + B)
+    W = (rng.standard_normal((N1, N0)) / np.sqrt(N0)).astype(np.float32)
+    X = rng.standard_normal((N0, B)).astype(np.float32)
+    DT = (rng.standard_normal((B, N1)) / B).astype(np.float32)
+    Delta = np.ascontiguousarray(DT.T)
+    code = GPCode(N1, N0, B, m, n, 1, 1, P)
+    cp = CodedProduct(code, precision=g.GPD_PREC_FP64_SLICED_TRAIN)
+    assert cp.plan.query(g.GPD_Q_PRECISION) == g.GPD_PREC_FP64_SLICED_TRAIN and cp.np_dtype == np.float64
+    M, K = N1 // m, N0 // n
+    Wsh = cp.encode_W(W)
+    assert Wsh.numel() > P * M * K                                 # FP64 shares plus the two sliced copies
+    Ws_o = op.encode_W(W, code)
+    master = host(Wsh)[:P * M * K].reshape(P, M, K)
+    assert np.abs(master - Ws_o).max() <= 4e-16 * np.abs(Ws_o).max() * m * n
+    # forward product: rows of W~_p (exact row maxima) x columns of X~_p
+    Xs_o = op.encode_X(X, code)
+    Z = cp.outputs_as_array(g.GPD_FWD, cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X)))
+    Zo = op.worker_products(Ws_o, Xs_o)
+    tol = _pair_tolerance(np.abs(Ws_o).max(axis=2), np.abs(Xs_o).max(axis=1), K)
+    assert np.isfinite(Z).all() and (np.abs(Z - Zo) <= tol).all(), float((np.abs(Z - Zo) / tol).max())
+    # backward product: rows of Delta~^T_p (scale from the bound over its m blocks) x columns of W~_p
+    Ds_o = op.encode_DeltaT(DT, code)
+    Zb_t = cp.products(g.GPD_BWD, cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT))
+    Zb = cp.outputs_as_array(g.GPD_BWD, Zb_t)
+    Zbo = op.worker_products(Ds_o, Ws_o)
+    blk = np.abs(DT.astype(np.float64)).reshape(B, m, M).max(axis=2)                        # [B][m]
+    bound = np.einsum("pi,bi->pb", np.abs(code.points)[:, None] ** code.exp_DeltaT()[0][None, :], blk)
+    tol = _pair_tolerance(bound, np.abs(Ws_o).max(axis=1), M)
+    assert np.isfinite(Zb).all() and (np.abs(Zb - Zbo) <= tol).all(), float((np.abs(Zb - Zbo) / tol).max())
+    # the backward outputs go through location and decoding like any others
+    nodes = np.zeros(P, dtype=bool)
+    nodes[[1, P - 2][:min(2, P - code.Q_b - 1)]] = True             # as many as the backward product can correct
+    mask = sum(1 << int(q) for q in np.flatnonzero(nodes))
+    g.gpd_inject(cp.plan, g.GPD_BWD, Zb_t, 21, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=mask, scale=1.0)
+    Zr = Zbo.copy()
+    oinj.inject_gauss(Zr, 21, 1.0, nodes=nodes)
+    ro = locate_subspace(Zr, code.points, code.Q_b, tolerances_for(np.float64))
+    r = cp.locate(g.GPD_BWD, Zb_t)
+    assert r.outcome == ro.outcome == CORRECTED and np.array_equal(cp.flags(r), ro.flagged) and np.array_equal(ro.flagged, nodes)
+    CT = cp.decode(g.GPD_BWD, Zb_t)
+    assert op.rel_fro(CT, op.ref_backward(DT, W)) < 1e-4
+    assert op.rel_fro(CT, op.decode(Zr, code, BWD, use=~ro.flagged)) < 1e-4
+    # coded update with weight decay (Eq. 10): FP64 shares, then audit through the re-cut copies' source
+    eta, lam = 0.0625, 0.125
+    Dh_o, Xh_o = op.encode_update_operands(Delta, X, code)
+    g.gpd_update_shares(cp.plan, Wsh, cp.encode(g.GPD_OPERAND_DELTA_UPD, Delta), cp.encode(g.GPD_OPERAND_X_UPD, X), eta, lam)
+    want = op.update_shares(Ws_o, Dh_o, Xh_o, eta=eta, lam=lam)
+    got = host(Wsh)[:P * M * K].reshape(P, M, K)
+    dmax = np.einsum("pi,ri->pr", np.abs(code.points)[:, None] ** code.exp_update()[0][None, :],
+                     np.abs(Delta.astype(np.float64)).reshape(m, M, B).max(axis=2).T)       # bound of |Delta^_p| rows
+    xmax = np.einsum("pj,rj->pr", np.abs(code.points)[:, None] ** code.exp_update()[1][None, :],
+                     np.abs(X.astype(np.float64)).reshape(n, K, B).max(axis=2).T)
+    tol = eta * _pair_tolerance(dmax, xmax, B) + 4e-16 * np.abs(want).max()
+    assert (np.abs(got - want) <= tol).all(), float((np.abs(got - want) / tol).max())
+    r = cp.locate(g.GPD_AUDIT, Wsh)
+    assert r.outcome == NO_ERROR
+    assert op.rel_fro(cp.decode(g.GPD_AUDIT, Wsh), op.ref_update(W, Delta, X, eta, lam)) < 1e-4
+    # the forward product after the update reads the re-cut row copy: it must see the new shares
+    Z2 = cp.outputs_as_array(g.GPD_FWD, cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X)))
+    Z2o = op.worker_products(want, Xs_o)
+    tol = _pair_tolerance(np.abs(want).max(axis=2), np.abs(Xs_o).max(axis=1), K)
+    assert (np.abs(Z2 - Z2o) <= tol).all()
+    # and so must the backward product (column copy)
+    Zb2 = cp.outputs_as_array(g.GPD_BWD, cp.products(g.GPD_BWD, cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT)))
+    tol = _pair_tolerance(bound, np.abs(want).max(axis=1), M)
+    assert (np.abs(Zb2 - op.worker_products(Ds_o, want)) <= tol).all()
+    # share errors: written into the FP64 shares, seen by the next forward product, repaired by regeneration
+    g.gpd_inject(cp.plan, g.GPD_AUDIT, Wsh, 22, g.GPD_INJECT_GAUSS, prob=-1.0, node_mask=1 << 3, scale=0.1)
+    Zf_t = cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))
+    r = cp.locate(g.GPD_FWD, Zf_t)
+    assert r.outcome == CORRECTED and list(np.flatnonzero(cp.flags(r))) == [3]
+    g.gpd_regenerate_shares(cp.plan, Wsh, cp.res, cp.ws)
+    got = host(Wsh)[:P * M * K].reshape(P, M, K)
+    assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()
+    Z3 = cp.outputs_as_array(g.GPD_FWD, cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X)))
+    assert np.abs(Z3 - Z2o).max() <= 1e-10 * np.sqrt(np.mean(Z2o ** 2))
+    assert g.gpd_device_status() == 0
+
+
+def test_training_mode_rejects_shapes_it_cannot_serve():
+    # N1/m = 40 is not a multiple of 16 (backward contraction length)
+    with pytest.raises(g.GpdError) as ei:
+        g.gpd_plan((80, 64, 32), (2, 2, 1, 1), 10, precision=g.GPD_PREC_FP64_SLICED_TRAIN)
+    assert ei.value.status == g.GPD_ERR_UNSUPPORTED
+    # a forward-only plan (P below the backward threshold) has no use for it
+    with pytest.raises(g.GpdError) as ei:
+        g.gpd_plan((96, 64, 48), (3, 2, 1, 3), 9, precision=g.GPD_PREC_FP64_SLICED_TRAIN)
+    assert ei.value.status in (g.GPD_ERR_UNSUPPORTED, g.GPD_ERR_P_TOO_SMALL)

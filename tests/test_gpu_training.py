@@ -24,10 +24,10 @@ REL_TOL = 1e-4
 class GpuLayer:
     """Device state of one coded layer: plan, shares, workspace, results, outputs."""
 
-    def __init__(self, W: np.ndarray, B: int, m: int, n: int, P: int):
+    def __init__(self, W: np.ndarray, B: int, m: int, n: int, P: int, precision: int = g.GPD_PREC_AUTO):
         N1, N0 = W.shape
         self.N1, self.N0, self.B, self.P = N1, N0, B, P
-        self.plan = g.gpd_plan((N1, N0, B), (m, n, 1, 1), P)
+        self.plan = g.gpd_plan((N1, N0, B), (m, n, 1, 1), P, precision=precision)
         self.np_dtype = np.float32 if self.plan.query(g.GPD_Q_ELEMENT_SIZE) == 4 else np.float64
         self.W_shares = self.plan.empty(g.GPD_Q_W_SHARE_ELEMS)
         g.gpd_encode_A(self.plan, dev(W), self.W_shares)
@@ -293,10 +293,12 @@ def test_training_with_share_errors_and_regeneration():
         assert op.rel_fro(layers[l].audit(), U[l]) < REL_TOL
 
 
-def test_config5_full_size_two_steps():
+@pytest.mark.parametrize("precision", [g.GPD_PREC_AUTO, g.GPD_PREC_FP64_SLICED_TRAIN])
+def test_config5_full_size_two_steps(precision):
     """The sparse-autoencoder workload at full size (1024 <-> 8192, batch 1024, split 4 x 4, P = 36,
-    thresholds 19 / 28 / 16, FP64 path), two coded SGD steps with Gaussian node errors."""
-    _run_autoencoder(wl.CONFIG_5_AUTOENCODER, 2)
+    thresholds 19 / 28 / 16), two coded SGD steps with Gaussian node errors: on the FP64 mma path the
+    precision rule picks, and with every product on int8 digit planes (training mode)."""
+    _run_autoencoder(wl.CONFIG_5_AUTOENCODER, 2, precision)
 
 
 def test_config5_ten_steps_half_size():
@@ -304,16 +306,17 @@ def test_config5_ten_steps_half_size():
     split, node count, thresholds and error probability): the oracle's ten full-size steps take minutes."""
     cfg = wl.scaled_down(wl.CONFIG_5_AUTOENCODER, 2)
     assert cfg.steps == 10 and cfg.P == 36
-    _run_autoencoder(cfg, cfg.steps)
+    _run_autoencoder(cfg, cfg.steps, g.GPD_PREC_FP64_SLICED_TRAIN)
 
 
-def _run_autoencoder(cfg, n_steps):
+def _run_autoencoder(cfg, n_steps, precision):
     W1, W2, X = wl.autoencoder_inputs(cfg)
     enc_o = odnn.CodedLayer.from_weights(W1, GPCode(cfg.n_hidden, cfg.n_visible, cfg.B, cfg.m, cfg.n, 1, 1, cfg.P),
                                          inject_mode="gauss", inject_prob=cfg.inject_prob)
     dec_o = odnn.CodedLayer.from_weights(W2, GPCode(cfg.n_visible, cfg.n_hidden, cfg.B, cfg.m, cfg.n, 1, 1, cfg.P),
                                          inject_mode="gauss", inject_prob=cfg.inject_prob)
-    enc, dec = GpuLayer(W1, cfg.B, cfg.m, cfg.n, cfg.P), GpuLayer(W2, cfg.B, cfg.m, cfg.n, cfg.P)
+    enc = GpuLayer(W1, cfg.B, cfg.m, cfg.n, cfg.P, precision)
+    dec = GpuLayer(W2, cfg.B, cfg.m, cfg.n, cfg.P, precision)
     assert enc.np_dtype == np.float64
     Xd = dev(X)
     U1, U2 = W1.astype(np.float64), W2.astype(np.float64)
