@@ -636,7 +636,8 @@ def run_layer(args, kind, steps):
       mlp_layer: hidden layer of the MLP, 4096 x 4096 weights, batch 256, split 2 x 2, P = 10; thresholds
                  5 / 6, so FP32 shares and tensor-core 3xTF32 products
       sae_layer: encoder of the sparse autoencoder, 8192 x 1024 weights, batch 1024, split 4 x 4, P = 36;
-                 thresholds 19 / 28, so FP64 shares and FP64 mma products"""
+                 thresholds 19 / 28: FP64-class arithmetic, with every product on int8 digit planes
+                 (training mode; --precision fp64: FP64 shares and FP64 mma products)"""
     import torch
     import paper_1811_10751_b200 as g
     import workloads as wl
@@ -653,7 +654,12 @@ def run_layer(args, kind, steps):
     X = torch.randn((N0, B), device="cuda", generator=gen).clamp_(min=0)
     D = torch.randn((N1, B), device="cuda", generator=gen) / B
     DT = D.t().contiguous()
-    plan = g.gpd_plan((N1, N0, B), (m, n, 1, 1), P)
+    # thresholds above 9 (the autoencoder): every product on int8 digit planes (training mode) unless
+    # --precision fp64 asks for the FP64 mma path; thresholds up to 9 (the MLP): FP32 shares, 3xTF32
+    sliced = kind == "sae_layer" and args.precision != "fp64"
+    plan = g.gpd_plan((N1, N0, B), (m, n, 1, 1), P,
+                      precision=g.GPD_PREC_FP64_SLICED_TRAIN if sliced else g.GPD_PREC_AUTO)
+    g.gpd_plan_upload(plan)
     f32 = plan.query(g.GPD_Q_ELEMENT_SIZE) == 4
     Wsh = plan.empty(g.GPD_Q_W_SHARE_ELEMS)
     g.gpd_encode_A(plan, W, Wsh)
@@ -705,17 +711,31 @@ def run_layer(args, kind, steps):
         kern[name] = a.elapsed_time(b) / steps
     status = g.gpd_device_status()
     outcomes = [int(r.outcome) for r in g.read_results(res)[:2]]
+    extra = {}
     if f32:
         peak = measure_tf32_matmul_peak(torch) / 3.0
         kernel = "sgemm_3xtf32_kernel (forward products)"
         src = "measured here: torch.matmul TF32 8192^3 best of 10, divided by 3 (3xTF32)"
         dtype = "f32 (3xTF32 products, FP64 encode/locate/decode arithmetic)"
+    elif sliced:
+        peak, src = measure_int8_matmul_peak(torch)
+        if not peak:
+            peak = load_peaks()["bf16_burst"] * NOMINAL_INT8_TOPS / NOMINAL_BF16_TFLOPS
+            src += "; bf16 burst x nominal int8:bf16 ratio 2"
+        kernel = "gemm_i8_sliced_kernel (forward products, 21 digit-plane pairs)"
+        dtype = "f64 (products: int8 digit planes, exact int32 accumulation; FP64 shares beside the planes)"
+        fp64_peak = measure_fp64_matmul_peak(torch)
+        extra = {"fp64_equivalent_tflops": {k: 2.0 * P * (N1 // m) * (N0 // n) * B / (v * 1e-3) / 1e12 for k, v in kern.items()},
+                 "fp64_peak_measured_here": fp64_peak, "frac_of_nominal": None}
     else:
         peak = measure_fp64_matmul_peak(torch)
         kernel = "dgemm_mma_kernel (forward products)"
         src = "measured here: torch.matmul FP64 8192^3, best of 10 (cuBLAS)"
         dtype = "f64"
     flops = 2.0 * P * (N1 // m) * (N0 // n) * B               # flops of one product over all nodes
+    if sliced:
+        flops *= 21                                           # executed int8 operations: 21 plane pairs per product
+        extra["frac_of_nominal"] = flops / (kern["forward"] * 1e-3) / 1e12 / NOMINAL_INT8_TOPS
     useful = 3 * 2.0 * N1 * N0 * B
     line = {"metric": METRIC, "value": useful / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1, "steps": steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
@@ -728,7 +748,8 @@ def run_layer(args, kind, steps):
             "roofline": {"bound": "tensor", "kernel": kernel,
                          "achieved": flops / (kern["forward"] * 1e-3) / 1e12, "peak": peak, "unit": "TFLOP/s",
                          "frac": flops / (kern["forward"] * 1e-3) / 1e12 / peak, "traffic": None,
-                         "peak_source": src}}
+                         "peak_source": src, **extra}}
+    plan.destroy()
     return line
 
 
@@ -904,11 +925,13 @@ def main():
         if world == 1 and args.scale_down == 1 and not args.no_secondary:
             # one short run each of the other paths, so that a single default run observes them all
             short = max(3, min(args.steps, 10))
+            fp64_args = argparse.Namespace(**dict(vars(args), precision="fp64"))
             sec = {}
             for name, fn in (("matmul_fp64_mma", lambda: run_ours(args, cfg, "fp64", short, 1, full=False)),
                              ("matvec", lambda: run_matvec(args, short)),
                              ("mlp_layer", lambda: run_layer(args, "mlp_layer", short)),
                              ("sae_layer", lambda: run_layer(args, "sae_layer", short)),
+                             ("sae_layer_fp64_mma", lambda: run_layer(fp64_args, "sae_layer", short)),
                              ("positions", lambda: run_positions(args, short))):
                 try:
                     sec[name] = brief(fn())
