@@ -10,9 +10,12 @@
 // of MMAs loses up to one ulp of the running sum per step, always towards zero: over K = 2048
 // (768 steps) that is 1.4e-5 of the output's rms, which a threshold-9 decoder amplifies beyond
 // the 1e-4 bar.  The chain is therefore kept short: tensor memory only holds the partial sum of
-// group_kb k-blocks (one k-block: K = 32, 12 steps); the epilogue warps pull every finished partial sum into
-// FP32 registers, where the groups are added with round-to-nearest, and two accumulators in
-// tensor memory alternate so that one group drains while the next one is being multiplied.
+// group_kb k-blocks (one k-block: K = 32, 12 steps).  Two accumulators in tensor memory alternate
+// between groups; the eight warps that split the operands also pull every finished partial sum
+// into FP32 registers (each owns a lane quarter and half of the columns: 64 values per thread)
+// and add the groups up with round-to-nearest.  At a tile's end they write the sums back into
+// the accumulator they drained last, from where the four epilogue warps take them while the next
+// tile's main loop is already running.
 // Warp roles:
 //   warp 0       : TMA producer (one lane) - raw FP32 tiles of A and B into a 4-stage ring that
 //                  runs on across tiles
@@ -20,11 +23,10 @@
 //   warps 2..9   : split every landed pair of tiles: B in place in shared memory (hi overwrites the
 //                  raw tile, lo goes to a second tile); A row by row into tensor memory (hi and lo, 32
 //                  columns each per stage), from where the MMAs take it: the A operand then costs
-//                  shared-memory bandwidth once (its raw read) instead of four times
-//   warps 10..17 : read every finished group's partial sum back (tcgen05.ld; a warp owns one lane
-//                  quarter and one half of the columns), hand the accumulator back to the MMA warp,
-//                  add the partial sums up in registers and write the tile at its end (plain
-//                  store, or read-modify-write for the coded update)
+//                  shared-memory bandwidth once (its raw read) instead of four times.  Two k-blocks
+//                  behind their conversions they drain the finished accumulation groups (above)
+//   warps 10..13 : read a finished tile back (tcgen05.ld), hand the accumulator back to the MMA
+//                  warp, and write the tile (plain store, or read-modify-write for the coded update)
 // Operand tiles use the 128-byte swizzle; A is K-major; B is K-major for the update (X^_p is
 // [N][K]) and MN-major for the forward / backward products (X~_p, W~_p are [K][N]).
 // Tensor memory (512 columns): accumulators in columns 0..255, the A stages behind them.
@@ -54,10 +56,14 @@ constexpr int STAGE_BYTES = A_TILE_BYTES + 2 * B_TILE_BYTES;   // raw A, B hi, B
 // one chain of up to 256 elements is accurate enough there and keeps a whole tile of lead for the
 // read-modify-write.
 constexpr int kGroupKbProduct = 2, kGroupKbProductLarge = 1, kGroupKbUpdate = 8;
-constexpr int kEpiWarps = 8;                         // warps 10..17: lane quarter = warp mod 4, column half = (warp - 10) / 4
-constexpr int EPI_COLS = 16;                         // columns of a staged chunk
-constexpr int EPI_PITCH = 20;                        // floats per staged row: 16-byte aligned, conflict-free for 16-byte accesses
-constexpr int EPI_STAGE_BYTES = kEpiWarps * 32 * EPI_PITCH * 4;   // one 32 x 16 chunk per epilogue warp
+constexpr int kDrainLag = 2;                         // update kernel: a group is drained this many conversions after its last k-block
+constexpr int kEpiWarps = 4;                         // update kernel, warps 10..13: drain a finished tile, one per lane quarter
+constexpr int EPI_PITCH = 36;                        // floats per staged row: 16-byte aligned, conflict-free for 16-byte accesses
+constexpr int kEpiWarpsD = 8;                        // product kernel, warps 10..17: drain every group (64 columns of a lane quarter each)
+constexpr int EPI_COLS_D = 16;                       // product kernel: columns of a staged chunk
+constexpr int EPI_PITCH_D = 20;
+constexpr int EPI_STAGE_BYTES = kEpiWarpsD * 32 * EPI_PITCH_D * 4;   // one 32 x 16 chunk per warp (update kernel: 32 x 32 for four warps fits too)
+static_assert(kEpiWarps * 32 * EPI_PITCH * 4 <= EPI_STAGE_BYTES, "staging area of the update kernel");
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_STAGE_BYTES + 1024;
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr int TMEM_ACC_COLS = 2 * BN;                // two 128-column accumulators: one fills while the other drains
@@ -66,7 +72,12 @@ constexpr int TMEM_COLS = 512;
 static_assert(TMEM_ACC_COLS + STAGES * TMEM_A_COLS <= TMEM_COLS, "tensor memory budget");
 constexpr int kConvWarps = 8;                        // warps 2..9: split tiles
 constexpr int kConvThreads = kConvWarps * 32;
-constexpr int kThreads = 64 + kConvThreads + kEpiWarps * 32;
+// Who adds the groups up: the product kernel has eight epilogue warps for it (18 warps, 96 registers a
+// thread); the update kernel, which has one group per tile for mini-batches up to 256 and whose
+// read-modify-write epilogue wants wide chunks and a whole tile of lead, lets the splitting warps do
+// it (14 warps, 128 registers).  Measured on 10 x [2048 x 2048] x [2048 x 256]: products 0.178 ms with
+// the first arrangement and 0.207 ms with the second; update 0.217 ms and 0.147 ms.
+template <bool UPDATE> constexpr int kThreadsOf = 64 + kConvThreads + (UPDATE ? kEpiWarps : kEpiWarpsD) * 32;
 
 __device__ int g_tf32_status = 0;                    // GPD_ERR_TIMEOUT if a bounded wait expired
 
@@ -127,15 +138,19 @@ __device__ __forceinline__ float to_tf32(float x) {
 __device__ __forceinline__ float trunc_tf32(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
 template <bool B_KMAJOR, bool UPDATE>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsOf<UPDATE>, 1)
 sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams prm,
                     int tiles_m, int tiles_n, int full_tiles, int split, int n_virtual, int group_kb) {
     if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
+    constexpr bool EPI_DRAINS = !UPDATE;             // the epilogue warps (not the splitting warps) add the groups up
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // full / conv / empty: operand ring, runs on across the tiles of this CTA; acc_full[b] / acc_empty[b]:
     // accumulator b (tensor-memory columns 128 b ..) complete / read back
-    __shared__ __align__(8) uint64_t full_bar[STAGES], conv_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
+    // tile_full[t & 1]: tile t's sums are back in tensor memory (written by the eight splitting warps); two
+    // barriers, because tile t + 1 (the other accumulator) can be complete before the epilogue warps, still
+    // storing tile t - 1, start to wait for tile t
+    __shared__ __align__(8) uint64_t full_bar[STAGES], conv_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2], tile_full[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
@@ -167,8 +182,12 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], kEpiWarps);
+            // a group's accumulator is handed back by the eight splitting warps, a tile's last one by
+            // the four epilogue warps arriving twice each
+            mbar_init(&acc_empty[b], kConvWarps);
         }
+        mbar_init(&tile_full[0], kConvWarps);
+        mbar_init(&tile_full[1], kConvWarps);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -266,12 +285,75 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
         }
     } else if (warp < 2 + kConvWarps) {
-        // ------------------------------ split hi / lo ------------------------------
+        // ------------------------------ split hi / lo, drain groups ------------------------------
         const int tc = threadIdx.x - 64;             // 0..kConvThreads-1
         // A: this warp may touch tensor-memory lanes 32 q .. 32 q + 31 (q = warp mod 4); the two warps
         // of a quarter take 16 of the 32 k-columns each.  A thread owns one row of the tile.
         const int q = warp & 3, khalf = (warp - 2) >> 2;
         const int arow = q * 32 + lane;
+        // Accumulation groups: this warp adds up columns 64 khalf .. 64 khalf + 63 of its lane quarter.
+        const int n_groups = (num_kb + group_kb - 1) / group_kb;
+        int n_tiles_mine = 0;
+        for (int vt = blockIdx.x; vt < n_virtual; vt += gridDim.x) ++n_tiles_mine;
+        const int total_groups = n_tiles_mine * n_groups;
+        float acc[BN / 2];
+        int drained = 0;                             // groups drained so far, over all tiles
+        // index (over all tiles of this CTA) of the last k-block of group g
+        auto last_kblock = [&](int g) {
+            const int t = g / n_groups, j = g - t * n_groups;
+            return t * num_kb + min((j + 1) * group_kb, num_kb) - 1;
+        };
+        // Pull group g's partial sum into the registers; after a tile's last group write the sums back.
+        auto drain = [&](int g) -> bool {
+            const int t = g / n_groups, j = g - t * n_groups, buf = g & 1;
+            int p, m0, n0, bn;
+            decode(blockIdx.x + t * (int)gridDim.x, p, m0, n0, bn);
+            const bool ready = mbar_wait(&acc_full[buf], (g >> 1) & 1, abort_p);
+            __syncwarp();
+            if (!__all_sync(0xffffffffu, ready)) return false;   // tcgen05.ld is warp-collective: all lanes or none
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + khalf * (BN / 2));
+#pragma unroll
+            for (int c = 0; c < BN / 2; c += 32) {
+                if (khalf * (BN / 2) + c < bn) {     // strips are 64 or 32 columns wide
+                    uint32_t r[32];
+                    asm volatile(
+                        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                        : "r"(tbase + (uint32_t)c));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        acc[c + i] = j == 0 ? __uint_as_float(r[i]) : acc[c + i] + __uint_as_float(r[i]);
+                }
+            }
+            if (j < n_groups - 1) {                  // hand the accumulator back to the MMA warp
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                return true;
+            }
+            // the tile is complete: its sums go back into the accumulator just read, for the epilogue warps
+#pragma unroll
+            for (int c = 0; c < BN / 2; c += 16) {
+                if (khalf * (BN / 2) + c < bn) {
+                    uint32_t r[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(acc[c + i]);
+                    tmem_st16(tbase + (uint32_t)c, r);
+                }
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tile_full[t & 1]);
+            return true;
+        };
         int it = 0;
         bool ok = true;
         for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
@@ -317,102 +399,202 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&conv_bar[s]);
+                // groups whose last k-block was converted kDrainLag conversions ago: their MMAs have
+                // (nearly) finished, so the wait inside drain() is short
+                if constexpr (!EPI_DRAINS) {
+                    while (ok && drained < total_groups && it >= last_kblock(drained) + kDrainLag) ok = drain(drained++);
+                    if (!ok) break;
+                }
             }
+        }
+        if constexpr (!EPI_DRAINS) {
+            while (ok && drained < total_groups) ok = drain(drained++);   // what the lag left over
         }
     } else {
         // ------------------------------ epilogue ------------------------------
-        const int ew = warp - (2 + kConvWarps);      // 0..7
-        const int q = warp & 3;                      // this warp may touch TMEM lanes 32q .. 32q+31
-        const int ch = (ew >> 2) * (BN / 2);         // first of this warp's 64 columns of the tile
-        const float shrink = (float)prm.shrink, eta = (float)prm.eta;
-        const bool vec = (prm.N % 4 == 0);
-        const int n_groups = (num_kb + group_kb - 1) / group_kb;
-        float* st = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES) + ew * (32 * EPI_PITCH);
-        const int col4 = (lane & 3) * 4, rsub = lane >> 2;    // this lane's part of a staged 32 x 16 chunk
-        int gi = 0;
-        bool ok = true;
-        for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
-            int p, m0, n0, bn;
-            decode(vt, p, m0, n0, bn);
-            float acc[BN / 2];                       // this thread's row, this warp's columns
-            for (int g = 0; g < n_groups; ++g, ++gi) {
-                const int buf = gi & 1;
-                const bool acc_ready = mbar_wait(&acc_full[buf], (gi >> 1) & 1, abort_p);
-                __syncwarp();
-                if (!__all_sync(0xffffffffu, acc_ready)) { ok = false; break; }   // tcgen05.ld is warp-collective: all lanes or none
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-                for (int c = 0; c < BN / 2; c += 16) {
-                    if (ch + c < bn) {               // strips are 64 or 32 columns wide
-                        uint32_t r[16];
-                        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + ch + c);
-                        asm volatile(
-                            "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-                            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                              "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-                            : "r"(taddr));
-                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            acc[c + j] = g == 0 ? __uint_as_float(r[j]) : acc[c + j] + __uint_as_float(r[j]);
+        if constexpr (EPI_DRAINS) {
+            // products: eight warps (lane quarter = warp mod 4, column half = (warp - 10) / 4) pull every
+            // finished group into registers, add the groups up and store the tile at its end
+            const int ew = warp - (2 + kConvWarps);      // 0..7
+            const int q = warp & 3;                      // this warp may touch TMEM lanes 32q .. 32q+31
+            const int ch = (ew >> 2) * (BN / 2);         // first of this warp's 64 columns of the tile
+            const float shrink = (float)prm.shrink, eta = (float)prm.eta;
+            const bool vec = (prm.N % 4 == 0);
+            const int n_groups = (num_kb + group_kb - 1) / group_kb;
+            float* st = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES) + ew * (32 * EPI_PITCH_D);
+            const int col4 = (lane & 3) * 4, rsub = lane >> 2;    // this lane's part of a staged 32 x 16 chunk
+            int gi = 0;
+            bool ok = true;
+            for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
+                int p, m0, n0, bn;
+                decode(vt, p, m0, n0, bn);
+                float acc[BN / 2];                       // this thread's row, this warp's columns
+                for (int g = 0; g < n_groups; ++g, ++gi) {
+                    const int buf = gi & 1;
+                    const bool acc_ready = mbar_wait(&acc_full[buf], (gi >> 1) & 1, abort_p);
+                    __syncwarp();
+                    if (!__all_sync(0xffffffffu, acc_ready)) { ok = false; break; }   // tcgen05.ld is warp-collective: all lanes or none
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    #pragma unroll
+                    for (int c = 0; c < BN / 2; c += 16) {
+                        if (ch + c < bn) {               // strips are 64 or 32 columns wide
+                            uint32_t r[16];
+                            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + ch + c);
+                            asm volatile(
+                                "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                                "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                                  "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                                : "r"(taddr));
+                            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    #pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                acc[c + j] = g == 0 ? __uint_as_float(r[j]) : acc[c + j] + __uint_as_float(r[j]);
+                        }
+                    }
+                    // this group's partial sum is in registers: hand the accumulator back
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                }
+                if (!ok) break;
+                const int64_t gm = (int64_t)m0 + q * 32 + lane;
+                float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
+    #pragma unroll
+                for (int c0 = 0; c0 < BN / 2; c0 += EPI_COLS_D) {
+                    if (ch + c0 >= bn) break;
+                    const int64_t gc = (int64_t)n0 + ch + c0;           // first global column of the chunk
+                    const bool whole = vec && gc + EPI_COLS_D <= prm.N;
+                    if (whole) {
+                        // A thread holds the columns of one row; written as they are, a store would touch 32
+                        // rows with 16 bytes each.  A 32 x 16 chunk goes through shared memory instead and
+                        // leaves as 64-byte row segments (four lanes per row, eight rows per store).  The
+                        // update asks for the stored share before it stages the chunk.
+                        float4 old[4];
+                        if (UPDATE) {
+    #pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int64_t grow = (int64_t)m0 + q * 32 + 8 * i + rsub;
+                                old[i] = grow < prm.M ? *reinterpret_cast<const float4*>(C + grow * prm.N + gc + col4)
+                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+                            }
+                        }
+    #pragma unroll
+                        for (int j = 0; j < EPI_COLS_D; j += 4)
+                            *reinterpret_cast<float4*>(st + lane * EPI_PITCH_D + j) =
+                                make_float4(acc[c0 + j], acc[c0 + j + 1], acc[c0 + j + 2], acc[c0 + j + 3]);
+                        __syncwarp();
+    #pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int row = 8 * i + rsub;
+                            const int64_t grow = (int64_t)m0 + q * 32 + row;
+                            float4 v = *reinterpret_cast<const float4*>(st + row * EPI_PITCH_D + col4);
+                            if (grow < prm.M) {
+                                if (UPDATE) {
+                                    const float4 o = old[i];
+                                    v.x = shrink * o.x + eta * v.x; v.y = shrink * o.y + eta * v.y;
+                                    v.z = shrink * o.z + eta * v.z; v.w = shrink * o.w + eta * v.w;
+                                }
+                                *reinterpret_cast<float4*>(C + grow * prm.N + gc + col4) = v;
+                            }
+                        }
+                        __syncwarp();                        // the next chunk reuses the staging rows
+                    } else if (gm < prm.M) {
+                        float* crow = C + gm * prm.N + gc;
+    #pragma unroll
+                        for (int j = 0; j < EPI_COLS_D; ++j) {
+                            if (gc + j < prm.N) {
+                                float v = acc[c0 + j];
+                                if (UPDATE) v = shrink * crow[j] + eta * v;
+                                crow[j] = v;
+                            }
+                        }
                     }
                 }
-                // this group's partial sum is in registers: hand the accumulator back
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[buf]);
             }
-            if (!ok) break;
-            const int64_t gm = (int64_t)m0 + q * 32 + lane;
-            float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
-#pragma unroll
-            for (int c0 = 0; c0 < BN / 2; c0 += EPI_COLS) {
-                if (ch + c0 >= bn) break;
-                const int64_t gc = (int64_t)n0 + ch + c0;           // first global column of the chunk
-                const bool whole = vec && gc + EPI_COLS <= prm.N;
-                if (whole) {
-                    // A thread holds the columns of one row; written as they are, a store would touch 32
-                    // rows with 16 bytes each.  A 32 x 16 chunk goes through shared memory instead and
-                    // leaves as 64-byte row segments (four lanes per row, eight rows per store).  The
-                    // update asks for the stored share before it stages the chunk.
-                    float4 old[4];
-                    if (UPDATE) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int64_t grow = (int64_t)m0 + q * 32 + 8 * i + rsub;
-                            old[i] = grow < prm.M ? *reinterpret_cast<const float4*>(C + grow * prm.N + gc + col4)
+        } else {
+            // update: four warps read a finished tile back from tensor memory and apply it to the shares
+            const int q = warp & 3;                      // this warp may touch TMEM lanes 32q .. 32q+31
+            const float shrink = (float)prm.shrink, eta = (float)prm.eta;
+            const bool vec = (prm.N % 4 == 0);
+            const int n_groups = (num_kb + group_kb - 1) / group_kb;
+            int ti = 0;
+            for (int vt = blockIdx.x; vt < n_virtual; vt += gridDim.x, ++ti) {
+                int p, m0, n0, bn;
+                decode(vt, p, m0, n0, bn);
+                const int buf = ((ti + 1) * n_groups - 1) & 1;      // the accumulator of the tile's last group holds its sums
+                const bool tile_ready = mbar_wait(&tile_full[ti & 1], (ti >> 1) & 1, abort_p);
+                __syncwarp();
+                if (!__all_sync(0xffffffffu, tile_ready)) break;   // tcgen05.ld is warp-collective: all lanes or none
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const int64_t gm = (int64_t)m0 + q * 32 + lane;
+                float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
+    #pragma unroll 1
+                for (int c0 = 0; c0 < bn; c0 += 32) {
+                    const bool whole = vec && n0 + c0 + 32 <= prm.N;     // the chunk leaves as 128-byte row segments
+                    const int col4 = (lane & 7) * 4, rsub = lane >> 3;   // this lane's part of a staged chunk
+                    float4 old[8];                                       // the stored share, asked for before the accumulator is read
+                    if (UPDATE && whole) {
+    #pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int64_t grow = (int64_t)m0 + q * 32 + 4 * i + rsub;
+                            old[i] = grow < prm.M ? *reinterpret_cast<const float4*>(C + grow * prm.N + n0 + c0 + col4)
                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
                     }
-#pragma unroll
-                    for (int j = 0; j < EPI_COLS; j += 4)
-                        *reinterpret_cast<float4*>(st + lane * EPI_PITCH + j) =
-                            make_float4(acc[c0 + j], acc[c0 + j + 1], acc[c0 + j + 2], acc[c0 + j + 3]);
-                    __syncwarp();
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int row = 8 * i + rsub;
-                        const int64_t grow = (int64_t)m0 + q * 32 + row;
-                        float4 v = *reinterpret_cast<const float4*>(st + row * EPI_PITCH + col4);
-                        if (grow < prm.M) {
-                            if (UPDATE) {
-                                const float4 o = old[i];
-                                v.x = shrink * o.x + eta * v.x; v.y = shrink * o.y + eta * v.y;
-                                v.z = shrink * o.z + eta * v.z; v.w = shrink * o.w + eta * v.w;
-                            }
-                            *reinterpret_cast<float4*>(C + grow * prm.N + gc + col4) = v;
-                        }
+                    uint32_t r[32];
+                    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0);
+                    asm volatile(
+                        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                        : "r"(taddr));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (c0 + 32 >= bn) {                 // last read of this accumulator: hand it back (two arrivals per warp)
+                        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) { mbar_arrive(&acc_empty[buf]); mbar_arrive(&acc_empty[buf]); }
                     }
-                    __syncwarp();                        // the next chunk reuses the staging rows
-                } else if (gm < prm.M) {
-                    float* crow = C + gm * prm.N + gc;
-#pragma unroll
-                    for (int j = 0; j < EPI_COLS; ++j) {
-                        if (gc + j < prm.N) {
-                            float v = acc[c0 + j];
-                            if (UPDATE) v = shrink * crow[j] + eta * v;
-                            crow[j] = v;
+                    if (whole) {
+                        // A thread holds 32 columns of one row; written as they are, a store would touch 32
+                        // rows with 16 bytes each.  The chunk goes through shared memory instead and
+                        // leaves as whole 128-byte row segments (eight lanes per row, four rows per store).
+                        float* st = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES) + (warp - 2 - kConvWarps) * (32 * EPI_PITCH);
+    #pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4*>(st + lane * EPI_PITCH + j) =
+                                make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
+                                            __uint_as_float(r[j + 3]));
+                        __syncwarp();
+    #pragma unroll
+                        for (int rr = 0; rr < 32; rr += 4) {
+                            const int row = rr + rsub;
+                            const int64_t grow = (int64_t)m0 + q * 32 + row;
+                            float4 v = *reinterpret_cast<const float4*>(st + row * EPI_PITCH + col4);
+                            if (grow < prm.M) {
+                                float* cp = C + grow * prm.N + n0 + c0 + col4;
+                                if (UPDATE) {
+                                    const float4 o = old[rr / 4];
+                                    v.x = shrink * o.x + eta * v.x; v.y = shrink * o.y + eta * v.y;
+                                    v.z = shrink * o.z + eta * v.z; v.w = shrink * o.w + eta * v.w;
+                                }
+                                *reinterpret_cast<float4*>(cp) = v;
+                            }
+                        }
+                        __syncwarp();                        // the next chunk reuses the staging rows
+                    } else if (gm < prm.M) {
+                        float* crow = C + gm * prm.N + n0 + c0;
+    #pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (n0 + c0 + j < prm.N) {
+                                float v = __uint_as_float(r[j]);
+                                if (UPDATE) v = shrink * crow[j] + eta * v;
+                                crow[j] = v;
+                            }
                         }
                     }
                 }
@@ -459,7 +641,7 @@ gpd_status launch(const GemmParams& prm, cudaStream_t st) {
     const int64_t n_virtual = full_tiles + (int64_t)(split > 1 ? rem : 0) * split;
     const unsigned grid = (unsigned)std::min<int64_t>(n_virtual, sms);   // persistent: one CTA per SM walks the list
     const int group_kb = UPDATE ? kGroupKbUpdate : (prm.max_threshold >= 7 ? kGroupKbProductLarge : kGroupKbProduct);
-    sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<grid, kThreads, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n, full_tiles,
+    sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<grid, kThreadsOf<UPDATE>, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n, full_tiles,
                                                                               split, (int)n_virtual, group_kb);
     return launch_ok();
 }

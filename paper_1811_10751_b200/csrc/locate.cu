@@ -115,6 +115,14 @@ __global__ void __launch_bounds__(kThreads, RT <= 8 ? 4 : (RT <= 24 ? 2 : 1)) sy
     const int64_t n_batches = (prm.L + kThreads - 1) / kThreads;
     for (int64_t batch = blockIdx.x; batch < n_batches; batch += gridDim.x) {
         const int64_t l = batch * kThreads + threadIdx.x;
+        {   // The syndrome registers leave room for few loads in flight per thread, so the codeword of this
+            // thread's next trip is asked for now and waits in L2 when its loads are issued.
+            const int64_t ln = l + (int64_t)gridDim.x * kThreads;
+            if (RT > 8 && ln < prm.L) {          // up to eight parity checks: nine loads in flight already, no gain
+                const T* zn = Z + ln;
+                for (int pn = 0; pn < prm.P; ++pn, zn += prm.L) asm volatile("prefetch.global.L2 [%0];" ::"l"(zn));
+            }
+        }
         double s[RT];
         double nz = 0.0;
         if (l < prm.L) {

@@ -78,6 +78,8 @@ def test_encode_matches_oracle(N1, N0, B, m, n, d1, d2, P, prec):
     (512, 512, 256, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),        # tcgen05 3xTF32 tiles, exact multiples
     (400, 272, 200, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),        # tcgen05 path with ragged M, N and K
     (2048, 1024, 256, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),      # many k-blocks: the stage ring wraps
+    (512, 768, 1000, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),       # mini-batch 1000: the update's contraction spans four
+                                                             # accumulation groups (the last one short)
     (10, 512, 64, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),          # 5-row blocks
     (1024, 512, 1, 4, 2, 1, 1, 13, g.GPD_PREC_FP32),         # matrix-vector
     (1024, 512, 1, 4, 2, 1, 1, 13, g.GPD_PREC_FP64),
