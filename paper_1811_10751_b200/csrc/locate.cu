@@ -82,7 +82,8 @@ __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P,
     }
 }
 
-// One thread per output position (codeword): the syndrome in RT registers, the zero test.  The
+// Streaming pass for up to eight parity checks.  One thread per output position (codeword): the
+// syndrome in RT registers, the zero test.  The
 // Gram matrix of the failing codewords is formed warp by warp on the FP64 tensor cores: the 32 scaled syndromes of a warp are staged in shared
 // memory and fed to mma.m8n8k4 as both operands (G += S S^T, four codewords per instruction), so
 // the accumulator costs two registers per 8 x 8 tile and the streaming loop needs no CTA barrier.
@@ -167,6 +168,219 @@ __global__ void __launch_bounds__(kThreads, RT <= 8 ? 4 : (RT <= 24 ? 2 : 1)) sy
             if (acc[a][b][0] != 0.0) atomicAdd(&sG[r * RT + c], acc[a][b][0]);
             if (acc[a][b][1] != 0.0) atomicAdd(&sG[r * RT + c + 1], acc[a][b][1]);
         }
+    unsigned int act = my_active;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        act += __shfl_xor_sync(0xffffffffu, act, o);
+        bad_all |= __shfl_xor_sync(0xffffffffu, bad_all, o);
+    }
+    if (lane == 0) {
+        if (act) atomicAdd(&prm.counts[0], (unsigned long long)act);
+        if (bad_all) atomicOr(&prm.counts[1], bad_all);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < prm.R * prm.R; i += kThreads) {
+        const int r = i / prm.R, c = i % prm.R;
+        if (r <= c && sG[r * RT + c] != 0.0) atomicAdd(&prm.gram[r * prm.R + c], sG[r * RT + c]);
+    }
+}
+
+// Streaming pass for more than eight parity checks (the syndrome no longer fits beside enough loads in
+// flight in one thread's registers).  A warp takes 32 consecutive output positions at a time and forms their syndromes
+// on the FP64 tensor cores: S (RT x 32) = H (RT x P) Z (P x 32) as mma.m8n8k4 tiles, H's fragments from
+// shared memory, Z's fragments loaded straight from global memory (a lane owns one node of a k-step
+// of four and one of eight positions of a tile; the four tiles of a k-step cover 4 rows x 256 bytes),
+// the accumulators in 2 * NT * 4 registers per lane.  Against one thread per codeword with the whole
+// syndrome in its registers this needs an eighth of the arithmetic instructions, no shared-memory
+// operand reads per node, and leaves registers for many loads in flight.  Squared norms of the
+// codewords and of the syndromes are met by shuffles; the zero test follows per position.  The Gram
+// matrix of the failing codewords is formed warp by warp on the tensor cores as well: the 32
+// scaled syndromes of a warp are staged in shared memory and fed to mma.m8n8k4 as both operands
+// (G += S S^T, four codewords per instruction).  A block of positions that holds a non-finite or
+// huge value, and every block when nodes are erased, is redone codeword by codeword with the checked
+// form above.
+template <typename T, int RT>
+__global__ void __launch_bounds__(kThreads, RT <= 24 ? 2 : 1) syndrome_gram_mma_kernel(SyndromeParams prm) {
+    constexpr int NT = RT / 8;                          // 8 x 8 tiles per side of the Gram matrix
+    constexpr int LD = RT + 4;                          // row pitch of the staging buffer (bank spread)
+    constexpr int kWarps = kThreads / 32;
+    constexpr int UK = 2;                               // k-steps (of four nodes) per chunk of loads; two chunks are in flight
+    constexpr int NG = NT * (NT + 1) / 2;               // 8 x 8 tiles of the Gram matrix's upper triangle
+    extern __shared__ __align__(16) double sm[];
+    double* sH = sm;                                    // [P4][RT] node-major, rows >= R and nodes >= P are zero
+    const int P4 = (prm.P + 3) & ~3;
+    double* sS = sm + RT * P4;                          // [kWarps][32][LD]
+    double* sA = sS + kWarps * 32 * LD;                 // [kWarps][NG][32][2] Gram fragments of every warp (kept out of the registers)
+    double* sG = sA + kWarps * NG * 64;                 // [RT][RT] CTA total
+    for (int i = threadIdx.x; i < RT * P4; i += kThreads) {
+        const int pnode = i / RT, r = i % RT;
+        sH[i] = (r < prm.R && pnode < prm.P) ? prm.H[r * prm.P + pnode] : 0.0;
+    }
+    for (int i = threadIdx.x; i < kWarps * NG * 64; i += kThreads) sA[i] = 0.0;
+    for (int i = threadIdx.x; i < RT * RT; i += kThreads) sG[i] = 0.0;
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int kq = lane & 3, nq = lane >> 2;            // node within a k-step / position within a tile (fragment coordinates)
+    double* myS = sS + warp * 32 * LD;
+    double2* myA = reinterpret_cast<double2*>(sA + warp * NG * 64) + lane;   // fragment g of this lane: myA[32 g]
+    unsigned long long bad_all = 0ULL;
+    unsigned int my_active = 0;
+    const T* Z = reinterpret_cast<const T*>(prm.Z);
+    const int n_ksteps = P4 >> 2;
+    const int n_chunks = (n_ksteps + UK - 1) / UK;
+    const int64_t n_blocks = (prm.L + 31) / 32;
+    const int64_t stride = (int64_t)gridDim.x * kWarps;
+    for (int64_t blk = (int64_t)blockIdx.x * kWarps + warp; blk < n_blocks; blk += stride) {
+        const int64_t base = blk * 32;
+        bool any_active = false;
+        bool redo = prm.erased != 0ULL;
+        if (!redo) {
+            {   // this warp's next block: asked for now, waiting in L2 when its loads are issued
+                const int64_t nb = (blk + stride) * 32 + 8 * kq;       // lane (kq, nq): 64-byte piece kq of node nq, nq + 8, ...
+                if (nb < prm.L)
+                    for (int pn = nq; pn < prm.P; pn += 8) asm volatile("prefetch.global.L2 [%0];" ::"l"(Z + (int64_t)pn * prm.L + nb));
+            }
+            double d[NT][4][2];                          // syndromes: rows 8 mt + nq, positions 8 t + 2 kq + {0, 1}
+            double pz[4] = {0.0, 0.0, 0.0, 0.0};         // this lane's share of ||z||^2 of position 8 t + nq
+#pragma unroll
+            for (int mt = 0; mt < NT; ++mt)
+#pragma unroll
+                for (int t = 0; t < 4; ++t) d[mt][t][0] = d[mt][t][1] = 0.0;
+            auto load_chunk = [&](int c, double (&z)[UK][4]) {
+#pragma unroll
+                for (int u = 0; u < UK; ++u) {
+                    const int ks = c * UK + u, node = 4 * ks + kq;
+                    const T* zp = Z + (int64_t)node * prm.L + base + nq;
+#pragma unroll
+                    for (int t = 0; t < 4; ++t)
+                        z[u][t] = (ks < n_ksteps && node < prm.P && base + 8 * t + nq < prm.L) ? (double)__ldcs(zp + 8 * t) : 0.0;
+                }
+            };
+            auto use_chunk = [&](int c, const double (&z)[UK][4]) {
+#pragma unroll
+                for (int u = 0; u < UK; ++u) {
+                    const int ks = c * UK + u;
+                    if (ks < n_ksteps) {                 // warp-uniform
+                        const double* hp = sH + (4 * ks + kq) * RT + nq;
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) pz[t] = fma(z[u][t], z[u][t], pz[t]);
+#pragma unroll
+                        for (int mt = 0; mt < NT; ++mt) {
+                            const double h = hp[8 * mt];
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) dmma_m8n8k4(d[mt][t][0], d[mt][t][1], h, z[u][t]);
+                        }
+                    }
+                }
+            };
+            double za[UK][4], zb[UK][4];                 // two chunks: one being multiplied, one in flight
+            load_chunk(0, za);
+            for (int c = 0; c < n_chunks; c += 2) {
+                if (c + 1 < n_chunks) load_chunk(c + 1, zb);
+                use_chunk(c, za);
+                if (c + 2 < n_chunks) load_chunk(c + 2, za);
+                if (c + 1 < n_chunks) use_chunk(c + 1, zb);
+            }
+            // ||z||^2 of position 8 t + nq: sum over the four lanes of the position
+            bool huge = false;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                pz[t] += __shfl_xor_sync(0xffffffffu, pz[t], 1);
+                pz[t] += __shfl_xor_sync(0xffffffffu, pz[t], 2);
+                huge |= !(pz[t] < kHugeSquared);
+            }
+            redo = __any_sync(0xffffffffu, huge);
+            if (!redo) {
+                bool act_any = false;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        double ns = 0.0;                 // ||s||^2 of position 8 t + 2 kq + e: over the tiles, then over the eight row lanes
+#pragma unroll
+                        for (int mt = 0; mt < NT; ++mt) ns = fma(d[mt][t][e], d[mt][t][e], ns);
+                        ns += __shfl_xor_sync(0xffffffffu, ns, 4);
+                        ns += __shfl_xor_sync(0xffffffffu, ns, 8);
+                        ns += __shfl_xor_sync(0xffffffffu, ns, 16);
+                        const double nz = __shfl_sync(0xffffffffu, pz[t], (2 * kq + e) * 4);
+                        const bool active = (nz > 0.0) && (ns > prm.tau2 * nz);
+                        act_any |= active;
+                        if (nq == 0) my_active += active ? 1u : 0u;     // one of the eight row lanes counts
+                        const double w = active ? rsqrt(nz) : 0.0;
+#pragma unroll
+                        for (int mt = 0; mt < NT; ++mt) d[mt][t][e] *= w;
+                    }
+                }
+                any_active = __any_sync(0xffffffffu, act_any);
+                if (any_active) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e)
+#pragma unroll
+                            for (int mt = 0; mt < NT; ++mt) myS[(8 * t + 2 * kq + e) * LD + 8 * mt + nq] = d[mt][t][e];
+                }
+            }
+        }
+        if (redo) {                                      // lane = position, checked values
+            const int64_t l = base + lane;
+            double s[RT];
+            double nz = 0.0;
+            if (l < prm.L) {
+                codeword_syndrome<T, RT, true>(Z + l, prm.L, prm.P, sH, prm.erased, s, nz, bad_all);
+            } else {
+#pragma unroll
+                for (int r = 0; r < RT; ++r) s[r] = 0.0;
+            }
+            double ns = 0.0;
+#pragma unroll
+            for (int r = 0; r < RT; ++r) ns = fma(s[r], s[r], ns);
+            const bool active = (nz > 0.0) && (ns > prm.tau2 * nz);
+            my_active += active ? 1u : 0u;
+            any_active = __any_sync(0xffffffffu, active);
+            if (any_active) {
+                const double w = active ? rsqrt(nz) : 0.0;
+                double2* row = reinterpret_cast<double2*>(myS + lane * LD);
+#pragma unroll
+                for (int r = 0; r < RT / 2; ++r) row[r] = make_double2(s[2 * r] * w, s[2 * r + 1] * w);
+            }
+        }
+        if (any_active) {                                // G += sum over the block's codewords of s s^T / ||z||^2
+            __syncwarp();
+            double acc[NG][2];
+#pragma unroll
+            for (int g = 0; g < NG; ++g) { const double2 v = myA[32 * g]; acc[g][0] = v.x; acc[g][1] = v.y; }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {                // codewords 4j .. 4j+3 of the block
+                const double* src = myS + (4 * j + (lane & 3)) * LD + (lane >> 2);
+                double f[NT];
+#pragma unroll
+                for (int a = 0; a < NT; ++a) f[a] = src[8 * a];
+                int g = 0;
+#pragma unroll
+                for (int a = 0; a < NT; ++a)
+#pragma unroll
+                    for (int b = a; b < NT; ++b, ++g) dmma_m8n8k4(acc[g][0], acc[g][1], f[a], f[b]);   // upper triangle
+            }
+#pragma unroll
+            for (int g = 0; g < NG; ++g) myA[32 * g] = make_double2(acc[g][0], acc[g][1]);
+            __syncwarp();
+        }
+    }
+    // warp fragments -> CTA total (shared atomics) -> global (one atomic per upper-triangle entry)
+    {
+        int g = 0;
+#pragma unroll
+        for (int a = 0; a < NT; ++a)
+#pragma unroll
+            for (int b = a; b < NT; ++b, ++g) {
+                const double2 v = myA[32 * g];
+                const int r = 8 * a + (lane >> 2), c = 8 * b + 2 * (lane & 3);
+                if (v.x != 0.0) atomicAdd(&sG[r * RT + c], v.x);
+                if (v.y != 0.0) atomicAdd(&sG[r * RT + c + 1], v.y);
+            }
+    }
     unsigned int act = my_active;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -656,15 +870,22 @@ inline gpd_status launch_finish(const FinishParams& fp, cudaStream_t st) {
 
 template <typename T, int RT>
 gpd_status launch_syndrome(const SyndromeParams& prm, cudaStream_t st) {
-    const size_t smem = sizeof(double) * ((size_t)RT * prm.P + (size_t)kThreads * (RT + 4) + (size_t)RT * RT);
-    if (smem > 48 * 1024) {
-        if (cudaFuncSetAttribute(syndrome_gram_kernel<T, RT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem) != cudaSuccess)
+    if constexpr (RT <= 8) {
+        const size_t smem = sizeof(double) * ((size_t)RT * prm.P + (size_t)kThreads * (RT + 4) + (size_t)RT * RT);
+        const int64_t batches = (prm.L + kThreads - 1) / kThreads;
+        const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(batches, sm_count() * 4));
+        syndrome_gram_kernel<T, RT><<<grid, kThreads, smem, st>>>(prm);
+    } else {
+        constexpr int NG = (RT / 8) * (RT / 8 + 1) / 2;
+        const size_t smem = sizeof(double) * ((size_t)RT * ((prm.P + 3) & ~3) + (size_t)kThreads * (RT + 4) +
+                                              (size_t)(kThreads / 32) * NG * 64 + (size_t)RT * RT);
+        if (smem > 48 * 1024 &&
+            cudaFuncSetAttribute(syndrome_gram_mma_kernel<T, RT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return GPD_ERR_CUDA;
+        const int64_t batches = (prm.L + kThreads - 1) / kThreads;
+        const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(batches, sm_count() * (RT <= 24 ? 2 : 1)));
+        syndrome_gram_mma_kernel<T, RT><<<grid, kThreads, smem, st>>>(prm);
     }
-    const int64_t batches = (prm.L + kThreads - 1) / kThreads;
-    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>(batches, sm_count() * 4));
-    syndrome_gram_kernel<T, RT><<<grid, kThreads, smem, st>>>(prm);
     return launch_ok();
 }
 
