@@ -92,6 +92,10 @@ using tc::umma_commit;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     return tc::mbar_wait(bar, parity, abort_flag, &g_tf32_status);
 }
+// for the epilogue warps: they wait most of the time, and a poll every 200 ns is early enough for them
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    return tc::mbar_wait(bar, parity, abort_flag, &g_tf32_status, kWaitCycles, 200);
+}
 
 // Shared-memory matrix descriptor: start address, leading / stride byte offsets in 16-byte units,
 // descriptor version 1, layout type (2 = 128-byte swizzle of 16-byte chunks, used for K-major
@@ -431,7 +435,7 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 float acc[BN / 2];                       // this thread's row, this warp's columns
                 for (int g = 0; g < n_groups; ++g, ++gi) {
                     const int buf = gi & 1;
-                    const bool acc_ready = mbar_wait(&acc_full[buf], (gi >> 1) & 1, abort_p);
+                    const bool acc_ready = mbar_wait_relaxed(&acc_full[buf], (gi >> 1) & 1, abort_p);
                     __syncwarp();
                     if (!__all_sync(0xffffffffu, acc_ready)) { ok = false; break; }   // tcgen05.ld is warp-collective: all lanes or none
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -523,7 +527,7 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 int p, m0, n0, bn;
                 decode(vt, p, m0, n0, bn);
                 const int buf = ((ti + 1) * n_groups - 1) & 1;      // the accumulator of the tile's last group holds its sums
-                const bool tile_ready = mbar_wait(&tile_full[ti & 1], (ti >> 1) & 1, abort_p);
+                const bool tile_ready = mbar_wait_relaxed(&tile_full[ti & 1], (ti >> 1) & 1, abort_p);
                 __syncwarp();
                 if (!__all_sync(0xffffffffu, tile_ready)) break;   // tcgen05.ld is warp-collective: all lanes or none
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");

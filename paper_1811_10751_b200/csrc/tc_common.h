@@ -35,11 +35,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait: false if the phase did not complete within `limit` cycles or the CTA is aborting.
 // On expiry the CTA's abort flag is set and GPD_ERR_TIMEOUT is written to *status (a __device__
 // word the host reads back), so that every other waiter of the CTA gives up as well.
+// backoff_ns > 0: sleep that long between polls (for waiters off the critical path, so that their polling
+// does not take issue slots from the warps that are on it).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          long long limit = kWaitCycles) {
+                                          long long limit = kWaitCycles, unsigned backoff_ns = 0) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
+        if (backoff_ns) __nanosleep(backoff_ns);
         if (*abort_flag) return false;
         if (clock64() - t0 > limit) {
             *abort_flag = 1;
