@@ -8,10 +8,9 @@
 // CTA through a shared-memory SYRK and added to global memory with one atomic per entry.
 // Non-finite values and erased nodes count as zero and their node is flagged up front.
 //
-// Pass 2 (one warp): eigen-decomposition of G (pivoted Cholesky down to its numerical rank, then
-// cyclic Jacobi on the small matrix L^T L); numerical rank rho; the error
-// support is the set of nodes whose parity-check column H_p lies in the span of the top-rho
-// eigenvectors (any P-Q columns of H are independent, so for at most P-Q-1 erroneous nodes no
+// Pass 2 (one warp): pivoted Cholesky factorisation of G: numerical rank rho (pivots above the
+// eigenvalue threshold) and range (its leading rho columns); the error
+// support is the set of nodes whose parity-check column H_p lies in that range (any P-Q columns of H are independent, so for at most P-Q-1 erroneous nodes no
 // other column does); the support is verified by the syndrome energy left outside span(H_A).
 // A rank-deficient error matrix (fewer columns of H in that span than its rank) is handled by
 // Algorithm 1's search over the supersets of the columns found, bounded in the number of supports.
@@ -411,34 +410,28 @@ struct FinishParams {
 // Shared memory of the finish kernel for R parity checks and P nodes (doubles first, then ints, bytes).
 __host__ __device__ inline size_t finish_smem_bytes(int R, int P) {
     const int ld = R | 1;
-    return sizeof(double) * ((size_t)5 * R * ld + 2 * (size_t)R * P + (size_t)R + 2 * (size_t)(R + 1) + (size_t)P) +
-           sizeof(int) * ((size_t)(R + 1) + (size_t)R + (size_t)P + (size_t)R) + (size_t)P;
+    return sizeof(double) * ((size_t)4 * R * ld + 2 * (size_t)R * P + (size_t)R + (size_t)P) +
+           sizeof(int) * ((size_t)P + (size_t)R) + (size_t)P;
 }
 
 // One warp.  The Gram matrix G of the failing codewords has rank = number of erroneous nodes (a
-// few) plus a noise floor far below the threshold, so its eigen-decomposition is done on a small
-// matrix: a diagonally pivoted Cholesky factorisation G = L L^T + (remainder below 2^-30 of the
-// eigenvalue threshold) gives k columns, the k x k matrix L^T L has the eigenvalues of L L^T, and
-// cyclic Jacobi runs on that.  The retained subspace is L w_i / sqrt(lambda_i) for the eigenpairs
-// above the threshold; the verification uses ||(I - Pi) L||_F^2 = tr((I - Pi) L L^T (I - Pi)).
+// few) plus a noise floor far below the threshold.  A diagonally pivoted Cholesky factorisation
+// G = L L^T + (remainder below 2^-30 of the eigenvalue threshold) gives its numerical rank (pivots
+// above the threshold) and its range (the leading columns of L); the verification uses
+// ||(I - Pi) L||_F^2 = tr((I - Pi) L L^T (I - Pi)).
 __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
     extern __shared__ __align__(16) double fs[];
     const int lane = threadIdx.x;
     const int R = prm.R, P = prm.P, ld = R | 1;
-    double* A = fs;                          // [R][ld] G -> Schur complement; then the second Jacobi buffer
+    double* A = fs;                          // [R][ld] G -> Schur complement; fallback search: L with span(H_base) projected out
     double* Lm = A + R * ld;                 // [R][ld] Cholesky columns
-    double* M = Lm + R * ld;                 // [R][ld] L^T L; after the eigen-decomposition: basis of span(H_A)
-    double* Wv = M + R * ld;                 // [R][ld] eigenvectors of L^T L in columns
-    double* U = Wv + R * ld;                 // [R][ld] orthonormal basis of the retained subspace in columns
+    double* M = Lm + R * ld;                 // [R][ld] orthonormal basis of span(H_A) (verification, fallback search)
+    double* U = M + R * ld;                  // [R][ld] orthonormal basis of the retained subspace in columns
     double* Hs = U + R * ld;                 // [R][P]
     double* Hp = Hs + R * P;                 // [R][P] fallback search: H with span(H_base) projected out
-    double* lam = Hp + R * P;                // [R]
-    double* rot_c = lam + R;                 // [R + 1] per index: row_i <- c row_i + s row_partner
-    double* rot_s = rot_c + (R + 1);         // [R + 1]
-    double* dist = rot_s + (R + 1);          // [P]
-    int* partner = reinterpret_cast<int*>(dist + P);   // [R + 1]
-    int* order = partner + (R + 1);          // [R]
-    int* free_nodes = order + R;             // [P] fallback search: nodes outside the base set, increasing
+    double* lam = Hp + R * P;                // [R] pivots of the factorisation
+    double* dist = lam + R;                  // [P]
+    int* free_nodes = reinterpret_cast<int*>(dist + P);   // [P] fallback search: nodes outside the base set, increasing
     int* comb = free_nodes + P;              // [R] fallback search: current combination (indices into free_nodes)
     unsigned char* inside = reinterpret_cast<unsigned char*>(comb + R);   // [P]
     gpd_locate_result* res = prm.result;
@@ -496,6 +489,7 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
                 if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
             }
             if (!(v > stop)) break;
+            if (lane == 0) lam[nl] = v;                                     // pivot of this step
             const double li = mine ? A[lane * ld + idx] * rsqrt(v) : 0.0;   // rows of earlier pivots are zero
             if (lane < R) Lm[lane * ld + nl] = li;
             __syncwarp();
@@ -513,108 +507,23 @@ __global__ void __launch_bounds__(32) locate_finish_kernel(FinishParams prm) {
             for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
             remainder = d;
         }
-        // ---- M = L^T L (nl x nl), W = I --------------------------------------------------------
-        for (int e = lane; e < nl * nl; e += 32) {
-            const int a = e / nl, b = e - a * nl;
-            double acc = 0.0;
-            for (int i = 0; i < R; ++i) acc = fma(Lm[i * ld + a], Lm[i * ld + b], acc);
-            M[a * ld + b] = acc;
-            Wv[a * ld + b] = a == b ? 1.0 : 0.0;
-        }
-        __syncwarp();
-        // ---- Jacobi on M: M <- J^T M J, W <- W J ----------------------------------------------
-        // Rotations of one round act on disjoint index pairs (round-robin pairing of n = nl or
-        // nl + 1 indices: n - 1 rounds of n / 2 pairs), so their angles are found side by side
-        // (lane = pair) and applied together: every index i gets its partner and the pair
-        // (c_i, s_i) with new row_i = c_i row_i + s_i row_partner, and J^T M J is written entry by
-        // entry into the other of two buffers (A is free by now), and so is W J (second buffer: U).
-        double* Ga = M;
-        double* Gb = A;
-        double* Wa = Wv;                     // eigenvectors, second buffer: U (not in use before the sweeps end)
-        double* Wb = U;
-        if (nl > 1) {
-            double tr = 0.0;
-            for (int i = 0; i < nl; ++i) tr += M[i * ld + i];
-            const int n = (nl + 1) & ~1, half = n >> 1;
-            const int ml_i = lane / nl, ml_j = lane % nl, ms_i = 32 / nl, ms_j = 32 % nl;
-            for (int sweep = 0; sweep < 40; ++sweep) {
-                double off = 0.0;
-                for (int e = lane, i = ml_i, c = ml_j; e < nl * nl; e += 32, i += ms_i, c += ms_j) {
-                    if (c >= nl) { c -= nl; ++i; }
-                    if (i != c) off += Ga[i * ld + c] * Ga[i * ld + c];
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xffffffffu, off, o);
-                if (off <= 1e-27 * tr * tr) break;          // off-diagonal mass at the FP64 rounding floor
-                for (int rd = 0; rd < n - 1; ++rd) {
-                    if (lane < half) {
-                        int a = rd + lane, b = rd + n - 1 - lane;            // both below 2 (n - 1)
-                        if (a >= n - 1) a -= n - 1;
-                        if (b >= n - 1) b -= n - 1;
-                        if (lane == 0) { a = n - 1; b = rd; }
-                        const int p = min(a, b), q = max(a, b);
-                        double c = 1.0, sn = 0.0;
-                        if (q < nl) {
-                            const double gpq = Ga[p * ld + q], gpp = Ga[p * ld + p], gqq = Ga[q * ld + q];
-                            if (!(fabs(gpq) <= 1e-300 || gpq * gpq <= 1e-40 * fabs(gpp * gqq))) {
-                                // tan of the rotation angle (the root of smaller magnitude) is o2 / den with
-                                // den = d + sign(d) hypot(d, o2); cosine and sine follow from (den, o2)
-                                // normalised, which takes two reciprocal square roots and no division
-                                const double d = gqq - gpp, o2 = 2.0 * gpq, h2 = d * d + o2 * o2;
-                                const double den = d + copysign(h2 * rsqrt(h2), d);
-                                const double rn = rsqrt(den * den + o2 * o2);
-                                c = fabs(den) * rn;
-                                sn = copysign(o2, o2 * den) * rn;
-                            }
-                            rot_c[q] = c; rot_s[q] = sn; partner[q] = p;
-                        }
-                        rot_c[p] = c; rot_s[p] = -sn; partner[p] = q < nl ? q : p;
-                    }
-                    __syncwarp();
-                    for (int e = lane, i = ml_i, jj = ml_j; e < nl * nl; e += 32, i += ms_i, jj += ms_j) {
-                        if (jj >= nl) { jj -= nl; ++i; }
-                        const int ip = partner[i], jp = partner[jj];
-                        const double ci = rot_c[i], si = rot_s[i], cj = rot_c[jj], sj = rot_s[jj];
-                        const double t0 = ci * Ga[i * ld + jj] + si * Ga[ip * ld + jj];
-                        const double t1 = ci * Ga[i * ld + jp] + si * Ga[ip * ld + jp];
-                        Gb[i * ld + jj] = (jj == ip && si != 0.0) ? 0.0 : cj * t0 + sj * t1;   // the rotated pair's entry is zero by construction
-                        Wb[i * ld + jj] = cj * Wa[i * ld + jj] + sj * Wa[i * ld + jp];          // W J: columns rotate like those of M
-                    }
-                    __syncwarp();
-                    double* tmp = Ga; Ga = Gb; Gb = tmp;
-                    tmp = Wa; Wa = Wb; Wb = tmp;
-                }
-            }
-        }
-        if (Wa != Wv) {                      // the last round left the eigenvectors in U's storage
-            for (int e = lane; e < nl * ld; e += 32) Wv[e] = Wa[e];
-            __syncwarp();
-        }
-        // ---- eigenvalues in descending order ---------------------------------------------
-        if (lane == 0) {
-            for (int i = 0; i < nl; ++i) { lam[i] = Ga[i * ld + i]; order[i] = i; }
-            for (int i = 1; i < nl; ++i) {                   // insertion sort, nl <= 32
-                const int oi = order[i];
-                int j = i - 1;
-                while (j >= 0 && lam[order[j]] < lam[oi]) { order[j + 1] = order[j]; --j; }
-                order[j + 1] = oi;
-            }
-        }
-        __syncwarp();
-        for (int i = 0; i < nl; ++i) rank += lam[order[i]] > theta ? 1 : 0;
+        // ---- numerical rank: pivots above the eigenvalue threshold ---------------------------------
+        // The pivots of the diagonally pivoted factorisation are non-increasing and bracket the
+        // eigenvalues from below up to the dimension: lambda_k / (R - k + 1) <= d_k, and the pivots past
+        // the true rank are at the level of what is left (the noise floor).  Erroneous nodes put
+        // eigenvalues orders of magnitude above the threshold and the floor lies orders below it, so
+        // counting pivots gives the count of eigenvalues above the threshold without an eigen-solver.
+        for (int k = 0; k < nl; ++k) rank += lam[k] > theta ? 1 : 0;
         if (lane == 0) res->rank = rank;
         if (rank > budget) {
             if (lane == 0) res->outcome = GPD_DECODE_FAILURE;
             return;
         }
-        // ---- retained subspace: u_e = L w_e / sqrt(lambda_e), then re-orthonormalised ---------
+        // ---- retained subspace: the first `rank` columns of L, orthonormalised --------------------
+        // (columns of the Gram matrix with earlier pivots projected out: they span its range up to
+        // the floor, as the leading eigenvectors do)
         for (int e = 0; e < rank; ++e) {
-            const int col = order[e];
-            double u = 0.0;
-            if (lane < R) {
-                for (int a = 0; a < nl; ++a) u = fma(Lm[lane * ld + a], Wv[a * ld + col], u);
-                u *= rsqrt(lam[col]);
-            }
+            double u = lane < R ? Lm[lane * ld + e] : 0.0;
             for (int pass = 0; pass < 2; ++pass) {
                 for (int f = 0; f < e; ++f) {
                     double part = lane < R ? U[lane * ld + f] * u : 0.0;
