@@ -19,7 +19,8 @@
 // Warp roles:
 //   warp 0       : TMA producer (one lane) - raw FP32 tiles of A and B into a 4-stage ring that
 //                  runs on across tiles
-//   warp 1       : allocates tensor memory; one lane issues the MMAs and commits them to mbarriers
+//   warp 1       : allocates tensor memory; one lane issues the MMAs of the even k-blocks and commits them
+//                  to mbarriers (the last warp's lane 0 does the same for the odd k-blocks)
 //   warps 2..9   : split every landed pair of tiles: B in place in shared memory (hi overwrites the
 //                  raw tile, lo goes to a second tile); A row by row into tensor memory (hi and lo, 32
 //                  columns each per stage), from where the MMAs take it: the A operand then costs
@@ -77,7 +78,7 @@ constexpr int kConvThreads = kConvWarps * 32;
 // read-modify-write epilogue wants wide chunks and a whole tile of lead, lets the splitting warps do
 // it (14 warps, 128 registers).  Measured on 10 x [2048 x 2048] x [2048 x 256]: products 0.178 ms with
 // the first arrangement and 0.207 ms with the second; update 0.217 ms and 0.147 ms.
-template <bool UPDATE> constexpr int kThreadsOf = 64 + kConvThreads + (UPDATE ? kEpiWarps : kEpiWarpsD) * 32;
+template <bool UPDATE> constexpr int kThreadsOf = 64 + kConvThreads + (UPDATE ? kEpiWarps : kEpiWarpsD) * 32 + 32;   // + second issuer
 
 __device__ int g_tf32_status = 0;                    // GPD_ERR_TIMEOUT if a bounded wait expired
 
@@ -91,6 +92,25 @@ using tc::tma_load_3d;
 using tc::umma_commit;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     return tc::mbar_wait(bar, parity, abort_flag, &g_tf32_status);
+}
+// Hand-over between the two MMA issuers: a counter in shared memory, written with release and read with
+// acquire semantics.  The wait is bounded like the barrier waits.
+__device__ __forceinline__ bool turn_wait(int* turn, int want, volatile int* abort_flag) {
+    const long long t0 = clock64();
+    for (;;) {
+        int v;
+        asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(turn)) : "memory");
+        if (v >= want) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicExch(&g_tf32_status, (int)GPD_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void turn_pass(int* turn, int next) {
+    asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(turn)), "r"(next) : "memory");
 }
 // for the epilogue warps: they wait most of the time, and a poll every 200 ns is early enough for them
 __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
@@ -157,8 +177,10 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __shared__ __align__(8) uint64_t full_bar[STAGES], conv_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2], tile_full[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ int issue_turn;                       // index of the k-block whose MMAs may be issued next
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kIssuer2Warp = kThreadsOf<UPDATE> / 32 - 1;   // the last warp: second MMA issuer
     const int num_kb = (int)((prm.K + BK - 1) / BK);
     // Virtual tile list: whole 128 x 128 tiles first; the tiles left over after the last full round
     // over the SMs follow as `split` column strips each (128 x 32 strips when split = 4), so that
@@ -193,6 +215,7 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         mbar_init(&tile_full[0], kConvWarps);
         mbar_init(&tile_full[1], kConvWarps);
         abort_flag = 0;
+        issue_turn = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -239,52 +262,67 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------ MMA issuer ------------------------------
+    } else if (warp == 1 || warp == kIssuer2Warp) {
+        // ------------------------------ MMA issuers ------------------------------
+        // Two threads take the k-blocks in turn (lane 0 of warp 1 the even ones, lane 0 of the last warp
+        // the odd ones).  Everything a k-block needs besides the MMAs themselves - waiting for its operands
+        // and for a free accumulator, building descriptors, committing to the barriers afterwards - costs
+        // a single thread as many cycles as issuing the twelve MMAs does (issue blocks while the tensor
+        // pipe is busy; measured 700 cycles of issue and 700-900 of the rest per k-block), and the pipe's
+        // queue is too short to bridge that.  With two issuers one thread's bookkeeping runs under the
+        // other's MMAs; only the hand-over (a release / acquire on a shared-memory counter, with the
+        // tcgen05 fences that order the two threads' MMAs) lies between the k-blocks.
         if (lane == 0) {
-            int it = 0, gi = 0;                   // k-blocks / accumulation groups issued so far, over all tiles
+            const int me = warp == 1 ? 0 : 1;
+            int it = 0, gi = 0;                   // k-blocks / accumulation groups so far, over all tiles (both issuers count alike)
             bool ok = true;
             for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
                 int p, m0, n0, bn;
                 decode(vt, p, m0, n0, bn);
                 const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
                                        ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                int kg = 0;                      // position of the k-block inside its accumulation group
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int buf = gi & 1, kg = kb % group_kb;
-                    if (kg == 0) {
-                        // the group before last used this accumulator: it must have been read back
-                        if (!mbar_wait(&acc_empty[buf], ((gi >> 1) & 1) ^ 1, abort_p)) { ok = false; break; }
+                    const int buf = gi & 1;
+                    const bool group_end = kg == group_kb - 1 || kb == num_kb - 1;
+                    if ((it & 1) == me) {
+                        if (kg == 0) {
+                            // the group before last used this accumulator: it must have been read back
+                            if (!mbar_wait(&acc_empty[buf], ((gi >> 1) & 1) ^ 1, abort_p)) { ok = false; break; }
+                        }
+                        const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1;
+                        if (!mbar_wait(&conv_bar[s], ph, abort_p)) { ok = false; break; }
+                        // the two B descriptors are built once per stage, a k-step only adds its offset to
+                        // their address field (16-byte units, no carry out of 14 bits: a stage lies inside
+                        // the 227 KB window)
+                        const uint32_t a_hi = A_tmem(s), a_lo = A_tmem(s) + BK;
+                        const uint64_t db_hi0 = B_KMAJOR ? desc_kmajor(smem_u32(B_hi(s))) : desc_mnmajor(smem_u32(B_hi(s)));
+                        const uint64_t db_lo0 = db_hi0 + (uint64_t)(B_TILE_BYTES >> 4);
+                        // my turn: the other issuer has handed over after its last MMA of k-block it - 1
+                        if (!turn_wait(&issue_turn, it, abort_p)) { ok = false; break; }
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    }
-                    const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
-                    const int s = it % STAGES;
-                    const uint32_t ph = (it / STAGES) & 1;
-                    if (!mbar_wait(&conv_bar[s], ph, abort_p)) { ok = false; break; }
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    // One thread issues everything, so its instruction count per k-block is on the
-                    // critical path: the two B descriptors are built once per stage, a k-step only
-                    // adds its offset to their address field (16-byte units, no carry out of 14 bits:
-                    // a stage lies inside the 227 KB window).
-                    const uint32_t a_hi = A_tmem(s), a_lo = A_tmem(s) + BK;
-                    const uint64_t db_hi0 = B_KMAJOR ? desc_kmajor(smem_u32(B_hi(s))) : desc_mnmajor(smem_u32(B_hi(s)));
-                    const uint64_t db_lo0 = db_hi0 + (uint64_t)(B_TILE_BYTES >> 4);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // A: the next 8 elements of K are 8 tensor-memory columns further.
-                        // B, K-major: 32 bytes further inside the swizzled row; MN-major: the next 8
-                        // k-rows are 8 * 128 bytes further in every 32-column chunk
-                        const uint32_t a_off = k * UMMA_K;
-                        const uint64_t b_off = (uint64_t)((B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128) >> 4);
-                        const uint32_t first = (kg > 0 || k > 0) ? 1u : 0u;    // a group starts from zero
-                        umma_tf32_ta(tmem_d, a_lo + a_off, db_hi0 + b_off, idesc, first);   // small terms first
-                        umma_tf32_ta(tmem_d, a_hi + a_off, db_lo0 + b_off, idesc, 1u);
-                        umma_tf32_ta(tmem_d, a_hi + a_off, db_hi0 + b_off, idesc, 1u);
+                        for (int k = 0; k < BK / UMMA_K; ++k) {
+                            // A: the next 8 elements of K are 8 tensor-memory columns further.
+                            // B, K-major: 32 bytes further inside the swizzled row; MN-major: the next 8
+                            // k-rows are 8 * 128 bytes further in every 32-column chunk
+                            const uint32_t a_off = k * UMMA_K;
+                            const uint64_t b_off = (uint64_t)((B_KMAJOR ? k * UMMA_K * 4 : k * UMMA_K * 128) >> 4);
+                            const uint32_t first = (kg > 0 || k > 0) ? 1u : 0u;    // a group starts from zero
+                            umma_tf32_ta(tmem_d, a_lo + a_off, db_hi0 + b_off, idesc, first);   // small terms first
+                            umma_tf32_ta(tmem_d, a_hi + a_off, db_lo0 + b_off, idesc, 1u);
+                            umma_tf32_ta(tmem_d, a_hi + a_off, db_hi0 + b_off, idesc, 1u);
+                        }
+                        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                        turn_pass(&issue_turn, it + 1);
+                        umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
+                        // this group's partial sum complete: the group's earlier MMAs (the other issuer's
+                        // among them) feed the same accumulator, so they have finished when these have
+                        if (group_end) umma_commit(&acc_full[buf]);
                     }
-                    umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
-                    if (kg == group_kb - 1 || kb == num_kb - 1) {
-                        umma_commit(&acc_full[buf]); // this group's partial sum complete
-                        ++gi;
-                    }
+                    if (group_end) { ++gi; kg = 0; } else { ++kg; }
                 }
             }
         }
