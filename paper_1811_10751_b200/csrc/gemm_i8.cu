@@ -32,13 +32,21 @@ namespace gpd {
 
 namespace {
 
-constexpr int BM = 128, BN = 64, BK = 64, STAGES = 3;
+// Output tiles are 128 x BN.  BN = 64 is the wide form: S accumulator groups of 64 columns fill 384 of
+// the 512 tensor-memory columns, so a tile's epilogue cannot run under the next tile's main loop.  That
+// costs about 4 us a tile, little against a long contraction and as much as the main loop itself when
+// K is a few hundred.  BN = 32 is the form for short contractions: two sets of S x 32 columns
+// alternate, the epilogue is hidden, and the price (the A planes are fetched per 32 instead of per 64
+// output columns) is smaller than what the exposed epilogue costs there.
+constexpr int BM = 128, BK = 64, STAGES = 3;
 constexpr int UMMA_K = 32;                            // int8 elements per MMA along K
 constexpr int A_PLANE_BYTES = BM * BK;                // 8 KB, rows of 64 B
-constexpr int B_PLANE_BYTES = BN * BK;                // 4 KB
-__host__ __device__ constexpr int stage_bytes(int S) { return S * (A_PLANE_BYTES + B_PLANE_BYTES); }   // 72 KB (60 KB)
-__host__ __device__ constexpr int smem_bytes(int S) { return STAGES * stage_bytes(S) + 1024; }
-constexpr int TMEM_COLS = 512;                        // S x 64 used; allocations are powers of two
+__host__ __device__ constexpr int b_plane_bytes(int BN) { return BN * BK; }                // 4 KB (2 KB)
+__host__ __device__ constexpr int stage_bytes(int S, int BN) { return S * (A_PLANE_BYTES + b_plane_bytes(BN)); }   // 72 KB (60 KB) at BN = 64
+__host__ __device__ constexpr int smem_bytes(int S, int BN) { return STAGES * stage_bytes(S, BN) + 1024; }
+__host__ __device__ constexpr int acc_sets(int S, int BN) { return 2 * S * BN <= 512 ? 2 : 1; }
+constexpr int TMEM_COLS = 512;                        // allocations are powers of two
+constexpr int64_t kNarrowTileMaxK = 512;              // contraction lengths served with BN = 32
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + kEpiWarps * 32;
 
@@ -50,7 +58,7 @@ using tc::mbar_expect_tx;
 using tc::mbar_init;
 using tc::mbar_try_wait;
 using tc::smem_u32;
-using tc::tma_load_3d;
+using tc::tma_load_4d;
 using tc::umma_commit;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     return tc::mbar_wait(bar, parity, abort_flag, &g_i8_status);
@@ -96,17 +104,38 @@ struct I8Params {
     const gpd_locate_result* gate;       // update: skipped when this reports a decoding failure
 };
 
-template <int S, bool UPDATE>
+// One warp reads 16 lanes x 32 (16) consecutive 32-bit columns of tensor memory in the 16 x 256-bit shape:
+// thread t gets, for each block k of 8 columns, registers 4k + 2i + e = (lane 8i + t / 4, column 8k + 2 (t % 4) + e),
+// lanes counted from the lane base of taddr.
+__device__ __forceinline__ void tmem_ld_16x256(uint32_t (&r)[16], uint32_t taddr) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_16x256(uint32_t (&r)[8], uint32_t taddr) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr));
+}
+
+template <int S, bool UPDATE, int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, I8Params prm,
                       int tiles_m, int tiles_n, int tiles) {
     if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
-    constexpr int STAGE_BYTES = stage_bytes(S);
+    constexpr int STAGE_BYTES = stage_bytes(S, BN);
+    constexpr int B_PLANE_BYTES = b_plane_bytes(BN);
+    constexpr int NSETS = acc_sets(S, BN);            // accumulator sets in tensor memory (S * BN columns each)
+    constexpr int CW = BN / 2;                        // columns an epilogue warp reads (two warps per lane quarter)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // full/empty: operand ring (runs on across the tiles of this CTA); acc_full: a tile's accumulators
     // are complete; acc_empty: the epilogue warps have read them, the next tile may overwrite them
-    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full, acc_empty;
+    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
@@ -118,8 +147,10 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&acc_full, 1);
-        mbar_init(&acc_empty, kEpiWarps);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], kEpiWarps);
+        }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -156,11 +187,9 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     const uint32_t ph = (it / STAGES) & 1;
                     if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) { ok = false; break; }
                     mbar_expect_tx(&full_bar[s], STAGE_BYTES);
-#pragma unroll
-                    for (int t = 0; t < S; ++t) {
-                        tma_load_3d(A_plane(s, t), &tmA, kb * BK, m0, t * prm.P + p, &full_bar[s]);
-                        tma_load_3d(B_plane(s, t), &tmB, kb * BK, n0, t * prm.P + p, &full_bar[s]);
-                    }
+                    // one copy per operand brings all S digit planes of the block (box K x rows x 1 node x S)
+                    tma_load_4d(A_plane(s, 0), &tmA, kb * BK, m0, p, 0, &full_bar[s]);
+                    tma_load_4d(B_plane(s, 0), &tmB, kb * BK, n0, p, 0, &full_bar[s]);
                 }
             }
             if (*abort_p) {                      // let copies still in flight land before the CTA exits
@@ -176,9 +205,11 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int it = 0, ti = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++ti) {
-                // the previous tile's accumulators must have been read
-                if (!mbar_wait(&acc_empty, (ti & 1) ^ 1, abort_p)) { ok = false; break; }
+                // the tile that used this accumulator set before must have been read
+                const int set = ti % NSETS;
+                if (!mbar_wait(&acc_empty[set], ((ti / NSETS) & 1) ^ 1, abort_p)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmem_acc = tmem_base + (uint32_t)(set * S * BN);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
@@ -196,94 +227,113 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                             const int n_first = n_total > 256 ? 256 : n_total;
                             // the plane-0 instruction of a tile's first k-step overwrites every group
                             const uint32_t acc = (kb > 0 || k > 0 || ta > 0) ? 1u : 0u;
-                            umma_i8(tmem_base + BN * ta, da, desc_sw64(b0 + k * UMMA_K), idesc_i8(n_first), acc);
+                            umma_i8(tmem_acc + BN * ta, da, desc_sw64(b0 + k * UMMA_K), idesc_i8(n_first), acc);
                             if (n_total > 256)
-                                umma_i8(tmem_base + BN * ta + 256, da, desc_sw64(b0 + 4 * B_PLANE_BYTES + k * UMMA_K),
+                                umma_i8(tmem_acc + BN * ta + 256, da, desc_sw64(b0 + (256 / BN) * B_PLANE_BYTES + k * UMMA_K),
                                         idesc_i8(n_total - 256), acc);
                         }
                     }
                     umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
                 }
-                if (ok) umma_commit(&acc_full);      // this tile's accumulators complete
+                if (ok) umma_commit(&acc_full[set]); // this tile's accumulators complete
             }
         }
     } else {
         // ------------------------------ epilogue ------------------------------
+        // Tensor memory is read in the 16 x 256-bit shape: a row of 8 columns is spread over 4 adjacent
+        // lanes, 2 columns each, so that a 16-byte store per lane writes 64 contiguous bytes of each of
+        // 8 rows (whole 32-byte sectors) instead of 16 bytes of each of 32 rows.
+        constexpr int NK = CW / 8;                   // 8-column blocks per warp
         const int q = warp & 3;                      // this warp may touch TMEM lanes 32q .. 32q+31
-        const int c0 = ((warp - 2) >> 2) * 32;       // two warps per lane quarter: 32 columns each
+        const int c0 = ((warp - 2) >> 2) * CW;       // two warps per lane quarter: CW columns each
+        const int rq = lane >> 2, cq = lane & 3;     // row within a block of 8 rows, column pair within 8 columns
         int ti = 0;
         for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++ti) {
             int p, m0, n0;
             tile_origin(tile, p, m0, n0);
-            const int64_t gm = (int64_t)m0 + q * 32 + lane;
-            const int64_t gn = (int64_t)n0 + c0 + lane;  // lane j keeps the scale of column c0 + j
-            const double row_scale = gm < prm.M ? exp2i(prm.ea[(int64_t)p * prm.M + gm] - 2 * kDigitBits) : 0.0;
-            const double col_scale = gn < prm.N ? exp2i(prm.eb[(int64_t)p * prm.N + gn]) : 0.0;
-            const bool acc_ready = mbar_wait(&acc_full, ti & 1, abort_p);
+            // this thread's outputs: rows r_base + 8 ri (ri = 0..3), columns c_base + 8 k + {0, 1} (k = 0..NK-1)
+            const int64_t r_base = (int64_t)m0 + q * 32 + rq;
+            const int64_t c_base = (int64_t)n0 + c0 + 2 * cq;
+            int era[4], ecb[NK][2];                  // exponents of the rows' and the columns' scales
+#pragma unroll
+            for (int ri = 0; ri < 4; ++ri)
+                era[ri] = r_base + 8 * ri < prm.M ? prm.ea[(int64_t)p * prm.M + r_base + 8 * ri] - 2 * kDigitBits : 0;
+#pragma unroll
+            for (int k = 0; k < NK; ++k)
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    ecb[k][e] = c_base + 8 * k + e < prm.N ? prm.eb[(int64_t)p * prm.N + c_base + 8 * k + e] : 0;
+            const int set = ti % NSETS;
+            const bool acc_ready = mbar_wait(&acc_full[set], (ti / NSETS) & 1, abort_p);
             __syncwarp();
             if (!__all_sync(0xffffffffu, acc_ready)) break;   // tcgen05.ld is warp-collective: all lanes or none
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            double v[32];
+            double v[4][NK][2];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = 0.0;
-            // smallest weight first; two groups are in flight per wait (one for the odd one out)
-            auto tmem_ld32 = [&](uint32_t (&r)[32], int g) {
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(BN * g + c0);
-                asm volatile(
-                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                    : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                      "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                      "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                      "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                    : "r"(taddr));
+            for (int ri = 0; ri < 4; ++ri)
+#pragma unroll
+                for (int k = 0; k < NK; ++k) v[ri][k][0] = v[ri][k][1] = 0.0;
+            // lanes 32q + 16h .. + 15 of group g; register 4k + 2i + e = (row 8i + rq, column 8k + 2cq + e)
+            auto group_addr = [&](int g, int h) {
+                return tmem_base + ((uint32_t)(q * 32 + 16 * h) << 16) + (uint32_t)(set * S * BN + BN * g + c0);
             };
+            // smallest weight first; two groups are in flight per wait (one for the odd one out)
 #pragma unroll
             for (int g = S - 1; g >= 0; g -= 2) {
-                uint32_t r0[32], r1[32];
-                tmem_ld32(r0, g);
-                if (g >= 1) tmem_ld32(r1, g - 1);
+                uint32_t r[2][2][4 * NK];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    tmem_ld_16x256(r[0][h], group_addr(g, h));
+                    if (g >= 1) tmem_ld_16x256(r[1][h], group_addr(g - 1, h));
+                }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                const double w0 = exp2i(-kDigitBits * g);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = fma(i2d(r0[j]), w0, v[j]);
-                if (g >= 1) {
-                    const double w1 = exp2i(-kDigitBits * (g - 1));
+                for (int u = 0; u < 2; ++u) {
+                    if (u == 1 && g < 1) break;
+                    const double w = exp2i(-kDigitBits * (g - u));
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = fma(i2d(r1[j]), w1, v[j]);
+                    for (int ri = 0; ri < 4; ++ri)
+#pragma unroll
+                        for (int k = 0; k < NK; ++k)
+#pragma unroll
+                            for (int e = 0; e < 2; ++e)
+                                v[ri][k][e] = fma(i2d(r[u][ri >> 1][4 * k + 2 * (ri & 1) + e]), w, v[ri][k][e]);
                 }
             }
             // the accumulators are in registers: hand tensor memory back to the MMA warp, then scale
             // and store while the next tile's main loop runs
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty);
-            double* crow = prm.C + (int64_t)p * prm.M * prm.N + gm * prm.N + n0 + c0;
-            const bool vec = (prm.N & 1) == 0 && n0 + c0 + 32 <= prm.N;
-            double2 old[16];                             // update: the stored shares this thread adds into
-            if (UPDATE && vec && gm < prm.M) {
+            if (lane == 0) mbar_arrive(&acc_empty[set]);
+            double* cbase = prm.C + (int64_t)p * prm.M * prm.N + r_base * prm.N + c_base;
+            const bool vec = (prm.N & 1) == 0;       // 16-byte stores: pairs start at even columns
 #pragma unroll
-                for (int j = 0; j < 16; ++j) old[j] = *reinterpret_cast<const double2*>(crow + 2 * j);
-            }
+            for (int ri = 0; ri < 4; ++ri) {
+                if (r_base + 8 * ri >= prm.M) continue;
+                double* crow = cbase + (int64_t)(8 * ri) * prm.N;
+                double2 old[NK];                     // update: the stored shares this thread adds into
+                if (UPDATE && vec) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-                double2 o;                               // column scales come from the lanes that hold them
-                o.x = v[j] * row_scale * __shfl_sync(0xffffffffu, col_scale, j);
-                o.y = v[j + 1] * row_scale * __shfl_sync(0xffffffffu, col_scale, j + 1);
-                if (gm < prm.M) {
-                    if (vec) {
+                    for (int k = 0; k < NK; ++k)
+                        if (c_base + 8 * k + 1 < prm.N) old[k] = *reinterpret_cast<const double2*>(crow + 8 * k);
+                }
+#pragma unroll
+                for (int k = 0; k < NK; ++k) {
+                    double2 o;
+                    o.x = v[ri][k][0] * exp2i(era[ri] + ecb[k][0]);
+                    o.y = v[ri][k][1] * exp2i(era[ri] + ecb[k][1]);
+                    if (vec && c_base + 8 * k + 1 < prm.N) {
                         if (UPDATE) {
-                            o.x = fma(prm.eta, o.x, prm.shrink * old[j >> 1].x);
-                            o.y = fma(prm.eta, o.y, prm.shrink * old[j >> 1].y);
-                            *reinterpret_cast<double2*>(crow + j) = o;      // read again soon: no streaming hint
+                            o.x = fma(prm.eta, o.x, prm.shrink * old[k].x);
+                            o.y = fma(prm.eta, o.y, prm.shrink * old[k].y);
+                            *reinterpret_cast<double2*>(crow + 8 * k) = o;      // read again soon: no streaming hint
                         } else {
-                            __stcs(reinterpret_cast<double2*>(crow + j), o);
+                            __stcs(reinterpret_cast<double2*>(crow + 8 * k), o);
                         }
                     } else {
-                        if (n0 + c0 + j < prm.N) crow[j] = UPDATE ? fma(prm.eta, o.x, prm.shrink * crow[j]) : o.x;
-                        if (n0 + c0 + j + 1 < prm.N)
-                            crow[j + 1] = UPDATE ? fma(prm.eta, o.y, prm.shrink * crow[j + 1]) : o.y;
+                        if (c_base + 8 * k < prm.N) crow[8 * k] = UPDATE ? fma(prm.eta, o.x, prm.shrink * crow[8 * k]) : o.x;
+                        if (c_base + 8 * k + 1 < prm.N)
+                            crow[8 * k + 1] = UPDATE ? fma(prm.eta, o.y, prm.shrink * crow[8 * k + 1]) : o.y;
                     }
                 }
             }
@@ -301,9 +351,25 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 // ---- host side -------------------------------------------------------------------------------------
 // 3-D byte tensor [batch][rows][K] (K contiguous), box {BK, box_rows, 1}, 64-byte swizzle,
 // out-of-range elements read as zero.
-bool make_map(CUtensorMap* map, const void* base, int64_t batch, int64_t rows, int64_t K, int box_rows) {
-    return tc::make_map_3d(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, base, batch, rows, K, BK, box_rows,
+// planes [S][P][rows][K] as a 4-d tensor; one box = a K-block of box_rows rows of one node in all S planes
+bool make_map(CUtensorMap* map, const void* base, int S, int64_t P, int64_t rows, int64_t K, int box_rows) {
+    return tc::make_map_4d(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, base, S, P, rows, K, BK, box_rows, 1, S,
                            CU_TENSOR_MAP_SWIZZLE_64B);
+}
+
+template <int S, bool UPDATE, int BN>
+gpd_status launch_i8(const I8Gemm& g, const I8Params& prm, cudaStream_t st) {
+    CUtensorMap tmA, tmB;
+    if (!make_map(&tmA, g.A, S, g.P, g.M, g.K, BM)) return GPD_ERR_CUDA;
+    if (!make_map(&tmB, g.B, S, g.P, g.N, g.K, BN)) return GPD_ERR_CUDA;
+    auto kernel = gemm_i8_sliced_kernel<S, UPDATE, BN>;
+    constexpr int smem = smem_bytes(S, BN);
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GPD_ERR_CUDA;
+    const int tiles_n = (int)((g.N + BN - 1) / BN), tiles_m = (int)((g.M + BM - 1) / BM);
+    const int64_t tiles = (int64_t)tiles_n * tiles_m * g.P;
+    const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());     // persistent: one CTA per SM walks the tiles
+    kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, prm, tiles_m, tiles_n, (int)tiles);
+    return launch_ok();
 }
 
 }  // namespace
@@ -317,20 +383,11 @@ gpd_status gemm_i8_launch(const I8Gemm& g, cudaStream_t st) {
     prm.P = g.P; prm.M = g.M; prm.N = g.N; prm.K = g.K;
     prm.ea = g.ea; prm.eb = g.eb; prm.C = g.C;
     prm.shrink = g.shrink; prm.eta = g.eta; prm.gate = g.gate;
-    const int S = g.slices;
-    CUtensorMap tmA, tmB;
-    if (!make_map(&tmA, g.A, (int64_t)S * g.P, g.M, g.K, BM)) return GPD_ERR_CUDA;
-    if (!make_map(&tmB, g.B, (int64_t)S * g.P, g.N, g.K, BN)) return GPD_ERR_CUDA;
-    auto kernel = g.update ? gemm_i8_sliced_kernel<6, true>
-                           : (S == 6 ? gemm_i8_sliced_kernel<6, false> : gemm_i8_sliced_kernel<5, false>);
-    if (g.update && S != 6) return GPD_ERR_UNSUPPORTED;
-    const int smem = S == 6 ? smem_bytes(6) : smem_bytes(5);
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GPD_ERR_CUDA;
-    const int tiles_n = (int)((g.N + BN - 1) / BN), tiles_m = (int)((g.M + BM - 1) / BM);
-    const int64_t tiles = (int64_t)tiles_n * tiles_m * g.P;
-    const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());     // persistent: one CTA per SM walks the tiles
-    kernel<<<grid, kThreads, smem, st>>>(tmA, tmB, prm, tiles_m, tiles_n, (int)tiles);
-    return launch_ok();
+    if (g.update) return g.slices == 6 ? launch_i8<6, true, 64>(g, prm, st) : GPD_ERR_UNSUPPORTED;
+    // short contractions: narrow tiles whose epilogue runs under the next tile's main loop
+    const bool narrow = g.K <= kNarrowTileMaxK;
+    if (g.slices == 6) return narrow ? launch_i8<6, false, 32>(g, prm, st) : launch_i8<6, false, 64>(g, prm, st);
+    return narrow ? launch_i8<5, false, 32>(g, prm, st) : launch_i8<5, false, 64>(g, prm, st);
 }
 
 gpd_status gemm_sliced_launch(gpd_plan_s* plan, gpd_product which, const void* W_shares, const void* other_sliced,
