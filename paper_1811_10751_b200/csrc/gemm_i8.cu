@@ -32,21 +32,17 @@ namespace gpd {
 
 namespace {
 
-// Output tiles are 128 x BN.  BN = 64 is the wide form: S accumulator groups of 64 columns fill 384 of
-// the 512 tensor-memory columns, so a tile's epilogue cannot run under the next tile's main loop.  That
-// costs about 4 us a tile, little against a long contraction and as much as the main loop itself when
-// K is a few hundred.  BN = 32 is the form for short contractions: two sets of S x 32 columns
-// alternate, the epilogue is hidden, and the price (the A planes are fetched per 32 instead of per 64
-// output columns) is smaller than what the exposed epilogue costs there.
-constexpr int BM = 128, BK = 64, STAGES = 3;
+// Output tiles are 128 x 64: S accumulator groups of 64 columns fill 384 of the 512 tensor-memory columns.
+// (Tiles of 128 x 32 with two alternating accumulator sets, which hide the epilogue's read of tensor
+// memory, were measured and are slower at every contraction length: the A planes are then fetched per
+// 32 instead of per 64 output columns.)
+constexpr int BM = 128, BN = 64, BK = 64, STAGES = 3;
 constexpr int UMMA_K = 32;                            // int8 elements per MMA along K
 constexpr int A_PLANE_BYTES = BM * BK;                // 8 KB, rows of 64 B
-__host__ __device__ constexpr int b_plane_bytes(int BN) { return BN * BK; }                // 4 KB (2 KB)
-__host__ __device__ constexpr int stage_bytes(int S, int BN) { return S * (A_PLANE_BYTES + b_plane_bytes(BN)); }   // 72 KB (60 KB) at BN = 64
-__host__ __device__ constexpr int smem_bytes(int S, int BN) { return STAGES * stage_bytes(S, BN) + 1024; }
-__host__ __device__ constexpr int acc_sets(int S, int BN) { return 2 * S * BN <= 512 ? 2 : 1; }
+constexpr int B_PLANE_BYTES = BN * BK;                // 4 KB
+__host__ __device__ constexpr int stage_bytes(int S) { return S * (A_PLANE_BYTES + B_PLANE_BYTES); }   // 72 KB (60 KB)
+__host__ __device__ constexpr int smem_bytes(int S) { return STAGES * stage_bytes(S) + 1024; }
 constexpr int TMEM_COLS = 512;                        // allocations are powers of two
-constexpr int64_t kNarrowTileMaxK = 512;              // contraction lengths served with BN = 32
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + kEpiWarps * 32;
 
@@ -104,7 +100,7 @@ struct I8Params {
     const gpd_locate_result* gate;       // update: skipped when this reports a decoding failure
 };
 
-// One warp reads 16 lanes x 32 (16) consecutive 32-bit columns of tensor memory in the 16 x 256-bit shape:
+// One warp reads 16 lanes x 32 consecutive 32-bit columns of tensor memory in the 16 x 256-bit shape:
 // thread t gets, for each block k of 8 columns, registers 4k + 2i + e = (lane 8i + t / 4, column 8k + 2 (t % 4) + e),
 // lanes counted from the lane base of taddr.
 __device__ __forceinline__ void tmem_ld_16x256(uint32_t (&r)[16], uint32_t taddr) {
@@ -115,27 +111,18 @@ __device__ __forceinline__ void tmem_ld_16x256(uint32_t (&r)[16], uint32_t taddr
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_ld_16x256(uint32_t (&r)[8], uint32_t taddr) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-        : "r"(taddr));
-}
-
-template <int S, bool UPDATE, int BN>
+template <int S, bool UPDATE>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, I8Params prm,
                       int tiles_m, int tiles_n, int tiles) {
     if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
-    constexpr int STAGE_BYTES = stage_bytes(S, BN);
-    constexpr int B_PLANE_BYTES = b_plane_bytes(BN);
-    constexpr int NSETS = acc_sets(S, BN);            // accumulator sets in tensor memory (S * BN columns each)
+    constexpr int STAGE_BYTES = stage_bytes(S);
     constexpr int CW = BN / 2;                        // columns an epilogue warp reads (two warps per lane quarter)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // full/empty: operand ring (runs on across the tiles of this CTA); acc_full: a tile's accumulators
     // are complete; acc_empty: the epilogue warps have read them, the next tile may overwrite them
-    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full[2], acc_empty[2];
+    __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], acc_full, acc_empty;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
@@ -147,10 +134,8 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&acc_full[b], 1);
-            mbar_init(&acc_empty[b], kEpiWarps);
-        }
+        mbar_init(&acc_full, 1);
+        mbar_init(&acc_empty, kEpiWarps);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -205,11 +190,9 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int it = 0, ti = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++ti) {
-                // the tile that used this accumulator set before must have been read
-                const int set = ti % NSETS;
-                if (!mbar_wait(&acc_empty[set], ((ti / NSETS) & 1) ^ 1, abort_p)) { ok = false; break; }
+                // the previous tile's accumulators must have been read
+                if (!mbar_wait(&acc_empty, (ti & 1) ^ 1, abort_p)) { ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t tmem_acc = tmem_base + (uint32_t)(set * S * BN);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
@@ -227,15 +210,15 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                             const int n_first = n_total > 256 ? 256 : n_total;
                             // the plane-0 instruction of a tile's first k-step overwrites every group
                             const uint32_t acc = (kb > 0 || k > 0 || ta > 0) ? 1u : 0u;
-                            umma_i8(tmem_acc + BN * ta, da, desc_sw64(b0 + k * UMMA_K), idesc_i8(n_first), acc);
+                            umma_i8(tmem_base + BN * ta, da, desc_sw64(b0 + k * UMMA_K), idesc_i8(n_first), acc);
                             if (n_total > 256)
-                                umma_i8(tmem_acc + BN * ta + 256, da, desc_sw64(b0 + (256 / BN) * B_PLANE_BYTES + k * UMMA_K),
+                                umma_i8(tmem_base + BN * ta + 256, da, desc_sw64(b0 + (256 / BN) * B_PLANE_BYTES + k * UMMA_K),
                                         idesc_i8(n_total - 256), acc);
                         }
                     }
                     umma_commit(&empty_bar[s]);      // stage reusable once these MMAs have read it
                 }
-                if (ok) umma_commit(&acc_full[set]); // this tile's accumulators complete
+                if (ok) umma_commit(&acc_full);      // this tile's accumulators complete
             }
         }
     } else {
@@ -263,8 +246,7 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
 #pragma unroll
                 for (int e = 0; e < 2; ++e)
                     ecb[k][e] = c_base + 8 * k + e < prm.N ? prm.eb[(int64_t)p * prm.N + c_base + 8 * k + e] : 0;
-            const int set = ti % NSETS;
-            const bool acc_ready = mbar_wait(&acc_full[set], (ti / NSETS) & 1, abort_p);
+            const bool acc_ready = mbar_wait(&acc_full, ti & 1, abort_p);
             __syncwarp();
             if (!__all_sync(0xffffffffu, acc_ready)) break;   // tcgen05.ld is warp-collective: all lanes or none
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -275,9 +257,10 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 for (int k = 0; k < NK; ++k) v[ri][k][0] = v[ri][k][1] = 0.0;
             // lanes 32q + 16h .. + 15 of group g; register 4k + 2i + e = (row 8i + rq, column 8k + 2cq + e)
             auto group_addr = [&](int g, int h) {
-                return tmem_base + ((uint32_t)(q * 32 + 16 * h) << 16) + (uint32_t)(set * S * BN + BN * g + c0);
+                return tmem_base + ((uint32_t)(q * 32 + 16 * h) << 16) + (uint32_t)(BN * g + c0);
             };
-            // smallest weight first; two groups are in flight per wait (one for the odd one out)
+            // smallest weight first; two groups are in flight per wait (one for the odd one out).
+            // (Summing the groups as 64-bit integers first, to spare the FP64 pipe, was measured: slower.)
 #pragma unroll
             for (int g = S - 1; g >= 0; g -= 2) {
                 uint32_t r[2][2][4 * NK];
@@ -304,7 +287,7 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             // and store while the next tile's main loop runs
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[set]);
+            if (lane == 0) mbar_arrive(&acc_empty);
             double* cbase = prm.C + (int64_t)p * prm.M * prm.N + r_base * prm.N + c_base;
             const bool vec = (prm.N & 1) == 0;       // 16-byte stores: pairs start at even columns
 #pragma unroll
@@ -357,13 +340,13 @@ bool make_map(CUtensorMap* map, const void* base, int S, int64_t P, int64_t rows
                            CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
-template <int S, bool UPDATE, int BN>
+template <int S, bool UPDATE>
 gpd_status launch_i8(const I8Gemm& g, const I8Params& prm, cudaStream_t st) {
     CUtensorMap tmA, tmB;
     if (!make_map(&tmA, g.A, S, g.P, g.M, g.K, BM)) return GPD_ERR_CUDA;
     if (!make_map(&tmB, g.B, S, g.P, g.N, g.K, BN)) return GPD_ERR_CUDA;
-    auto kernel = gemm_i8_sliced_kernel<S, UPDATE, BN>;
-    constexpr int smem = smem_bytes(S, BN);
+    auto kernel = gemm_i8_sliced_kernel<S, UPDATE>;
+    constexpr int smem = smem_bytes(S);
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return GPD_ERR_CUDA;
     const int tiles_n = (int)((g.N + BN - 1) / BN), tiles_m = (int)((g.M + BM - 1) / BM);
     const int64_t tiles = (int64_t)tiles_n * tiles_m * g.P;
@@ -383,11 +366,8 @@ gpd_status gemm_i8_launch(const I8Gemm& g, cudaStream_t st) {
     prm.P = g.P; prm.M = g.M; prm.N = g.N; prm.K = g.K;
     prm.ea = g.ea; prm.eb = g.eb; prm.C = g.C;
     prm.shrink = g.shrink; prm.eta = g.eta; prm.gate = g.gate;
-    if (g.update) return g.slices == 6 ? launch_i8<6, true, 64>(g, prm, st) : GPD_ERR_UNSUPPORTED;
-    // short contractions: narrow tiles whose epilogue runs under the next tile's main loop
-    const bool narrow = g.K <= kNarrowTileMaxK;
-    if (g.slices == 6) return narrow ? launch_i8<6, false, 32>(g, prm, st) : launch_i8<6, false, 64>(g, prm, st);
-    return narrow ? launch_i8<5, false, 32>(g, prm, st) : launch_i8<5, false, 64>(g, prm, st);
+    if (g.update) return g.slices == 6 ? launch_i8<6, true>(g, prm, st) : GPD_ERR_UNSUPPORTED;
+    return g.slices == 6 ? launch_i8<6, false>(g, prm, st) : launch_i8<5, false>(g, prm, st);
 }
 
 gpd_status gemm_sliced_launch(gpd_plan_s* plan, gpd_product which, const void* W_shares, const void* other_sliced,
