@@ -6,6 +6,8 @@
 //
 //   1. position_scan_kernel: one thread per position; syndrome r = H z (orthonormal H in shared
 //      memory), zero test ||r||^2 <= tau^2 ||z||^2; positions that fail it are appended to a list.
+//      The syndromes of the first listed positions are kept beside the list, so that their
+//      repair does not read the codeword a second time.
 //   2. position_fix_kernel: one thread per listed position.  The code is a polynomial code, so the
 //      sparsest solution is found the Reed-Solomon way in real arithmetic: power-sum syndromes
 //      S_j = sum_p w_p b_p^j z_p (w the barycentric weights), and for nu = 1 .. t the locator
@@ -13,7 +15,8 @@
 //      values over the points name the support A; the error values are the least-squares solution
 //      of H_A e = r; the support is accepted when what is left of r passes the zero test.  The
 //      accepted errors are subtracted in place.
-//   3. position_finish_kernel: outcome and counters into the result struct.
+//   3. Outcome and counters go into the result struct: written by the last block of the repair
+//      kernel to finish (position_finish_kernel when the code has no parity check to scan with).
 #include "gpd_internal.h"
 
 namespace gpd {
@@ -26,8 +29,10 @@ struct PosParams {
     const double* Hg;                     // [R][P] power-sum parity check
     const double* points;                 // [P]
     unsigned long long* counters;         // [0] listed, [1] active, [2] corrected, [3] failed, [4] entries,
-                                          // [5] largest support, [6] touched-node mask
+                                          // [5] largest support, [6] touched-node mask, [7] finished blocks
     unsigned int* list;                   // positions that failed the zero test
+    double* rec;                          // [rec_cap][R + 1]: syndrome r and ||z||^2 of the first listed positions
+    unsigned long long rec_cap;
     gpd_position_result* result;
     int64_t L;
     int P, R;
@@ -95,7 +100,17 @@ __global__ void __launch_bounds__(256, RT <= 8 ? 4 : 1) position_scan_kernel(Pos
                 if (m_list) slot = atomicAdd(&prm.counters[0], (unsigned long long)__popc(m_list));
             }
             slot = __shfl_sync(0xffffffffu, slot, 0);
-            if (listed) prm.list[slot + __popc(m_list & ((1u << lane) - 1u))] = (unsigned int)pos;
+            if (listed) {
+                const unsigned long long mine = slot + __popc(m_list & ((1u << lane) - 1u));
+                prm.list[mine] = (unsigned int)pos;
+                if (mine < prm.rec_cap) {             // hand the syndrome over: the repair then needs no second read of z
+                    double* rec = prm.rec + mine * (unsigned long long)(prm.R + 1);
+#pragma unroll
+                    for (int j = 0; j < RT; ++j)
+                        if (j < prm.R) rec[j] = r[j];
+                    rec[prm.R] = z2;
+                }
+            }
         }
     }
 }
@@ -114,6 +129,7 @@ __device__ __forceinline__ bool solve_small(double (&a)[TT][TT + 1], int n, doub
             if (i < n && j < n) amax = fmax(amax, fabs(a[i][j]));
     if (!(amax > 0.0)) return false;
     bool ok = true;
+    double pinv[TT];                         // reciprocal pivots, used again by the back substitution
 #pragma unroll UF
     for (int k = 0; k < TT; ++k) {
         if (k < n) {
@@ -126,6 +142,7 @@ __device__ __forceinline__ bool solve_small(double (&a)[TT][TT + 1], int n, doub
             }
             if (fabs(a[k][k]) <= 1e-13 * amax) ok = false;
             const double inv = 1.0 / a[k][k];
+            pinv[k] = inv;
 #pragma unroll UF
             for (int i = k + 1; i < TT; ++i) {
                 if (i < n) {
@@ -145,24 +162,78 @@ __device__ __forceinline__ bool solve_small(double (&a)[TT][TT + 1], int n, doub
 #pragma unroll UF
             for (int j = 0; j < TT; ++j)
                 if (j > i && j < n) s -= a[i][j] * x[j];
-            x[i] = s / a[i][i];
+            x[i] = s * pinv[i];
         }
     }
     return true;
+}
+
+// Outcome and counters into the result struct, by the threads tid = 0 .. nthr-1 of one block.  The
+// counters are read past L1: other blocks' atomics filled them.
+__device__ __forceinline__ void write_position_result(const PosParams& prm, int tid, int nthr) {
+    gpd_position_result* res = prm.result;
+    const unsigned long long active = __ldcg(&prm.counters[1]), failed = __ldcg(&prm.counters[3]);
+    if (tid == 0) {
+        res->outcome = active == 0ULL ? GPD_NO_ERROR : (failed ? GPD_DECODE_FAILURE : GPD_CORRECTED);
+        res->max_errors = (int32_t)__ldcg(&prm.counters[5]);
+        res->device_status = 0;
+        res->reserved = 0;
+        res->n_active = (int64_t)active;
+        res->n_corrected = (int64_t)__ldcg(&prm.counters[2]);
+        res->n_failed = (int64_t)failed;
+        res->n_entries = (int64_t)__ldcg(&prm.counters[4]);
+    }
+    const unsigned long long touched = __ldcg(&prm.counters[6]);
+    for (int p = tid; p < kMaxNodes; p += nthr) res->touched[p] = (p < prm.P && ((touched >> p) & 1ULL)) ? 1 : 0;
+}
+
+// A block that has finished takes a ticket; the last one of the grid writes the result.
+__device__ __forceinline__ void finish_by_last_block(const PosParams& prm) {
+    __shared__ bool s_last;
+    __threadfence();                                  // this thread's counter updates and repairs are visible ...
+    __syncthreads();                                  // ... and so are those of the whole block
+    if (threadIdx.x == 0) {
+        s_last = atomicAdd(&prm.counters[7], 1ULL) + 1ULL == (unsigned long long)gridDim.x;
+        __threadfence();
+    }
+    __syncthreads();
+    if (s_last) write_position_result(prm, threadIdx.x, blockDim.x);
 }
 
 // RT: parity checks rounded up (8 or 32); TT: errors per codeword rounded up (4 or 16).  The
 // right-hand side of a system sits in column TT of its rows.
 template <typename T, int RT, int TT>
 __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
-    extern __shared__ double sm[];        // H [R][P], Hg [R][P], points [P]
+    extern __shared__ double sm[];        // H [R][P], Hg [R][P], points [P], small codes: H^T H [P][P]
     double* sH = sm;
     double* sHg = sm + prm.R * prm.P;
     double* sPts = sHg + prm.R * prm.P;
+    double* sT = sPts + prm.P;            // [R][R] = Hg H^T: S = T r, since the rows of Hg lie in the row space of H
+    double* sG = sT + prm.R * prm.R;
+    if ((unsigned long long)blockIdx.x * 64 >= prm.counters[0]) {          // nothing listed for this block
+        finish_by_last_block(prm);
+        return;
+    }
     for (int i = threadIdx.x; i < prm.R * prm.P; i += 64) { sH[i] = prm.H[i]; sHg[i] = prm.Hg[i]; }
     for (int i = threadIdx.x; i < prm.P; i += 64) sPts[i] = prm.points[i];
     __syncthreads();
     constexpr int UF = TT <= 4 ? 32 : 1;     // small codes: loops fully unrolled, everything in registers
+    constexpr bool kGramTable = TT <= 4;     // normal equations read their entries from H^T H
+    for (int i = threadIdx.x; i < prm.R * prm.R; i += 64) {
+        const int a = i / prm.R, b = i - a * prm.R;
+        double s2 = 0.0;
+        for (int p = 0; p < prm.P; ++p) s2 = fma(sHg[a * prm.P + p], sH[b * prm.P + p], s2);
+        sT[i] = s2;
+    }
+    if (kGramTable) {
+        for (int i = threadIdx.x; i < prm.P * prm.P; i += 64) {
+            const int a = i / prm.P, b = i - a * prm.P;
+            double s2 = 0.0;
+            for (int q = 0; q < prm.R; ++q) s2 = fma(sH[q * prm.P + a], sH[q * prm.P + b], s2);
+            sG[i] = s2;
+        }
+        __syncthreads();
+    }
     T* Z = reinterpret_cast<T*>(prm.Z);
     const int P = prm.P, R = prm.R, t = R / 2;
     const unsigned long long listed = prm.counters[0];
@@ -176,14 +247,46 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
 #pragma unroll UF
         for (int j = 0; j < RT; ++j) { r[j] = 0.0; S[j] = 0.0; }
         double z2 = 0.0;
-        for (int p = 0; p < P; ++p) {
-            const double z = (double)Z[(int64_t)p * prm.L + pos];
-            z2 = fma(z, z, z2);
+        if (it < prm.rec_cap) {
+            // the scan left r and ||z||^2 of this position behind
+            const double* rec = prm.rec + it * (unsigned long long)(R + 1);
+            if (valid) {
+#pragma unroll UF
+                for (int j = 0; j < RT; ++j)
+                    if (j < R) r[j] = rec[j];
+                z2 = rec[R];
+            }
 #pragma unroll UF
             for (int j = 0; j < RT; ++j) {
                 if (j < R) {
-                    r[j] = fma(sH[j * P + p], z, r[j]);
-                    S[j] = fma(sHg[j * P + p], z, S[j]);
+                    double s2 = 0.0;
+#pragma unroll UF
+                    for (int k = 0; k < RT; ++k)
+                        if (k < R) s2 = fma(sT[j * R + k], r[k], s2);
+                    S[j] = s2;
+                }
+            }
+        }
+        // beyond the records: read the codeword again.  Its P values lie L elements apart: several loads
+        // are issued before the first is used
+        constexpr int U = 9;
+        for (int p0 = 0; p0 < P && it >= prm.rec_cap; p0 += U) {
+            double zv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) zv[u] = p0 + u < P ? (double)Z[(int64_t)(p0 + u) * prm.L + pos] : 0.0;
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (p0 + u < P) {
+                    const double z = zv[u];
+                    const int p = p0 + u;
+                    z2 = fma(z, z, z2);
+#pragma unroll UF
+                    for (int j = 0; j < RT; ++j) {
+                        if (j < R) {
+                            r[j] = fma(sH[j * P + p], z, r[j]);
+                            S[j] = fma(sHg[j * P + p], z, S[j]);
+                        }
+                    }
                 }
             }
         }
@@ -227,27 +330,47 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
                 }
             }
             if (!solve_small<TT>(a, nu, lam)) continue;
-            // the nu points where the locator is smallest
-            unsigned long long taken = 0ULL;
+            // the nu points where the locator is smallest, smallest first (of equal values the lower
+            // point): one pass over the points with an insertion into the sorted list kept so far
+            {
+                double small_v[TT];
 #pragma unroll UF
-            for (int k = 0; k < TT; ++k) {
-                if (k < nu) {
-                    int best = -1;
-                    double best_v = 0.0;
-                    for (int p = 0; p < P; ++p) {
-                        if ((taken >> p) & 1ULL) continue;
-                        const double x = sPts[p];
-                        double v = 1.0;
+                for (int k = 0; k < TT; ++k) { small_v[k] = __longlong_as_double(0x7ff0000000000000LL); nodes[k] = 0; }
+#pragma unroll 5
+                for (int p = 0; p < P; ++p) {
+                    const double x = sPts[p];
+                    double v = 1.0;
 #pragma unroll UF
-                        for (int i = TT - 1; i >= 0; --i)
-                            if (i < nu) v = fma(v, x, lam[i]);
-                        v = fabs(v);
-                        if (best < 0 || v < best_v) { best = p; best_v = v; }
+                    for (int i = TT - 1; i >= 0; --i)
+                        if (i < nu) v = fma(v, x, lam[i]);
+                    v = fabs(v);
+                    double cv = v < kHuge ? v : kHuge;       // every point is finite in the list, so each enters once
+                    int cn = p;
+#pragma unroll UF
+                    for (int k = 0; k < TT; ++k) {
+                        if (k < nu && cv < small_v[k]) {
+                            const double tv = small_v[k]; small_v[k] = cv; cv = tv;
+                            const int tn = nodes[k]; nodes[k] = cn; cn = tn;
+                        }
                     }
-                    nodes[k] = best;
-                    taken |= 1ULL << best;
                 }
             }
+            // normal equations of H_A e = r: H_A^T H_A does not change between the two passes below
+            double gram[TT][TT];
+#pragma unroll UF
+            for (int i = 0; i < TT; ++i)
+#pragma unroll UF
+                for (int j = 0; j < TT; ++j) {
+                    double s2 = 0.0;
+                    if (i < nu && j < nu) {
+                        if (kGramTable) {
+                            s2 = sG[nodes[i] * P + nodes[j]];
+                        } else {
+                            for (int q = 0; q < R; ++q) s2 = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s2);
+                        }
+                    }
+                    gram[i][j] = s2;
+                }
             // least squares H_A e = r through the normal equations, then one step of refinement on the
             // residual (neighbouring nodes make H_A ill-conditioned; the refinement brings the error
             // values back to the accuracy of an orthogonal factorisation)
@@ -273,13 +396,8 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
                     for (int j = 0; j <= TT; ++j) a[i][j] = 0.0;
                     if (i < nu) {
 #pragma unroll UF
-                        for (int j = 0; j < TT; ++j) {
-                            if (j < nu) {
-                                double s2 = 0.0;
-                                for (int q = 0; q < R; ++q) s2 = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s2);
-                                a[i][j] = s2;
-                            }
-                        }
+                        for (int j = 0; j < TT; ++j)
+                            if (j < nu) a[i][j] = gram[i][j];
                         double s2 = 0.0;
 #pragma unroll UF
                         for (int q = 0; q < RT; ++q)
@@ -336,34 +454,28 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
             }
         }
     }
+    finish_by_last_block(prm);
 }
 
-__global__ void position_finish_kernel(PosParams prm) {
-    gpd_position_result* res = prm.result;
-    const unsigned long long active = prm.counters[1], failed = prm.counters[3];
-    if (threadIdx.x == 0) {
-        res->outcome = active == 0ULL ? GPD_NO_ERROR : (failed ? GPD_DECODE_FAILURE : GPD_CORRECTED);
-        res->max_errors = (int32_t)prm.counters[5];
-        res->device_status = 0;
-        res->reserved = 0;
-        res->n_active = (int64_t)active;
-        res->n_corrected = (int64_t)prm.counters[2];
-        res->n_failed = (int64_t)failed;
-        res->n_entries = (int64_t)prm.counters[4];
-    }
-    for (int p = threadIdx.x; p < kMaxNodes; p += blockDim.x)
-        res->touched[p] = (p < prm.P && ((prm.counters[6] >> p) & 1ULL)) ? 1 : 0;
-}
+__global__ void position_finish_kernel(PosParams prm) { write_position_result(prm, threadIdx.x, blockDim.x); }
 
 constexpr int64_t kPosHeaderBytes = 256;  // counters
 
 }  // namespace
 
+// Listed positions whose syndrome the scan keeps for the repair: one in sixteen (at least 4096); a run
+// with more failures than that reads the remaining codewords a second time.
+int64_t position_records(int64_t L) { return std::min<int64_t>(L, std::max<int64_t>(4096, L / 16)); }
+
 int64_t position_workspace_bytes(const gpd_plan_s* plan) {
-    int64_t L = 0;
-    for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT})
-        if (plan->prod[w].Q > 0) L = std::max<int64_t>(L, plan->prod[w].br * plan->prod[w].bc);
-    return kPosHeaderBytes + (L * 4 + 255) / 256 * 256;
+    int64_t L = 0, rec = 0;
+    for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT}) {
+        if (plan->prod[w].Q == 0) continue;
+        const int64_t Lw = plan->prod[w].br * plan->prod[w].bc;
+        L = std::max<int64_t>(L, Lw);
+        rec = std::max<int64_t>(rec, position_records(Lw) * (plan->prod[w].R + 1) * (int64_t)sizeof(double));
+    }
+    return kPosHeaderBytes + (L * 4 + 255) / 256 * 256 + rec;
 }
 
 gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* outputs, gpd_position_result* result,
@@ -385,6 +497,8 @@ gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* o
     prm.points = plan->dev.base + plan->dev.off_points;
     prm.counters = reinterpret_cast<unsigned long long*>(workspace);
     prm.list = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(workspace) + kPosHeaderBytes);
+    prm.rec = reinterpret_cast<double*>(reinterpret_cast<char*>(workspace) + kPosHeaderBytes + (L * 4 + 255) / 256 * 256);
+    prm.rec_cap = (unsigned long long)position_records(L);
     prm.result = result;
     prm.L = L; prm.P = plan->P; prm.R = pi.R;
     prm.tau2 = plan->tau_col * plan->tau_col;
@@ -401,15 +515,15 @@ gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* o
         else f32 ? position_scan_kernel<float, 32><<<grid1, 256, smem1, st>>>(prm)
                  : position_scan_kernel<double, 32><<<grid1, 256, smem1, st>>>(prm);
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
-        const size_t smem2 = sizeof(double) * (2 * pi.R * plan->P + plan->P);
+        const size_t smem2 = sizeof(double) * (2 * pi.R * plan->P + plan->P + pi.R * pi.R + (pi.R <= 8 ? plan->P * plan->P : 0));
         const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 63) / 64, sm_count() * 8));
         if (pi.R <= 8) f32 ? position_fix_kernel<float, 8, 4><<<grid2, 64, smem2, st>>>(prm)
                            : position_fix_kernel<double, 8, 4><<<grid2, 64, smem2, st>>>(prm);
         else f32 ? position_fix_kernel<float, 32, 16><<<grid2, 64, smem2, st>>>(prm)
                  : position_fix_kernel<double, 32, 16><<<grid2, 64, smem2, st>>>(prm);
-        if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+        return launch_ok();                          // the last block of the repair kernel writes the result
     }
-    position_finish_kernel<<<1, 64, 0, st>>>(prm);
+    position_finish_kernel<<<1, 64, 0, st>>>(prm);   // no parity checks: nothing was scanned
     return launch_ok();
 }
 

@@ -41,6 +41,17 @@ def _scatter_errors(Z, t_max, frac, seed, scale):
     (128, 128, 32, 2, 2, 2, 20, g.GPD_PREC_FP64),            # Q = 9,  R = 11, t = 5: the general (not unrolled) form
 ])
 def test_positions_repaired_like_the_oracle(N1, N0, B, m, n, d1, P, prec):
+    _check_against_oracle(N1, N0, B, m, n, d1, P, prec, frac=0.05)
+
+
+def test_positions_more_failures_than_kept_syndromes():
+    """The scan keeps the syndromes of the first 4096 failing positions for the repair (16384 positions
+    here); with 40 % of the positions hit the repair reads the other codewords a second time.  Both routes
+    must decide like the oracle."""
+    _check_against_oracle(512, 512, 128, 2, 4, 2, 25, g.GPD_PREC_FP64, frac=0.4)
+
+
+def _check_against_oracle(N1, N0, B, m, n, d1, P, prec, frac):
     rng = np.random.default_rng(N1 + P)
     W = (rng.standard_normal((N1, N0)) / np.sqrt(N0)).astype(np.float32)
     X = rng.standard_normal((N0, B)).astype(np.float32)
@@ -52,7 +63,7 @@ def test_positions_repaired_like_the_oracle(N1, N0, B, m, n, d1, P, prec):
     t = (P - code.Q_f) // 2
     scale = float(np.sqrt(np.mean(clean ** 2)))
     bad = clean.copy()
-    sizes = _scatter_errors(bad, max(t, 1), 0.05, seed=7, scale=scale)
+    sizes = _scatter_errors(bad, max(t, 1), frac, seed=7, scale=scale)
     Zg = dev(bad.astype(cp.np_dtype).reshape(-1))
     tol = tolerances_for(cp.np_dtype)
     ro = correct_positions(bad.astype(cp.np_dtype), code.points, code.Q_f, tol)
