@@ -303,7 +303,9 @@ gpd_status gpd_locate_errors(gpd_plan_t plan, gpd_product which, const void* out
  * Q of them) reads the repaired outputs.  Positions that cannot be repaired are left as they are
  * and counted; the outcome is then GPD_DECODE_FAILURE.  Meant for small floor((P-Q)/2) (the
  * locator is found in the monomial basis).
- * result_dev: device gpd_position_result.  workspace_dev: GPD_Q_POSITION_WORKSPACE_BYTES bytes.
+ * result_dev: device gpd_position_result.  workspace_dev: GPD_Q_POSITION_WORKSPACE_BYTES bytes
+ * (counters, a 4-byte index per position, and the syndromes of up to one position in 32 (at least 4096);
+ * when more positions than that fail, the codewords of the others are read a second time).
  */
 gpd_status gpd_correct_positions(gpd_plan_t plan, gpd_product which, void* outputs_dev,
                                  gpd_position_result* result_dev, void* workspace_dev, void* stream);

@@ -463,9 +463,9 @@ constexpr int64_t kPosHeaderBytes = 256;  // counters
 
 }  // namespace
 
-// Listed positions whose syndrome the scan keeps for the repair: one in sixteen (at least 4096); a run
+// Listed positions whose syndrome the scan keeps for the repair: one in 32 (at least 4096); a run
 // with more failures than that reads the remaining codewords a second time.
-int64_t position_records(int64_t L) { return std::min<int64_t>(L, std::max<int64_t>(4096, L / 16)); }
+int64_t position_records(int64_t L) { return std::min<int64_t>(L, std::max<int64_t>(4096, L / 32)); }
 
 int64_t position_workspace_bytes(const gpd_plan_s* plan) {
     int64_t L = 0, rec = 0;

@@ -43,7 +43,9 @@ def test_position_result_layout_workspace_query_and_argument_checks():
     c = wl.CONFIG_3_MATMUL
     plan = g.gpd_plan((c.N1, c.N0, c.B), (c.m, c.n, c.d, 1), c.P)
     L = (c.N1 // c.m) * max(c.B // c.d, c.N0 // c.n)             # largest product of the plan (audit: N1/m x N0/n)
-    assert plan.query(g.GPD_Q_POSITION_WORKSPACE_BYTES) == 256 + 4 * L
+    # counters, the list of failing positions, and R + 1 doubles (syndrome, squared norm) for one position
+    # in 32 of the product that needs most: here the audit product, R = P - Q_w = 17
+    assert plan.query(g.GPD_Q_POSITION_WORKSPACE_BYTES) == 256 + 4 * L + (L // 32) * (17 + 1) * 8
     one = C.c_void_p(4096)                                        # never dereferenced: the checks come first
     assert g.lib.gpd_correct_positions(plan.handle, g.GPD_FWD, one, one, None, None) == g.GPD_ERR_WORKSPACE
     assert g.lib.gpd_correct_positions(plan.handle, g.GPD_FWD, None, one, one, None) == g.GPD_ERR_ARG
