@@ -67,6 +67,8 @@ struct gpd_plan_s {
     bool train = false;          // GPD_PREC_FP64_SLICED_TRAIN: W's buffer holds FP64 shares and two sliced copies
     double tau_col = 0, tau_in = 0;
     std::vector<double> points;
+    bool points_symmetric = false;   // b_{P-1-p} = -b_p exactly (always so for the built-in Chebyshev points)
+    bool alt_subst = false;          // GPD_SUBST_V_EQ_UM: the exponent of W's block (i, j) is i + m j instead of n i + j
     std::vector<double> coefW, coefX, coefDT, coefDup, coefXup;   // [P][blocks]
     gpd::ProductInfo prod[4];    // indexed by gpd_product (GPD_UPD unused)
     // device side

@@ -217,6 +217,9 @@ extern "C" gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* sp
         for (int q = 0; q < p; ++q)
             if (plan->points[p] == plan->points[q]) { delete plan; return GPD_ERR_POINTS; }
     }
+    plan->alt_subst = alt;
+    plan->points_symmetric = true;
+    for (int p = 0; p < P; ++p) plan->points_symmetric &= plan->points[P - 1 - p] == -plan->points[p];
     const bool bwd_ok = (P >= Qb) && (Qb <= kMaxQ) && (P - Qb <= kMaxR);
     const bool audit_ok = (P - Qw <= kMaxR);
     const int64_t q_for_prec = bwd_ok ? std::max(Qf, Qb) : Qf;

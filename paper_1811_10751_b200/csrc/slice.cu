@@ -27,6 +27,10 @@ struct SliceParams {
     int64_t ld;            // leading dimension of src
     int64_t br, bc;        // block rows / cols of src
     int gc, nblk, P;
+    // W only: the share of node p is a polynomial of degree nblk - 1 in its point b_p, and the points come
+    // in pairs b_{P-1-p} = -b_p.  blk_of_exp[e] is the block whose coefficient is b_p^e.
+    bool poly;
+    int blk_of_exp[16];
 };
 
 // Largest magnitudes are tracked as the high 32 bits of |a| (non-negative doubles order like
@@ -177,7 +181,7 @@ inline size_t fused_smem_bytes(int P, int nblk, int64_t bc) {
     return head + 2 * sizeof(float) * (size_t)nblk * (size_t)bc;
 }
 
-template <int NBLK, int S>
+template <int NBLK, int S, bool POLY>
 __global__ void __launch_bounds__(kFusedMaxThreads, 1) rowslice_fused_kernel(SliceParams prm) {
     extern __shared__ __align__(16) unsigned char s_raw[];
     const int P = prm.P, tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31;
@@ -242,27 +246,63 @@ __global__ void __launch_bounds__(kFusedMaxThreads, 1) rowslice_fused_kernel(Sli
         __syncthreads();
         if (tid < NBLK) blk[tid] = 0u;               // next read two rows from now, barriers in between
         for (int it = tid; it < bc4; it += nthr) {
-            double x[NBLK][4];
+            double x[NBLK][4];                       // POLY: indexed by the exponent, else by the block
 #pragma unroll
             for (int b = 0; b < NBLK; ++b) {
-                const float4 v = *reinterpret_cast<const float4*>(xb + b * bc + 4 * it);
+                const int blk = POLY ? prm.blk_of_exp[b] : b;
+                const float4 v = *reinterpret_cast<const float4*>(xb + blk * bc + 4 * it);
                 x[b][0] = v.x; x[b][1] = v.y; x[b][2] = v.z; x[b][3] = v.w;
             }
             unsigned int off = (unsigned int)((r * bc) >> 2) + (unsigned int)it;   // word offset inside plane 0, node 0
-#pragma unroll 2
-            for (int p = 0; p < P; ++p, off += node_words) {
-                const double* cf = s_cf + p * NBLK;
-                double a[4] = {0, 0, 0, 0};
+            if constexpr (POLY) {
+                // sum_e x_e b^e = E(b^2) + b O(b^2) with E, O the even and odd halves: nodes p and P-1-p
+                // (b and -b) share E and O, which halves the FP64 work of the evaluation
+                constexpr int LE = (NBLK - 1) & ~1, LO = ((NBLK - 2) & ~1) + 1;
+                const int blk1 = prm.blk_of_exp[1];
+                for (int p = 0; 2 * p < P; ++p) {
+                    const int p2 = P - 1 - p;
+                    const double b1 = s_cf[p * NBLK + blk1], b2 = s_cf[p2 * NBLK + blk1], y = b1 * b1;
+                    double E[4], O[4], a[4];
 #pragma unroll
-                for (int b = 0; b < NBLK; ++b) {
-                    const double k = cf[b];
-                    a[0] = fma(k, x[b][0], a[0]); a[1] = fma(k, x[b][1], a[1]);
-                    a[2] = fma(k, x[b][2], a[2]); a[3] = fma(k, x[b][3], a[3]);
+                    for (int v = 0; v < 4; ++v) {
+                        E[v] = x[LE][v];
+                        O[v] = x[LO][v];
+#pragma unroll
+                        for (int e = LE - 2; e >= 0; e -= 2) E[v] = fma(E[v], y, x[e][v]);
+#pragma unroll
+                        for (int e = LO - 2; e >= 1; e -= 2) O[v] = fma(O[v], y, x[e][v]);
+                        a[v] = fma(b1, O[v], E[v]);
+                    }
+                    unsigned int word[S];
+                    digits4<S>(a, s_scale[p], word);
+                    const unsigned int o1 = off + (unsigned int)p * node_words;
+#pragma unroll
+                    for (int s = 0; s < S; ++s) __stcs(planes_w + (o1 + (unsigned int)s * plane_words), word[s]);
+                    if (p2 != p) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) a[v] = fma(b2, O[v], E[v]);
+                        digits4<S>(a, s_scale[p2], word);
+                        const unsigned int o2 = off + (unsigned int)p2 * node_words;
+#pragma unroll
+                        for (int s = 0; s < S; ++s) __stcs(planes_w + (o2 + (unsigned int)s * plane_words), word[s]);
+                    }
                 }
-                unsigned int word[S];
-                digits4<S>(a, s_scale[p], word);
+            } else {
+#pragma unroll 2
+                for (int p = 0; p < P; ++p, off += node_words) {
+                    const double* cf = s_cf + p * NBLK;
+                    double a[4] = {0, 0, 0, 0};
 #pragma unroll
-                for (int s = 0; s < S; ++s) __stcs(planes_w + (off + (unsigned int)s * plane_words), word[s]);
+                    for (int b = 0; b < NBLK; ++b) {
+                        const double k = cf[b];
+                        a[0] = fma(k, x[b][0], a[0]); a[1] = fma(k, x[b][1], a[1]);
+                        a[2] = fma(k, x[b][2], a[2]); a[3] = fma(k, x[b][3], a[3]);
+                    }
+                    unsigned int word[S];
+                    digits4<S>(a, s_scale[p], word);
+#pragma unroll
+                    for (int s = 0; s < S; ++s) __stcs(planes_w + (off + (unsigned int)s * plane_words), word[s]);
+                }
             }
         }
         __syncthreads();                             // row buffer `buf` is refilled by the next trip's copies
@@ -434,7 +474,10 @@ gpd_status launch_rows_fused(const SliceParams& prm, int slices, size_t smem, cu
         kernel<<<grid, threads, smem, st>>>(prm);
         return launch_ok();
     };
-    return slices == 6 ? go(rowslice_fused_kernel<NBLK, 6>) : go(rowslice_fused_kernel<NBLK, 5>);
+    if constexpr (NBLK >= 2) {
+        if (prm.poly) return slices == 6 ? go(rowslice_fused_kernel<NBLK, 6, true>) : go(rowslice_fused_kernel<NBLK, 5, true>);
+    }
+    return slices == 6 ? go(rowslice_fused_kernel<NBLK, 6, false>) : go(rowslice_fused_kernel<NBLK, 5, false>);
 }
 
 template <int NBLK>
@@ -572,7 +615,12 @@ gpd_status encode_sliced_launch(gpd_plan_s* plan, int operand, const float* src,
     switch (operand) {
         case -1:                  // W: m x n blocks of (N1/m) x (N0/n); operand rows = share rows, K = N0/n
             gr = c.m; prm.gc = c.n; prm.ld = s.N0; prm.br = s.N1 / c.m; prm.bc = s.N0 / c.n;
-            prm.coef = plan->dev.base + plan->dev.off_coefW; break;
+            prm.coef = plan->dev.base + plan->dev.off_coefW;
+            prm.poly = c.m * c.n <= 16 && plan->points_symmetric;
+            for (int i = 0; i < c.m; ++i)
+                for (int j = 0; j < c.n; ++j)
+                    if (prm.poly) prm.blk_of_exp[plan->alt_subst ? i + c.m * j : c.n * i + j] = i * c.n + j;
+            break;
         case GPD_OPERAND_X_FWD:   // X: n x d1 blocks of (N0/n) x (B/d1); operand rows = share columns, K = N0/n
             gr = c.n; prm.gc = c.d1; prm.ld = s.B; prm.br = s.N0 / c.n; prm.bc = s.B / c.d1;
             prm.coef = plan->dev.base + plan->dev.off_coefX; by_rows = false; break;

@@ -115,6 +115,25 @@ def test_sliced_products_with_the_library_points(N1, N0, B, m, n, d1, P, S):
     assert op.rel_fro(cp.decode(g.GPD_FWD, Z), op.ref_forward(W, X)) < 1e-4
 
 
+def test_sliced_products_alternate_substitution_with_the_library_points():
+    """The substitution v = u^m, w = u^(mn) gives W's block (i, j) the exponent i + m j; with mirrored
+    points the encoder evaluates the share polynomial of nodes p and P-1-p from shared even and odd halves
+    and has to pick the blocks in the order of their exponents."""
+    from oracle.code import SUBST_V_UM
+    N1, N0, B, m, n, d1, P = 192, 256, 64, 3, 2, 2, 21
+    plan0 = g.gpd_plan((N1, N0, B), (m, n, d1, 1), P)
+    pts = plan0.table(g.GPD_TABLE_POINTS)
+    plan0.destroy()
+    W, X = _inputs(N1, N0, B, seed=77)
+    code = GPCode(N1, N0, B, m, n, d1, 1, P, points=pts, subst=SUBST_V_UM)
+    assert P >= code.Q_f
+    cp, Z = _sliced_products(code, W, X)
+    Wsh, Xsh = op.encode_W(W, code), op.encode_X(X, code)
+    got = cp.outputs_as_array(g.GPD_FWD, Z)
+    assert (np.abs(got - op.worker_products(Wsh, Xsh)) <= _output_tolerance(W, code, Wsh, Xsh)).all()
+    assert op.rel_fro(cp.decode(g.GPD_FWD, Z), op.ref_forward(W, X)) < 1e-4
+
+
 def test_sliced_scales_zero_rows_and_tiny_values():
     """Row / column scales: rows of zeros, columns of zeros and operands 1e-30 and 1e+20 times the
     usual size decode to the same relative accuracy (the digits carry no absolute scale)."""
