@@ -200,6 +200,94 @@ __device__ __forceinline__ void finish_by_last_block(const PosParams& prm) {
     if (s_last) write_position_result(prm, threadIdx.x, blockDim.x);
 }
 
+// One round of the repair for a support of exactly NU nodes, everything sized by NU at compile time
+// (small codes): locator from the Hankel system, its NU smallest values over the points, least
+// squares H_A e = r through the normal equations with one step of refinement, zero test of what is
+// left of r.  Same arithmetic, in the same order, as the general form inside position_fix_kernel.
+template <int NU, int RT, int TT>
+__device__ __forceinline__ bool try_support(const double (&S)[RT], const double (&r)[RT], const double* sH,
+                                            const double* sPts, const double* sG, int P, int R, double limit,
+                                            int (&nodes)[TT], double (&err)[TT]) {
+    static_assert(2 * NU <= RT && NU <= TT, "support size against the parity checks");
+    double a[NU][NU + 1], lam[NU];
+#pragma unroll
+    for (int j = 0; j < NU; ++j) {
+#pragma unroll
+        for (int i = 0; i < NU; ++i) a[j][i] = S[j + i];
+        a[j][NU] = -S[j + NU];
+    }
+    if (!solve_small<NU>(a, NU, lam)) return false;
+    double small_v[NU];
+    int nd[NU];
+#pragma unroll
+    for (int k = 0; k < NU; ++k) { small_v[k] = __longlong_as_double(0x7ff0000000000000LL); nd[k] = 0; }
+#pragma unroll 5
+    for (int p = 0; p < P; ++p) {
+        const double x = sPts[p];
+        double v = 1.0;
+#pragma unroll
+        for (int i = NU - 1; i >= 0; --i) v = fma(v, x, lam[i]);
+        v = fabs(v);
+        double cv = v < kHuge ? v : kHuge;
+        int cn = p;
+#pragma unroll
+        for (int k = 0; k < NU; ++k) {
+            if (cv < small_v[k]) {
+                const double tv = small_v[k]; small_v[k] = cv; cv = tv;
+                const int tn = nd[k]; nd[k] = cn; cn = tn;
+            }
+        }
+    }
+    double gram[NU][NU];
+#pragma unroll
+    for (int i = 0; i < NU; ++i)
+#pragma unroll
+        for (int j = 0; j < NU; ++j) gram[i][j] = sG[nd[i] * P + nd[j]];
+    double e[NU];
+#pragma unroll
+    for (int i = 0; i < NU; ++i) e[i] = 0.0;
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+        double v[RT];
+#pragma unroll
+        for (int q = 0; q < RT; ++q) {
+            double w = r[q];
+            if (q < R) {
+#pragma unroll
+                for (int i = 0; i < NU; ++i) w = fma(-sH[q * P + nd[i]], e[i], w);
+            }
+            v[q] = w;
+        }
+#pragma unroll
+        for (int i = 0; i < NU; ++i) {
+#pragma unroll
+            for (int j = 0; j < NU; ++j) a[i][j] = gram[i][j];
+            double s2 = 0.0;
+#pragma unroll
+            for (int q = 0; q < RT; ++q)
+                if (q < R) s2 = fma(sH[q * P + nd[i]], v[q], s2);
+            a[i][NU] = s2;
+        }
+        double delta[NU];
+        if (!solve_small<NU>(a, NU, delta)) return false;
+#pragma unroll
+        for (int i = 0; i < NU; ++i) e[i] += delta[i];
+    }
+    double left = 0.0;
+#pragma unroll
+    for (int q = 0; q < RT; ++q) {
+        if (q < R) {
+            double w = r[q];
+#pragma unroll
+            for (int i = 0; i < NU; ++i) w = fma(-sH[q * P + nd[i]], e[i], w);
+            left = fma(w, w, left);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < NU; ++i) { nodes[i] = nd[i]; err[i] = e[i]; }
+    return left <= limit;
+}
+
 // RT: parity checks rounded up (8 or 32); TT: errors per codeword rounded up (4 or 16).  The
 // right-hand side of a system sits in column TT of its rows.
 template <typename T, int RT, int TT>
@@ -298,6 +386,16 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
         for (int i = 0; i < TT; ++i) { nodes[i] = 0; err[i] = 0.0; }
 #pragma unroll 1
         for (int nu = 1; valid && nu <= t && accepted == 0; ++nu) {
+            if constexpr (TT <= 4 && RT == 8) {       // small codes: one instantiation per support size
+                bool ok = false;
+                switch (nu) {
+                    case 1: ok = try_support<1, RT, TT>(S, r, sH, sPts, sG, P, R, limit, nodes, err); break;
+                    case 2: ok = try_support<2, RT, TT>(S, r, sH, sPts, sG, P, R, limit, nodes, err); break;
+                    case 3: ok = try_support<3, RT, TT>(S, r, sH, sPts, sG, P, R, limit, nodes, err); break;
+                    default: ok = try_support<4, RT, TT>(S, r, sH, sPts, sG, P, R, limit, nodes, err); break;
+                }
+                if (ok) accepted = nu;
+            } else {
             double a[TT][TT + 1], lam[TT];
 #pragma unroll UF
             for (int j = 0; j < TT; ++j) {
@@ -428,6 +526,7 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
                 }
             }
             if (left <= limit) accepted = nu;
+            }
         }
         unsigned long long mask = 0ULL;
 #pragma unroll UF
