@@ -14,8 +14,9 @@
 // accumulators are adjacent in tensor memory, so one tcgen05.mma of N = 64 (S - s) columns
 // (two when that exceeds 256) covers all pairs of plane s: 8 (6) instructions per 32 elements of K.
 //
-// One CTA per SM walks the output tiles.  Warp roles: warp 0 one lane issues the TMA copies (2 S per
-// 64-element k-block, 3-stage ring that runs on across tiles), warp 1 allocates tensor memory and
+// One CTA per SM walks the output tiles.  Warp roles: warp 0 one lane issues the TMA copies (two per
+// 64-element k-block: the planes are a 4-d tensor [S][P][rows][K] and one box holds all S planes of an
+// operand; 3-stage ring that runs on across tiles), warp 1 allocates tensor memory and
 // one lane issues the MMAs, warps 2..9 read the accumulators back and combine them in FP64
 // (sum_g acc_g 2^-8g), release tensor memory to the next tile's MMAs, then apply the row and column
 // powers of two and store while that tile's main loop is already running.

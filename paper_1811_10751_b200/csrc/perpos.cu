@@ -396,136 +396,136 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
                 }
                 if (ok) accepted = nu;
             } else {
-            double a[TT][TT + 1], lam[TT];
-#pragma unroll UF
-            for (int j = 0; j < TT; ++j) {
-                lam[j] = 0.0;
-#pragma unroll UF
-                for (int i = 0; i <= TT; ++i) a[j][i] = 0.0;
-            }
-            // Hankel system of the locator: sum_i l_i S_{j+i} = -S_{j+nu}, j = 0 .. nu-1
-            if constexpr (TT <= 4) {                              // S_{j+i} without a dynamic index
-#pragma unroll
-                for (int j = 0; j < TT; ++j)
-#pragma unroll
-                    for (int i = 0; i < TT; ++i)
-                        if (j < nu && i < nu) {
-#pragma unroll
-                            for (int q = 0; q < RT; ++q)
-                                if (q == j + i) a[j][i] = S[q];
-                        }
-#pragma unroll
-                for (int j = 0; j < TT; ++j)
-                    if (j < nu) {
-#pragma unroll
-                        for (int q = 0; q < RT; ++q)
-                            if (q == j + nu) a[j][TT] = -S[q];
-                    }
-            } else {
-                for (int j = 0; j < nu; ++j) {
-                    for (int i = 0; i < nu; ++i) a[j][i] = S[j + i];
-                    a[j][TT] = -S[j + nu];
-                }
-            }
-            if (!solve_small<TT>(a, nu, lam)) continue;
-            // the nu points where the locator is smallest, smallest first (of equal values the lower
-            // point): one pass over the points with an insertion into the sorted list kept so far
-            {
-                double small_v[TT];
-#pragma unroll UF
-                for (int k = 0; k < TT; ++k) { small_v[k] = __longlong_as_double(0x7ff0000000000000LL); nodes[k] = 0; }
-#pragma unroll 5
-                for (int p = 0; p < P; ++p) {
-                    const double x = sPts[p];
-                    double v = 1.0;
-#pragma unroll UF
-                    for (int i = TT - 1; i >= 0; --i)
-                        if (i < nu) v = fma(v, x, lam[i]);
-                    v = fabs(v);
-                    double cv = v < kHuge ? v : kHuge;       // every point is finite in the list, so each enters once
-                    int cn = p;
-#pragma unroll UF
-                    for (int k = 0; k < TT; ++k) {
-                        if (k < nu && cv < small_v[k]) {
-                            const double tv = small_v[k]; small_v[k] = cv; cv = tv;
-                            const int tn = nodes[k]; nodes[k] = cn; cn = tn;
-                        }
-                    }
-                }
-            }
-            // normal equations of H_A e = r: H_A^T H_A does not change between the two passes below
-            double gram[TT][TT];
-#pragma unroll UF
-            for (int i = 0; i < TT; ++i)
+                double a[TT][TT + 1], lam[TT];
 #pragma unroll UF
                 for (int j = 0; j < TT; ++j) {
-                    double s2 = 0.0;
-                    if (i < nu && j < nu) {
-                        if (kGramTable) {
-                            s2 = sG[nodes[i] * P + nodes[j]];
-                        } else {
-                            for (int q = 0; q < R; ++q) s2 = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s2);
+                    lam[j] = 0.0;
+#pragma unroll UF
+                    for (int i = 0; i <= TT; ++i) a[j][i] = 0.0;
+                }
+                // Hankel system of the locator: sum_i l_i S_{j+i} = -S_{j+nu}, j = 0 .. nu-1
+                if constexpr (TT <= 4) {                              // S_{j+i} without a dynamic index
+#pragma unroll
+                    for (int j = 0; j < TT; ++j)
+#pragma unroll
+                        for (int i = 0; i < TT; ++i)
+                            if (j < nu && i < nu) {
+#pragma unroll
+                                for (int q = 0; q < RT; ++q)
+                                    if (q == j + i) a[j][i] = S[q];
+                            }
+#pragma unroll
+                    for (int j = 0; j < TT; ++j)
+                        if (j < nu) {
+#pragma unroll
+                            for (int q = 0; q < RT; ++q)
+                                if (q == j + nu) a[j][TT] = -S[q];
+                        }
+                } else {
+                    for (int j = 0; j < nu; ++j) {
+                        for (int i = 0; i < nu; ++i) a[j][i] = S[j + i];
+                        a[j][TT] = -S[j + nu];
+                    }
+                }
+                if (!solve_small<TT>(a, nu, lam)) continue;
+                // the nu points where the locator is smallest, smallest first (of equal values the lower
+                // point): one pass over the points with an insertion into the sorted list kept so far
+                {
+                    double small_v[TT];
+#pragma unroll UF
+                    for (int k = 0; k < TT; ++k) { small_v[k] = __longlong_as_double(0x7ff0000000000000LL); nodes[k] = 0; }
+#pragma unroll 5
+                    for (int p = 0; p < P; ++p) {
+                        const double x = sPts[p];
+                        double v = 1.0;
+#pragma unroll UF
+                        for (int i = TT - 1; i >= 0; --i)
+                            if (i < nu) v = fma(v, x, lam[i]);
+                        v = fabs(v);
+                        double cv = v < kHuge ? v : kHuge;       // every point is finite in the list, so each enters once
+                        int cn = p;
+#pragma unroll UF
+                        for (int k = 0; k < TT; ++k) {
+                            if (k < nu && cv < small_v[k]) {
+                                const double tv = small_v[k]; small_v[k] = cv; cv = tv;
+                                const int tn = nodes[k]; nodes[k] = cn; cn = tn;
+                            }
                         }
                     }
-                    gram[i][j] = s2;
                 }
-            // least squares H_A e = r through the normal equations, then one step of refinement on the
-            // residual (neighbouring nodes make H_A ill-conditioned; the refinement brings the error
-            // values back to the accuracy of an orthogonal factorisation)
-            bool solved = true;
+                // normal equations of H_A e = r: H_A^T H_A does not change between the two passes below
+                double gram[TT][TT];
 #pragma unroll UF
-            for (int i = 0; i < TT; ++i) err[i] = 0.0;
+                for (int i = 0; i < TT; ++i)
+#pragma unroll UF
+                    for (int j = 0; j < TT; ++j) {
+                        double s2 = 0.0;
+                        if (i < nu && j < nu) {
+                            if (kGramTable) {
+                                s2 = sG[nodes[i] * P + nodes[j]];
+                            } else {
+                                for (int q = 0; q < R; ++q) s2 = fma(sH[q * P + nodes[i]], sH[q * P + nodes[j]], s2);
+                            }
+                        }
+                        gram[i][j] = s2;
+                    }
+                // least squares H_A e = r through the normal equations, then one step of refinement on the
+                // residual (neighbouring nodes make H_A ill-conditioned; the refinement brings the error
+                // values back to the accuracy of an orthogonal factorisation)
+                bool solved = true;
+#pragma unroll UF
+                for (int i = 0; i < TT; ++i) err[i] = 0.0;
 #pragma unroll 1
-            for (int pass = 0; pass < 2 && solved; ++pass) {
-                double v[RT];
+                for (int pass = 0; pass < 2 && solved; ++pass) {
+                    double v[RT];
+#pragma unroll UF
+                    for (int q = 0; q < RT; ++q) {
+                        double w = r[q];
+                        if (q < R) {
+#pragma unroll UF
+                            for (int i = 0; i < TT; ++i)
+                                if (i < nu) w = fma(-sH[q * P + nodes[i]], err[i], w);
+                        }
+                        v[q] = w;
+                    }
+#pragma unroll UF
+                    for (int i = 0; i < TT; ++i) {
+#pragma unroll UF
+                        for (int j = 0; j <= TT; ++j) a[i][j] = 0.0;
+                        if (i < nu) {
+#pragma unroll UF
+                            for (int j = 0; j < TT; ++j)
+                                if (j < nu) a[i][j] = gram[i][j];
+                            double s2 = 0.0;
+#pragma unroll UF
+                            for (int q = 0; q < RT; ++q)
+                                if (q < R) s2 = fma(sH[q * P + nodes[i]], v[q], s2);
+                            a[i][TT] = s2;
+                        }
+                    }
+                    double delta[TT];
+#pragma unroll UF
+                    for (int i = 0; i < TT; ++i) delta[i] = 0.0;
+                    solved = solve_small<TT>(a, nu, delta);
+                    if (solved) {
+#pragma unroll UF
+                        for (int i = 0; i < TT; ++i)
+                            if (i < nu) err[i] += delta[i];
+                    }
+                }
+                if (!solved) continue;
+                double left = 0.0;
 #pragma unroll UF
                 for (int q = 0; q < RT; ++q) {
-                    double w = r[q];
                     if (q < R) {
+                        double w = r[q];
 #pragma unroll UF
                         for (int i = 0; i < TT; ++i)
                             if (i < nu) w = fma(-sH[q * P + nodes[i]], err[i], w);
-                    }
-                    v[q] = w;
-                }
-#pragma unroll UF
-                for (int i = 0; i < TT; ++i) {
-#pragma unroll UF
-                    for (int j = 0; j <= TT; ++j) a[i][j] = 0.0;
-                    if (i < nu) {
-#pragma unroll UF
-                        for (int j = 0; j < TT; ++j)
-                            if (j < nu) a[i][j] = gram[i][j];
-                        double s2 = 0.0;
-#pragma unroll UF
-                        for (int q = 0; q < RT; ++q)
-                            if (q < R) s2 = fma(sH[q * P + nodes[i]], v[q], s2);
-                        a[i][TT] = s2;
+                        left = fma(w, w, left);
                     }
                 }
-                double delta[TT];
-#pragma unroll UF
-                for (int i = 0; i < TT; ++i) delta[i] = 0.0;
-                solved = solve_small<TT>(a, nu, delta);
-                if (solved) {
-#pragma unroll UF
-                    for (int i = 0; i < TT; ++i)
-                        if (i < nu) err[i] += delta[i];
-                }
-            }
-            if (!solved) continue;
-            double left = 0.0;
-#pragma unroll UF
-            for (int q = 0; q < RT; ++q) {
-                if (q < R) {
-                    double w = r[q];
-#pragma unroll UF
-                    for (int i = 0; i < TT; ++i)
-                        if (i < nu) w = fma(-sH[q * P + nodes[i]], err[i], w);
-                    left = fma(w, w, left);
-                }
-            }
-            if (left <= limit) accepted = nu;
+                if (left <= limit) accepted = nu;
             }
         }
         unsigned long long mask = 0ULL;
