@@ -17,8 +17,9 @@
  *     calls only enqueue work and never synchronise; the return value reports host-detectable
  *     errors only.  Data-dependent outcomes (no error / corrected / decoding failure) are
  *     written to a gpd_locate_result in device memory.
- *   - The library allocates device memory only for the plan's small coefficient tables
- *     (uploaded by gpd_plan_upload or on the plan's first compute call, freed by gpd_plan_destroy).
+ *   - The library allocates device memory only for the plan's small coefficient tables and, on
+ *     FP32 plans, a scratch area of 64 KB per SM behind them (one allocation, made by
+ *     gpd_plan_upload or on the plan's first compute call, freed by gpd_plan_destroy).
  *   - Storage type of shares and worker outputs: float (GPD_PREC_FP32) or double
  *     (GPD_PREC_FP64); inputs W, X, Delta and decoded results are always float.
  *   - A plan is immutable after creation; concurrent calls on different streams need distinct
@@ -211,8 +212,8 @@ gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, int32_t P,
  * u^(mn k + m-1-i), update operands Delta_i at u^i and X_j at u^(m j). */
 gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* split, gpd_substitution subst, int32_t P,
                           const double* points_host, gpd_precision precision, gpd_plan_t* out);
-/* Uploads the plan's coefficient tables to the current device now (one cudaMalloc and one synchronous
- * copy of a few KB) instead of at the plan's first compute call; a second call does nothing.  Lets a
+/* Uploads the plan's coefficient tables to the current device now (one cudaMalloc - tables, plus the
+ * scratch area of FP32 plans - and one synchronous copy of a few KB) instead of at the plan's first compute call; a second call does nothing.  Lets a
  * caller keep allocation and synchronisation out of its timed or captured region. */
 gpd_status gpd_plan_upload(gpd_plan_t plan);
 gpd_status gpd_plan_destroy(gpd_plan_t plan);
@@ -239,6 +240,9 @@ gpd_status gpd_encode_B(gpd_plan_t plan, gpd_operand operand, const float* src_d
  *   GPD_FWD: out[p] = W~_p X~_p        ([N1/m x N0/n] [N0/n x B/d1])
  *   GPD_BWD: out[p] = Delta~^T_p W~_p  ([B/d2 x N1/m] [N1/m x N0/n])
  * outputs_dev: [P][rows][cols] in the plan's storage type.
+ * FP32 plans: the tensor-core products keep partial sums in scratch memory that belongs to the plan
+ * (allocated with its tables, see gpd_plan_upload), so two such calls on one plan must not run at the
+ * same time on different streams; calls ordered on one stream, or on one plan per stream, are fine.
  */
 gpd_status gpd_worker_gemm(gpd_plan_t plan, gpd_product which, const void* W_shares_dev,
                            const void* other_shares_dev, void* outputs_dev, void* stream);

@@ -22,6 +22,8 @@ struct GemmParams {
     const gpd_locate_result* gate;
     int max_threshold;      // largest recovery threshold the result will be decoded with (0: unknown);
                             // the FP32 tensor-core path shortens its accumulation chains for large ones
+    void* splitk_scratch;   // device scratch for the FP32 tensor-core path's split contraction (may be null)
+    int64_t splitk_bytes;
 };
 
 gpd_status gemm_generic_launch(const GemmParams& prm, int elem_size, cudaStream_t st);
@@ -30,6 +32,8 @@ bool dgemm_mma_supported(const GemmParams& prm);
 gpd_status dgemm_mma_launch(const GemmParams& prm, cudaStream_t st);
 bool sgemm_3xtf32_supported(const GemmParams& prm);
 gpd_status sgemm_3xtf32_launch(const GemmParams& prm, cudaStream_t st);
+// Scratch the FP32 tensor-core path wants for cutting `pieces` parts out of its left-over tiles (pieces <= SM count).
+int64_t sgemm_3xtf32_scratch_bytes(int64_t pieces);
 gpd_status bounded_wait_selftest_launch(long long limit_cycles, cudaStream_t st);
 int tf32_device_status_fetch_and_clear();   // synchronous read of the tensor-path status word
 

@@ -160,7 +160,13 @@ gpd_status worker_gemm_launch(gpd_plan_s* plan, gpd_product which, const void* W
     prm.max_threshold = plan->prod[which].Q;
     if (prm.N == 1) return gemv_launch(prm, plan->elem_size, st);
     if (plan->elem_size == 8 && dgemm_mma_supported(prm)) return dgemm_mma_launch(prm, st);
-    if (plan->elem_size == 4 && sgemm_3xtf32_supported(prm)) return sgemm_3xtf32_launch(prm, st);
+    if (plan->elem_size == 4 && sgemm_3xtf32_supported(prm)) {
+        const gpd_status rc = ensure_device(plan);       // the plan's allocation carries the split-contraction scratch
+        if (rc != GPD_OK) return rc;
+        prm.splitk_scratch = plan->dev.splitk;
+        prm.splitk_bytes = plan->dev.splitk_bytes;
+        return sgemm_3xtf32_launch(prm, st);
+    }
     return gemm_generic_launch(prm, plan->elem_size, st);
 }
 

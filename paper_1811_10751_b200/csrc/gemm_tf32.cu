@@ -3,8 +3,12 @@
 // shared memory by TMA, and 3xTF32 splitting so that the result keeps FP32-level accuracy:
 //     a = a_hi + a_lo (both exactly representable in TF32),   a*b ~ a_lo*b_hi + a_hi*b_lo + a_hi*b_hi.
 //
-// One CTA per SM walks a list of 128 x 128 tiles of the nodes' products (column strips of them for
-// the tiles left over after the last full round over the SMs).
+// One CTA per SM walks a list of 128 x 128 tiles of the nodes' products.  The tiles left over after
+// the last full round over the SMs are cut into pieces that fit one more, short round: products into
+// parts of their contraction, whose sums meet in a scratch buffer of the plan (a part costs its share
+// of a tile's time, where a column strip still pays for all of A: cut into four strips, 24 left-over
+// tiles of the 4096 x 4096 layer cost 0.73 of a full round, cut into six parts 0.4); the update, whose
+// output is read-modify-write, into column strips.
 //
 // Accumulation.  The tensor cores add into their FP32 accumulator with truncation, so a long chain
 // of MMAs loses up to one ulp of the running sum per step, always towards zero: over K = 2048
@@ -34,6 +38,8 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises a status word, drains its copies,
 // frees its tensor memory and returns.
 #include <cuda.h>
+
+#include <type_traits>
 
 #include "gemm_common.h"
 #include "tc_common.h"
@@ -161,10 +167,58 @@ __device__ __forceinline__ float to_tf32(float x) {
 // What the tensor core makes of a raw FP32 word in a TF32 operand: the 13 low mantissa bits dropped.
 __device__ __forceinline__ float trunc_tf32(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
-template <bool B_KMAJOR, bool UPDATE>
+// Split contraction, after a warp has written its 32 x 64 piece of one part's sum into the scratch
+// buffer: the warp takes a ticket on the piece; the warps with the same index in the other parts' CTAs
+// do the same.  Whoever draws the last ticket adds the parts up in the order of the parts (so the sum
+// does not depend on who came last) and stores the piece into C.  Kept out of line: it runs once per
+// left-over tile and must not cost the main loop registers.
+__device__ __noinline__ void splitk_finish(const float* kscratch, unsigned int* kcount, int left, int ksplit, int ew,
+                                           float* Cg, int64_t M, int64_t N, int m0, int n0) {
+    const int lane = threadIdx.x & 31;
+    const int q = (threadIdx.x >> 5) & 3, ch = (ew >> 2) * (BN / 2);
+    const int col4 = (lane & 3) * 4, rsub = lane >> 2;
+    __threadfence();
+    __syncwarp();
+    unsigned int ticket = 0;
+    if (lane == 0) ticket = atomicAdd(&kcount[left * kEpiWarpsD + ew], 1u);
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    if (ticket != (unsigned int)(ksplit - 1)) return;            // another part will finish this piece
+    __threadfence();
+    const float* parts = kscratch + (size_t)left * ksplit * (size_t)(BM * BN);
+    const bool vec_c = (N % 4 == 0);
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN / 2; c0 += EPI_COLS_D) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = q * 32 + 8 * i + rsub, col = ch + c0 + col4;
+            float4 sum = __ldcg(reinterpret_cast<const float4*>(parts + (size_t)row * BN + col));
+            for (int pp = 1; pp < ksplit; ++pp) {
+                const float4 v = __ldcg(reinterpret_cast<const float4*>(parts + (size_t)pp * (BM * BN) + (size_t)row * BN + col));
+                sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+            }
+            const int64_t grow = (int64_t)m0 + row, gcol = (int64_t)n0 + col;
+            if (grow < M) {
+                float* dst = Cg + grow * N + gcol;
+                if (vec_c && gcol + 4 <= N) {
+                    *reinterpret_cast<float4*>(dst) = sum;
+                } else {
+                    if (gcol < N) dst[0] = sum.x;
+                    if (gcol + 1 < N) dst[1] = sum.y;
+                    if (gcol + 2 < N) dst[2] = sum.z;
+                    if (gcol + 3 < N) dst[3] = sum.w;
+                }
+            }
+        }
+    }
+}
+
+// KSPLIT: the instantiation that cuts left-over tiles along the contraction (products only; launched
+// only when there is something to cut, so that the plain walk over whole tiles keeps its registers).
+template <bool B_KMAJOR, bool UPDATE, bool KSPLIT>
 __global__ void __launch_bounds__(kThreadsOf<UPDATE>, 1)
 sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmParams prm,
-                    int tiles_m, int tiles_n, int full_tiles, int split, int n_virtual, int group_kb) {
+                    int tiles_m, int tiles_n, int full_tiles, int split, int ksplit, int n_virtual, int group_kb,
+                    float* kscratch, unsigned int* kcount) {
     if (UPDATE && prm.gate && prm.gate->outcome == GPD_DECODE_FAILURE) return;
     constexpr bool EPI_DRAINS = !UPDATE;             // the epilogue warps (not the splitting warps) add the groups up
     extern __shared__ uint8_t smem_raw[];
@@ -183,8 +237,35 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     constexpr int kIssuer2Warp = kThreadsOf<UPDATE> / 32 - 1;   // the last warp: second MMA issuer
     const int num_kb = (int)((prm.K + BK - 1) / BK);
     // Virtual tile list: whole 128 x 128 tiles first; the tiles left over after the last full round
-    // over the SMs follow as `split` column strips each (128 x 32 strips when split = 4), so that
-    // the last, partly filled round is short.  CTA b takes virtual tiles b, b + grid, ...
+    // over the SMs follow in pieces, so that the last, partly filled round is short.  Products
+    // (ksplit > 1): `ksplit` parts of the contraction each - a part costs its share of a tile's time;
+    // the parts' sums meet in a scratch buffer and the last part to arrive adds them up in the order
+    // of the parts.  Update (split > 1): `split` column strips each (128 x 32 strips when split = 4;
+    // a strip still pays for all of A, so the gain is smaller).  CTA b takes virtual tiles b, b + grid, ...
+    // kb0, nkb: the piece's k-blocks; part: its index among the tile's parts; left: index of the
+    // left-over tile (-1 for a whole tile or a strip).
+    auto decode_k = [&](int vt, int& p, int& m0, int& n0, int& bn, int& kb0, int& nkb, int& part, int& left) {
+        int tile = vt, sub = 0;
+        bn = BN; kb0 = 0; nkb = num_kb; part = 0; left = -1;
+        if (vt >= full_tiles) {
+            const int piece = vt - full_tiles;
+            if (KSPLIT) {
+                left = piece / ksplit;
+                part = piece - left * ksplit;
+                tile = full_tiles + left;
+                kb0 = (int)((long long)part * num_kb / ksplit);
+                nkb = (int)((long long)(part + 1) * num_kb / ksplit) - kb0;
+            } else {
+                tile = full_tiles + piece / split;
+                sub = piece % split;
+                bn = BN / split;
+            }
+        }
+        const int tn = tile % tiles_n, tm = (tile / tiles_n) % tiles_m;
+        p = tile / (tiles_n * tiles_m);
+        m0 = tm * BM;
+        n0 = tn * BN + sub * bn;
+    };
     auto decode = [&](int vt, int& p, int& m0, int& n0, int& bn) {
         int tile = vt, sub = 0;
         bn = BN;
@@ -239,19 +320,21 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             int it = 0;                          // k-blocks issued so far, over all tiles
             bool ok = true;
             for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
-                int p, m0, n0, bn;
-                decode(vt, p, m0, n0, bn);
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                int p, m0, n0, bn, kb0 = 0, nkb = num_kb, part = 0, left = -1;
+                if constexpr (KSPLIT) decode_k(vt, p, m0, n0, bn, kb0, nkb, part, left);
+                else decode(vt, p, m0, n0, bn);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1;
+                    const int k0 = (kb0 + kb) * BK;
                     if (!mbar_wait(&empty_bar[s], ph ^ 1, abort_p)) { ok = false; break; }
                     mbar_expect_tx(&full_bar[s], A_TILE_BYTES + bn * BK * 4);
-                    tma_load_3d(A_raw(s), &tmA, kb * BK, m0, p, &full_bar[s]);
+                    tma_load_3d(A_raw(s), &tmA, k0, m0, p, &full_bar[s]);
                     for (int c = 0; c < bn / 32; ++c) {      // B arrives in boxes of 32 columns (or 32 rows of X^_p)
                         if (B_KMAJOR)
-                            tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, kb * BK, n0 + 32 * c, p, &full_bar[s]);
+                            tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, k0, n0 + 32 * c, p, &full_bar[s]);
                         else
-                            tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, n0 + 32 * c, kb * BK, p, &full_bar[s]);
+                            tma_load_3d(B_hi(s) + c * (BK * 128), &tmB, n0 + 32 * c, k0, p, &full_bar[s]);
                     }
                 }
             }
@@ -277,14 +360,15 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             int it = 0, gi = 0;                   // k-blocks / accumulation groups so far, over all tiles (both issuers count alike)
             bool ok = true;
             for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
-                int p, m0, n0, bn;
-                decode(vt, p, m0, n0, bn);
+                int p, m0, n0, bn, kb0 = 0, nkb = num_kb, part = 0, left = -1;
+                if constexpr (KSPLIT) decode_k(vt, p, m0, n0, bn, kb0, nkb, part, left);
+                else decode(vt, p, m0, n0, bn);
                 const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((B_KMAJOR ? 0u : 1u) << 16) |
                                        ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
                 int kg = 0;                      // position of the k-block inside its accumulation group
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int buf = gi & 1;
-                    const bool group_end = kg == group_kb - 1 || kb == num_kb - 1;
+                    const bool group_end = kg == group_kb - 1 || kb == nkb - 1;
                     if ((it & 1) == me) {
                         if (kg == 0) {
                             // the group before last used this accumulator: it must have been read back
@@ -399,10 +483,11 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int it = 0;
         bool ok = true;
         for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
-            int p, m0, n0, bn;
-            decode(vt, p, m0, n0, bn);
+            int p, m0, n0, bn, kb0 = 0, nkb = num_kb, part = 0, left = -1;
+            if constexpr (KSPLIT) decode_k(vt, p, m0, n0, bn, kb0, nkb, part, left);
+            else decode(vt, p, m0, n0, bn);
             const int b_float4 = bn * BK / 4;        // 16-byte units of one B tile
-            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % STAGES;
                 const uint32_t ph = (it / STAGES) & 1;
                 const bool landed = mbar_wait(&full_bar[s], ph, abort_p);
@@ -460,16 +545,17 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int ew = warp - (2 + kConvWarps);      // 0..7
             const int q = warp & 3;                      // this warp may touch TMEM lanes 32q .. 32q+31
             const int ch = (ew >> 2) * (BN / 2);         // first of this warp's 64 columns of the tile
-            const float shrink = (float)prm.shrink, eta = (float)prm.eta;
-            const bool vec = (prm.N % 4 == 0);
-            const int n_groups = (num_kb + group_kb - 1) / group_kb;
+            [[maybe_unused]] const float shrink = (float)prm.shrink, eta = (float)prm.eta;
+            [[maybe_unused]] const bool vec = (prm.N % 4 == 0);
             float* st = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES) + ew * (32 * EPI_PITCH_D);
             const int col4 = (lane & 3) * 4, rsub = lane >> 2;    // this lane's part of a staged 32 x 16 chunk
             int gi = 0;
             bool ok = true;
             for (int vt = blockIdx.x; vt < n_virtual && ok; vt += gridDim.x) {
-                int p, m0, n0, bn;
-                decode(vt, p, m0, n0, bn);
+                int p, m0, n0, bn, kb0 = 0, nkb = num_kb, part = 0, left = -1;
+                if constexpr (KSPLIT) decode_k(vt, p, m0, n0, bn, kb0, nkb, part, left);
+                else decode(vt, p, m0, n0, bn);
+                const int n_groups = (nkb + group_kb - 1) / group_kb;
                 float acc[BN / 2];                       // this thread's row, this warp's columns
                 for (int g = 0; g < n_groups; ++g, ++gi) {
                     const int buf = gi & 1;
@@ -500,57 +586,108 @@ sgemm_3xtf32_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 }
                 if (!ok) break;
-                const int64_t gm = (int64_t)m0 + q * 32 + lane;
-                float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
+                if constexpr (!KSPLIT) {
+                    const int64_t gm = (int64_t)m0 + q * 32 + lane;
+                    float* C = reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
     #pragma unroll
-                for (int c0 = 0; c0 < BN / 2; c0 += EPI_COLS_D) {
-                    if (ch + c0 >= bn) break;
-                    const int64_t gc = (int64_t)n0 + ch + c0;           // first global column of the chunk
-                    const bool whole = vec && gc + EPI_COLS_D <= prm.N;
-                    if (whole) {
-                        // A thread holds the columns of one row; written as they are, a store would touch 32
-                        // rows with 16 bytes each.  A 32 x 16 chunk goes through shared memory instead and
-                        // leaves as 64-byte row segments (four lanes per row, eight rows per store).  The
-                        // update asks for the stored share before it stages the chunk.
-                        float4 old[4];
-                        if (UPDATE) {
+                    for (int c0 = 0; c0 < BN / 2; c0 += EPI_COLS_D) {
+                        if (ch + c0 >= bn) break;
+                        const int64_t gc = (int64_t)n0 + ch + c0;           // first global column of the chunk
+                        const bool whole = vec && gc + EPI_COLS_D <= prm.N;
+                        if (whole) {
+                            // A thread holds the columns of one row; written as they are, a store would touch 32
+                            // rows with 16 bytes each.  A 32 x 16 chunk goes through shared memory instead and
+                            // leaves as 64-byte row segments (four lanes per row, eight rows per store).  The
+                            // update asks for the stored share before it stages the chunk.
+                            float4 old[4];
+                            if (UPDATE) {
+    #pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const int64_t grow = (int64_t)m0 + q * 32 + 8 * i + rsub;
+                                    old[i] = grow < prm.M ? *reinterpret_cast<const float4*>(C + grow * prm.N + gc + col4)
+                                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+                                }
+                            }
+    #pragma unroll
+                            for (int j = 0; j < EPI_COLS_D; j += 4)
+                                *reinterpret_cast<float4*>(st + lane * EPI_PITCH_D + j) =
+                                    make_float4(acc[c0 + j], acc[c0 + j + 1], acc[c0 + j + 2], acc[c0 + j + 3]);
+                            __syncwarp();
     #pragma unroll
                             for (int i = 0; i < 4; ++i) {
-                                const int64_t grow = (int64_t)m0 + q * 32 + 8 * i + rsub;
-                                old[i] = grow < prm.M ? *reinterpret_cast<const float4*>(C + grow * prm.N + gc + col4)
-                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
-                            }
-                        }
-    #pragma unroll
-                        for (int j = 0; j < EPI_COLS_D; j += 4)
-                            *reinterpret_cast<float4*>(st + lane * EPI_PITCH_D + j) =
-                                make_float4(acc[c0 + j], acc[c0 + j + 1], acc[c0 + j + 2], acc[c0 + j + 3]);
-                        __syncwarp();
-    #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int row = 8 * i + rsub;
-                            const int64_t grow = (int64_t)m0 + q * 32 + row;
-                            float4 v = *reinterpret_cast<const float4*>(st + row * EPI_PITCH_D + col4);
-                            if (grow < prm.M) {
-                                if (UPDATE) {
-                                    const float4 o = old[i];
-                                    v.x = shrink * o.x + eta * v.x; v.y = shrink * o.y + eta * v.y;
-                                    v.z = shrink * o.z + eta * v.z; v.w = shrink * o.w + eta * v.w;
+                                const int row = 8 * i + rsub;
+                                const int64_t grow = (int64_t)m0 + q * 32 + row;
+                                float4 v = *reinterpret_cast<const float4*>(st + row * EPI_PITCH_D + col4);
+                                if (grow < prm.M) {
+                                    if (UPDATE) {
+                                        const float4 o = old[i];
+                                        v.x = shrink * o.x + eta * v.x; v.y = shrink * o.y + eta * v.y;
+                                        v.z = shrink * o.z + eta * v.z; v.w = shrink * o.w + eta * v.w;
+                                    }
+                                    *reinterpret_cast<float4*>(C + grow * prm.N + gc + col4) = v;
                                 }
-                                *reinterpret_cast<float4*>(C + grow * prm.N + gc + col4) = v;
                             }
-                        }
-                        __syncwarp();                        // the next chunk reuses the staging rows
-                    } else if (gm < prm.M) {
-                        float* crow = C + gm * prm.N + gc;
+                            __syncwarp();                        // the next chunk reuses the staging rows
+                        } else if (gm < prm.M) {
+                            float* crow = C + gm * prm.N + gc;
     #pragma unroll
-                        for (int j = 0; j < EPI_COLS_D; ++j) {
-                            if (gc + j < prm.N) {
-                                float v = acc[c0 + j];
-                                if (UPDATE) v = shrink * crow[j] + eta * v;
-                                crow[j] = v;
+                            for (int j = 0; j < EPI_COLS_D; ++j) {
+                                if (gc + j < prm.N) {
+                                    float v = acc[c0 + j];
+                                    if (UPDATE) v = shrink * crow[j] + eta * v;
+                                    crow[j] = v;
+                                }
                             }
                         }
+                    }
+                } else {
+                    // Where the tile goes: into C, or - one part of a left-over tile's contraction - into that
+                    // part's 128 x 128 slot of the scratch buffer (same code; base, pitch and limits are
+                    // compile-time constants there).
+                    auto store_tile = [&](auto part_tag) {
+                        constexpr bool PART = decltype(part_tag)::value;
+                        float* C = PART ? kscratch + ((size_t)left * ksplit + part) * (size_t)(BM * BN)
+                                        : reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N;
+                        const int64_t ldc = PART ? BN : prm.N, row_lim = PART ? BM : prm.M, col_lim = PART ? BN : prm.N;
+                        const int64_t row0 = PART ? 0 : m0, col0 = PART ? 0 : n0;
+                        const bool vec = (ldc % 4 == 0);
+                        const int64_t gm = row0 + q * 32 + lane;
+    #pragma unroll
+                        for (int c0 = 0; c0 < BN / 2; c0 += EPI_COLS_D) {
+                            if (ch + c0 >= bn) break;
+                            const int64_t gc = col0 + ch + c0;                  // first column of the chunk
+                            const bool whole = vec && gc + EPI_COLS_D <= col_lim;
+                            if (whole) {
+                                // A thread holds the columns of one row; written as they are, a store would touch
+                                // 32 rows with 16 bytes each.  A 32 x 16 chunk goes through shared memory instead
+                                // and leaves as 64-byte row segments (four lanes per row, eight rows per store).
+    #pragma unroll
+                                for (int j = 0; j < EPI_COLS_D; j += 4)
+                                    *reinterpret_cast<float4*>(st + lane * EPI_PITCH_D + j) =
+                                        make_float4(acc[c0 + j], acc[c0 + j + 1], acc[c0 + j + 2], acc[c0 + j + 3]);
+                                __syncwarp();
+    #pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const int row = 8 * i + rsub;
+                                    const int64_t grow = row0 + q * 32 + row;
+                                    const float4 v = *reinterpret_cast<const float4*>(st + row * EPI_PITCH_D + col4);
+                                    if (grow < row_lim) *reinterpret_cast<float4*>(C + grow * ldc + gc + col4) = v;
+                                }
+                                __syncwarp();                        // the next chunk reuses the staging rows
+                            } else if (gm < row_lim) {
+                                float* crow = C + gm * ldc + gc;
+    #pragma unroll
+                                for (int j = 0; j < EPI_COLS_D; ++j)
+                                    if (gc + j < col_lim) crow[j] = acc[c0 + j];
+                            }
+                        }
+                    };
+                    if (left < 0) {
+                        store_tile(std::false_type{});
+                    } else {
+                        store_tile(std::true_type{});
+                        splitk_finish(kscratch, kcount, left, ksplit, ew, reinterpret_cast<float*>(prm.C) + (int64_t)p * prm.M * prm.N,
+                                      prm.M, prm.N, m0, n0);
                     }
                 }
             }
@@ -660,6 +797,9 @@ bool make_map(CUtensorMap* map, const void* base, int64_t batch, int64_t rows, i
     return tc::make_map_3d(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, batch, rows, cols, box_cols, box_rows, swizzle);
 }
 
+// Scratch of the split contraction: counters of `rem` left-over tiles, then `pieces` part sums of one tile each.
+constexpr int64_t kSplitKHeaderBytes(int64_t rem) { return (rem * kEpiWarpsD * (int64_t)sizeof(unsigned int) + 255) / 256 * 256; }
+
 template <bool B_KMAJOR, bool UPDATE>
 gpd_status launch(const GemmParams& prm, cudaStream_t st) {
     CUtensorMap tmA, tmB;
@@ -667,28 +807,57 @@ gpd_status launch(const GemmParams& prm, cudaStream_t st) {
     const bool okB = B_KMAJOR ? make_map(&tmB, prm.B, prm.P, prm.N, prm.K, BK, 32, CU_TENSOR_MAP_SWIZZLE_128B)
                               : make_map(&tmB, prm.B, prm.P, prm.K, prm.N, 32, BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
     if (!okB) return GPD_ERR_CUDA;
-    if (cudaFuncSetAttribute(sgemm_3xtf32_kernel<B_KMAJOR, UPDATE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(sgemm_3xtf32_kernel<B_KMAJOR, UPDATE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(sgemm_3xtf32_kernel<B_KMAJOR, UPDATE, !UPDATE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              SMEM_BYTES) != cudaSuccess)
         return GPD_ERR_CUDA;
     const int tiles_n = (int)((prm.N + BN - 1) / BN), tiles_m = (int)((prm.M + BM - 1) / BM);
     const int64_t tiles = (int64_t)tiles_n * tiles_m * prm.P;
-    // One CTA per SM at a time.  After the last full round, `rem` tiles are left: cutting them into
-    // 2 or 4 strips shortens that last round if the strips still fit in one round.
+    // One CTA per SM at a time.  After the last full round, `rem` tiles are left.  Products: each is cut
+    // into as many parts of its contraction as still fit in one round (at least four k-blocks per part),
+    // if the caller gave a scratch buffer for the parts' sums.  Otherwise (and for the update, whose
+    // output is read-modify-write): 2 or 4 column strips each, if the strips still fit in one round.
     const int sms = sm_count();
     const int rem = (int)(tiles % sms);
-    int split = 1;
-    if (rem > 0 && rem * 4 <= sms) split = 4;
-    else if (rem > 0 && rem * 2 <= sms) split = 2;
-    const int full_tiles = (int)(tiles - (split > 1 ? rem : 0));
-    const int64_t n_virtual = full_tiles + (int64_t)(split > 1 ? rem : 0) * split;
+    const int num_kb = (int)((prm.K + BK - 1) / BK);
+    int split = 1, ksplit = 1;
+    if (!UPDATE && rem > 0 && prm.splitk_scratch) {
+        ksplit = std::min(std::min(sms / rem, num_kb / 4), 32);
+        while (ksplit > 1 && sgemm_3xtf32_scratch_bytes(rem * ksplit) > prm.splitk_bytes) --ksplit;
+        if (ksplit < 2) ksplit = 1;
+    }
+    if (ksplit == 1) {
+        if (rem > 0 && rem * 4 <= sms) split = 4;
+        else if (rem > 0 && rem * 2 <= sms) split = 2;
+    }
+    const int pieces = ksplit > 1 ? ksplit : split;
+    const int full_tiles = (int)(tiles - (pieces > 1 ? rem : 0));
+    const int64_t n_virtual = full_tiles + (int64_t)(pieces > 1 ? rem : 0) * pieces;
     const unsigned grid = (unsigned)std::min<int64_t>(n_virtual, sms);   // persistent: one CTA per SM walks the list
     const int group_kb = UPDATE ? kGroupKbUpdate : (prm.max_threshold >= 7 ? kGroupKbProductLarge : kGroupKbProduct);
-    sgemm_3xtf32_kernel<B_KMAJOR, UPDATE><<<grid, kThreadsOf<UPDATE>, SMEM_BYTES, st>>>(tmA, tmB, prm, tiles_m, tiles_n, full_tiles,
-                                                                              split, (int)n_virtual, group_kb);
+    float* kscratch = nullptr;
+    unsigned int* kcount = nullptr;
+    if (ksplit > 1) {
+        // counters first (one per left-over tile and epilogue warp), the parts' sums 256 bytes further on
+        kcount = reinterpret_cast<unsigned int*>(prm.splitk_scratch);
+        kscratch = reinterpret_cast<float*>(reinterpret_cast<char*>(prm.splitk_scratch) + kSplitKHeaderBytes(rem));
+        if (cudaMemsetAsync(kcount, 0, sizeof(unsigned int) * rem * kEpiWarpsD, st) != cudaSuccess) return GPD_ERR_CUDA;
+    }
+    if (ksplit > 1)
+        sgemm_3xtf32_kernel<B_KMAJOR, UPDATE, !UPDATE><<<grid, kThreadsOf<UPDATE>, SMEM_BYTES, st>>>(
+            tmA, tmB, prm, tiles_m, tiles_n, full_tiles, split, ksplit, (int)n_virtual, group_kb, kscratch, kcount);
+    else
+        sgemm_3xtf32_kernel<B_KMAJOR, UPDATE, false><<<grid, kThreadsOf<UPDATE>, SMEM_BYTES, st>>>(
+            tmA, tmB, prm, tiles_m, tiles_n, full_tiles, split, ksplit, (int)n_virtual, group_kb, kscratch, kcount);
     return launch_ok();
 }
 
 }  // namespace
+
+int64_t sgemm_3xtf32_scratch_bytes(int64_t pieces) {
+    return kSplitKHeaderBytes(pieces) + pieces * (int64_t)(BM * BN * sizeof(float));
+}
 
 bool sgemm_3xtf32_supported(const GemmParams& prm) {
     // TMA: 16-byte aligned bases and row pitches; big enough that a 128 x 128 tile is not mostly padding

@@ -51,6 +51,10 @@ struct DeviceTables {
     int64_t n_doubles = 0;
     int64_t off_points = 0;
     int64_t off_coefW = 0, off_coefX = 0, off_coefDT = 0, off_coefDup = 0, off_coefXup = 0;
+    // FP32 plans: scratch behind the tables (same allocation) in which the tensor-core products add up the
+    // parts of a split contraction; one product launch of a plan uses it at a time
+    void* splitk = nullptr;
+    int64_t splitk_bytes = 0;
 };
 
 }  // namespace gpd

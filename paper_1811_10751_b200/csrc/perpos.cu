@@ -404,28 +404,9 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
                     for (int i = 0; i <= TT; ++i) a[j][i] = 0.0;
                 }
                 // Hankel system of the locator: sum_i l_i S_{j+i} = -S_{j+nu}, j = 0 .. nu-1
-                if constexpr (TT <= 4) {                              // S_{j+i} without a dynamic index
-#pragma unroll
-                    for (int j = 0; j < TT; ++j)
-#pragma unroll
-                        for (int i = 0; i < TT; ++i)
-                            if (j < nu && i < nu) {
-#pragma unroll
-                                for (int q = 0; q < RT; ++q)
-                                    if (q == j + i) a[j][i] = S[q];
-                            }
-#pragma unroll
-                    for (int j = 0; j < TT; ++j)
-                        if (j < nu) {
-#pragma unroll
-                            for (int q = 0; q < RT; ++q)
-                                if (q == j + nu) a[j][TT] = -S[q];
-                        }
-                } else {
-                    for (int j = 0; j < nu; ++j) {
-                        for (int i = 0; i < nu; ++i) a[j][i] = S[j + i];
-                        a[j][TT] = -S[j + nu];
-                    }
+                for (int j = 0; j < nu; ++j) {
+                    for (int i = 0; i < nu; ++i) a[j][i] = S[j + i];
+                    a[j][TT] = -S[j + nu];
                 }
                 if (!solve_small<TT>(a, nu, lam)) continue;
                 // the nu points where the locator is smallest, smallest first (of equal values the lower

@@ -5,6 +5,7 @@
 #include <new>
 
 #include "gpd_internal.h"
+#include "gemm_common.h"
 #include "slice_common.h"
 
 namespace gpd {
@@ -127,7 +128,11 @@ gpd_status ensure_device(gpd_plan_s* plan) {
     for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT}) plan->prod[w].off_Hg = push(plan->prod[w].Hg);
     d.n_doubles = (int64_t)host.size();
     if (cudaGetDevice(&plan->device) != cudaSuccess) return GPD_ERR_CUDA;
-    if (cudaMalloc(&d.base, sizeof(double) * host.size()) != cudaSuccess) return GPD_ERR_CUDA;
+    const int64_t table_bytes = (int64_t)sizeof(double) * (int64_t)host.size();      // a multiple of 256
+    const int64_t scratch_bytes = (plan->elem_size == 4 && !plan->sliced) ? sgemm_3xtf32_scratch_bytes(sm_count()) : 0;
+    if (cudaMalloc(&d.base, (size_t)(table_bytes + scratch_bytes)) != cudaSuccess) return GPD_ERR_CUDA;
+    d.splitk = scratch_bytes ? reinterpret_cast<char*>(d.base) + table_bytes : nullptr;
+    d.splitk_bytes = scratch_bytes;
     if (cudaMemcpy(d.base, host.data(), sizeof(double) * host.size(), cudaMemcpyHostToDevice) !=
         cudaSuccess) {
         cudaFree(d.base);

@@ -77,7 +77,10 @@ def test_encode_matches_oracle(N1, N0, B, m, n, d1, d2, P, prec):
     (66, 50, 14, 2, 2, 2, 2, 16, g.GPD_PREC_FP64),           # odd sizes -> CUDA-core kernel
     (512, 512, 256, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),        # tcgen05 3xTF32 tiles, exact multiples
     (400, 272, 200, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),        # tcgen05 path with ragged M, N and K
-    (2048, 1024, 256, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),      # many k-blocks: the stage ring wraps
+    (2048, 1024, 256, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),      # many k-blocks: the stage ring wraps; 160 tiles on 148
+                                                             # SMs: the 12 left over are cut into four parts of K
+    (600, 1024, 200, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),       # 60 ragged tiles (300 x 200 per node), each cut into two
+                                                             # parts of K = 512 whose sums meet in the plan's scratch
     (512, 768, 1000, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),       # mini-batch 1000: the update's contraction spans four
                                                              # accumulation groups (the last one short)
     (10, 512, 64, 2, 2, 1, 1, 10, g.GPD_PREC_FP32),          # 5-row blocks
