@@ -230,6 +230,8 @@ __global__ void __launch_bounds__(kThreads, RT <= 24 ? 2 : 1) syndrome_gram_mma_
     const int n_chunks = (n_ksteps + UK - 1) / UK;
     const int64_t n_blocks = (prm.L + 31) / 32;
     const int64_t stride = (int64_t)gridDim.x * kWarps;
+    double za[UK][4], zb[UK][4];                         // two chunks of loads: one being multiplied, one in flight
+    bool have_first = false;                             // za already holds (or awaits) chunk 0 of the current block
     for (int64_t blk = (int64_t)blockIdx.x * kWarps + warp; blk < n_blocks; blk += stride) {
         const int64_t base = blk * 32;
         bool any_active = false;
@@ -246,14 +248,14 @@ __global__ void __launch_bounds__(kThreads, RT <= 24 ? 2 : 1) syndrome_gram_mma_
             for (int mt = 0; mt < NT; ++mt)
 #pragma unroll
                 for (int t = 0; t < 4; ++t) d[mt][t][0] = d[mt][t][1] = 0.0;
-            auto load_chunk = [&](int c, double (&z)[UK][4]) {
+            auto load_chunk = [&](int64_t b0, int c, double (&z)[UK][4]) {
 #pragma unroll
                 for (int u = 0; u < UK; ++u) {
                     const int ks = c * UK + u, node = 4 * ks + kq;
-                    const T* zp = Z + (int64_t)node * prm.L + base + nq;
+                    const T* zp = Z + (int64_t)node * prm.L + b0 + nq;
 #pragma unroll
                     for (int t = 0; t < 4; ++t)
-                        z[u][t] = (ks < n_ksteps && node < prm.P && base + 8 * t + nq < prm.L) ? (double)__ldcs(zp + 8 * t) : 0.0;
+                        z[u][t] = (ks < n_ksteps && node < prm.P && b0 + 8 * t + nq < prm.L) ? (double)__ldcs(zp + 8 * t) : 0.0;
                 }
             };
             auto use_chunk = [&](int c, const double (&z)[UK][4]) {
@@ -273,12 +275,19 @@ __global__ void __launch_bounds__(kThreads, RT <= 24 ? 2 : 1) syndrome_gram_mma_
                     }
                 }
             };
-            double za[UK][4], zb[UK][4];                 // two chunks: one being multiplied, one in flight
-            load_chunk(0, za);
+            if (!have_first) load_chunk(base, 0, za);
+            have_first = false;
             for (int c = 0; c < n_chunks; c += 2) {
-                if (c + 1 < n_chunks) load_chunk(c + 1, zb);
+                if (c + 1 < n_chunks) load_chunk(base, c + 1, zb);
                 use_chunk(c, za);
-                if (c + 2 < n_chunks) load_chunk(c + 2, za);
+                if (c + 2 < n_chunks) {
+                    load_chunk(base, c + 2, za);
+                } else if (blk + stride < n_blocks) {
+                    // za is free: the first chunk of this warp's next block travels while the rest of
+                    // this block is multiplied, tested and added to the Gram matrix
+                    load_chunk((blk + stride) * 32, 0, za);
+                    have_first = true;
+                }
                 if (c + 1 < n_chunks) use_chunk(c + 1, zb);
             }
             // ||z||^2 of position 8 t + nq: sum over the four lanes of the position
