@@ -921,7 +921,7 @@ def relaunch_under_torchrun(args):
 
 def brief(line):
     """What the `secondary` object keeps of a secondary workload's line."""
-    keep = ("value", "unit", "ms_per_step", "dtype", "kernel_ms", "gemv_ms", "encode_W_once_ms", "encode_W_hbm_frac",
+    keep = ("value", "unit", "ms_per_step", "graph_replay_ms_per_step", "dtype", "kernel_ms", "gemv_ms", "encode_W_once_ms", "encode_W_hbm_frac",
             "correct_positions_ms", "check", "last_outcomes_fwd_bwd", "device_status", "stage_ms", "path_roofline")
     out = {"workload": line["config"]["workload"], "metric": line["metric"]}
     out.update({k: line[k] for k in keep if k in line})
