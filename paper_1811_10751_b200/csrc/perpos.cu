@@ -290,31 +290,42 @@ __device__ __forceinline__ bool try_support(const double (&S)[RT], const double 
 
 // RT: parity checks rounded up (8 or 32); TT: errors per codeword rounded up (4 or 16).  The
 // right-hand side of a system sits in column TT of its rows.
+// Small codes (TT <= 4): a block takes 32 positions at a time and has one warp per support size; warp
+// nu - 1 tries supports of nu nodes for all 32 (the sizes are tried side by side instead of one after
+// the other: a position's repair is a serial chain, and the chain for the largest size is a little over
+// half of the sum), and warp 0 then takes, for every position, the smallest size that passed - the
+// decision of the sequential search.  Larger codes: 64 positions per block, sizes in turn.
 template <typename T, int RT, int TT>
-__global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
+__global__ void __launch_bounds__(128) position_fix_kernel(PosParams prm) {
+    constexpr bool kSizesSideBySide = TT <= 4 && RT == 8;
+    constexpr int kPerBlock = kSizesSideBySide ? 32 : 64;     // positions a block takes per trip
+    __shared__ int s_nodes[kSizesSideBySide ? 4 : 1][32][4];
+    __shared__ double s_err[kSizesSideBySide ? 4 : 1][32][4];
+    __shared__ unsigned char s_ok[kSizesSideBySide ? 4 : 1][32];
+    const int nthr = blockDim.x;
     extern __shared__ double sm[];        // H [R][P], Hg [R][P], points [P], small codes: H^T H [P][P]
     double* sH = sm;
     double* sHg = sm + prm.R * prm.P;
     double* sPts = sHg + prm.R * prm.P;
     double* sT = sPts + prm.P;            // [R][R] = Hg H^T: S = T r, since the rows of Hg lie in the row space of H
     double* sG = sT + prm.R * prm.R;
-    if ((unsigned long long)blockIdx.x * 64 >= prm.counters[0]) {          // nothing listed for this block
+    if ((unsigned long long)blockIdx.x * kPerBlock >= prm.counters[0]) {   // nothing listed for this block
         finish_by_last_block(prm);
         return;
     }
-    for (int i = threadIdx.x; i < prm.R * prm.P; i += 64) { sH[i] = prm.H[i]; sHg[i] = prm.Hg[i]; }
-    for (int i = threadIdx.x; i < prm.P; i += 64) sPts[i] = prm.points[i];
+    for (int i = threadIdx.x; i < prm.R * prm.P; i += nthr) { sH[i] = prm.H[i]; sHg[i] = prm.Hg[i]; }
+    for (int i = threadIdx.x; i < prm.P; i += nthr) sPts[i] = prm.points[i];
     __syncthreads();
     constexpr int UF = TT <= 4 ? 32 : 1;     // small codes: loops fully unrolled, everything in registers
     constexpr bool kGramTable = TT <= 4;     // normal equations read their entries from H^T H
-    for (int i = threadIdx.x; i < prm.R * prm.R; i += 64) {
+    for (int i = threadIdx.x; i < prm.R * prm.R; i += nthr) {
         const int a = i / prm.R, b = i - a * prm.R;
         double s2 = 0.0;
         for (int p = 0; p < prm.P; ++p) s2 = fma(sHg[a * prm.P + p], sH[b * prm.P + p], s2);
         sT[i] = s2;
     }
     if (kGramTable) {
-        for (int i = threadIdx.x; i < prm.P * prm.P; i += 64) {
+        for (int i = threadIdx.x; i < prm.P * prm.P; i += nthr) {
             const int a = i / prm.P, b = i - a * prm.P;
             double s2 = 0.0;
             for (int q = 0; q < prm.R; ++q) s2 = fma(sH[q * prm.P + a], sH[q * prm.P + b], s2);
@@ -326,9 +337,9 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
     const int P = prm.P, R = prm.R, t = R / 2;
     const unsigned long long listed = prm.counters[0];
     // all lanes of a warp run the same rounds (the counters are updated once per warp and round)
-    for (unsigned long long base = (unsigned long long)blockIdx.x * 64; base < listed;
-         base += (unsigned long long)gridDim.x * 64) {
-        const unsigned long long it = base + threadIdx.x;
+    for (unsigned long long base = (unsigned long long)blockIdx.x * kPerBlock; base < listed;
+         base += (unsigned long long)gridDim.x * kPerBlock) {
+        const unsigned long long it = base + (kSizesSideBySide ? (threadIdx.x & 31) : threadIdx.x);
         const bool valid = it < listed;
         const int64_t pos = valid ? prm.list[it] : 0;
         double r[RT], S[RT];
@@ -384,17 +395,34 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
         double err[TT];
 #pragma unroll UF
         for (int i = 0; i < TT; ++i) { nodes[i] = 0; err[i] = 0.0; }
-#pragma unroll 1
-        for (int nu = 1; valid && nu <= t && accepted == 0; ++nu) {
-            if constexpr (TT <= 4 && RT == 8) {       // small codes: one instantiation per support size
-                bool ok = false;
-                switch (nu) {
+        if constexpr (kSizesSideBySide) {
+            const int wv = threadIdx.x >> 5, ln = threadIdx.x & 31, nu = wv + 1;     // this warp's support size
+            bool ok = false;
+            if (valid && nu <= t) {
+                switch (nu) {                          // one instantiation per support size
                     case 1: ok = try_support<1, RT, TT>(S, r, sH, sPts, sG, P, R, limit, nodes, err); break;
                     case 2: ok = try_support<2, RT, TT>(S, r, sH, sPts, sG, P, R, limit, nodes, err); break;
                     case 3: ok = try_support<3, RT, TT>(S, r, sH, sPts, sG, P, R, limit, nodes, err); break;
                     default: ok = try_support<4, RT, TT>(S, r, sH, sPts, sG, P, R, limit, nodes, err); break;
                 }
-                if (ok) accepted = nu;
+            }
+            s_ok[wv][ln] = ok ? 1 : 0;
+#pragma unroll
+            for (int i = 0; i < TT; ++i) { s_nodes[wv][ln][i] = nodes[i]; s_err[wv][ln][i] = err[i]; }
+            __syncthreads();
+            if (wv == 0) {                             // the smallest size that passed, as the search in turn would find
+                for (int w2 = 0; w2 < t && accepted == 0; ++w2) {
+                    if (s_ok[w2][ln]) {
+                        accepted = w2 + 1;
+#pragma unroll
+                        for (int i = 0; i < TT; ++i) { nodes[i] = s_nodes[w2][ln][i]; err[i] = s_err[w2][ln][i]; }
+                    }
+                }
+            }
+        }
+#pragma unroll 1
+        for (int nu = 1; !kSizesSideBySide && valid && nu <= t && accepted == 0; ++nu) {
+            if constexpr (kSizesSideBySide) {
             } else {
                 double a[TT][TT + 1], lam[TT];
 #pragma unroll UF
@@ -518,6 +546,10 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
                 mask |= 1ULL << nodes[i];
             }
         }
+        if (kSizesSideBySide && threadIdx.x >= 32) {   // the other sizes' warps: nothing to write back or count
+            __syncthreads();                           // (pairs with the barrier at the end of warp 0's trip)
+            continue;
+        }
         const unsigned int n_fixed = __popc(__ballot_sync(0xffffffffu, valid && accepted > 0));
         const unsigned int n_lost = __popc(__ballot_sync(0xffffffffu, valid && accepted == 0));
         const unsigned int n_ent = __reduce_add_sync(0xffffffffu, (unsigned int)accepted);
@@ -533,6 +565,7 @@ __global__ void __launch_bounds__(64) position_fix_kernel(PosParams prm) {
                 atomicOr(&prm.counters[6], ((unsigned long long)m_hi << 32) | m_lo);
             }
         }
+        if (kSizesSideBySide) __syncthreads();         // the result slots are written again in the next trip
     }
     finish_by_last_block(prm);
 }
@@ -596,9 +629,16 @@ gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* o
                  : position_scan_kernel<double, 32><<<grid1, 256, smem1, st>>>(prm);
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
         const size_t smem2 = sizeof(double) * (2 * pi.R * plan->P + plan->P + pi.R * pi.R + (pi.R <= 8 ? plan->P * plan->P : 0));
-        const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + 63) / 64, sm_count() * 8));
-        if (pi.R <= 8) f32 ? position_fix_kernel<float, 8, 4><<<grid2, 64, smem2, st>>>(prm)
-                           : position_fix_kernel<double, 8, 4><<<grid2, 64, smem2, st>>>(prm);
+        const int per_block = pi.R <= 8 ? 32 : 64;                       // positions a block takes per trip
+        const int grid2 = (int)std::max<int64_t>(1, std::min<int64_t>((L + per_block - 1) / per_block, sm_count() * 8));
+        const int threads_small = 32 * std::max(1, pi.R / 2);            // one warp per support size
+        if (pi.R <= 8 && smem2 > 40 * 1024) {                            // beside 6 KB of static shared memory: past the default limit
+            const cudaError_t e = f32 ? cudaFuncSetAttribute(position_fix_kernel<float, 8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)
+                                      : cudaFuncSetAttribute(position_fix_kernel<double, 8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+            if (e != cudaSuccess) return GPD_ERR_CUDA;
+        }
+        if (pi.R <= 8) f32 ? position_fix_kernel<float, 8, 4><<<grid2, threads_small, smem2, st>>>(prm)
+                           : position_fix_kernel<double, 8, 4><<<grid2, threads_small, smem2, st>>>(prm);
         else f32 ? position_fix_kernel<float, 32, 16><<<grid2, 64, smem2, st>>>(prm)
                  : position_fix_kernel<double, 32, 16><<<grid2, 64, smem2, st>>>(prm);
         return launch_ok();                          // the last block of the repair kernel writes the result
