@@ -42,7 +42,8 @@ __device__ __forceinline__ void dmma_m8n8k4(double& d0, double& d1, double a, do
                  : "d"(a), "d"(b));
 }
 
-// Syndrome s = H z and squared norm of one codeword: P loads at stride L, issued in equal groups of up to nine.
+// Syndrome s = H z and squared norm of one codeword: P loads at stride L, issued in equal groups of up to ten
+// (ten nodes, the MLP layers' code, then cost one trip to memory instead of two).
 // CHECKED = false is the plain form: no per-value tests; a non-finite value, or one of magnitude
 // >= kHuge (its square would leave the FP64 range and turn the zero test into inf > inf), shows up
 // as a norm >= kHugeSquared and the caller repeats the codeword with CHECKED = true, which zeroes
@@ -51,7 +52,7 @@ template <typename T, int RT, bool CHECKED>
 __device__ __forceinline__ void codeword_syndrome(const T* zp, int64_t L, int P, const double* sH,
                                                   unsigned long long erased, double (&s)[RT], double& nz,
                                                   unsigned long long& bad) {
-    constexpr int U = RT <= 8 ? 9 : 4;                   // most loads issued together (fewer where the syndrome fills the registers)
+    constexpr int U = RT <= 8 ? 10 : 4;                  // most loads issued together (fewer where the syndrome fills the registers)
 #pragma unroll
     for (int r = 0; r < RT; ++r) s[r] = 0.0;
     nz = 0.0;

@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(256, RT <= 8 ? 4 : 1) position_scan_kernel(Pos
     __syncthreads();
     const T* Z = reinterpret_cast<const T*>(prm.Z);
     const int lane = threadIdx.x & 31;
-    constexpr int U = RT <= 8 ? 9 : 4;            // loads issued together, in groups of equal size
+    constexpr int U = RT <= 8 ? 10 : 4;           // loads issued together, in groups of equal size
     const int n_groups = (prm.P + U - 1) / U, gs = (prm.P + n_groups - 1) / n_groups;
     // all lanes of a warp run the same rounds (the counters are updated once per warp and round)
     for (int64_t base = (int64_t)blockIdx.x * 256; base < prm.L; base += (int64_t)gridDim.x * 256) {
