@@ -18,7 +18,8 @@
  *     errors only.  Data-dependent outcomes (no error / corrected / decoding failure) are
  *     written to a gpd_locate_result in device memory.  With the plan uploaded beforehand
  *     (gpd_plan_upload) the compute calls below, gpd_locate_errors_static excepted, may be issued
- *     on a stream that is being captured into a CUDA graph.
+ *     on a stream that is being captured into a CUDA graph; the graph's kernels read the plan's
+ *     device tables, so the plan must outlive every replay.
  *   - The library allocates device memory only for the plan's small coefficient tables and, on
  *     FP32 plans, a scratch area of 64 KB per SM behind them (one allocation, made by
  *     gpd_plan_upload or on the plan's first compute call, freed by gpd_plan_destroy).
