@@ -216,7 +216,8 @@ gpd_status gpd_plan(const gpd_shape* shape, const gpd_split* split, int32_t P,
 gpd_status gpd_plan_subst(const gpd_shape* shape, const gpd_split* split, gpd_substitution subst, int32_t P,
                           const double* points_host, gpd_precision precision, gpd_plan_t* out);
 /* Uploads the plan's coefficient tables to the current device now (one cudaMalloc - tables, plus the
- * scratch area of FP32 plans - and one synchronous copy of a few KB) instead of at the plan's first compute call; a second call does nothing.  Lets a
+ * scratch area of FP32 plans -, one synchronous copy of a few KB, and three one-block kernels that
+ * precompute the decoding matrices of the error-free case, waited for) instead of at the plan's first compute call; a second call does nothing.  Lets a
  * caller keep allocation and synchronisation out of its timed or captured region. */
 gpd_status gpd_plan_upload(gpd_plan_t plan);
 gpd_status gpd_plan_destroy(gpd_plan_t plan);

@@ -55,6 +55,11 @@ struct DeviceTables {
     // parts of a split contraction; one product launch of a plan uses it at a time
     void* splitk = nullptr;
     int64_t splitk_bytes = 0;
+    // decoding matrices of the error-free case (every node in use), one per product, computed once at
+    // upload by the kernel that otherwise computes them per call: [wanted][P] doubles at these offsets
+    // (in doubles from base; -1: none), and one int of scratch for that kernel's gate
+    int64_t off_dcache[4] = {-1, -1, -1, -1};
+    int64_t off_dcache_gate = -1;
 };
 
 }  // namespace gpd
@@ -134,6 +139,8 @@ gpd_status regenerate_launch(gpd_plan_s* plan, void* shares, const gpd_locate_re
 gpd_status correct_positions_launch(gpd_plan_s* plan, gpd_product which, void* outputs, gpd_position_result* result,
                                     void* workspace, cudaStream_t st);
 int64_t position_workspace_bytes(const gpd_plan_s* plan);
+// Fills the plan's cache of error-free decoding matrices (called once, from the upload, on the default stream).
+gpd_status decode_cache_fill(gpd_plan_s* plan);
 gpd_status decode_launch(gpd_plan_s* plan, gpd_product which, const void* outputs, bool have_mask,
                          uint64_t use_mask, const gpd_locate_result* result, float* out, float* act_out,
                          int activation, void* workspace, cudaStream_t st);

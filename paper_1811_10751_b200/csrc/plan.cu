@@ -126,6 +126,11 @@ gpd_status ensure_device(gpd_plan_s* plan) {
     d.off_coefXup = push(plan->coefXup);
     for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT}) plan->prod[w].off_H = push(plan->prod[w].H);
     for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT}) plan->prod[w].off_Hg = push(plan->prod[w].Hg);
+    for (int w : {GPD_FWD, GPD_BWD, GPD_AUDIT}) {
+        if (plan->prod[w].Q == 0) continue;
+        d.off_dcache[w] = push(std::vector<double>((size_t)plan->prod[w].grid_rows * plan->prod[w].grid_cols * plan->P, 0.0));
+    }
+    d.off_dcache_gate = push(std::vector<double>(1, 0.0));
     d.n_doubles = (int64_t)host.size();
     if (cudaGetDevice(&plan->device) != cudaSuccess) return GPD_ERR_CUDA;
     const int64_t table_bytes = (int64_t)sizeof(double) * (int64_t)host.size();      // a multiple of 256
@@ -135,6 +140,11 @@ gpd_status ensure_device(gpd_plan_s* plan) {
     d.splitk_bytes = scratch_bytes;
     if (cudaMemcpy(d.base, host.data(), sizeof(double) * host.size(), cudaMemcpyHostToDevice) !=
         cudaSuccess) {
+        cudaFree(d.base);
+        d.base = nullptr;
+        return GPD_ERR_CUDA;
+    }
+    if (decode_cache_fill(plan) != GPD_OK || cudaDeviceSynchronize() != cudaSuccess) {
         cudaFree(d.base);
         d.base = nullptr;
         return GPD_ERR_CUDA;
