@@ -99,6 +99,7 @@ struct I8Params {
     int P;
     double shrink, eta;                  // update: C <- shrink * C + eta * A B^T
     const gpd_locate_result* gate;       // update: skipped when this reports a decoding failure
+    unsigned int* colmax;                // update, optional: [P][N] largest |new C| per column (high words)
 };
 
 // One warp reads 16 lanes x 32 consecutive 32-bit columns of tensor memory in the 16 x 256-bit shape:
@@ -291,6 +292,9 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             if (lane == 0) mbar_arrive(&acc_empty);
             double* cbase = prm.C + (int64_t)p * prm.M * prm.N + r_base * prm.N + c_base;
             const bool vec = (prm.N & 1) == 0;       // 16-byte stores: pairs start at even columns
+            unsigned int cmax[NK][2];                // update: largest |new value| of this thread's rows, per column
+#pragma unroll
+            for (int k = 0; k < NK; ++k) cmax[k][0] = cmax[k][1] = 0u;
 #pragma unroll
             for (int ri = 0; ri < 4; ++ri) {
                 if (r_base + 8 * ri >= prm.M) continue;
@@ -310,16 +314,40 @@ gemm_i8_sliced_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                         if (UPDATE) {
                             o.x = fma(prm.eta, o.x, prm.shrink * old[k].x);
                             o.y = fma(prm.eta, o.y, prm.shrink * old[k].y);
+                            cmax[k][0] = max(cmax[k][0], (unsigned int)__double2hiint(o.x) & 0x7FFFFFFFu);
+                            cmax[k][1] = max(cmax[k][1], (unsigned int)__double2hiint(o.y) & 0x7FFFFFFFu);
                             *reinterpret_cast<double2*>(crow + 8 * k) = o;      // read again soon: no streaming hint
                         } else {
                             __stcs(reinterpret_cast<double2*>(crow + 8 * k), o);
                         }
                     } else {
-                        if (c_base + 8 * k < prm.N) crow[8 * k] = UPDATE ? fma(prm.eta, o.x, prm.shrink * crow[8 * k]) : o.x;
-                        if (c_base + 8 * k + 1 < prm.N)
-                            crow[8 * k + 1] = UPDATE ? fma(prm.eta, o.y, prm.shrink * crow[8 * k + 1]) : o.y;
+                        if (c_base + 8 * k < prm.N) {
+                            const double nx = UPDATE ? fma(prm.eta, o.x, prm.shrink * crow[8 * k]) : o.x;
+                            if (UPDATE) cmax[k][0] = max(cmax[k][0], (unsigned int)__double2hiint(nx) & 0x7FFFFFFFu);
+                            crow[8 * k] = nx;
+                        }
+                        if (c_base + 8 * k + 1 < prm.N) {
+                            const double ny = UPDATE ? fma(prm.eta, o.y, prm.shrink * crow[8 * k + 1]) : o.y;
+                            if (UPDATE) cmax[k][1] = max(cmax[k][1], (unsigned int)__double2hiint(ny) & 0x7FFFFFFFu);
+                            crow[8 * k + 1] = ny;
+                        }
                     }
                 }
+            }
+            if (UPDATE && prm.colmax) {
+                // column maxima of the new shares for the column-sliced copy: over this thread's four rows
+                // (above), then over the eight lanes that hold the same columns, one atomic per column
+#pragma unroll
+                for (int k = 0; k < NK; ++k)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        unsigned int v = cmax[k][e];
+                        v = max(v, __shfl_xor_sync(0xffffffffu, v, 4));
+                        v = max(v, __shfl_xor_sync(0xffffffffu, v, 8));
+                        v = max(v, __shfl_xor_sync(0xffffffffu, v, 16));
+                        if (rq == 0 && v && c_base + 8 * k + e < prm.N)
+                            atomicMax(prm.colmax + (int64_t)p * prm.N + c_base + 8 * k + e, v);
+                    }
             }
         }
     }
@@ -366,7 +394,7 @@ gpd_status gemm_i8_launch(const I8Gemm& g, cudaStream_t st) {
     I8Params prm{};
     prm.P = g.P; prm.M = g.M; prm.N = g.N; prm.K = g.K;
     prm.ea = g.ea; prm.eb = g.eb; prm.C = g.C;
-    prm.shrink = g.shrink; prm.eta = g.eta; prm.gate = g.gate;
+    prm.shrink = g.shrink; prm.eta = g.eta; prm.gate = g.gate; prm.colmax = g.colmax;
     if (g.update) return g.slices == 6 ? launch_i8<6, true>(g, prm, st) : GPD_ERR_UNSUPPORTED;
     return g.slices == 6 ? launch_i8<6, false>(g, prm, st) : launch_i8<5, false>(g, prm, st);
 }
@@ -427,9 +455,13 @@ gpd_status update_sliced_launch(gpd_plan_s* plan, void* W_shares, const void* Dh
     g.eb = reinterpret_cast<const int*>(reinterpret_cast<const char*>(Xhat_sliced) + lb.expo_offset);
     g.C = reinterpret_cast<double*>(W_shares);                     // the FP64 shares lead the buffer
     g.update = true; g.shrink = shrink; g.eta = eta; g.gate = gate;
+    // the epilogue meets the column maxima of the new shares, which the re-cut of the column copy needs
+    const TrainLayout tl = train_layout(plan);
+    g.colmax = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(W_shares) + tl.cols_offset + tl.cols.amax_offset);
+    if (cudaMemsetAsync(g.colmax, 0, sizeof(unsigned int) * g.P * g.N, st) != cudaSuccess) return GPD_ERR_CUDA;
     gpd_status rc = gemm_i8_launch(g, st);
     if (rc != GPD_OK) return rc;
-    return reslice_launch(plan, W_shares, st);
+    return reslice_launch(plan, W_shares, st, gate, true);
 }
 
 int i8_device_status_fetch_and_clear() {

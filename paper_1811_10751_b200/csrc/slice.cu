@@ -387,7 +387,9 @@ __global__ void __launch_bounds__(256) colpass_kernel(SliceParams prm) {
 // per plane at a time.
 template <int S>
 __global__ void __launch_bounds__(256) reslice_rows_kernel(const double* __restrict__ master, int8_t* planes, int* expo,
-                                                          int64_t n_rows, int64_t K, int64_t plane_stride) {
+                                                          int64_t n_rows, int64_t K, int64_t plane_stride,
+                                                          const gpd_locate_result* gate) {
+    if (gate && gate->outcome == GPD_DECODE_FAILURE) return;      // the update was skipped: the copies still hold the shares
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     if (row >= n_rows) return;                                     // whole warp
@@ -432,8 +434,9 @@ constexpr int RC_ROWS = 128, RC_COLS = 32, RC_PITCH = RC_ROWS + 1;
 template <int S>
 __global__ void __launch_bounds__(256) reslice_cols_kernel(const double* __restrict__ master, const unsigned int* amax,
                                                           int8_t* planes, int* expo, int64_t M, int64_t K,
-                                                          int64_t plane_stride) {
+                                                          int64_t plane_stride, const gpd_locate_result* gate) {
     __shared__ double xs[RC_COLS * RC_PITCH];
+    if (gate && gate->outcome == GPD_DECODE_FAILURE) return;      // the update was skipped: the copies still hold the shares
     const int64_t c0 = (int64_t)blockIdx.x * RC_COLS, r0 = (int64_t)blockIdx.y * RC_ROWS, p = blockIdx.z;
     const double* src = master + p * M * K;
     for (int idx = threadIdx.x; idx < RC_ROWS * RC_COLS; idx += 256) {
@@ -572,7 +575,8 @@ SlicedLayout sliced_layout(int slices, int64_t P, int64_t rows, int64_t K) {
     return l;
 }
 
-gpd_status reslice_launch(gpd_plan_s* plan, void* W_shares, cudaStream_t st) {
+gpd_status reslice_launch(gpd_plan_s* plan, void* W_shares, cudaStream_t st, const gpd_locate_result* gate,
+                          bool cols_amax_ready) {
     if (!plan->train) return GPD_ERR_UNSUPPORTED;
     const gpd_shape& s = plan->shape;
     const gpd_split& c = plan->split;
@@ -584,18 +588,20 @@ gpd_status reslice_launch(gpd_plan_s* plan, void* W_shares, cudaStream_t st) {
         int8_t* planes = reinterpret_cast<int8_t*>(base + tl.rows_offset);
         int* expo = reinterpret_cast<int*>(base + tl.rows_offset + tl.rows.expo_offset);
         const int64_t n_rows = P * M;
-        reslice_rows_kernel<6><<<(unsigned)((n_rows + 7) / 8), 256, 0, st>>>(master, planes, expo, n_rows, K, P * M * K);
+        reslice_rows_kernel<6><<<(unsigned)((n_rows + 7) / 8), 256, 0, st>>>(master, planes, expo, n_rows, K, P * M * K, gate);
         if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
     }
     {   // columns of the shares
         int8_t* planes = reinterpret_cast<int8_t*>(base + tl.cols_offset);
         int* expo = reinterpret_cast<int*>(base + tl.cols_offset + tl.cols.expo_offset);
         unsigned int* amax = reinterpret_cast<unsigned int*>(base + tl.cols_offset + tl.cols.amax_offset);
-        if (cudaMemsetAsync(amax, 0, sizeof(unsigned int) * P * K, st) != cudaSuccess) return GPD_ERR_CUDA;
-        colmax_kernel<<<dim3((unsigned)((K + 255) / 256), (unsigned)((M + 63) / 64), (unsigned)P), 256, 0, st>>>(master, amax, M, K);
-        if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+        if (!cols_amax_ready) {
+            if (cudaMemsetAsync(amax, 0, sizeof(unsigned int) * P * K, st) != cudaSuccess) return GPD_ERR_CUDA;
+            colmax_kernel<<<dim3((unsigned)((K + 255) / 256), (unsigned)((M + 63) / 64), (unsigned)P), 256, 0, st>>>(master, amax, M, K);
+            if (launch_ok() != GPD_OK) return GPD_ERR_CUDA;
+        }
         reslice_cols_kernel<6><<<dim3((unsigned)((K + RC_COLS - 1) / RC_COLS), (unsigned)((M + RC_ROWS - 1) / RC_ROWS), (unsigned)P),
-                                 256, 0, st>>>(master, amax, planes, expo, M, K, P * M * K);
+                                 256, 0, st>>>(master, amax, planes, expo, M, K, P * M * K, gate);
     }
     return launch_ok();
 }

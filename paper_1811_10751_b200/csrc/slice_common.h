@@ -43,7 +43,10 @@ bool sliced_supported(const gpd_plan_s* plan);
 // Encoders.  operand: -1 = W (gpd_encode_A), else a gpd_operand.  dst: the caller's share buffer.
 gpd_status encode_sliced_launch(gpd_plan_s* plan, int operand, const float* src, void* dst, cudaStream_t st);
 // Training mode: cut both sliced copies of W's shares from the FP64 shares at the start of the buffer.
-gpd_status reslice_launch(gpd_plan_s* plan, void* W_shares, cudaStream_t st);
+// gate (optional): a result whose decoding failure means the shares were left as they were: nothing is re-cut.
+// cols_amax_ready: the column maxima already sit in the column copy's scratch (the update's epilogue met them).
+gpd_status reslice_launch(gpd_plan_s* plan, void* W_shares, cudaStream_t st, const gpd_locate_result* gate = nullptr,
+                          bool cols_amax_ready = false);
 
 // One batched int8 digit-plane product with FP64 recombination:
 //   C[p] (M x N, FP64, row-major) = A[p] (M x K) * B[p] (N x K)^T      for p = 0 .. P-1,
@@ -58,6 +61,7 @@ struct I8Gemm {
     bool update;
     double shrink, eta;
     const gpd_locate_result* gate;
+    unsigned int* colmax;       // update, optional: [P][N] largest |new C| per column (high words, zero on entry)
 };
 gpd_status gemm_i8_launch(const I8Gemm& g, cudaStream_t st);
 

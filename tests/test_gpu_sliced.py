@@ -336,6 +336,17 @@ def test_training_mode_products_update_and_audit_match_oracle(N1, N0, B, m, n, P
     assert np.abs(got - want).max() <= 1e-12 * np.abs(want).max()
     Z3 = cp.outputs_as_array(g.GPD_FWD, cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X)))
     assert np.abs(Z3 - Z2o).max() <= 1e-10 * np.sqrt(np.mean(Z2o ** 2))
+    # an update gated by a failed decode of the backward product changes nothing: neither the FP64 shares
+    # nor the two sliced copies (the forward and the backward product read them)
+    gate = g.new_results(1)
+    gate.view(torch.int32)[0] = g.GPD_DECODE_FAILURE
+    before = host(Wsh).copy()
+    Zb3 = cp.outputs_as_array(g.GPD_BWD, cp.products(g.GPD_BWD, cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT)))
+    g.gpd_update_shares(cp.plan, Wsh, cp.encode(g.GPD_OPERAND_DELTA_UPD, Delta), cp.encode(g.GPD_OPERAND_X_UPD, X),
+                        eta, lam, gate=gate)
+    assert np.array_equal(host(Wsh)[:P * M * K], before[:P * M * K])
+    assert np.array_equal(cp.outputs_as_array(g.GPD_FWD, cp.products(g.GPD_FWD, cp.encode(g.GPD_OPERAND_X_FWD, X))), Z3)
+    assert np.array_equal(cp.outputs_as_array(g.GPD_BWD, cp.products(g.GPD_BWD, cp.encode(g.GPD_OPERAND_DELTAT_BWD, DT))), Zb3)
     assert g.gpd_device_status() == 0
 
 
