@@ -593,6 +593,8 @@ def run_matvec(args, steps):
     # stream they are given).  Reported beside the eager figure, never instead of it.
     graph_ms = None
     try:
+        if getattr(args, "no_graph", False):
+            raise RuntimeError("graph replay switched off")
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=stream):
             g.gpd_encode_B(plan, g.GPD_OPERAND_X_FWD, Xd, Xsh, stream=stream)
@@ -728,6 +730,8 @@ def run_layer(args, kind, steps):
     # the same step captured once into a CUDA graph and replayed (reported beside the eager figure)
     graph_ms = None
     try:
+        if getattr(args, "no_graph", False):
+            raise RuntimeError("graph replay switched off")
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=stream):
             step(0)
@@ -919,6 +923,12 @@ def relaunch_under_torchrun(args):
     return subprocess.call(cmd)
 
 
+def under_profiler() -> bool:
+    """True when a CUDA profiler has injected itself into this process (ncu, nsys, compute-sanitizer)."""
+    return any(k in os.environ for k in ("CUDA_INJECTION64_PATH", "NV_COMPUTE_PROFILER_PERFWORKS_DIR",
+                                         "NVTX_INJECTION64_PATH", "NV_NSIGHT_INJECTION_PORT_BASE"))
+
+
 def brief(line):
     """What the `secondary` object keeps of a secondary workload's line."""
     keep = ("value", "unit", "ms_per_step", "graph_replay_ms_per_step", "dtype", "kernel_ms", "gemv_ms", "encode_W_once_ms", "encode_W_hbm_frac",
@@ -951,7 +961,11 @@ def main():
     ap.add_argument("--repeats", type=int, default=5, help="timed regions of --steps steps each (the median is reported)")
     ap.add_argument("--no-secondary", action="store_true",
                     help="leave the short runs of the other workloads out of the default line")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="leave the CUDA-graph replay figures out (set by itself under a profiler: ncu "
+                         "ends a process that launches into a stream capture)")
     args = ap.parse_args()
+    args.no_graph = args.no_graph or under_profiler()
     if args.gpus > 1 and "RANK" not in os.environ:
         sys.exit(relaunch_under_torchrun(args))
     import workloads as wl
