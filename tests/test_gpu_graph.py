@@ -12,6 +12,11 @@ torch = pytest.importorskip("torch")
 if not torch.cuda.is_available():
     pytest.skip("needs a CUDA device", allow_module_level=True)
 
+import os                                    # noqa: E402
+
+if any(k in os.environ for k in ("CUDA_INJECTION64_PATH", "NV_COMPUTE_PROFILER_PERFWORKS_DIR", "NV_NSIGHT_INJECTION_PORT_BASE")):
+    pytest.skip("a profiler is attached: ncu ends a process that launches into a stream capture", allow_module_level=True)
+
 import paper_1811_10751_b200 as g            # noqa: E402
 
 
