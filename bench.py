@@ -47,9 +47,9 @@ FALLBACK_BF16_SUSTAINED = 1400.0
 FALLBACK_HBM_GBS = 6650.0
 CPU_SAMPLE_ROWS = 1024              # rows of W in the CPU sample (1/8 of the workload)
 TRAFFIC_BYTES_PER_LAUNCH = None     # dram read+write bytes of the dominant kernel from ncu (see profiles/)
-TRAFFIC_BYTES_PER_LAUNCH_SLICED = {6: 1552644000,   # gemm_i8_sliced_kernel<6>: dram read 1.355699 GB + write 0.196945 GB (profiles/)
+TRAFFIC_BYTES_PER_LAUNCH_SLICED = {6: 1541924000,   # gemm_i8_sliced_kernel<6>: dram read 1.345208 GB + write 0.196716 GB (profiles/)
                                    5: None}         # five planes: no counters taken
-TENSOR_PIPE_PCT_NCU = {6: 79.0, 5: None}            # sm__pipe_tensor_cycles_active, % of elapsed (profiles/)
+TENSOR_PIPE_PCT_NCU = {6: 79.3, 5: None}            # sm__pipe_tensor_cycles_active, % of elapsed (profiles/)
 
 
 def load_peaks():
